@@ -1,0 +1,738 @@
+// Host side of libconflayers.so: context, weight arena, and the sequencing of the kernels that make
+// up a draft step, a verify pass, acceptance and the confidence scoring.  All arithmetic of the
+// method runs in the kernels; this file only lays out memory and enqueues launches on one stream.
+#include <math.h>
+#include <stdarg.h>
+#include <stddef.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "cl_internal.h"
+
+struct ClLayer {
+    char *wqkv, *wo, *wgu, *wd;   // [3d,d] [d,d] [2F,d] (gate/up rows interleaved) [d,F]
+    float *n1, *n2;
+    char *kc, *vc;                // this layer's K and V cache [max_seq, d]
+};
+
+struct cl_ctx {
+    cl_model_cfg cfg;
+    cudaStream_t stream;
+    int device, n_sm;
+    char err[512];
+    size_t esz;                   // bytes per stored element (weights, KV, taps)
+    int loaded, head_only, prefilled;
+    // device memory
+    char *wbuf;                   // all layer matrices, one allocation, in execution order
+    char *embed, *lm_head;
+    float *final_norm, *norms;
+    char *kv;
+    float2 *rope_cs;
+    float *x, *xn, *qkv, *att, *hff, *att_part, *logits;
+    unsigned *tickets;            // [0] LM head ticket, [1 ..] attention tickets
+    ClHeadPartial *head_part;
+    int head_grid;
+    ClDevState *st;
+    ClDevState *h_st;             // pinned host mirror
+    int *prompt_dev;              // [max_seq]
+    int *out_dev;                 // generated tokens
+    int out_cap;
+    char *ring;                   // [L, P, d] storage type
+    // scoring scratch
+    float *sc_conf, *sc_pmax, *sc_clayer;
+    int *sc_arg;
+    size_t sc_cap;                // rows*P capacity
+    uint8_t *sel_mask;            // device [iters_cap, L]
+    double *sel_margins;          // device [L]
+    float *sel_clayers;           // device [iters_cap, L]
+    int sel_iters_cap;
+    std::vector<ClLayer> layers;
+    std::vector<uint8_t> mask;    // host copy of the skip set
+    int nsplit, per_max;
+    // host view of the device state (exact after every call that synchronises)
+    int h_ctx, h_ndraft, tapped;
+    uint64_t launches;
+};
+
+static char g_err[512] = "";
+
+static int fail(cl_ctx *c, int code, const char *fmt, ...) __attribute__((format(printf, 3, 4)));
+static int fail(cl_ctx *c, int code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(c ? c->err : g_err, 512, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define CU(call)                                                                                          \
+    do {                                                                                                  \
+        cudaError_t e_ = (call);                                                                          \
+        if (e_ != cudaSuccess) return fail(c, CL_ECUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+#define KL(call)                                                                                          \
+    do {                                                                                                  \
+        cudaError_t e_ = (call);                                                                          \
+        ++c->launches;                                                                                    \
+        if (e_ != cudaSuccess) return fail(c, CL_ECUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+#define ST_FIELD(c, type, field) ((type *)((char *)(c)->st + offsetof(ClDevState, field)))
+
+namespace {
+
+struct ClPoke {
+    int ctx, pending, n_drafted, done, n_out, max_new;   // -1 = leave unchanged
+    int n_force;
+    int force[CL_MAX_K];
+};
+
+__global__ void k_poke(ClDevState *st, ClPoke p) {
+    if (threadIdx.x != 0) return;
+    if (p.ctx >= 0) st->ctx = p.ctx;
+    if (p.pending >= 0) st->cyc_tok[0] = p.pending;
+    for (int i = 0; i < p.n_force; ++i) st->cyc_tok[1 + i] = p.force[i];
+    if (p.n_drafted >= 0) st->n_drafted = p.n_drafted;
+    if (p.done >= 0) st->done = p.done;
+    if (p.n_out >= 0) st->n_out = p.n_out;
+    if (p.max_new >= 0) st->max_new = p.max_new;
+}
+
+ClPoke poke_none() {
+    ClPoke p;
+    p.ctx = p.pending = p.n_drafted = p.done = p.n_out = p.max_new = -1;
+    p.n_force = 0;
+    return p;
+}
+
+}  // namespace
+
+static int poke(cl_ctx *c, const ClPoke &p) {
+    k_poke<<<1, 32, 0, c->stream>>>(c->st, p);
+    KL(cudaGetLastError());
+    return CL_OK;
+}
+
+static int sync_state(cl_ctx *c) {
+    CU(cudaMemcpyAsync(c->h_st, c->st, sizeof(ClDevState), cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    c->h_ctx = c->h_st->ctx;
+    return CL_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+
+extern "C" const char *cl_last_error(cl_ctx *c) { return c ? c->err : g_err; }
+
+extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **out) {
+    cl_ctx *c = nullptr;
+    if (!cfg || !out) return fail(c, CL_EINVAL, "cl_create: null argument");
+    *out = nullptr;
+    if (cfg->n_layers < 0 || cfg->d_model <= 0 || cfg->n_heads <= 0 || cfg->vocab < 2 || cfg->max_seq <= 0)
+        return fail(c, CL_EINVAL, "cl_create: non-positive dimension");
+    if (cfg->n_heads * cfg->head_dim != cfg->d_model) return fail(c, CL_EINVAL, "cl_create: d_model != n_heads * head_dim");
+    if (cfg->n_kv_heads != cfg->n_heads) return fail(c, CL_EINVAL, "cl_create: only n_kv_heads == n_heads is supported");
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return fail(c, CL_EINVAL, "cl_create: head_dim must be 64 or 128");
+    if (cfg->d_model % 8 || (cfg->n_layers > 0 && (cfg->d_ffn <= 0 || cfg->d_ffn % 8)))
+        return fail(c, CL_EINVAL, "cl_create: d_model and d_ffn must be multiples of 8");
+    if (cfg->weight_dtype != 0 && cfg->weight_dtype != 1) return fail(c, CL_EINVAL, "cl_create: weight_dtype must be 0 or 1");
+    if (cfg->tap_positions < 0) return fail(c, CL_EINVAL, "cl_create: tap_positions < 0");
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(c, CL_ECUDA, "cl_create: no CUDA device: %s", cudaGetErrorString(e));
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) return fail(c, CL_ECUDA, "cl_create: cudaGetDeviceProperties: %s", cudaGetErrorString(e));
+    if (prop.major < 10) return fail(c, CL_ECUDA, "cl_create: compute capability %d.%d, built for sm_100a only", prop.major, prop.minor);
+    c = new (std::nothrow) cl_ctx();
+    if (!c) return fail(nullptr, CL_ENOMEM, "cl_create: host allocation failed");
+    c->cfg = *cfg;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->device = dev;
+    c->n_sm = prop.multiProcessorCount;
+    c->esz = cfg->weight_dtype == 1 ? 2 : 4;
+    c->err[0] = 0;
+    c->mask.assign((size_t)cfg->n_layers, 0);
+    *out = c;
+    return CL_OK;
+}
+
+static void free_all(cl_ctx *c) {
+    void *ptrs[] = {c->wbuf, c->embed, c->lm_head, c->final_norm, c->norms, c->kv, c->rope_cs, c->x, c->xn, c->qkv,
+                    c->att, c->hff, c->att_part, c->logits, c->tickets, c->head_part, c->st, c->prompt_dev, c->out_dev,
+                    c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sel_mask, c->sel_margins, c->sel_clayers};
+    for (void *p : ptrs)
+        if (p) cudaFree(p);
+    if (c->h_st) cudaFreeHost(c->h_st);
+}
+
+extern "C" int cl_destroy(cl_ctx *c) {
+    if (!c) return CL_OK;
+    cudaStreamSynchronize(c->stream);
+    free_all(c);
+    delete c;
+    return CL_OK;
+}
+
+template <typename T>
+static cudaError_t dmalloc(T **p, size_t bytes) {
+    return cudaMalloc((void **)p, bytes ? bytes : 16);
+}
+
+#define DM(ptr, bytes)                                                                                          \
+    do {                                                                                                        \
+        cudaError_t e_ = dmalloc(&(ptr), (bytes));                                                              \
+        if (e_ != cudaSuccess) {                                                                                \
+            cudaGetLastError();                                                                                 \
+            return fail(c, e_ == cudaErrorMemoryAllocation ? CL_ENOMEM : CL_ECUDA, "cudaMalloc(%zu) for %s: %s", \
+                        (size_t)(bytes), #ptr, cudaGetErrorString(e_));                                         \
+        }                                                                                                       \
+    } while (0)
+
+extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
+    if (!c || !w) return fail(c, CL_EINVAL, "cl_load: null argument");
+    if (c->loaded) return fail(c, CL_ESTATE, "cl_load: weights already loaded");
+    const cl_model_cfg &g = c->cfg;
+    const size_t d = g.d_model, F = g.d_ffn, V = g.vocab, L = g.n_layers, es = c->esz;
+    c->head_only = w->head_only ? 1 : 0;
+    if (!w->lm_head || !w->final_norm) return fail(c, CL_EINVAL, "cl_load: lm_head / final_norm missing");
+    if (!c->head_only) {
+        if (!w->embed || !w->wq || !w->wk || !w->wv || !w->wo || !w->wg || !w->wu || !w->wd || !w->norm1 || !w->norm2)
+            return fail(c, CL_EINVAL, "cl_load: null weight array");
+        for (size_t l = 0; l < L; ++l)
+            if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->wg[l] || !w->wu[l] || !w->wd[l] || !w->norm1[l] ||
+                !w->norm2[l])
+                return fail(c, CL_EINVAL, "cl_load: null weight pointer in layer %zu", l);
+    }
+    const cudaMemcpyKind kind = cudaMemcpyDefault;
+
+    // ---- head, norms, state (needed by every context)
+    DM(c->lm_head, V * d * es);
+    DM(c->final_norm, d * 4);
+    CU(cudaMemcpyAsync(c->lm_head, w->lm_head, V * d * es, kind, c->stream));
+    CU(cudaMemcpyAsync(c->final_norm, w->final_norm, d * 4, kind, c->stream));
+    DM(c->st, sizeof(ClDevState));
+    CU(cudaMemsetAsync(c->st, 0, sizeof(ClDevState), c->stream));
+    CU(cudaMallocHost((void **)&c->h_st, sizeof(ClDevState)));
+    memset(c->h_st, 0, sizeof(ClDevState));
+    DM(c->xn, (size_t)CL_MAX_T * d * 4);
+    DM(c->logits, (size_t)CL_MAX_T * V * 4);
+    c->head_grid = c->n_sm * 4;
+    DM(c->head_part, (size_t)c->head_grid * CL_MAX_T * sizeof(ClHeadPartial));
+    const size_t n_tickets = 1 + (size_t)CL_MAX_T * g.n_heads;
+    DM(c->tickets, n_tickets * 4);
+    CU(cudaMemsetAsync(c->tickets, 0, n_tickets * 4, c->stream));
+    DM(c->sel_margins, (L ? L : 1) * sizeof(double));
+    DM(c->sc_clayer, (L ? L : 1) * 4);
+
+    if (!c->head_only) {
+        // ---- weights: per layer [Wqkv | Wo | Wgu | Wd], contiguous in execution order
+        const size_t b_qkv = 3 * d * d * es, b_o = d * d * es, b_gu = 2 * F * d * es, b_d = d * F * es;
+        const size_t per_layer = b_qkv + b_o + b_gu + b_d;
+        DM(c->wbuf, per_layer * L);
+        DM(c->norms, 2 * L * d * 4);
+        DM(c->embed, V * d * es);
+        CU(cudaMemcpyAsync(c->embed, w->embed, V * d * es, kind, c->stream));
+        const size_t kv_layer = (size_t)g.max_seq * d * es;
+        DM(c->kv, 2 * L * kv_layer);
+        CU(cudaMemsetAsync(c->kv, 0, 2 * L * kv_layer, c->stream));
+        char *stage_g = nullptr, *stage_u = nullptr;
+        if (!w->on_device) {
+            DM(stage_g, F * d * es);
+            DM(stage_u, F * d * es);
+        }
+        c->layers.resize(L);
+        for (size_t l = 0; l < L; ++l) {
+            ClLayer &y = c->layers[l];
+            y.wqkv = c->wbuf + l * per_layer;
+            y.wo = y.wqkv + b_qkv;
+            y.wgu = y.wo + b_o;
+            y.wd = y.wgu + b_gu;
+            y.n1 = c->norms + (2 * l) * d;
+            y.n2 = c->norms + (2 * l + 1) * d;
+            y.kc = c->kv + (2 * l) * kv_layer;
+            y.vc = c->kv + (2 * l + 1) * kv_layer;
+            CU(cudaMemcpyAsync(y.wqkv, w->wq[l], d * d * es, kind, c->stream));
+            CU(cudaMemcpyAsync(y.wqkv + d * d * es, w->wk[l], d * d * es, kind, c->stream));
+            CU(cudaMemcpyAsync(y.wqkv + 2 * d * d * es, w->wv[l], d * d * es, kind, c->stream));
+            CU(cudaMemcpyAsync(y.wo, w->wo[l], b_o, kind, c->stream));
+            CU(cudaMemcpyAsync(y.wd, w->wd[l], b_d, kind, c->stream));
+            CU(cudaMemcpyAsync(y.n1, w->norm1[l], d * 4, kind, c->stream));
+            CU(cudaMemcpyAsync(y.n2, w->norm2[l], d * 4, kind, c->stream));
+            const void *sg = w->wg[l], *su = w->wu[l];
+            if (!w->on_device) {
+                CU(cudaMemcpyAsync(stage_g, sg, F * d * es, kind, c->stream));
+                CU(cudaMemcpyAsync(stage_u, su, F * d * es, kind, c->stream));
+                sg = stage_g;
+                su = stage_u;
+            }
+            KL(cl_launch_interleave(g.weight_dtype, sg, su, y.wgu, (int)F, (int)d, c->stream));
+        }
+        // ---- rotary table cos/sin(pos * theta^(-2i/hd)), evaluated in double on the host
+        const int half = g.head_dim / 2;
+        std::vector<float2> cs((size_t)g.max_seq * half);
+        for (int p = 0; p < g.max_seq; ++p)
+            for (int i = 0; i < half; ++i) {
+                const double ang = (double)p * pow((double)g.rope_theta, -2.0 * i / g.head_dim);
+                cs[(size_t)p * half + i] = make_float2((float)cos(ang), (float)sin(ang));
+            }
+        DM(c->rope_cs, cs.size() * sizeof(float2));
+        CU(cudaMemcpyAsync(c->rope_cs, cs.data(), cs.size() * sizeof(float2), cudaMemcpyHostToDevice, c->stream));
+        // ---- activations and scratch
+        DM(c->x, (size_t)CL_MAX_T * d * 4);
+        DM(c->qkv, (size_t)CL_MAX_T * 3 * d * 4);
+        DM(c->att, (size_t)CL_MAX_T * d * 4);
+        DM(c->hff, (size_t)CL_MAX_T * F * 4);
+        c->nsplit = 4;
+        c->per_max = (g.max_seq + c->nsplit - 1) / c->nsplit;
+        DM(c->att_part, (size_t)CL_MAX_T * g.n_heads * c->nsplit * (g.head_dim + 2) * 4);
+        DM(c->prompt_dev, (size_t)g.max_seq * 4);
+        if (g.tap_positions > 0) {
+            DM(c->ring, L * (size_t)g.tap_positions * d * es);
+            CU(cudaMemsetAsync(c->ring, 0, L * (size_t)g.tap_positions * d * es, c->stream));
+        }
+        CU(cudaStreamSynchronize(c->stream));   // host staging vector and borrowed pointers are released after this
+        if (stage_g) cudaFree(stage_g);
+        if (stage_u) cudaFree(stage_u);
+    } else {
+        CU(cudaStreamSynchronize(c->stream));
+    }
+    c->loaded = 1;
+    return CL_OK;
+}
+
+// ---- one pass of T rows through the kept layers ------------------------------------------------
+
+static int gemv(cl_ctx *c, int T, int epi, const void *W, int rows, int cols, const float *xin, float *out, int ld) {
+    ClGemvArgs a;
+    memset(&a, 0, sizeof(a));
+    a.W = W; a.rows = rows; a.cols = cols; a.xin = xin; a.out = out; a.ld = ld; a.st = c->st;
+    const int ngroups = (rows + 1) / 2;
+    int grid = (ngroups + 7) / 8;
+    if (grid > c->n_sm * 4) grid = c->n_sm * 4;
+    KL(cl_launch_gemv(c->cfg.weight_dtype, T, epi, a, grid, c->stream));
+    return CL_OK;
+}
+
+static int head(cl_ctx *c, int T, const float *xin, const ClDevState *st, int *out_tok, float *out_pmax, float *out_conf,
+                float *logits) {
+    ClGemvArgs a;
+    memset(&a, 0, sizeof(a));
+    a.W = c->lm_head; a.rows = c->cfg.vocab; a.cols = c->cfg.d_model; a.xin = xin; a.st = st;
+    a.logits = logits; a.partials = c->head_part; a.ticket = c->tickets;
+    a.out_tok = out_tok; a.out_pmax = out_pmax; a.out_conf = out_conf;
+    a.inv_log_v = (float)(1.0 / log((double)c->cfg.vocab));
+    const int ngroups = (a.rows + 1) / 2;
+    int grid = (ngroups + 7) / 8;
+    if (grid > c->head_grid) grid = c->head_grid;
+    KL(cl_launch_gemv(c->cfg.weight_dtype, T, CL_EPI_HEAD, a, grid, c->stream));
+    return CL_OK;
+}
+
+// tok: device pointer to the T token ids; rows sit at positions st->ctx + row0 + t.
+static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_t *mask, int tap, int want_head,
+                        int *out_tok, float *out_pmax, float *out_conf, float *logits) {
+    const cl_model_cfg &g = c->cfg;
+    const int d = g.d_model, F = g.d_ffn, wd = g.weight_dtype;
+    int rc;
+    KL(cl_launch_embed(wd, c->embed, tok, T, d, c->x, c->st, c->stream));
+    for (int l = 0; l < g.n_layers; ++l) {
+        if (mask && mask[l]) continue;
+        const ClLayer &y = c->layers[l];
+        // attention half: RMSNorm -> QKV -> rotary + cache append -> attention over the cache -> output projection + residual
+        KL(cl_launch_rmsnorm(c->x, y.n1, T, d, g.rms_eps, c->xn, c->st, c->stream));
+        if ((rc = gemv(c, T, CL_EPI_STORE, y.wqkv, 3 * d, d, c->xn, c->qkv, 3 * d))) return rc;
+        KL(cl_launch_rope_append(wd, c->qkv, T, row0, g.n_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq, c->st,
+                                 c->stream));
+        ClAttnArgs a;
+        a.q = c->qkv; a.ld_q = 3 * d; a.kcache = y.kc; a.vcache = y.vc; a.part = c->att_part; a.tickets = c->tickets + 1;
+        a.out = c->att; a.st = c->st; a.row0 = row0; a.n_heads = g.n_heads; a.head_dim = g.head_dim; a.d_model = d;
+        a.nsplit = c->nsplit; a.per_max = c->per_max; a.max_seq = g.max_seq;
+        KL(cl_launch_attn(wd, T, a, c->stream));
+        if ((rc = gemv(c, T, CL_EPI_RESID, y.wo, d, d, c->att, c->x, d))) return rc;
+        // FFN half: RMSNorm -> gate/up + SiLU -> down projection + residual
+        KL(cl_launch_rmsnorm(c->x, y.n2, T, d, g.rms_eps, c->xn, c->st, c->stream));
+        if ((rc = gemv(c, T, CL_EPI_SILU, y.wgu, 2 * F, d, c->xn, c->hff, F))) return rc;
+        if ((rc = gemv(c, T, CL_EPI_RESID, y.wd, d, F, c->hff, c->x, d))) return rc;
+        if (tap && c->ring)
+            KL(cl_launch_tap(wd, c->x, T, row0, d, c->ring + (size_t)l * g.tap_positions * d * c->esz, g.tap_positions, c->st,
+                             c->stream));
+    }
+    if (want_head) {
+        KL(cl_launch_rmsnorm(c->x, c->final_norm, T, d, g.rms_eps, c->xn, c->st, c->stream));
+        if ((rc = head(c, T, c->xn, c->st, out_tok, out_pmax, out_conf, logits))) return rc;
+    }
+    return CL_OK;
+}
+
+static int need_model(cl_ctx *c, const char *fn, bool need_prefill) {
+    if (!c) return fail(c, CL_EINVAL, "%s: null context", fn);
+    if (!c->loaded) return fail(c, CL_ESTATE, "%s: no weights loaded", fn);
+    if (c->head_only) return fail(c, CL_ESTATE, "%s: context was loaded head-only", fn);
+    if (need_prefill && !c->prefilled) return fail(c, CL_ESTATE, "%s: call cl_prefill first", fn);
+    return CL_OK;
+}
+
+extern "C" int cl_prefill(cl_ctx *c, const int32_t *tokens, int n, int tap_hidden, int32_t *first_token) {
+    int rc = need_model(c, "cl_prefill", false);
+    if (rc) return rc;
+    if (!tokens || n <= 0) return fail(c, CL_EINVAL, "cl_prefill: empty prompt");
+    if (n + 1 > c->cfg.max_seq) return fail(c, CL_ERANGE, "cl_prefill: prompt of %d tokens exceeds max_seq %d", n, c->cfg.max_seq);
+    for (int i = 0; i < n; ++i)
+        if (tokens[i] < 0 || tokens[i] >= c->cfg.vocab) return fail(c, CL_EINVAL, "cl_prefill: token %d out of range at %d", tokens[i], i);
+    CU(cudaMemcpyAsync(c->prompt_dev, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, c->stream));
+    ClPoke p = poke_none();
+    p.ctx = 0; p.n_drafted = 0; p.done = 0;
+    if ((rc = poke(c, p))) return rc;
+    for (int c0 = 0; c0 < n; c0 += CL_PREFILL_CHUNK) {
+        const int T = (n - c0 < CL_PREFILL_CHUNK) ? n - c0 : CL_PREFILL_CHUNK;
+        const bool last = c0 + T >= n;
+        rc = forward_rows(c, c->prompt_dev + c0, T, 0, nullptr, tap_hidden, last, ST_FIELD(c, int, tgt_tok),
+                          ST_FIELD(c, float, v_pmax), ST_FIELD(c, float, v_conf), nullptr);
+        if (rc) return rc;
+        KL(cl_launch_advance(c->st, T, last ? 1 : 0, c->stream));
+    }
+    if ((rc = sync_state(c))) return rc;
+    c->prefilled = 1;
+    c->h_ndraft = 0;
+    c->tapped = tap_hidden ? n : 0;
+    if (first_token) *first_token = c->h_st->cyc_tok[0];
+    return CL_OK;
+}
+
+extern "C" int cl_set_skip_set(cl_ctx *c, const uint8_t *mask) {
+    if (!c || !mask) return fail(c, CL_EINVAL, "cl_set_skip_set: null argument");
+    for (int l = 0; l < c->cfg.n_layers; ++l)
+        if (mask[l] != 0 && mask[l] != 3)
+            return fail(c, CL_EINVAL, "cl_set_skip_set: layer %d has mask %d; only 0 (kept) and 3 (whole layer) are supported", l, mask[l]);
+    c->mask.assign(mask, mask + c->cfg.n_layers);
+    return CL_OK;
+}
+
+extern "C" int cl_get_skip_set(cl_ctx *c, uint8_t *mask) {
+    if (!c || !mask) return fail(c, CL_EINVAL, "cl_get_skip_set: null argument");
+    memcpy(mask, c->mask.data(), c->mask.size());
+    return CL_OK;
+}
+
+extern "C" int cl_draft(cl_ctx *c, int K, float stop_p, int32_t *toks, float *p_max, float *conf, float *logits,
+                        int *n_drafted) {
+    int rc = need_model(c, "cl_draft", true);
+    if (rc) return rc;
+    if (K < 1 || K > CL_MAX_K) return fail(c, CL_ERANGE, "cl_draft: K = %d outside 1..%d", K, CL_MAX_K);
+    if (c->h_ctx + K + 1 > c->cfg.max_seq) return fail(c, CL_ERANGE, "cl_draft: position %d exceeds max_seq", c->h_ctx + K);
+    int n = 0;
+    for (int i = 0; i < K; ++i) {
+        rc = forward_rows(c, ST_FIELD(c, int, cyc_tok) + i, 1, i, c->mask.data(), 0, 1, ST_FIELD(c, int, cyc_tok) + i + 1,
+                          ST_FIELD(c, float, d_pmax) + i, ST_FIELD(c, float, d_conf) + i,
+                          logits ? c->logits + (size_t)i * c->cfg.vocab : nullptr);
+        if (rc) return rc;
+        n = i + 1;
+        if (stop_p > 0.f) {   // confidence-aware early stop needs the probability on the host
+            if ((rc = sync_state(c))) return rc;
+            if (c->h_st->d_pmax[i] < stop_p) break;
+        }
+    }
+    ClPoke p = poke_none();
+    p.n_drafted = n;
+    if ((rc = poke(c, p))) return rc;
+    if ((rc = sync_state(c))) return rc;
+    c->h_ndraft = n;
+    if (logits) CU(cudaMemcpy(logits, c->logits, (size_t)n * c->cfg.vocab * 4, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < n; ++i) {
+        if (toks) toks[i] = c->h_st->cyc_tok[1 + i];
+        if (p_max) p_max[i] = c->h_st->d_pmax[i];
+        if (conf) conf[i] = c->h_st->d_conf[i];
+    }
+    if (n_drafted) *n_drafted = n;
+    return CL_OK;
+}
+
+extern "C" int cl_force_tokens(cl_ctx *c, const int32_t *toks, int n) {
+    int rc = need_model(c, "cl_force_tokens", true);
+    if (rc) return rc;
+    if (n < 0 || n > CL_MAX_K || (n > 0 && !toks)) return fail(c, CL_ERANGE, "cl_force_tokens: n = %d outside 0..%d", n, CL_MAX_K);
+    if (c->h_ctx + n + 1 > c->cfg.max_seq) return fail(c, CL_ERANGE, "cl_force_tokens: position exceeds max_seq");
+    ClPoke p = poke_none();
+    p.n_drafted = n;
+    p.n_force = n;
+    for (int i = 0; i < n; ++i) {
+        if (toks[i] < 0 || toks[i] >= c->cfg.vocab) return fail(c, CL_EINVAL, "cl_force_tokens: token out of range");
+        p.force[i] = toks[i];
+    }
+    if ((rc = poke(c, p))) return rc;
+    c->h_ndraft = n;
+    return CL_OK;
+}
+
+extern "C" int cl_verify(cl_ctx *c, int tap_hidden, int32_t *target_toks, float *logits) {
+    int rc = need_model(c, "cl_verify", true);
+    if (rc) return rc;
+    const int T = c->h_ndraft + 1;
+    if (c->h_ctx + T > c->cfg.max_seq) return fail(c, CL_ERANGE, "cl_verify: position exceeds max_seq");
+    rc = forward_rows(c, ST_FIELD(c, int, cyc_tok), T, 0, nullptr, tap_hidden, 1, ST_FIELD(c, int, tgt_tok),
+                      ST_FIELD(c, float, v_pmax), ST_FIELD(c, float, v_conf), logits ? c->logits : nullptr);
+    if (rc) return rc;
+    if ((rc = sync_state(c))) return rc;
+    if (tap_hidden) c->tapped += 1;
+    if (logits) CU(cudaMemcpy(logits, c->logits, (size_t)T * c->cfg.vocab * 4, cudaMemcpyDeviceToHost));
+    if (target_toks)
+        for (int i = 0; i < T; ++i) target_toks[i] = c->h_st->tgt_tok[i];
+    return CL_OK;
+}
+
+extern "C" int cl_accept(cl_ctx *c, int *n_accepted, int32_t *emitted) {
+    int rc = need_model(c, "cl_accept", true);
+    if (rc) return rc;
+    KL(cl_launch_accept(c->st, -1, nullptr, c->stream));
+    if ((rc = sync_state(c))) return rc;
+    c->h_ndraft = 0;
+    const int n = c->h_st->n_acc_last;
+    if (n_accepted) *n_accepted = n;
+    if (emitted)
+        for (int i = 0; i <= n; ++i) emitted[i] = c->h_st->emitted[i];
+    return CL_OK;
+}
+
+extern "C" int cl_step_vanilla(cl_ctx *c, int32_t *tok) {
+    int rc = need_model(c, "cl_step_vanilla", true);
+    if (rc) return rc;
+    if (c->h_ctx + 1 > c->cfg.max_seq) return fail(c, CL_ERANGE, "cl_step_vanilla: position exceeds max_seq");
+    ClPoke p = poke_none();
+    p.n_drafted = 0;
+    if ((rc = poke(c, p))) return rc;
+    rc = forward_rows(c, ST_FIELD(c, int, cyc_tok), 1, 0, nullptr, 0, 1, ST_FIELD(c, int, tgt_tok), ST_FIELD(c, float, v_pmax),
+                      ST_FIELD(c, float, v_conf), nullptr);
+    if (rc) return rc;
+    KL(cl_launch_accept(c->st, 0, nullptr, c->stream));
+    if ((rc = sync_state(c))) return rc;
+    c->h_ndraft = 0;
+    if (tok) *tok = c->h_st->emitted[0];
+    return CL_OK;
+}
+
+static int enqueue_cycle(cl_ctx *c, int K) {
+    int rc;
+    for (int i = 0; i < K; ++i) {
+        rc = forward_rows(c, ST_FIELD(c, int, cyc_tok) + i, 1, i, c->mask.data(), 0, 1, ST_FIELD(c, int, cyc_tok) + i + 1,
+                          ST_FIELD(c, float, d_pmax) + i, ST_FIELD(c, float, d_conf) + i, nullptr);
+        if (rc) return rc;
+    }
+    rc = forward_rows(c, ST_FIELD(c, int, cyc_tok), K + 1, 0, nullptr, 0, 1, ST_FIELD(c, int, tgt_tok),
+                      ST_FIELD(c, float, v_pmax), ST_FIELD(c, float, v_conf), nullptr);
+    if (rc) return rc;
+    KL(cl_launch_accept(c->st, K, c->out_dev, c->stream));
+    return CL_OK;
+}
+
+extern "C" int cl_generate(cl_ctx *c, int K, int max_new, int32_t *out, int *n_out, cl_stats *stats) {
+    int rc = need_model(c, "cl_generate", true);
+    if (rc) return rc;
+    if (K < 0 || K > CL_MAX_K) return fail(c, CL_ERANGE, "cl_generate: K = %d outside 0..%d", K, CL_MAX_K);
+    if (max_new <= 0 || !out) return fail(c, CL_EINVAL, "cl_generate: nothing to generate");
+    if (c->h_ctx + max_new + K > c->cfg.max_seq)
+        return fail(c, CL_ERANGE, "cl_generate: %d + %d + %d tokens exceed max_seq %d", c->h_ctx, max_new, K, c->cfg.max_seq);
+    if (max_new > c->out_cap) {
+        if (c->out_dev) cudaFree(c->out_dev);
+        c->out_dev = nullptr;
+        c->out_cap = 0;
+        DM(c->out_dev, (size_t)max_new * 4);
+        c->out_cap = max_new;
+    }
+    ClPoke p = poke_none();
+    p.n_out = 0; p.max_new = max_new; p.done = 0; p.n_drafted = 0;
+    if ((rc = poke(c, p))) return rc;
+    int remaining = max_new;
+    while (remaining > 0) {
+        // the fewest cycles that can finish the job; cycles enqueued past the end exit at once on the device
+        const int ncyc = (remaining + K) / (K + 1);
+        for (int i = 0; i < ncyc; ++i)
+            if ((rc = enqueue_cycle(c, K))) return rc;
+        if ((rc = sync_state(c))) return rc;
+        remaining = max_new - c->h_st->n_out;
+    }
+    CU(cudaMemcpy(out, c->out_dev, (size_t)max_new * 4, cudaMemcpyDeviceToHost));
+    p = poke_none();
+    p.done = 0;
+    if ((rc = poke(c, p))) return rc;
+    if ((rc = sync_state(c))) return rc;
+    c->h_ndraft = 0;
+    if (n_out) *n_out = max_new;
+    if (stats) cl_get_stats(c, stats);
+    return CL_OK;
+}
+
+extern "C" int cl_rollback(cl_ctx *c, int ctx_len, int32_t pending_token) {
+    int rc = need_model(c, "cl_rollback", true);
+    if (rc) return rc;
+    if (ctx_len < 0 || ctx_len > c->cfg.max_seq - 1) return fail(c, CL_ERANGE, "cl_rollback: ctx_len %d out of range", ctx_len);
+    if (pending_token < 0 || pending_token >= c->cfg.vocab) return fail(c, CL_EINVAL, "cl_rollback: token out of range");
+    ClPoke p = poke_none();
+    p.ctx = ctx_len; p.pending = pending_token; p.n_drafted = 0; p.done = 0;
+    if ((rc = poke(c, p))) return rc;
+    if ((rc = sync_state(c))) return rc;
+    c->h_ndraft = 0;
+    return CL_OK;
+}
+
+// ---- confidence scoring and selection -----------------------------------------------------------
+
+static int ensure_score_cap(cl_ctx *c, size_t n) {
+    if (n <= c->sc_cap) return CL_OK;
+    void *old[] = {c->sc_conf, c->sc_pmax, c->sc_arg};
+    for (void *q : old)
+        if (q) cudaFree(q);
+    c->sc_conf = c->sc_pmax = nullptr;
+    c->sc_arg = nullptr;
+    c->sc_cap = 0;
+    DM(c->sc_conf, n * 4);
+    DM(c->sc_pmax, n * 4);
+    DM(c->sc_arg, n * 4);
+    c->sc_cap = n;
+    return CL_OK;
+}
+
+// Scores rows*P hidden rows; leaves conf / p_max / argmax in the scoring scratch and the per-layer mean in c_layer_dev.
+static int score_rows(cl_ctx *c, const void *hidden, int rows, int P, float *c_layer_dev) {
+    const size_t n = (size_t)rows * P, d = c->cfg.d_model;
+    int rc = ensure_score_cap(c, n);
+    if (rc) return rc;
+    for (size_t r0 = 0; r0 < n; r0 += 8) {
+        const int T = (n - r0 < 8) ? (int)(n - r0) : 8;
+        KL(cl_launch_rmsnorm_rows(c->cfg.weight_dtype, (const char *)hidden + r0 * d * c->esz, c->final_norm, T, (int)d,
+                                  c->cfg.rms_eps, c->xn, c->stream));
+        if ((rc = head(c, T, c->xn, nullptr, c->sc_arg + r0, c->sc_pmax + r0, c->sc_conf + r0, nullptr))) return rc;
+    }
+    KL(cl_launch_mean_rows(c->sc_conf, rows, P, c_layer_dev, c->stream));
+    return CL_OK;
+}
+
+extern "C" int cl_layer_confidences(cl_ctx *c, const void *hidden, int rows, int P, float *conf_rows, float *p_max,
+                                    int32_t *argmax, float *c_layer) {
+    if (!c) return fail(c, CL_EINVAL, "cl_layer_confidences: null context");
+    if (!c->loaded) return fail(c, CL_ESTATE, "cl_layer_confidences: no weights loaded");
+    if (!hidden) {
+        if (!c->ring) return fail(c, CL_ESTATE, "cl_layer_confidences: no hidden-state ring (tap_positions = 0)");
+        if (c->tapped < c->cfg.tap_positions)
+            return fail(c, CL_ESTATE, "cl_layer_confidences: ring holds %d of %d positions", c->tapped, c->cfg.tap_positions);
+        hidden = c->ring;
+        rows = c->cfg.n_layers;
+        P = c->cfg.tap_positions;
+    }
+    if (rows <= 0 || P <= 0) return fail(c, CL_EINVAL, "cl_layer_confidences: rows and P must be positive");
+    if (rows > c->cfg.n_layers && c->cfg.n_layers > 0) {
+        // c_layer scratch is sized by n_layers; larger row counts use a temporary
+    }
+    float *cl_dev = c->sc_clayer;
+    float *tmp = nullptr;
+    if (rows > (c->cfg.n_layers ? c->cfg.n_layers : 1)) {
+        DM(tmp, (size_t)rows * 4);
+        cl_dev = tmp;
+    }
+    int rc = score_rows(c, hidden, rows, P, cl_dev);
+    if (!rc) {
+        const size_t n = (size_t)rows * P;
+        cudaError_t e = cudaStreamSynchronize(c->stream);
+        if (e == cudaSuccess && conf_rows) e = cudaMemcpy(conf_rows, c->sc_conf, n * 4, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess && p_max) e = cudaMemcpy(p_max, c->sc_pmax, n * 4, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess && argmax) e = cudaMemcpy(argmax, c->sc_arg, n * 4, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess && c_layer) e = cudaMemcpy(c_layer, cl_dev, (size_t)rows * 4, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) rc = fail(c, CL_ECUDA, "cl_layer_confidences: %s", cudaGetErrorString(e));
+    }
+    if (tmp) cudaFree(tmp);
+    return rc;
+}
+
+static int check_select(cl_ctx *c, const cl_select_cfg *s) {
+    if (!s) return fail(c, CL_EINVAL, "selection config is null");
+    if (s->lo < 0 || s->hi >= c->cfg.n_layers || s->hi - s->lo + 1 > 256)
+        return fail(c, CL_EINVAL, "selection range %d..%d outside the model's %d layers (or more than 256 eligible)", s->lo, s->hi, c->cfg.n_layers);
+    return CL_OK;
+}
+
+static int ensure_sel_iters(cl_ctx *c, int iters) {
+    if (iters <= c->sel_iters_cap) return CL_OK;
+    if (c->sel_mask) cudaFree(c->sel_mask);
+    if (c->sel_clayers) cudaFree(c->sel_clayers);
+    c->sel_mask = nullptr;
+    c->sel_clayers = nullptr;
+    c->sel_iters_cap = 0;
+    const size_t L = c->cfg.n_layers ? c->cfg.n_layers : 1;
+    DM(c->sel_mask, (size_t)iters * L);
+    DM(c->sel_clayers, (size_t)iters * L * 4);
+    c->sel_iters_cap = iters;
+    return CL_OK;
+}
+
+extern "C" int cl_select_skip_set(cl_ctx *c, const cl_select_cfg *s, const float *c_layer, uint8_t *mask, double *margins) {
+    if (!c || !mask) return fail(c, CL_EINVAL, "cl_select_skip_set: null argument");
+    if (!c->loaded) return fail(c, CL_ESTATE, "cl_select_skip_set: no weights loaded");
+    int rc = check_select(c, s);
+    if (rc) return rc;
+    if ((rc = ensure_sel_iters(c, 1))) return rc;
+    const int L = c->cfg.n_layers;
+    if (c_layer) CU(cudaMemcpyAsync(c->sc_clayer, c_layer, (size_t)L * 4, cudaMemcpyHostToDevice, c->stream));
+    KL(cl_launch_select(*s, L, c->sc_clayer, c->sel_mask, c->sel_margins, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    CU(cudaMemcpy(mask, c->sel_mask, (size_t)L, cudaMemcpyDeviceToHost));
+    if (margins) CU(cudaMemcpy(margins, c->sel_margins, (size_t)L * sizeof(double), cudaMemcpyDeviceToHost));
+    return CL_OK;
+}
+
+extern "C" int cl_score_loop(cl_ctx *c, const cl_select_cfg *s, const void *const *hidden_iters, int iters, int P,
+                             const float *scores, uint8_t *best_mask, int *best_iter, uint8_t *masks_all,
+                             float *c_layers_all) {
+    if (!c || !hidden_iters || !scores || iters <= 0 || P <= 0) return fail(c, CL_EINVAL, "cl_score_loop: bad argument");
+    if (!c->loaded) return fail(c, CL_ESTATE, "cl_score_loop: no weights loaded");
+    int rc = check_select(c, s);
+    if (rc) return rc;
+    if ((rc = ensure_sel_iters(c, iters))) return rc;
+    const int L = c->cfg.n_layers;
+    for (int it = 0; it < iters; ++it) {
+        if (!hidden_iters[it]) return fail(c, CL_EINVAL, "cl_score_loop: hidden_iters[%d] is null", it);
+        float *cl_dev = c->sel_clayers + (size_t)it * L;
+        if ((rc = score_rows(c, hidden_iters[it], L, P, cl_dev))) return rc;
+        KL(cl_launch_select(*s, L, cl_dev, c->sel_mask + (size_t)it * L, nullptr, c->stream));
+    }
+    std::vector<uint8_t> all((size_t)iters * L);
+    CU(cudaMemcpyAsync(all.data(), c->sel_mask, all.size(), cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    if (c_layers_all) CU(cudaMemcpy(c_layers_all, c->sel_clayers, (size_t)iters * L * 4, cudaMemcpyDeviceToHost));
+    int best = 0;   // round with the highest score; the earliest wins ties
+    for (int it = 1; it < iters; ++it)
+        if (scores[it] > scores[best]) best = it;
+    if (best_iter) *best_iter = best;
+    if (best_mask) memcpy(best_mask, all.data() + (size_t)best * L, (size_t)L);
+    if (masks_all) memcpy(masks_all, all.data(), all.size());
+    return CL_OK;
+}
+
+extern "C" int cl_read_hidden_ring(cl_ctx *c, void *out) {
+    if (!c || !out) return fail(c, CL_EINVAL, "cl_read_hidden_ring: null argument");
+    if (!c->ring) return fail(c, CL_ESTATE, "cl_read_hidden_ring: no ring (tap_positions = 0 or head-only context)");
+    CU(cudaStreamSynchronize(c->stream));
+    CU(cudaMemcpy(out, c->ring, (size_t)c->cfg.n_layers * c->cfg.tap_positions * c->cfg.d_model * c->esz, cudaMemcpyDeviceToHost));
+    return CL_OK;
+}
+
+extern "C" int cl_get_stats(cl_ctx *c, cl_stats *out) {
+    if (!c || !out) return fail(c, CL_EINVAL, "cl_get_stats: null argument");
+    memset(out, 0, sizeof(*out));
+    if (c->loaded && c->h_st) {
+        int rc = sync_state(c);
+        if (rc) return rc;
+        out->cycles = c->h_st->cycles;
+        out->drafted = c->h_st->drafted;
+        out->accepted = c->h_st->accepted;
+        out->emitted = c->h_st->emitted_total;
+        out->ctx_len = c->h_st->ctx;
+    }
+    for (uint8_t m : c->mask) out->n_skipped += (m != 0);
+    out->kernel_launches = c->launches;
+    return CL_OK;
+}

@@ -1,0 +1,88 @@
+// Internal declarations shared by the CUDA translation units of libconflayers.so.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "conflayers.h"
+
+#define CL_MAX_T (CL_MAX_K + 1)   // rows of the widest pass (verify)
+#define CL_PREFILL_CHUNK 8        // prompt tokens per prefill pass
+#define CL_LOGIT_CLAMP 1.0e4f     // clamp bound applied to fp32 logits (Section 3.1; the paper gives no bound)
+#define CL_SLOTS 16
+
+// Device-resident state of one context: everything a cycle needs so that no kernel argument
+// depends on values only the device knows (positions, pending tokens, counters).
+struct ClDevState {
+    int ctx;          // committed KV length; rows of a pass sit at positions ctx + row0 + t
+    int done;         // set by accept once max_new tokens are out: later kernels of the batch exit at once
+    int n_out;        // tokens written to the output buffer
+    int max_new;
+    int n_drafted;    // drafts of the current cycle
+    int n_acc_last;   // result of the last accept
+    int err;          // sticky device-side error flags
+    int pad;
+    int cyc_tok[CL_SLOTS];    // [0] pending token, [1..K] drafts
+    int tgt_tok[CL_SLOTS];    // [t] greedy token after verify row t
+    float d_pmax[CL_SLOTS], d_conf[CL_SLOTS];   // per draft step
+    float v_pmax[CL_SLOTS], v_conf[CL_SLOTS];   // per verify row
+    int emitted[CL_SLOTS];    // tokens emitted by the last accept
+    unsigned long long cycles, drafted, accepted, emitted_total;
+};
+
+// Partial softmax statistics of a slice of the vocabulary, relative to the slice maximum m:
+// z = sum exp(l - m), s = sum (l - m) exp(l - m); idx = position of m (lowest index on ties).
+struct ClHeadPartial {
+    float m, z, s;
+    int idx;
+};
+
+enum { CL_EPI_STORE = 0, CL_EPI_RESID = 1, CL_EPI_SILU = 2, CL_EPI_HEAD = 3 };
+
+struct ClGemvArgs {
+    const void *W;        // [rows, cols] storage type
+    int rows, cols;
+    const float *xin;     // [T, cols] fp32 activations
+    float *out;           // STORE: out[t*ld + r] = y; RESID: out[t*ld + r] += y; SILU: out[t*ld + r/2] = silu(y_r) * y_{r+1}
+    int ld;
+    const ClDevState *st;
+    // HEAD epilogue
+    float *logits;              // optional [T, rows]
+    ClHeadPartial *partials;    // [grid, T]
+    unsigned *ticket;
+    int *out_tok;               // [T] device
+    float *out_pmax, *out_conf; // [T] device
+    float inv_log_v;
+};
+
+struct ClAttnArgs {
+    const float *q;       // [T, ld_q] rotary-embedded queries (fp32)
+    int ld_q;
+    const void *kcache;   // this layer's K rows [max_seq, d] storage type
+    const void *vcache;
+    float *part;          // [T, H, nsplit, hd + 2] partial (m, l, o[hd])
+    unsigned *tickets;    // [T, H]
+    float *out;           // [T, d]
+    const ClDevState *st;
+    int row0, n_heads, head_dim, d_model, nsplit, per_max, max_seq;
+};
+
+// launchers (each returns the CUDA launch status)
+cudaError_t cl_launch_gemv(int wdtype, int T, int epi, const ClGemvArgs &a, int grid, cudaStream_t s);
+cudaError_t cl_launch_embed(int wdtype, const void *embed, const int *tok, int T, int d, float *x, const ClDevState *st,
+                            cudaStream_t s);
+cudaError_t cl_launch_rmsnorm(const float *x, const float *g, int T, int d, float eps, float *out, const ClDevState *st,
+                              cudaStream_t s);
+cudaError_t cl_launch_rmsnorm_rows(int in_dtype, const void *x, const float *g, int T, int d, float eps, float *out,
+                                   cudaStream_t s);
+cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H, int hd, int d, const float2 *rope_cs,
+                                  void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
+cudaError_t cl_launch_attn(int wdtype, int T, const ClAttnArgs &a, cudaStream_t s);
+cudaError_t cl_launch_tap(int wdtype, const float *x, int T, int row0, int d, void *ring_layer, int P,
+                          const ClDevState *st, cudaStream_t s);
+cudaError_t cl_launch_accept(ClDevState *st, int K, int *out_tokens, cudaStream_t s);
+cudaError_t cl_launch_advance(ClDevState *st, int n, int set_pending_from_tgt, cudaStream_t s);
+cudaError_t cl_launch_mean_rows(const float *conf_rows, int rows, int P, float *c_layer, cudaStream_t s);
+cudaError_t cl_launch_select(const cl_select_cfg &cfg, int n_layers, const float *c_layer, uint8_t *mask, double *margins,
+                             cudaStream_t s);
+cudaError_t cl_launch_interleave(int wdtype, const void *wg, const void *wu, void *dst, int F, int d, cudaStream_t s);

@@ -1,0 +1,253 @@
+"""GPU-vs-oracle parity through the C ABI (run on a B200): every step of the hot path on the five
+workloads (the two small ones in full; the 7B / 13B shapes with fewer layers and shorter runs so the
+CPU oracle finishes, plus properties that hold at any size; the scoring workload on sampled rows)."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2604_14612_b200 as cl
+import synth
+from oracle.selection import SelectConfig, select_skip_set, selection_details
+
+pytestmark = pytest.mark.gpu
+
+from harness import (NEAR_TIE, TOL, Report, lockstep_generate, make_pair, oracle_prefill_hidden,  # noqa: E402
+                     ring_in_position_order)
+
+
+def _select_cfgs(w, n_skip):
+    sc = cl.SelectCfg.make(w.lo, w.hi, n_skip=n_skip)
+    oc = SelectConfig(n_layers=w.shape.n_layers, lo=w.lo, hi=w.hi, n_skip=n_skip)
+    return sc, oc
+
+
+def _confidence_selected(om, ctx, w, prompt, P):
+    """Prefill with taps -> ring -> per-layer confidence -> Eq. 5-10 selection, both sides."""
+    first = ctx.cl_prefill(prompt, tap_hidden=True)
+    ring = ctx.cl_read_hidden_ring()
+    want_h = oracle_prefill_hidden(om, prompt, P)
+    got_h = ring_in_position_order(ring, len(prompt) - 1)
+    scale = max(1.0, float(np.abs(want_h).max()))
+    assert np.abs(got_h - want_h).max() <= 2 ** -7 * scale          # one storage-type ulp at the top of the range
+    g = ctx.cl_layer_confidences()
+    hid = torch.tensor(want_h).to(synth.torch_dtype(w.shape.weight_dtype))
+    o = oracle.layer_confidences(hid, om._keep["lm_head"], om._keep["final_norm"], w.shape.rms_eps)
+    # ring slots are position mod P; compare per-layer means and the per-row values after reordering
+    order = [(p % P) for p in range(len(prompt) - P, len(prompt))]
+    assert np.abs(g["conf"][:, order] - o["conf"]).max() <= TOL
+    assert np.abs(g["p_max"][:, order] - o["p_max"]).max() <= TOL
+    assert np.abs(g["c_layer"] - o["c_layer"]).max() <= TOL
+    bad = (g["argmax"][:, order] != o["argmax"]) & (o["margin"] >= NEAR_TIE)
+    assert not bad.any()
+    sc, oc = _select_cfgs(w, w.n_skip_conf)
+    mask, margins = ctx.cl_select_skip_set(sc)                       # on the device's own confidences
+    want = selection_details(list(o["c_layer"]), oc)
+    got_set = [l for l in range(w.shape.n_layers) if mask[l]]
+    # the same confidences give the same set bit for bit
+    mask2, margins2 = ctx.cl_select_skip_set(sc, c_layer=o["c_layer"].astype(np.float32))
+    want32 = selection_details([float(np.float32(v)) for v in o["c_layer"]], oc)
+    assert [l for l in range(w.shape.n_layers) if mask2[l]] == want32["skip"]
+    assert np.array_equal(margins2[w.lo:w.hi + 1], np.array(want32["margin"]))
+    # on its own confidences the set may only differ where two margins nearly tie
+    if got_set != want["skip"]:
+        m = sorted(want["margin"])
+        gap = m[w.n_skip_conf] - m[w.n_skip_conf - 1]
+        assert gap < 1e-3, (got_set, want["skip"], gap)
+    return first, synth.layers_to_mask(want["skip"], w.shape.n_layers), o
+
+
+def test_c1_tiny_fp32_full():
+    w = synth.WORKLOADS["C1"]
+    P = min(64, w.prompt_len)
+    om, ctx, _ = make_pair(w.shape, w.seed, tap_positions=P)
+    prompt = synth.make_prompt(w.seed, w.prompt_len, w.shape.vocab)
+    _, mask, _ = _confidence_selected(om, ctx, w, prompt, P)
+    assert int(mask.sum()) == 3 * w.n_skip_conf
+    rep = lockstep_generate(om, ctx, prompt, mask, 4, w.gen_len)
+    assert rep.max_logit_err < 1e-3          # fp32 weights: far inside the tolerance
+    print("C1", rep)
+
+
+def test_c1_free_running_generate_is_lossless_and_matches_oracle():
+    w = synth.WORKLOADS["C1"]
+    om, ctx, _ = make_pair(w.shape, w.seed)
+    prompt = synth.make_prompt(w.seed, w.prompt_len, w.shape.vocab)
+    van = oracle.generate_vanilla(om, prompt, w.gen_len)
+    first = ctx.cl_prefill(prompt)
+    g_van, st0 = ctx.cl_generate(0, w.gen_len - 1)
+    assert st0.cycles == w.gen_len - 1 and st0.drafted == 0
+    outs = {}
+    for layers, K in (([], 4), ([1], 4), ([1, 2], 3), ([2], 8), ([1], 1)):
+        ctx.cl_prefill(prompt)
+        ctx.cl_set_skip_set(synth.layers_to_mask(layers, w.shape.n_layers))
+        toks, st = ctx.cl_generate(K, w.gen_len - 1)
+        outs[(tuple(layers), K)] = (toks, st)
+        if not layers:
+            assert st.accepted == st.drafted                     # empty skip set: everything accepted
+        assert st.emitted == st.accepted + st.cycles
+    # lossless on the device, and equal to the oracle up to its first near tie
+    lim = next((i for i, m in enumerate(van["margins"]) if m < NEAR_TIE), w.gen_len)
+    assert [first] + list(g_van[:lim - 1]) == van["tokens"][:lim]
+    if lim == w.gen_len:
+        for key, (toks, _) in outs.items():
+            assert list(toks) == list(g_van), key
+
+
+def test_c2_12layer_bf16_full():
+    w = synth.WORKLOADS["C2"]
+    P = 64
+    om, ctx, _ = make_pair(w.shape, w.seed, tap_positions=P)
+    prompt = synth.make_prompt(w.seed, w.prompt_len, w.shape.vocab)
+    _, mask, _ = _confidence_selected(om, ctx, w, prompt, P)
+    assert int(np.count_nonzero(mask)) == 3
+    rep = lockstep_generate(om, ctx, prompt, mask, 4, w.gen_len, tap=True)
+    print("C2", rep)
+    assert rep.near_ties <= rep.tokens_compared // 10
+
+
+@pytest.mark.parametrize("name,L,prompt_len,gen_len,K,ratio", [("C3", 4, 40, 12, 4, 0.5), ("C3", 3, 19, 9, 8, 0.25),
+                                                                 ("C4", 3, 24, 8, 6, 0.4)])
+def test_large_shapes_reduced_depth(name, L, prompt_len, gen_len, K, ratio):
+    """7B / 13B layer shapes (every kernel at its full-size matrix shapes) with few layers."""
+    w = synth.reduced(synth.WORKLOADS[name], n_layers=L, prompt_len=prompt_len, gen_len=gen_len)
+    om, ctx, _ = make_pair(w.shape, w.seed, gen_device="cuda")
+    prompt = synth.make_prompt(w.seed, prompt_len, w.shape.vocab)
+    n_skip = max(1, synth.n_skip_for_ratio(w.lo, w.hi, ratio))
+    mask = synth.layers_to_mask(synth.uniform_skip_layers(w.lo, w.hi, n_skip), L)
+    rep = lockstep_generate(om, ctx, prompt, mask, K, gen_len)
+    print(w.name, rep)
+
+
+def test_c5_scoring_sampled_rows_and_loop():
+    c5 = synth.C5
+    L, P, d, V = c5["n_layers"], c5["positions"], c5["d_model"], c5["vocab"]
+    head = synth.make_lm_head(c5["seed"], V, d, device="cuda")
+    gain = torch.ones(d)
+    ctx = cl.Context(L, d, d // 128, 11008, V, 8, "bf16", rms_eps=c5["rms_eps"])
+    ctx.cl_load(dict(lm_head=head, final_norm=gain.cuda()), head_only=True)
+    hiddens = [synth.make_hidden(c5["seed"], t, L, P, d, device="cuda") for t in range(c5["iters"])]
+    g = ctx.cl_layer_confidences(hiddens[0])
+    rows, pos = [0, 13, 31], [0, 7, 33, 63]
+    o = oracle.layer_confidences(hiddens[0].cpu(), head.cpu(), gain, c5["rms_eps"], rows=rows, positions=pos)
+    ix = np.ix_(rows, pos)
+    assert np.abs(g["conf"][ix] - o["conf"]).max() <= TOL
+    assert np.abs(g["p_max"][ix] - o["p_max"]).max() <= TOL
+    assert not ((g["argmax"][ix] != o["argmax"]) & (o["margin"] >= NEAR_TIE)).any()
+    assert np.abs(g["c_layer"] - g["conf"].astype(np.float64).mean(axis=1)).max() < 1e-6
+    full = oracle.layer_confidences(hiddens[0].cpu(), head.cpu(), gain, c5["rms_eps"], rows=[5])
+    assert abs(full["c_layer"][0] - g["c_layer"][5]) <= TOL
+    assert (g["conf"] >= -1e-6).all() and (g["conf"] <= 1 + 1e-6).all()
+    # the search-round loop: per-round selection equals the oracle's on the same confidences; best round by score
+    scores = synth.make_round_scores(c5["seed"], c5["iters"])
+    sc = cl.SelectCfg.make(c5["lo"], c5["hi"], n_skip=c5["n_skip"])
+    oc = SelectConfig(n_layers=L, lo=c5["lo"], hi=c5["hi"], n_skip=c5["n_skip"])
+    out = ctx.cl_score_loop(sc, hiddens, scores)
+    assert np.abs(out["c_layers"][0] - g["c_layer"]).max() == 0.0
+    ref = oracle.score_loop([[float(v) for v in out["c_layers"][t]] for t in range(c5["iters"])], scores, oc)
+    for t in range(c5["iters"]):
+        assert [l for l in range(L) if out["masks"][t][l]] == ref["sets"][t]
+    assert out["best_iter"] == ref["best_iter"] == int(np.argmax(scores))
+    assert [l for l in range(L) if out["best_mask"][l]] == ref["best_set"]
+
+
+def test_selection_kernel_bit_exact_on_random_profiles():
+    w = synth.WORKLOADS["C1"]
+    L = 40
+    sh = dataclasses.replace(w.shape, n_layers=L, vocab=64, d_model=128, n_heads=2, d_ffn=64, max_seq=8)
+    ctx = cl.Context.from_shape(sh)
+    ctx.cl_load(dict(lm_head=torch.zeros(64, 128).cuda(), final_norm=torch.ones(128).cuda()), head_only=True)
+    rng = np.random.default_rng(0)
+    for trial in range(60):
+        c = (0.3 + 0.2 * rng.standard_normal(L)).astype(np.float32)
+        if trial % 5 == 0:
+            c[1:1 + rng.integers(2, 9)] = c[1]                         # leading flat run -> w_max > 1
+        lo, hi = (1, L - 2) if trial % 3 else (int(rng.integers(0, 5)), int(rng.integers(20, L)))
+        kw = dict(n_skip=int(rng.integers(0, hi - lo + 2)) if trial % 2 else -1, lam=float(rng.uniform(0.0, 0.6)),
+                  fixed_window=(10 if trial % 7 == 0 else 0), min_ratio=float(rng.choice([0.0, 0.4, 0.6])))
+        mask, marg = ctx.cl_select_skip_set(cl.SelectCfg.make(lo, hi, **kw), c_layer=c)
+        d = selection_details([float(v) for v in c], SelectConfig(n_layers=L, lo=lo, hi=hi, **kw))
+        assert [l for l in range(L) if mask[l]] == d["skip"], (trial, kw)
+        assert np.array_equal(marg[lo:hi + 1], np.array(d["margin"])), trial
+        assert mask[:lo].sum() == 0 and mask[hi + 1:].sum() == 0
+
+
+def test_edge_cases_and_errors():
+    w = synth.WORKLOADS["C1"]
+    sh = dataclasses.replace(w.shape, max_seq=40)
+    om, ctx, _ = make_pair(sh, 9, tap_positions=4)
+    V = sh.vocab
+    with pytest.raises(cl.ConfLayersError) as e:
+        ctx.cl_draft(4)
+    assert e.value.code == 4                                           # draft before prefill
+    # one-token prompt; ragged prefill (not a multiple of the chunk)
+    for n in (1, 9, 17):
+        p = synth.make_prompt(n, n, V)
+        first = ctx.cl_prefill(p)
+        ref = oracle.prefill(om, p)
+        assert first == ref[0] or ref[1] < NEAR_TIE
+    p = synth.make_prompt(3, 17, V)
+    ctx.cl_prefill(p)
+    # all four layers skipped: the draft model is embedding -> head
+    ctx.cl_set_skip_set([3, 3, 3, 3])
+    d = ctx.cl_draft(2, want_logits=True)
+    t0 = oracle.prefill(om, p)[0]
+    lg = om.forward([t0], 17, np.array([3, 3, 3, 3], np.uint8))["logits"][0]
+    assert np.abs(d["logits"][0] - lg).max() <= TOL
+    # zero drafts: verify of the pending token alone == vanilla step
+    ctx.cl_force_tokens([])
+    v = ctx.cl_verify(1, want_logits=True)
+    n, em = ctx.cl_accept()
+    assert n == 0 and em[0] == v["targets"][0]
+    ctx.cl_rollback(17, t0)
+    assert ctx.cl_step_vanilla() == v["targets"][0]
+    # early stop: a threshold of 1.0 stops after the first draft
+    ctx.cl_rollback(17, t0)
+    ctx.cl_set_skip_set([0, 3, 0, 0])
+    d = ctx.cl_draft(4, stop_p=1.0)
+    assert d["n_drafted"] == 1
+    # range errors: K too large, sequence overflow, bad mask, bad token
+    for bad in (0, cl.CL_MAX_K + 1):
+        with pytest.raises(cl.ConfLayersError) as e:
+            ctx.cl_draft(bad)
+        assert e.value.code == 5
+    with pytest.raises(cl.ConfLayersError) as e:
+        ctx.cl_generate(4, 30)
+    assert e.value.code == 5
+    with pytest.raises(cl.ConfLayersError) as e:
+        ctx.cl_set_skip_set([1, 0, 0, 0])
+    assert e.value.code == 1
+    with pytest.raises(cl.ConfLayersError) as e:
+        ctx.cl_prefill([V])
+    assert e.value.code == 1
+    with pytest.raises(cl.ConfLayersError) as e:
+        ctx.cl_prefill(np.zeros(40, np.int32))
+    assert e.value.code == 5
+    # the ring refuses to be scored before it is full
+    ctx.cl_prefill(synth.make_prompt(1, 3, V), tap_hidden=True)
+    with pytest.raises(cl.ConfLayersError) as e:
+        ctx.cl_layer_confidences()
+    assert e.value.code == 4
+    st = ctx.cl_get_stats()
+    assert st.kernel_launches > 0 and st.ctx_len == 3
+
+
+def test_generate_to_the_last_cache_slot():
+    w = synth.WORKLOADS["C1"]
+    sh = dataclasses.replace(w.shape, max_seq=16 + 20 + 4)
+    om, ctx, _ = make_pair(sh, 4)
+    p = synth.make_prompt(4, 16, sh.vocab)
+    ctx.cl_prefill(p)
+    ctx.cl_set_skip_set([0, 3, 0, 0])
+    toks, st = ctx.cl_generate(4, 20)                                  # 16 + 20 + 4 == max_seq exactly
+    assert len(toks) == 20 and st.ctx_len <= sh.max_seq
+    ctx.cl_prefill(p)
+    van, _ = ctx.cl_generate(0, 20)
+    ref = oracle.generate_vanilla(om, p, 21)
+    lim = next((i for i, m in enumerate(ref["margins"]) if m < NEAR_TIE), 21)
+    assert list(van[:lim - 1]) == ref["tokens"][1:lim]
+    if lim == 21:
+        assert list(toks) == list(van)
