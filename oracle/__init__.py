@@ -11,6 +11,7 @@ Parts:
   * ``scoring.py``   -- all-layer confidence scoring and the search-round loop (Sections 3.1, 3.3).
 """
 from .model import OracleModel, build_oracle, confidence_of_logits, lib  # noqa: F401
-from .cycle import accept_greedy, generate_speculative, generate_vanilla, speculative_cycle  # noqa: F401
+from .cycle import (accept_greedy, generate_speculative, generate_vanilla, prefill, speculative_cycle,  # noqa: F401
+                    top2_margin)
 from .selection import SelectConfig, select_skip_set, selection_details  # noqa: F401
 from .scoring import layer_confidences, score_loop  # noqa: F401
