@@ -50,6 +50,14 @@ struct cl_ctx {
     double *sel_margins;          // device [L]
     float *sel_clayers;           // device [iters_cap, L]
     int sel_iters_cap;
+    // token-step kernel (persistent single-token step)
+    ClLayerDev *layers_dev;
+    int *kept_dev, *kept_all_dev;
+    int n_kept, use_step, max_blk;
+    unsigned *bar_dev;
+    float *att_part2;
+    unsigned *att_tickets2;
+    ClHeadPartial *head_part2;
     std::vector<ClLayer> layers;
     std::vector<uint8_t> mask;    // host copy of the skip set
     int nsplit, per_max;
@@ -165,7 +173,8 @@ extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **ou
 static void free_all(cl_ctx *c) {
     void *ptrs[] = {c->wbuf, c->embed, c->lm_head, c->final_norm, c->norms, c->kv, c->rope_cs, c->x, c->xn, c->qkv,
                     c->att, c->hff, c->att_part, c->logits, c->tickets, c->head_part, c->st, c->prompt_dev, c->out_dev,
-                    c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sel_mask, c->sel_margins, c->sel_clayers};
+                    c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sel_mask, c->sel_margins, c->sel_clayers,
+                    c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->att_tickets2, c->head_part2};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->h_st) cudaFreeHost(c->h_st);
@@ -296,6 +305,35 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
             DM(c->ring, L * (size_t)g.tap_positions * d * es);
             CU(cudaMemsetAsync(c->ring, 0, L * (size_t)g.tap_positions * d * es, c->stream));
         }
+        // ---- token-step kernel: per-layer pointer table, kept-layer lists, barrier, attention / head partials
+        {
+            std::vector<ClLayerDev> ld(L);
+            std::vector<int> all(L);
+            for (size_t l = 0; l < L; ++l) {
+                const ClLayer &y = c->layers[l];
+                ld[l] = ClLayerDev{y.wqkv, y.wo, y.wgu, y.wd, y.n1, y.n2, y.kc, y.vc};
+                all[l] = (int)l;
+            }
+            DM(c->layers_dev, (L ? L : 1) * sizeof(ClLayerDev));
+            DM(c->kept_dev, (L ? L : 1) * sizeof(int));
+            DM(c->kept_all_dev, (L ? L : 1) * sizeof(int));
+            CU(cudaMemcpy(c->layers_dev, ld.data(), L * sizeof(ClLayerDev), cudaMemcpyHostToDevice));
+            CU(cudaMemcpy(c->kept_dev, all.data(), L * sizeof(int), cudaMemcpyHostToDevice));
+            CU(cudaMemcpy(c->kept_all_dev, all.data(), L * sizeof(int), cudaMemcpyHostToDevice));
+            c->n_kept = (int)L;
+            c->max_blk = (g.max_seq + 31) / 32;
+            DM(c->bar_dev, 2 * sizeof(unsigned));
+            CU(cudaMemsetAsync(c->bar_dev, 0, 2 * sizeof(unsigned), c->stream));
+            DM(c->att_part2, (size_t)g.n_heads * c->max_blk * (g.head_dim + 2) * 4);
+            DM(c->att_tickets2, (size_t)g.n_heads * 4);
+            CU(cudaMemsetAsync(c->att_tickets2, 0, (size_t)g.n_heads * 4, c->stream));
+            DM(c->head_part2, (size_t)c->n_sm * sizeof(ClHeadPartial));
+            const int maxc = cl_step_max_cols(g.weight_dtype);
+            int coop = 0;
+            cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
+            const char *off = getenv("CL_DISABLE_STEP_KERNEL");
+            c->use_step = coop && d <= (size_t)maxc && F <= (size_t)maxc && !(off && off[0] == '1');
+        }
         CU(cudaStreamSynchronize(c->stream));   // host staging vector and borrowed pointers are released after this
         if (stage_g) cudaFree(stage_g);
         if (stage_u) cudaFree(stage_u);
@@ -370,6 +408,39 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
     return CL_OK;
 }
 
+// n_steps consecutive single-token steps in one persistent launch (draft steps with the skip set, or
+// vanilla full-model steps that emit and advance on the device).
+static int run_steps(cl_ctx *c, int mode, int n_steps, int row0, bool full_model, float *logits, int *out_tokens) {
+    const cl_model_cfg &g = c->cfg;
+    ClStepArgs a;
+    memset(&a, 0, sizeof(a));
+    a.layers = c->layers_dev;
+    a.kept = full_model ? c->kept_all_dev : c->kept_dev;
+    a.n_kept = full_model ? g.n_layers : c->n_kept;
+    a.embed = c->embed; a.lm_head = c->lm_head; a.final_norm = c->final_norm;
+    a.d = g.d_model; a.F = g.d_ffn; a.V = g.vocab; a.H = g.n_heads; a.max_seq = g.max_seq; a.max_blk = c->max_blk;
+    a.eps = g.rms_eps; a.inv_log_v = (float)(1.0 / log((double)g.vocab));
+    a.rope_cs = c->rope_cs; a.st = c->st;
+    a.x = c->x; a.qkv = c->qkv; a.att = c->att; a.hff = c->hff;
+    a.att_part = c->att_part2; a.att_tickets = c->att_tickets2; a.head_part = c->head_part2; a.bar = c->bar_dev;
+    a.n_steps = n_steps; a.mode = mode; a.row0 = row0; a.out_tokens = out_tokens; a.logits = logits;
+    KL(cl_launch_token_steps(g.weight_dtype, g.head_dim, a, c->n_sm, c->stream));
+    return CL_OK;
+}
+
+// After a synchronisation: did a bounded device-side wait expire?
+static int check_device_err(cl_ctx *c, const char *fn) {
+    if (c->h_st->err) {
+        const int e = c->h_st->err;
+        cudaMemsetAsync(c->bar_dev, 0, 2 * sizeof(unsigned), c->stream);
+        cudaMemsetAsync(&c->st->err, 0, sizeof(int), c->stream);
+        cudaMemsetAsync(c->att_tickets2, 0, (size_t)c->cfg.n_heads * 4, c->stream);
+        cudaStreamSynchronize(c->stream);
+        return fail(c, CL_ETIMEOUT, "%s: a bounded device-side wait expired (flags %d); results of this call are invalid", fn, e);
+    }
+    return CL_OK;
+}
+
 static int need_model(cl_ctx *c, const char *fn, bool need_prefill) {
     if (!c) return fail(c, CL_EINVAL, "%s: null context", fn);
     if (!c->loaded) return fail(c, CL_ESTATE, "%s: no weights loaded", fn);
@@ -411,6 +482,14 @@ extern "C" int cl_set_skip_set(cl_ctx *c, const uint8_t *mask) {
         if (mask[l] != 0 && mask[l] != 3)
             return fail(c, CL_EINVAL, "cl_set_skip_set: layer %d has mask %d; only 0 (kept) and 3 (whole layer) are supported", l, mask[l]);
     c->mask.assign(mask, mask + c->cfg.n_layers);
+    if (c->kept_dev) {
+        std::vector<int> kept;
+        for (int l = 0; l < c->cfg.n_layers; ++l)
+            if (!mask[l]) kept.push_back(l);
+        CU(cudaStreamSynchronize(c->stream));
+        if (!kept.empty()) CU(cudaMemcpy(c->kept_dev, kept.data(), kept.size() * sizeof(int), cudaMemcpyHostToDevice));
+        c->n_kept = (int)kept.size();
+    }
     return CL_OK;
 }
 
@@ -427,21 +506,31 @@ extern "C" int cl_draft(cl_ctx *c, int K, float stop_p, int32_t *toks, float *p_
     if (K < 1 || K > CL_MAX_K) return fail(c, CL_ERANGE, "cl_draft: K = %d outside 1..%d", K, CL_MAX_K);
     if (c->h_ctx + K + 1 > c->cfg.max_seq) return fail(c, CL_ERANGE, "cl_draft: position %d exceeds max_seq", c->h_ctx + K);
     int n = 0;
-    for (int i = 0; i < K; ++i) {
-        rc = forward_rows(c, ST_FIELD(c, int, cyc_tok) + i, 1, i, c->mask.data(), 0, 1, ST_FIELD(c, int, cyc_tok) + i + 1,
-                          ST_FIELD(c, float, d_pmax) + i, ST_FIELD(c, float, d_conf) + i,
-                          logits ? c->logits + (size_t)i * c->cfg.vocab : nullptr);
-        if (rc) return rc;
-        n = i + 1;
-        if (stop_p > 0.f) {   // confidence-aware early stop needs the probability on the host
-            if ((rc = sync_state(c))) return rc;
-            if (c->h_st->d_pmax[i] < stop_p) break;
+    if (c->use_step && stop_p <= 0.f) {
+        if ((rc = run_steps(c, CL_STEP_DRAFT, K, 0, false, logits ? c->logits : nullptr, nullptr))) return rc;
+        n = K;
+    } else {
+        for (int i = 0; i < K; ++i) {
+            float *lg = logits ? c->logits + (size_t)i * c->cfg.vocab : nullptr;
+            if (c->use_step)
+                rc = run_steps(c, CL_STEP_DRAFT, 1, i, false, lg, nullptr);
+            else
+                rc = forward_rows(c, ST_FIELD(c, int, cyc_tok) + i, 1, i, c->mask.data(), 0, 1,
+                                  ST_FIELD(c, int, cyc_tok) + i + 1, ST_FIELD(c, float, d_pmax) + i,
+                                  ST_FIELD(c, float, d_conf) + i, lg);
+            if (rc) return rc;
+            n = i + 1;
+            if (stop_p > 0.f) {   // confidence-aware early stop needs the probability on the host
+                if ((rc = sync_state(c))) return rc;
+                if (c->h_st->d_pmax[i] < stop_p) break;
+            }
         }
     }
     ClPoke p = poke_none();
     p.n_drafted = n;
     if ((rc = poke(c, p))) return rc;
     if ((rc = sync_state(c))) return rc;
+    if ((rc = check_device_err(c, "cl_draft"))) return rc;
     c->h_ndraft = n;
     if (logits) CU(cudaMemcpy(logits, c->logits, (size_t)n * c->cfg.vocab * 4, cudaMemcpyDeviceToHost));
     for (int i = 0; i < n; ++i) {
@@ -506,11 +595,16 @@ extern "C" int cl_step_vanilla(cl_ctx *c, int32_t *tok) {
     ClPoke p = poke_none();
     p.n_drafted = 0;
     if ((rc = poke(c, p))) return rc;
-    rc = forward_rows(c, ST_FIELD(c, int, cyc_tok), 1, 0, nullptr, 0, 1, ST_FIELD(c, int, tgt_tok), ST_FIELD(c, float, v_pmax),
-                      ST_FIELD(c, float, v_conf), nullptr);
-    if (rc) return rc;
-    KL(cl_launch_accept(c->st, 0, nullptr, c->stream));
+    if (c->use_step) {
+        if ((rc = run_steps(c, CL_STEP_VANILLA, 1, 0, true, nullptr, nullptr))) return rc;
+    } else {
+        rc = forward_rows(c, ST_FIELD(c, int, cyc_tok), 1, 0, nullptr, 0, 1, ST_FIELD(c, int, tgt_tok),
+                          ST_FIELD(c, float, v_pmax), ST_FIELD(c, float, v_conf), nullptr);
+        if (rc) return rc;
+        KL(cl_launch_accept(c->st, 0, nullptr, c->stream));
+    }
     if ((rc = sync_state(c))) return rc;
+    if ((rc = check_device_err(c, "cl_step_vanilla"))) return rc;
     c->h_ndraft = 0;
     if (tok) *tok = c->h_st->emitted[0];
     return CL_OK;
@@ -518,10 +612,15 @@ extern "C" int cl_step_vanilla(cl_ctx *c, int32_t *tok) {
 
 static int enqueue_cycle(cl_ctx *c, int K) {
     int rc;
-    for (int i = 0; i < K; ++i) {
-        rc = forward_rows(c, ST_FIELD(c, int, cyc_tok) + i, 1, i, c->mask.data(), 0, 1, ST_FIELD(c, int, cyc_tok) + i + 1,
-                          ST_FIELD(c, float, d_pmax) + i, ST_FIELD(c, float, d_conf) + i, nullptr);
-        if (rc) return rc;
+    if (c->use_step && K > 0) {
+        if ((rc = run_steps(c, CL_STEP_DRAFT, K, 0, false, nullptr, nullptr))) return rc;
+    } else {
+        for (int i = 0; i < K; ++i) {
+            rc = forward_rows(c, ST_FIELD(c, int, cyc_tok) + i, 1, i, c->mask.data(), 0, 1,
+                              ST_FIELD(c, int, cyc_tok) + i + 1, ST_FIELD(c, float, d_pmax) + i,
+                              ST_FIELD(c, float, d_conf) + i, nullptr);
+            if (rc) return rc;
+        }
     }
     rc = forward_rows(c, ST_FIELD(c, int, cyc_tok), K + 1, 0, nullptr, 0, 1, ST_FIELD(c, int, tgt_tok),
                       ST_FIELD(c, float, v_pmax), ST_FIELD(c, float, v_conf), nullptr);
@@ -548,6 +647,12 @@ extern "C" int cl_generate(cl_ctx *c, int K, int max_new, int32_t *out, int *n_o
     p.n_out = 0; p.max_new = max_new; p.done = 0; p.n_drafted = 0;
     if ((rc = poke(c, p))) return rc;
     int remaining = max_new;
+    if (K == 0 && c->use_step) {
+        // vanilla decoding: all max_new steps in one persistent launch, tokens emitted on the device
+        if ((rc = run_steps(c, CL_STEP_VANILLA, max_new, 0, true, nullptr, c->out_dev))) return rc;
+        if ((rc = sync_state(c))) return rc;
+        remaining = 0;
+    }
     while (remaining > 0) {
         // the fewest cycles that can finish the job; cycles enqueued past the end exit at once on the device
         const int ncyc = (remaining + K) / (K + 1);
@@ -556,6 +661,7 @@ extern "C" int cl_generate(cl_ctx *c, int K, int max_new, int32_t *out, int *n_o
         if ((rc = sync_state(c))) return rc;
         remaining = max_new - c->h_st->n_out;
     }
+    if ((rc = check_device_err(c, "cl_generate"))) return rc;
     CU(cudaMemcpy(out, c->out_dev, (size_t)max_new * 4, cudaMemcpyDeviceToHost));
     p = poke_none();
     p.done = 0;

@@ -67,6 +67,39 @@ struct ClAttnArgs {
     int row0, n_heads, head_dim, d_model, nsplit, per_max, max_seq;
 };
 
+// Per-layer device pointers as the token-step kernel sees them.
+struct ClLayerDev {
+    const char *wqkv, *wo, *wgu, *wd;
+    const float *n1, *n2;
+    char *kc, *vc;
+};
+
+enum { CL_STEP_DRAFT = 0, CL_STEP_VANILLA = 1 };
+
+struct ClStepArgs {
+    const ClLayerDev *layers;   // device [n_layers]
+    const int *kept;            // device [n_kept] indices of the layers that run
+    int n_kept;
+    const void *embed, *lm_head;
+    const float *final_norm;
+    int d, F, V, H, max_seq, max_blk;
+    float eps, inv_log_v;
+    const float2 *rope_cs;
+    ClDevState *st;
+    float *x, *qkv, *att, *hff;          // global activation vectors [d] [3d] [d] [F]
+    float *att_part;                     // [H, max_blk, hd + 2]
+    unsigned *att_tickets;               // [H]
+    ClHeadPartial *head_part;            // [grid]
+    unsigned *bar;                       // grid barrier: [0] arrivals, [1] generation
+    int n_steps, mode, row0;
+    int *out_tokens;                     // vanilla mode: emitted tokens (may be null)
+    float *logits;                       // optional [n_steps, V]
+};
+
+size_t cl_step_smem_bytes();
+int cl_step_max_cols(int wdtype);
+cudaError_t cl_launch_token_steps(int wdtype, int head_dim, const ClStepArgs &a, int grid, cudaStream_t s);
+
 // launchers (each returns the CUDA launch status)
 cudaError_t cl_launch_gemv(int wdtype, int T, int epi, const ClGemvArgs &a, int grid, cudaStream_t s);
 cudaError_t cl_launch_embed(int wdtype, const void *embed, const int *tok, int T, int d, float *x, const ClDevState *st,

@@ -1,0 +1,684 @@
+// Persistent single-token decoder step ("token-step kernel"): the skip-masked draft step and the
+// vanilla full-model step at batch 1, one cooperative launch for up to CL_MAX_K (draft) or many
+// (vanilla) consecutive tokens.
+//
+// One CTA per SM.  Warp 8 (one elected thread) is the weight producer: it walks the static schedule
+// (steps x kept layers x {QKV, O, gate/up, down} + LM head), and for this CTA's contiguous block of
+// rows of each matrix issues bulk asynchronous copies (cp.async.bulk, completion on an mbarrier) into
+// a ring of 8 KB shared-memory slots.  It never waits for activations, so the HBM stream runs ahead
+// of the grid barriers that separate the phases.  Warps 0..7 are consumers: each thread keeps its
+// fixed columns of the activation vector in registers for a whole phase, every warp reads its 512-byte
+// stripes of each row from the ring (conflict-free 16-byte reads), partial dot products are reduced
+// with warp shuffles and a small shared-memory table, and the phase epilogue (store / residual add /
+// SiLU*up / LM head with online softmax-entropy-argmax) runs with one thread per row.
+// Skipped layers are simply absent from the schedule: they stream nothing and touch no KV entry.
+//
+// Every wait (mbarrier or grid barrier) is bounded in time; on expiry an error flag is set, every later
+// wait falls through, the kernel runs to its end with meaningless data and the host reports CL_ETIMEOUT.
+#include "cl_internal.h"
+
+namespace {
+
+constexpr int NCW = 8;                 // consumer warps
+constexpr int NCT = NCW * 32;          // consumer threads
+constexpr int SLOT_BYTES = 8192;       // ring slot: 512 chunks of 16 bytes = 2 chunks per consumer thread
+constexpr int NSLOT = 24;              // 192 KB in flight per SM
+constexpr int MAXIT = 8;               // 16-byte chunks per thread per row: rows up to 32 KB (C <= 16384 bf16)
+constexpr int MAXSEG = MAXIT / 2;
+constexpr int RB = 256;                // rows per epilogue block
+constexpr unsigned long long WAIT_NS = 2000000000ull;   // 2 s bound on any single wait
+
+struct Smem {
+    unsigned long long full[NSLOT];
+    unsigned long long empty[NSLOT];
+    float partial[RB * NCW];
+    float red[NCW];
+    ClHeadPartial hp[NCT];
+    int abort;
+    int next_tok;
+};
+
+__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long gtime() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(unsigned long long *bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the abort flags) if the phase did not complete in time.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, Smem *sm, ClDevState *st) {
+    if (mbar_try(bar, parity)) return true;
+    if (*(volatile int *)&sm->abort) return false;
+    const unsigned long long t0 = gtime();
+    for (unsigned i = 1;; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if ((i & 63u) == 0u) {
+            if (*(volatile int *)&sm->abort) return false;
+            if (gtime() - t0 > WAIT_NS) {
+                *(volatile int *)&sm->abort = 1;
+                atomicOr(&st->err, 1);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NCT) : "memory"); }
+
+__device__ __forceinline__ float ldcg_f(const float *p) { return __ldcg(p); }
+__device__ __forceinline__ float4 ldcg_f4(const float *p) { return __ldcg((const float4 *)p); }
+
+// Sense-reversing grid barrier on (count, generation) in global memory, called by every consumer
+// thread of every CTA; bounded in time.
+__device__ __forceinline__ void grid_barrier(unsigned *bar, Smem *sm, ClDevState *st) {
+    consumer_sync();
+    if (threadIdx.x == 0 && !*(volatile int *)&sm->abort) {
+        volatile unsigned *gen = bar + 1;
+        const unsigned my_gen = *gen;
+        __threadfence();
+        const unsigned arrived = atomicAdd(bar, 1u);
+        if (arrived == gridDim.x - 1) {
+            *(volatile unsigned *)bar = 0u;
+            __threadfence();
+            atomicAdd(bar + 1, 1u);
+        } else {
+            const unsigned long long t0 = gtime();
+            unsigned i = 0;
+            while (*gen == my_gen) {
+                if ((++i & 255u) == 0u) {
+                    if (*(volatile int *)&st->err || gtime() - t0 > WAIT_NS) {
+                        *(volatile int *)&sm->abort = 1;
+                        atomicOr(&st->err, 2);
+                        break;
+                    }
+                }
+            }
+        }
+        __threadfence();
+    }
+    consumer_sync();
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ ClHeadPartial hp_merge(const ClHeadPartial &a, const ClHeadPartial &b) {
+    if (b.z == 0.f) return a;
+    if (a.z == 0.f) return b;
+    ClHeadPartial r;
+    r.m = fmaxf(a.m, b.m);
+    const float ea = expf(a.m - r.m), eb = expf(b.m - r.m);
+    r.z = a.z * ea + b.z * eb;
+    r.s = ea * (a.s + (a.m - r.m) * a.z) + eb * (b.s + (b.m - r.m) * b.z);
+    r.idx = (a.m > b.m) ? a.idx : (b.m > a.m) ? b.idx : min(a.idx, b.idx);
+    return r;
+}
+
+__device__ __forceinline__ ClHeadPartial hp_shfl_xor(const ClHeadPartial &a, int o) {
+    ClHeadPartial r;
+    r.m = __shfl_xor_sync(0xffffffffu, a.m, o);
+    r.z = __shfl_xor_sync(0xffffffffu, a.z, o);
+    r.s = __shfl_xor_sync(0xffffffffu, a.s, o);
+    r.idx = __shfl_xor_sync(0xffffffffu, a.idx, o);
+    return r;
+}
+
+// Fixed-order reduction of one ClHeadPartial per consumer thread; result valid in every thread.
+__device__ ClHeadPartial hp_block_reduce(ClHeadPartial v, Smem *sm) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const ClHeadPartial other = hp_shfl_xor(v, o);
+        // combine in a lane-independent order so every lane ends with identical bits
+        v = ((threadIdx.x & o) == 0) ? hp_merge(v, other) : hp_merge(other, v);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    consumer_sync();
+    if (lane == 0) sm->hp[warp] = v;
+    consumer_sync();
+    ClHeadPartial r = sm->hp[0];
+#pragma unroll
+    for (int w = 1; w < NCW; ++w) r = hp_merge(r, sm->hp[w]);
+    return r;
+}
+
+template <typename WT>
+struct Chunk;   // one 16-byte chunk of weights against the matching activation registers
+template <>
+struct Chunk<__nv_bfloat16> {
+    static constexpr int EPC = 8;
+    static __device__ __forceinline__ float dot(const uint4 &w, const float (&x)[8], float acc) {
+        acc = fmaf(__uint_as_float(w.x << 16), x[0], acc);
+        acc = fmaf(__uint_as_float(w.x & 0xffff0000u), x[1], acc);
+        acc = fmaf(__uint_as_float(w.y << 16), x[2], acc);
+        acc = fmaf(__uint_as_float(w.y & 0xffff0000u), x[3], acc);
+        acc = fmaf(__uint_as_float(w.z << 16), x[4], acc);
+        acc = fmaf(__uint_as_float(w.z & 0xffff0000u), x[5], acc);
+        acc = fmaf(__uint_as_float(w.w << 16), x[6], acc);
+        acc = fmaf(__uint_as_float(w.w & 0xffff0000u), x[7], acc);
+        return acc;
+    }
+};
+template <>
+struct Chunk<float> {
+    static constexpr int EPC = 4;
+    static __device__ __forceinline__ float dot(const uint4 &w, const float (&x)[4], float acc) {
+        acc = fmaf(__uint_as_float(w.x), x[0], acc);
+        acc = fmaf(__uint_as_float(w.y), x[1], acc);
+        acc = fmaf(__uint_as_float(w.z), x[2], acc);
+        acc = fmaf(__uint_as_float(w.w), x[3], acc);
+        return acc;
+    }
+};
+
+template <typename ST>
+__device__ __forceinline__ float st_to_f32(ST v);
+template <>
+__device__ __forceinline__ float st_to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float st_to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename ST>
+__device__ __forceinline__ ST st_from_f32(float v);
+template <>
+__device__ __forceinline__ float st_from_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 st_from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// VPL consecutive stored elements -> fp32, read through L2.
+template <typename ST, int VPL>
+__device__ __forceinline__ void load_vals(const ST *p, float (&o)[VPL]) {
+    constexpr int BYTES = VPL * (int)sizeof(ST);
+    if (BYTES == 4) {
+        const unsigned u = __ldcg((const unsigned *)p);
+        if (sizeof(ST) == 2) {
+            o[0] = __uint_as_float(u << 16);
+            o[VPL - 1] = __uint_as_float(u & 0xffff0000u);
+        } else {
+            o[0] = __uint_as_float(u);
+        }
+    } else if (BYTES == 8) {
+        const uint2 u = __ldcg((const uint2 *)p);
+        if (sizeof(ST) == 2) {
+            o[0] = __uint_as_float(u.x << 16);
+            o[1 % VPL] = __uint_as_float(u.x & 0xffff0000u);
+            o[2 % VPL] = __uint_as_float(u.y << 16);
+            o[3 % VPL] = __uint_as_float(u.y & 0xffff0000u);
+        } else {
+            o[0] = __uint_as_float(u.x);
+            o[1 % VPL] = __uint_as_float(u.y);
+        }
+    } else {
+        const uint4 u = __ldcg((const uint4 *)p);
+        o[0] = __uint_as_float(u.x);
+        o[1 % VPL] = __uint_as_float(u.y);
+        o[2 % VPL] = __uint_as_float(u.z);
+        o[3 % VPL] = __uint_as_float(u.w);
+    }
+}
+
+struct Ring {
+    unsigned slot, par;   // position in the ring and the parity of the phase to wait for
+    __device__ __forceinline__ void advance() {
+        if (++slot == NSLOT) {
+            slot = 0;
+            par ^= 1u;
+        }
+    }
+};
+
+// This CTA's share of `units` row units (a unit is `unit` consecutive rows).
+__device__ __forceinline__ void my_rows(int rows, int unit, int &r0, int &r1) {
+    const long long units = rows / unit;
+    r0 = (int)(units * blockIdx.x / gridDim.x) * unit;
+    r1 = (int)(units * (blockIdx.x + 1) / gridDim.x) * unit;
+}
+
+// ---- producer -------------------------------------------------------------------------------------
+template <typename WT>
+__device__ void produce_matrix(const char *W, int rows, int cols, int unit, Ring &rg, unsigned char *ring, Smem *sm,
+                               ClDevState *st, unsigned *last_par) {
+    int r0, r1;
+    my_rows(rows, unit, r0, r1);
+    const size_t rowbytes = (size_t)cols * sizeof(WT);
+    const int nseg = (int)((rowbytes + SLOT_BYTES - 1) / SLOT_BYTES);
+    for (int r = r0; r < r1; ++r) {
+        const char *src = W + (size_t)r * rowbytes;
+        for (int s = 0; s < nseg; ++s) {
+            const unsigned bytes = (unsigned)min((size_t)SLOT_BYTES, rowbytes - (size_t)s * SLOT_BYTES);
+            mbar_wait(&sm->empty[rg.slot], rg.par ^ 1u, sm, st);
+            if (!*(volatile int *)&sm->abort) {
+                mbar_expect_tx(&sm->full[rg.slot], bytes);
+                bulk_g2s(ring + (size_t)rg.slot * SLOT_BYTES, src + (size_t)s * SLOT_BYTES, bytes, &sm->full[rg.slot]);
+                last_par[rg.slot] = rg.par;
+            }
+            rg.advance();
+        }
+    }
+}
+
+// ---- consumer: one matrix phase ------------------------------------------------------------------------
+// xr: this thread's activation registers, xr[it][e] = x[(it * NCT + tid) * EPC + e].
+// Calls epi(row_local_index_in_block, first_row_of_block, rows_in_block) with the partial table ready.
+template <typename WT, typename Epi>
+__device__ __forceinline__ void consume_matrix(int rows, int cols, int unit, const float (&xr)[MAXIT][Chunk<WT>::EPC],
+                                               Ring &rg, const unsigned char *ring, Smem *sm, ClDevState *st, Epi epi) {
+    constexpr int EPC = Chunk<WT>::EPC;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int r0, r1;
+    my_rows(rows, unit, r0, r1);
+    const int nchunks = cols / EPC;
+    const int nseg = (nchunks + 511) / 512;
+    for (int rb0 = r0; rb0 < r1; rb0 += RB) {
+        const int nrb = min(RB, r1 - rb0);
+        for (int r = 0; r < nrb; ++r) {
+            float acc = 0.f;
+#pragma unroll
+            for (int s = 0; s < MAXSEG; ++s) {
+                if (s < nseg) {
+                    mbar_wait(&sm->full[rg.slot], rg.par, sm, st);
+                    const unsigned char *base = ring + (size_t)rg.slot * SLOT_BYTES;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const int it = 2 * s + j;
+                        if (it * NCT + tid < nchunks) {
+                            const uint4 w = *(const uint4 *)(base + (size_t)(j * NCT + tid) * 16);
+                            acc = Chunk<WT>::dot(w, xr[it], acc);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->empty[rg.slot]);
+                    rg.advance();
+                }
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) sm->partial[r * NCW + warp] = acc;
+        }
+        consumer_sync();
+        epi(rb0, nrb);
+        consumer_sync();
+    }
+}
+
+__device__ __forceinline__ float row_sum(const Smem *sm, int r) {
+    const float *p = sm->partial + r * NCW;
+    float s = p[0];
+#pragma unroll
+    for (int w = 1; w < NCW; ++w) s += p[w];
+    return s;
+}
+
+// Load this thread's columns of a global fp32 vector into registers (L2 reads: written by other CTAs).
+template <int EPC>
+__device__ __forceinline__ void load_x(const float *x, int cols, float (&xr)[MAXIT][EPC]) {
+    const int nchunks = cols / EPC;
+#pragma unroll
+    for (int it = 0; it < MAXIT; ++it) {
+        const int ch = it * NCT + threadIdx.x;
+        if (ch < nchunks) {
+#pragma unroll
+            for (int q = 0; q < EPC / 4; ++q) {
+                const float4 v = ldcg_f4(x + (size_t)ch * EPC + 4 * q);
+                xr[it][4 * q] = v.x; xr[it][4 * q + 1] = v.y; xr[it][4 * q + 2] = v.z; xr[it][4 * q + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < EPC; ++e) xr[it][e] = 0.f;
+        }
+    }
+}
+
+// RMSNorm in registers: xr <- x * rsqrt(mean(x^2) + eps) * g.
+template <int EPC>
+__device__ __forceinline__ void load_x_rmsnorm(const float *x, const float *g, int cols, float eps, float (&xr)[MAXIT][EPC],
+                                               Smem *sm) {
+    load_x<EPC>(x, cols, xr);
+    float ss = 0.f;
+#pragma unroll
+    for (int it = 0; it < MAXIT; ++it)
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) ss = fmaf(xr[it][e], xr[it][e], ss);
+    ss = warp_sum(ss);
+    consumer_sync();
+    if ((threadIdx.x & 31) == 0) sm->red[threadIdx.x >> 5] = ss;
+    consumer_sync();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < NCW; ++w) tot += sm->red[w];
+    const float sc = 1.0f / sqrtf(tot / (float)cols + eps);
+    const int nchunks = cols / EPC;
+#pragma unroll
+    for (int it = 0; it < MAXIT; ++it) {
+        const int ch = it * NCT + threadIdx.x;
+        if (ch < nchunks) {
+#pragma unroll
+            for (int q = 0; q < EPC / 4; ++q) {
+                const float4 gv = __ldg((const float4 *)(g + (size_t)ch * EPC + 4 * q));
+                xr[it][4 * q] *= sc * gv.x; xr[it][4 * q + 1] *= sc * gv.y;
+                xr[it][4 * q + 2] *= sc * gv.z; xr[it][4 * q + 3] *= sc * gv.w;
+            }
+        }
+    }
+}
+
+// ---- attention phase: one warp per (head, block of 32 keys) ------------------------------------------
+template <typename ST, int HD>
+__device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int pos, Smem *sm) {
+    constexpr int EPL = 16 / (int)sizeof(ST);   // elements per lane per key
+    constexpr int LPK = HD / EPL;               // lanes per key
+    constexpr int KPW = 32 / LPK;               // keys per warp pass
+    constexpr int VPL = HD / 32;                // value elements per lane
+    constexpr int PSTRIDE = HD + 2;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nkeys = pos + 1;
+    const int nblk = (nkeys + 31) >> 5;
+    const int nitems = a.H * nblk;
+    const int d = a.d;
+    const int sub = lane / LPK, li = lane % LPK;
+    const float scale = rsqrtf((float)HD);
+    ST *Kc = (ST *)L.kc;
+    ST *Vc = (ST *)L.vc;
+    for (int item = blockIdx.x * NCW + warp; item < nitems; item += gridDim.x * NCW) {
+        const int h = item / nblk, kb = item % nblk;
+        const int j0 = kb << 5, n = min(32, nkeys - j0);
+        const float *qraw = a.qkv + h * HD;
+        // the block that holds the new position first appends its rotated key and its value to the cache
+        if (j0 + n == nkeys) {
+            const float *kraw = a.qkv + d + h * HD, *vraw = a.qkv + 2 * d + h * HD;
+            for (int i = lane; i < HD / 2; i += 32) {
+                const float2 cs = a.rope_cs[(size_t)pos * (HD / 2) + i];
+                const float ka = ldcg_f(kraw + i), kb2 = ldcg_f(kraw + i + HD / 2);
+                Kc[(size_t)pos * d + h * HD + i] = st_from_f32<ST>(ka * cs.x - kb2 * cs.y);
+                Kc[(size_t)pos * d + h * HD + i + HD / 2] = st_from_f32<ST>(kb2 * cs.x + ka * cs.y);
+                Vc[(size_t)pos * d + h * HD + i] = st_from_f32<ST>(ldcg_f(vraw + i));
+                Vc[(size_t)pos * d + h * HD + i + HD / 2] = st_from_f32<ST>(ldcg_f(vraw + i + HD / 2));
+            }
+            __syncwarp();
+        }
+        // rotated query, this lane's EPL elements
+        float qr[EPL];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            const int idx = li * EPL + e;
+            const int i = idx < HD / 2 ? idx : idx - HD / 2;
+            const float2 cs = a.rope_cs[(size_t)pos * (HD / 2) + i];
+            const float qa = ldcg_f(qraw + i), qb = ldcg_f(qraw + i + HD / 2);
+            qr[e] = idx < HD / 2 ? qa * cs.x - qb * cs.y : qb * cs.x + qa * cs.y;
+        }
+        // scores of up to 32 keys; lane j ends up holding the score of key j0 + j
+        float my_score = -INFINITY;
+#pragma unroll
+        for (int jb = 0; jb < 32; jb += KPW) {
+            const int j = jb + sub;
+            float s = 0.f;
+            if (j < n) {
+                const uint4 raw = __ldcg((const uint4 *)(Kc + (size_t)(j0 + j) * d + h * HD + li * EPL));
+                if (sizeof(ST) == 2) {
+                    const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        s = fmaf(qr[2 * e], __uint_as_float(u[e] << 16), s);
+                        s = fmaf(qr[2 * e + 1], __uint_as_float(u[e] & 0xffff0000u), s);
+                    }
+                } else {
+                    s = fmaf(qr[0], __uint_as_float(raw.x), s);
+                    s = fmaf(qr[1], __uint_as_float(raw.y), s);
+                    s = fmaf(qr[2], __uint_as_float(raw.z), s);
+                    s = fmaf(qr[3], __uint_as_float(raw.w), s);
+                }
+            }
+#pragma unroll
+            for (int o = LPK >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            s *= scale;
+            // key jb + k sits in lanes [k * LPK, (k + 1) * LPK): hand it to lane jb + k
+#pragma unroll
+            for (int k = 0; k < KPW; ++k) {
+                const float v = __shfl_sync(0xffffffffu, s, k * LPK);
+                if (lane == jb + k && jb + k < n) my_score = v;
+            }
+        }
+        float m = my_score;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        const float p = (lane < n) ? expf(my_score - m) : 0.f;
+        const float l = warp_sum(p);
+        float o_acc[VPL];
+#pragma unroll
+        for (int e = 0; e < VPL; ++e) o_acc[e] = 0.f;
+        for (int j = 0; j < n; ++j) {
+            const float pj = __shfl_sync(0xffffffffu, p, j);
+            float vv[VPL];
+            load_vals<ST, VPL>(Vc + (size_t)(j0 + j) * d + h * HD + lane * VPL, vv);
+#pragma unroll
+            for (int e = 0; e < VPL; ++e) o_acc[e] = fmaf(pj, vv[e], o_acc[e]);
+        }
+        float *part = a.att_part + ((size_t)h * a.max_blk + kb) * PSTRIDE;
+        if (lane == 0) {
+            part[0] = m;
+            part[1] = l;
+        }
+#pragma unroll
+        for (int e = 0; e < VPL; ++e) part[2 + lane * VPL + e] = o_acc[e];
+        __threadfence();
+        __syncwarp();
+        unsigned prev = 0;
+        if (lane == 0) prev = atomicAdd(a.att_tickets + h, 1u);
+        prev = __shfl_sync(0xffffffffu, prev, 0);
+        if (prev == (unsigned)nblk - 1) {
+            // last block of this head to finish: merge all blocks in order, normalise, write the head's output
+            __threadfence();
+            const float *p0 = a.att_part + (size_t)h * a.max_blk * PSTRIDE;
+            float M = -INFINITY;
+            for (int b = 0; b < nblk; ++b) M = fmaxf(M, ldcg_f(p0 + (size_t)b * PSTRIDE));
+            float Ls = 0.f, O[VPL];
+#pragma unroll
+            for (int e = 0; e < VPL; ++e) O[e] = 0.f;
+            for (int b = 0; b < nblk; ++b) {
+                const float w = expf(ldcg_f(p0 + (size_t)b * PSTRIDE) - M);
+                Ls = fmaf(ldcg_f(p0 + (size_t)b * PSTRIDE + 1), w, Ls);
+#pragma unroll
+                for (int e = 0; e < VPL; ++e) O[e] = fmaf(ldcg_f(p0 + (size_t)b * PSTRIDE + 2 + lane * VPL + e), w, O[e]);
+            }
+#pragma unroll
+            for (int e = 0; e < VPL; ++e) a.att[h * HD + lane * VPL + e] = O[e] / Ls;
+            if (lane == 0) a.att_tickets[h] = 0u;
+        }
+    }
+}
+
+// ---- the kernel ----------------------------------------------------------------------------------------
+template <typename WT, int HD>
+__global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char *ring = smem_raw;
+    Smem *sm = (Smem *)(smem_raw + (size_t)NSLOT * SLOT_BYTES);
+    ClDevState *st = a.st;
+    if (st->done) return;   // written only between launches: uniform over the grid
+    constexpr int EPC = Chunk<WT>::EPC;
+    const int tid = threadIdx.x;
+
+    if (tid == 0) {
+        for (int i = 0; i < NSLOT; ++i) {
+            mbar_init(&sm->full[i], 1);
+            mbar_init(&sm->empty[i], NCW);
+        }
+        sm->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int ctx0 = st->ctx;
+    const int d = a.d, F = a.F, V = a.V;
+
+    if (tid >= NCT) {
+        // ------------------------------ producer warp ------------------------------
+        if (tid == NCT) {
+            Ring rg{0u, 0u};
+            unsigned last_par[NSLOT];
+            for (int i = 0; i < NSLOT; ++i) last_par[i] = 2u;
+            for (int step = 0; step < a.n_steps; ++step) {
+                for (int ki = 0; ki < a.n_kept; ++ki) {
+                    const ClLayerDev L = a.layers[a.kept[ki]];
+                    produce_matrix<WT>(L.wqkv, 3 * d, d, 1, rg, ring, sm, st, last_par);
+                    produce_matrix<WT>(L.wo, d, d, 1, rg, ring, sm, st, last_par);
+                    produce_matrix<WT>(L.wgu, 2 * F, d, 2, rg, ring, sm, st, last_par);
+                    produce_matrix<WT>(L.wd, d, F, 1, rg, ring, sm, st, last_par);
+                }
+                produce_matrix<WT>((const char *)a.lm_head, V, d, 1, rg, ring, sm, st, last_par);
+            }
+            // Drain: every copy this thread issued must have landed before the CTA may exit.  In the normal
+            // path the consumers have already waited for all of them; after an abort this is the bounded wait
+            // for copies still in flight.
+            for (int i = 0; i < NSLOT; ++i) {
+                if (last_par[i] < 2u) {
+                    const unsigned long long t0 = gtime();
+                    while (!mbar_try(&sm->full[i], last_par[i]))
+                        if (gtime() - t0 > WAIT_NS) break;
+                }
+            }
+        }
+        return;
+    }
+
+    // ------------------------------ consumer warps ------------------------------
+    Ring rg{0u, 0u};
+    float xr[MAXIT][EPC];
+    int tok = st->cyc_tok[a.row0];
+    for (int step = 0; step < a.n_steps; ++step) {
+        const int pos = ctx0 + a.row0 + step;
+        // phase 0: embedding row -> residual stream (each CTA writes its slice)
+        {
+            const WT *erow = (const WT *)a.embed + (size_t)tok * d;
+            for (int i = blockIdx.x * NCT + tid; i < d; i += gridDim.x * NCT) a.x[i] = st_to_f32<WT>(erow[i]);
+        }
+        grid_barrier(a.bar, sm, st);
+        for (int ki = 0; ki < a.n_kept; ++ki) {
+            const ClLayerDev L = a.layers[a.kept[ki]];
+            // QKV projection of the normalised stream
+            load_x_rmsnorm<EPC>(a.x, L.n1, d, a.eps, xr, sm);
+            consume_matrix<WT>(3 * d, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
+                for (int r = tid; r < nrb; r += NCT) a.qkv[rb0 + r] = row_sum(sm, r);
+            });
+            grid_barrier(a.bar, sm, st);
+            attention_phase<WT, HD>(a, L, pos, sm);
+            grid_barrier(a.bar, sm, st);
+            // attention output projection + residual
+            load_x<EPC>(a.att, d, xr);
+            consume_matrix<WT>(d, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
+                for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
+            });
+            grid_barrier(a.bar, sm, st);
+            // gate/up projections (rows interleaved) + SiLU(gate) * up
+            load_x_rmsnorm<EPC>(a.x, L.n2, d, a.eps, xr, sm);
+            consume_matrix<WT>(2 * F, d, 2, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
+                for (int pr = tid; pr < nrb / 2; pr += NCT) {
+                    const float gt = row_sum(sm, 2 * pr), up = row_sum(sm, 2 * pr + 1);
+                    a.hff[rb0 / 2 + pr] = gt / (1.f + expf(-gt)) * up;
+                }
+            });
+            grid_barrier(a.bar, sm, st);
+            // down projection + residual
+            load_x<EPC>(a.hff, F, xr);
+            consume_matrix<WT>(d, F, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
+                for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
+            });
+            grid_barrier(a.bar, sm, st);
+        }
+        // LM head on the normalised stream, fused with clamp + online softmax / entropy / argmax
+        load_x_rmsnorm<EPC>(a.x, a.final_norm, d, a.eps, xr, sm);
+        ClHeadPartial run{0.f, 0.f, 0.f, 0x7fffffff};
+        float *lg = a.logits ? a.logits + (size_t)step * V : nullptr;
+        consume_matrix<WT>(V, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
+            for (int r = tid; r < nrb; r += NCT) {
+                const float l = fminf(fmaxf(row_sum(sm, r), -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
+                if (lg) lg[rb0 + r] = l;
+                run = hp_merge(run, ClHeadPartial{l, 1.f, 0.f, rb0 + r});
+            }
+        });
+        run = hp_block_reduce(run, sm);
+        if (tid == 0) a.head_part[blockIdx.x] = run;
+        grid_barrier(a.bar, sm, st);
+        // every CTA reduces the per-CTA partials itself (same order everywhere), so all know the token
+        ClHeadPartial fin{0.f, 0.f, 0.f, 0x7fffffff};
+        for (int b = tid; b < (int)gridDim.x; b += NCT) {
+            const ClHeadPartial *p = a.head_part + b;
+            ClHeadPartial q;
+            q.m = ldcg_f(&p->m); q.z = ldcg_f(&p->z); q.s = ldcg_f(&p->s); q.idx = __ldcg(&p->idx);
+            fin = hp_merge(fin, q);
+        }
+        fin = hp_block_reduce(fin, sm);
+        tok = fin.idx;
+        if (blockIdx.x == 0 && tid == 0) {
+            const float Hh = logf(fin.z) - fin.s / fin.z;   // entropy of the softmax (Eq. 2), from sums relative to the max
+            const float conf = 1.f - Hh * a.inv_log_v;      // Eq. 3-4
+            const float pm = 1.f / fin.z;
+            if (a.mode == CL_STEP_DRAFT) {
+                st->cyc_tok[a.row0 + step + 1] = tok;
+                st->d_pmax[a.row0 + step] = pm;
+                st->d_conf[a.row0 + step] = conf;
+            } else {
+                // vanilla decoding: the token is emitted at once and becomes the next pending token
+                if (a.out_tokens && st->n_out < st->max_new) a.out_tokens[st->n_out] = tok;
+                st->n_out = min(st->n_out + 1, st->max_new);
+                st->tgt_tok[0] = tok;
+                st->emitted[0] = tok;
+                st->cyc_tok[0] = tok;
+                st->v_pmax[0] = pm;
+                st->v_conf[0] = conf;
+                st->ctx = pos + 1;
+                st->n_acc_last = 0;
+                st->cycles += 1ull;
+                st->emitted_total += 1ull;
+            }
+        }
+        // the next step's phase 0 writes x, which nobody reads any more in this step: no barrier needed here,
+        // and head_part is rewritten only after the next step's grid barriers
+    }
+}
+
+}  // namespace
+
+size_t cl_step_smem_bytes() { return (size_t)NSLOT * SLOT_BYTES + sizeof(Smem); }
+
+int cl_step_max_cols(int wdtype) { return MAXIT * NCT * (wdtype == 1 ? 8 : 4); }
+
+cudaError_t cl_launch_token_steps(int wdtype, int head_dim, const ClStepArgs &a, int grid, cudaStream_t s) {
+    const void *fn = nullptr;
+    if (wdtype == 1 && head_dim == 64) fn = (const void *)k_token_steps<__nv_bfloat16, 64>;
+    else if (wdtype == 1 && head_dim == 128) fn = (const void *)k_token_steps<__nv_bfloat16, 128>;
+    else if (wdtype == 0 && head_dim == 64) fn = (const void *)k_token_steps<float, 64>;
+    else if (wdtype == 0 && head_dim == 128) fn = (const void *)k_token_steps<float, 128>;
+    else return cudaErrorInvalidValue;
+    const size_t smem = cl_step_smem_bytes();
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    void *params[] = {(void *)&a};
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(NCT + 32), params, smem, s);
+}
