@@ -634,7 +634,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             fin = hp_merge(fin, q);
         }
         fin = hp_block_reduce(fin, sm);
-        tok = fin.idx;
+        tok = min(max(fin.idx, 0), V - 1);   // (only an aborted run can leave the range; keep the next gather in bounds)
         if (blockIdx.x == 0 && tid == 0) {
             const float Hh = logf(fin.z) - fin.s / fin.z;   // entropy of the softmax (Eq. 2), from sums relative to the max
             const float conf = 1.f - Hh * a.inv_log_v;      // Eq. 3-4
