@@ -15,6 +15,7 @@ independent units to shard); value is the aggregate over ranks, time is the max 
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -150,6 +151,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="fewer layers of the same shape (profiling captures only)")
+    ap.add_argument("--gen", type=int, default=0, help="fewer generated tokens per step (profiling captures only)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -172,6 +174,8 @@ def main():
     w = synth.WORKLOADS[WORKLOAD]
     if args.layers:
         w = synth.reduced(w, n_layers=args.layers, prompt_len=w.prompt_len, gen_len=w.gen_len, max_seq=w.shape.max_seq)
+    if args.gen:
+        w = dataclasses.replace(w, gen_len=args.gen)
     shape = w.shape
     W = synth.make_weights(shape, w.seed, device="cuda")
     ctx = cl.Context.from_shape(shape)
