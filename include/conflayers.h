@@ -178,6 +178,33 @@ int cl_score_loop(cl_ctx *ctx, const cl_select_cfg *cfg, const void *const *hidd
  * type, position slot = absolute position modulo tap_positions. */
 int cl_read_hidden_ring(cl_ctx *ctx, void *out);
 
+/* Confidence scoring for callers that cannot allocate device memory.  The paper has no counterpart of
+ * this call: it is cl_layer_confidences() (final RMSNorm -> shared LM head -> clamp -> entropy confidence,
+ * top-1 probability, greedy token per row) without a context and without a single cudaMalloc / cudaFree.
+ * It is meant for processes in which this library may not allocate: a server whose framework has already
+ * reserved the whole GPU for its own caching allocator (a cudaMalloc here would fail or eat into that
+ * pool), or a latency-critical loop in which cudaMalloc's device-wide synchronisation is not acceptable.
+ *
+ * All working memory (normalised rows, per-block softmax partials, the completion ticket, the result
+ * staging) lives in one fixed array compiled into the library: about 0.5 MB that every GPU which loads the
+ * library holds until the process exits.  Hence the fixed limits below; larger sizes return CL_ERANGE.
+ *   lm_head    DEVICE [vocab, d_model] row-major, weight_dtype 0 = fp32 / 1 = bf16
+ *   final_norm DEVICE float[d_model]
+ *   hidden     DEVICE [n_rows, d_model] in the same storage type as lm_head
+ *   conf, p_max, argmax   HOST [n_rows], caller-owned, each may be NULL
+ * The call enqueues on cuda_stream (a cudaStream_t or NULL) and synchronises it before returning.
+ * The first call on each device looks up the array's device address; make that first call outside any
+ * stream capture.  Every call on a device uses the same array, which keeps whatever the previous call
+ * left (the call clears the part that must start at zero itself): two calls whose kernels overlap on the
+ * GPU, from different streams or threads, race and give wrong results.  Serialise them.
+ * Errors: CL_EINVAL (null input, bad dtype or shape), CL_ERANGE (beyond the limits), CL_ECUDA;
+ * the message is read with cl_last_error(NULL). */
+#define CL_STATIC_MAX_ROWS 4096
+#define CL_STATIC_MAX_D 8192
+int cl_layer_confidences_static(const void *lm_head, const float *final_norm, int vocab, int d_model, int weight_dtype,
+                                float rms_eps, const void *hidden, int n_rows, void *cuda_stream, float *conf,
+                                float *p_max, int32_t *argmax);
+
 /* ---- bookkeeping ----------------------------------------------------------------------------- */
 
 int cl_get_stats(cl_ctx *ctx, cl_stats *out);      /* alpha, beta, M of Section 4.1.2 derive from these */

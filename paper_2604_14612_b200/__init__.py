@@ -5,5 +5,5 @@
 ``libconflayers.so``).  There is no CPU fallback: if the library has not been built, or no CUDA
 device is present, calls raise.
 """
-from .binding import (CL_MAX_K, ConfLayersError, Context, SelectCfg, Stats, exported_symbols, library_path,  # noqa: F401
-                      load_library)
+from .binding import (CL_MAX_K, ConfLayersError, Context, SelectCfg, Stats, cl_layer_confidences_static,  # noqa: F401
+                      exported_symbols, library_path, load_library)

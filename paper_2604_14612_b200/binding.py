@@ -92,6 +92,7 @@ def load_library():
         "cl_score_loop": [vp, C.POINTER(SelectCfg), C.POINTER(vp), C.c_int, C.c_int, vp, vp, C.POINTER(C.c_int), vp, vp],
         "cl_read_hidden_ring": [vp, vp],
         "cl_get_stats": [vp, C.POINTER(Stats)],
+        "cl_layer_confidences_static": [vp, vp, C.c_int, C.c_int, C.c_int, C.c_float, vp, C.c_int, vp, vp, vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -105,6 +106,32 @@ def load_library():
 
 def _np_ptr(a: Optional[np.ndarray]):
     return None if a is None else a.ctypes.data
+
+
+def cl_layer_confidences_static(lm_head, final_norm, hidden, rms_eps: float = 1e-5, stream: Optional[int] = None):
+    """Context-free confidence scoring that allocates no device memory (see the header for who needs it).
+
+    lm_head [V, d], hidden [..., d] (same dtype, bf16 or fp32) and final_norm fp32 [d] are CUDA tensors;
+    returns dict(conf, p_max, argmax) as numpy arrays with hidden's leading shape."""
+    L = load_library()
+    import torch
+    assert lm_head.is_cuda and hidden.is_cuda and final_norm.is_cuda
+    assert lm_head.is_contiguous() and hidden.is_contiguous() and final_norm.is_contiguous()
+    assert lm_head.dtype == hidden.dtype and final_norm.dtype == torch.float32
+    V, d = lm_head.shape
+    lead = tuple(hidden.shape[:-1])
+    n = int(np.prod(lead))
+    conf = np.zeros(n, np.float32)
+    pm = np.zeros(n, np.float32)
+    am = np.zeros(n, np.int32)
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = L.cl_layer_confidences_static(lm_head.data_ptr(), final_norm.data_ptr(), V, d,
+                                       1 if lm_head.dtype == torch.bfloat16 else 0, rms_eps, hidden.data_ptr(), n,
+                                       C.c_void_p(stream), _np_ptr(conf), _np_ptr(pm), _np_ptr(am))
+    if rc:
+        raise ConfLayersError(rc, L.cl_last_error(None).decode())
+    return dict(conf=conf.reshape(lead), p_max=pm.reshape(lead), argmax=am.reshape(lead))
 
 
 class Context:

@@ -77,6 +77,13 @@ static int fail(cl_ctx *c, int code, const char *fmt, ...) {
     return code;
 }
 
+void cl_set_global_error(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
 #define CU(call)                                                                                          \
     do {                                                                                                  \
         cudaError_t e_ = (call);                                                                          \

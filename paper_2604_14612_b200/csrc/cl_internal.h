@@ -96,6 +96,9 @@ struct ClStepArgs {
     float *logits;                       // optional [n_steps, V]
 };
 
+// Records a message that cl_last_error(NULL) returns (for entry points that have no context).
+void cl_set_global_error(const char *fmt, ...) __attribute__((format(printf, 1, 2)));
+
 size_t cl_step_smem_bytes();
 int cl_step_max_cols(int wdtype);
 cudaError_t cl_launch_token_steps(int wdtype, int head_dim, const ClStepArgs &a, int grid, cudaStream_t s);

@@ -9,6 +9,11 @@
 //   HEAD   LM head fused with the clamp, an online softmax / entropy reduction, top-1 probability and
 //          argmax (Section 3.1, Eq. 1-4): logits are never written unless asked for.
 // This is the general path (any T, fp32 or bf16 weights); it is bound by HBM weight streaming for T = 1.
+#include <math.h>
+#include <string.h>
+
+#include <mutex>
+
 #include "cl_internal.h"
 
 namespace {
@@ -219,4 +224,123 @@ cudaError_t launch_w(int T, int epi, const ClGemvArgs &a, int grid, cudaStream_t
 cudaError_t cl_launch_gemv(int wdtype, int T, int epi, const ClGemvArgs &a, int grid, cudaStream_t s) {
     if (wdtype == 1) return launch_w<__nv_bfloat16>(T, epi, a, grid, s);
     return launch_w<float>(T, epi, a, grid, s);
+}
+
+// ---- confidence scoring without any allocation ------------------------------------------------------
+// Scratch of cl_layer_confidences_static(): one file-scope array that every GPU loading this library holds until
+// the process exits.  Layout (bytes): [0, 256) the LM-head kernel's ticket counter; then the normalised rows
+// xn [CL_MAX_T, CL_STATIC_MAX_D] fp32; the per-block softmax partials [SC_MAX_GRID, CL_MAX_T]; and the three
+// per-row results (confidence, top-1 probability, greedy token) [CL_STATIC_MAX_ROWS] each.
+namespace {
+
+constexpr int SC_MAX_GRID = 1024;
+constexpr int SC_CHUNK = 8;   // rows per LM-head pass
+constexpr size_t SC_OFF_XN = 256;
+constexpr size_t SC_OFF_PART = SC_OFF_XN + (size_t)SC_CHUNK * CL_STATIC_MAX_D * sizeof(float);
+constexpr size_t SC_OFF_CONF = SC_OFF_PART + (size_t)SC_MAX_GRID * SC_CHUNK * sizeof(ClHeadPartial);
+constexpr size_t SC_OFF_PMAX = SC_OFF_CONF + (size_t)CL_STATIC_MAX_ROWS * sizeof(float);
+constexpr size_t SC_OFF_ARG = SC_OFF_PMAX + (size_t)CL_STATIC_MAX_ROWS * sizeof(float);
+constexpr size_t SC_BYTES = SC_OFF_ARG + (size_t)CL_STATIC_MAX_ROWS * sizeof(int);
+
+static __device__ __align__(256) unsigned char g_static_scratch[SC_BYTES];
+
+constexpr int SC_MAX_DEVICES = 64;
+std::mutex g_sc_mutex;
+unsigned char *g_sc_addr[SC_MAX_DEVICES];   // device address of g_static_scratch on each device, once looked up
+int g_sc_sms[SC_MAX_DEVICES];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address: the address a kernel
+// may use comes from cudaGetSymbolAddress, asked once per device with that device current.
+int static_scratch(unsigned char **addr, int *n_sm) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) {
+        cl_set_global_error("cl_layer_confidences_static: no CUDA device: %s", cudaGetErrorString(e));
+        return CL_ECUDA;
+    }
+    if (dev < 0 || dev >= SC_MAX_DEVICES) {
+        cl_set_global_error("cl_layer_confidences_static: device ordinal %d not supported (max %d)", dev, SC_MAX_DEVICES - 1);
+        return CL_ERANGE;
+    }
+    std::lock_guard<std::mutex> lock(g_sc_mutex);
+    if (!g_sc_addr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p) {
+            cl_set_global_error("cl_layer_confidences_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+            return CL_ECUDA;
+        }
+        int sms = 0, major = 0;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (major < 10 || sms <= 0) {
+            cl_set_global_error("cl_layer_confidences_static: compute capability %d.x, built for sm_100a only", major);
+            return CL_ECUDA;
+        }
+        g_sc_sms[dev] = sms;
+        g_sc_addr[dev] = (unsigned char *)p;
+    }
+    *addr = g_sc_addr[dev];
+    *n_sm = g_sc_sms[dev];
+    return CL_OK;
+}
+
+}  // namespace
+
+extern "C" int cl_layer_confidences_static(const void *lm_head, const float *final_norm, int vocab, int d_model,
+                                           int weight_dtype, float rms_eps, const void *hidden, int n_rows,
+                                           void *cuda_stream, float *conf, float *p_max, int32_t *argmax) {
+    if (!lm_head || !final_norm || !hidden) {
+        cl_set_global_error("cl_layer_confidences_static: null input pointer");
+        return CL_EINVAL;
+    }
+    if (weight_dtype != 0 && weight_dtype != 1) {
+        cl_set_global_error("cl_layer_confidences_static: weight_dtype must be 0 or 1");
+        return CL_EINVAL;
+    }
+    if (vocab < 2 || d_model <= 0 || d_model % 8 || n_rows <= 0) {
+        cl_set_global_error("cl_layer_confidences_static: need vocab >= 2, d_model a positive multiple of 8, n_rows > 0");
+        return CL_EINVAL;
+    }
+    if (d_model > CL_STATIC_MAX_D || n_rows > CL_STATIC_MAX_ROWS) {
+        cl_set_global_error("cl_layer_confidences_static: d_model %d / n_rows %d beyond the fixed scratch (max %d / %d)", d_model,
+                            n_rows, CL_STATIC_MAX_D, CL_STATIC_MAX_ROWS);
+        return CL_ERANGE;
+    }
+    unsigned char *sc = nullptr;
+    int n_sm = 0;
+    int rc = static_scratch(&sc, &n_sm);
+    if (rc) return rc;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    float *xn = (float *)(sc + SC_OFF_XN);
+    float *d_conf = (float *)(sc + SC_OFF_CONF), *d_pmax = (float *)(sc + SC_OFF_PMAX);
+    int *d_arg = (int *)(sc + SC_OFF_ARG);
+    const size_t es = weight_dtype == 1 ? 2 : 4;
+    cudaError_t e = cudaMemsetAsync(sc, 0, SC_OFF_XN, s);   // the ticket must start at zero whatever the last call left
+    ClGemvArgs a;
+    memset(&a, 0, sizeof(a));
+    a.W = lm_head; a.rows = vocab; a.cols = d_model; a.xin = xn;
+    a.partials = (ClHeadPartial *)(sc + SC_OFF_PART);
+    a.ticket = (unsigned *)sc;
+    a.inv_log_v = (float)(1.0 / log((double)vocab));
+    int grid = ((vocab + 1) / 2 + 7) / 8;
+    if (grid > n_sm * 4) grid = n_sm * 4;
+    if (grid > SC_MAX_GRID) grid = SC_MAX_GRID;
+    for (int r0 = 0; r0 < n_rows && e == cudaSuccess; r0 += SC_CHUNK) {
+        const int T = n_rows - r0 < SC_CHUNK ? n_rows - r0 : SC_CHUNK;
+        e = cl_launch_rmsnorm_rows(weight_dtype, (const char *)hidden + (size_t)r0 * d_model * es, final_norm, T, d_model, rms_eps,
+                                   xn, s);
+        if (e != cudaSuccess) break;
+        a.out_tok = d_arg + r0; a.out_pmax = d_pmax + r0; a.out_conf = d_conf + r0;
+        e = cl_launch_gemv(weight_dtype, T, CL_EPI_HEAD, a, grid, s);
+    }
+    if (e == cudaSuccess && conf) e = cudaMemcpyAsync(conf, d_conf, (size_t)n_rows * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && p_max) e = cudaMemcpyAsync(p_max, d_pmax, (size_t)n_rows * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && argmax) e = cudaMemcpyAsync(argmax, d_arg, (size_t)n_rows * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        cl_set_global_error("cl_layer_confidences_static: %s", cudaGetErrorString(e));
+        return CL_ECUDA;
+    }
+    return CL_OK;
 }
