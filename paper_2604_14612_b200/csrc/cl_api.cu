@@ -331,7 +331,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
             c->max_blk = (g.max_seq + 31) / 32;
             DM(c->bar_dev, 2 * sizeof(unsigned));
             CU(cudaMemsetAsync(c->bar_dev, 0, 2 * sizeof(unsigned), c->stream));
-            DM(c->att_part2, (size_t)g.n_heads * c->max_blk * (g.head_dim + 2) * 4);
+            DM(c->att_part2, (size_t)g.n_heads * c->max_blk * (g.head_dim + 4) * 4);
             DM(c->att_tickets2, (size_t)g.n_heads * 4);
             CU(cudaMemsetAsync(c->att_tickets2, 0, (size_t)g.n_heads * 4, c->stream));
             DM(c->head_part2, (size_t)c->n_sm * sizeof(ClHeadPartial));

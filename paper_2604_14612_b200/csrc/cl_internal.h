@@ -87,7 +87,7 @@ struct ClStepArgs {
     const float2 *rope_cs;
     ClDevState *st;
     float *x, *qkv, *att, *hff;          // global activation vectors [d] [3d] [d] [F]
-    float *att_part;                     // [H, max_blk, hd + 2]
+    float *att_part;                     // [H, max_blk, hd + 4]
     unsigned *att_tickets;               // [H]
     ClHeadPartial *head_part;            // [grid]
     unsigned *bar;                       // grid barrier: [0] arrivals, [1] generation

@@ -21,10 +21,9 @@ namespace {
 
 constexpr int NCW = 8;                 // consumer warps
 constexpr int NCT = NCW * 32;          // consumer threads
-constexpr int SLOT_BYTES = 8192;       // ring slot: 512 chunks of 16 bytes = 2 chunks per consumer thread
-constexpr int NSLOT = 24;              // 192 KB in flight per SM
+constexpr int SLOT_BYTES = 32768;      // ring slot: as many whole weight rows as fit (at least one)
+constexpr int NSLOT = 6;               // 192 KB in flight per SM
 constexpr int MAXIT = 8;               // 16-byte chunks per thread per row: rows up to 32 KB (C <= 16384 bf16)
-constexpr int MAXSEG = MAXIT / 2;
 constexpr int RB = 256;                // rows per epilogue block
 constexpr unsigned long long WAIT_NS = 2000000000ull;   // 2 s bound on any single wait
 
@@ -261,70 +260,135 @@ __device__ __forceinline__ void my_rows(int rows, int unit, int &r0, int &r1) {
     r1 = (int)(units * (blockIdx.x + 1) / gridDim.x) * unit;
 }
 
+// Rows per ring slot for a matrix with `rowbytes` bytes per row.  Phases whose epilogue pairs rows (unit 2) keep
+// pairs inside a slot.  Producer and consumers derive the same slot <-> rows mapping from this.
+__device__ __forceinline__ int rows_per_slot(size_t rowbytes, int unit) {
+    int rps = (int)((size_t)SLOT_BYTES / rowbytes);
+    if (rps < 1) rps = 1;
+    if (unit == 2 && (rps & 1) && rps > 1) rps -= 1;
+    return rps;
+}
+
 // ---- producer -------------------------------------------------------------------------------------
+// One bulk copy per slot: the next rps rows of this CTA's block, which are contiguous in memory.
 template <typename WT>
 __device__ void produce_matrix(const char *W, int rows, int cols, int unit, Ring &rg, unsigned char *ring, Smem *sm,
                                ClDevState *st, unsigned *last_par) {
     int r0, r1;
     my_rows(rows, unit, r0, r1);
     const size_t rowbytes = (size_t)cols * sizeof(WT);
-    const int nseg = (int)((rowbytes + SLOT_BYTES - 1) / SLOT_BYTES);
-    for (int r = r0; r < r1; ++r) {
-        const char *src = W + (size_t)r * rowbytes;
-        for (int s = 0; s < nseg; ++s) {
-            const unsigned bytes = (unsigned)min((size_t)SLOT_BYTES, rowbytes - (size_t)s * SLOT_BYTES);
-            mbar_wait(&sm->empty[rg.slot], rg.par ^ 1u, sm, st);
-            if (!*(volatile int *)&sm->abort) {
-                mbar_expect_tx(&sm->full[rg.slot], bytes);
-                bulk_g2s(ring + (size_t)rg.slot * SLOT_BYTES, src + (size_t)s * SLOT_BYTES, bytes, &sm->full[rg.slot]);
-                last_par[rg.slot] = rg.par;
-            }
-            rg.advance();
+    const int rps = rows_per_slot(rowbytes, unit);
+    for (int r = r0; r < r1; r += rps) {
+        const unsigned bytes = (unsigned)((size_t)min(rps, r1 - r) * rowbytes);
+        mbar_wait(&sm->empty[rg.slot], rg.par ^ 1u, sm, st);
+        if (!*(volatile int *)&sm->abort) {
+            mbar_expect_tx(&sm->full[rg.slot], bytes);
+            bulk_g2s(ring + (size_t)rg.slot * SLOT_BYTES, W + (size_t)r * rowbytes, bytes, &sm->full[rg.slot]);
+            last_par[rg.slot] = rg.par;
         }
+        rg.advance();
     }
 }
 
 // ---- consumer: one matrix phase ------------------------------------------------------------------------
-// xr: this thread's activation registers, xr[it][e] = x[(it * NCT + tid) * EPC + e].
-// Calls epi(row_local_index_in_block, first_row_of_block, rows_in_block) with the partial table ready.
-template <typename WT, typename Epi>
-__device__ __forceinline__ void consume_matrix(int rows, int cols, int unit, const float (&xr)[MAXIT][Chunk<WT>::EPC],
-                                               Ring &rg, const unsigned char *ring, Smem *sm, ClDevState *st, Epi epi) {
+// Sums R per-thread values across the warp at once ("transposing" butterfly): log2(R) exchange steps halve the
+// number of values each lane carries, the remaining steps are plain butterflies.  On return acc[0] holds the
+// warp total of row (lane >> (5 - log2 R)) & (R - 1) in every lane; the combine order is fixed.
+template <int R>
+__device__ __forceinline__ void warp_reduce_rows(float (&acc)[R], int lane) {
+    int off = 16;
+#pragma unroll
+    for (int half = R / 2; half >= 1; half >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            const float send = upper ? acc[i] : acc[i + half];
+            const float keep = upper ? acc[i + half] : acc[i];
+            acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+        off >>= 1;
+    }
+#pragma unroll
+    for (; off >= 1; off >>= 1) acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], off);
+}
+
+template <int R>
+struct Log2;
+template <> struct Log2<1> { static constexpr int v = 0; };
+template <> struct Log2<2> { static constexpr int v = 1; };
+template <> struct Log2<4> { static constexpr int v = 2; };
+template <> struct Log2<8> { static constexpr int v = 3; };
+
+// xr: this thread's activation registers, xr[it][e] = x[(it * NCT + tid) * EPC + e]; NIT = chunks per thread per
+// row (rounded up to a supported count).  One wait per slot; inside a slot rows are taken R at a time in
+// straight-line code: all of a group's 16-byte reads are issued before the first multiply-add, every row has
+// its own accumulation chain, and the R row sums are reduced across the warp together.
+// Calls epi(first_row_of_block, rows_in_block) once the partial table of a block of up to RB rows is ready.
+template <typename WT, int NIT, int R, typename Epi>
+__device__ __forceinline__ void consume_rows(int r0, int r1, int nchunks, int rps, const float (&xr)[MAXIT][Chunk<WT>::EPC],
+                                             Ring &rg, const unsigned char *ring, Smem *sm, ClDevState *st, Epi epi) {
     constexpr int EPC = Chunk<WT>::EPC;
+    constexpr int SH = 5 - Log2<R>::v;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int r0, r1;
-    my_rows(rows, unit, r0, r1);
-    const int nchunks = cols / EPC;
-    const int nseg = (nchunks + 511) / 512;
-    for (int rb0 = r0; rb0 < r1; rb0 += RB) {
-        const int nrb = min(RB, r1 - rb0);
-        for (int r = 0; r < nrb; ++r) {
-            float acc = 0.f;
+    const size_t rowbytes = (size_t)nchunks * 16;
+    const int blockrows = max(1, RB / rps) * rps;
+    for (int rb0 = r0; rb0 < r1; rb0 += blockrows) {
+        const int nrb = min(blockrows, r1 - rb0);
+        for (int sr = 0; sr < nrb; sr += rps) {
+            const int ns = min(rps, nrb - sr);   // rows in this slot
+            mbar_wait(&sm->full[rg.slot], rg.par, sm, st);
+            const unsigned char *base = ring + (size_t)rg.slot * SLOT_BYTES + (size_t)tid * 16;
+            for (int g = 0; g < ns; g += R) {
+                uint4 w[R][NIT];
 #pragma unroll
-            for (int s = 0; s < MAXSEG; ++s) {
-                if (s < nseg) {
-                    mbar_wait(&sm->full[rg.slot], rg.par, sm, st);
-                    const unsigned char *base = ring + (size_t)rg.slot * SLOT_BYTES;
+                for (int i = 0; i < R; ++i) {
+                    // rows past the end of the slot re-read its last row (their sums are dropped below)
+                    const unsigned char *rowp = base + (size_t)min(g + i, ns - 1) * rowbytes;
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const int it = 2 * s + j;
-                        if (it * NCT + tid < nchunks) {
-                            const uint4 w = *(const uint4 *)(base + (size_t)(j * NCT + tid) * 16);
-                            acc = Chunk<WT>::dot(w, xr[it], acc);
-                        }
+                    for (int it = 0; it < NIT; ++it) {
+                        if (it * NCT + tid < nchunks) w[i][it] = *(const uint4 *)(rowp + (size_t)it * (NCT * 16));
+                        else w[i][it] = make_uint4(0u, 0u, 0u, 0u);
                     }
+                }
+                float acc[R];
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    float a0 = 0.f, a1 = 0.f;   // two chains per row: even and odd chunks
+#pragma unroll
+                    for (int it = 0; it < NIT; ++it) {
+                        if (it & 1) a1 = Chunk<WT>::dot(w[i][it], xr[it], a1);
+                        else a0 = Chunk<WT>::dot(w[i][it], xr[it], a0);
+                    }
+                    acc[i] = a0 + a1;
+                }
+                if (g + R >= ns) {   // every read of this slot has returned: hand it back to the producer
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm->empty[rg.slot]);
-                    rg.advance();
                 }
+                warp_reduce_rows<R>(acc, lane);
+                const int row = sr + g + ((lane >> SH) & (R - 1));
+                if ((lane & ((1 << SH) - 1)) == 0 && row < sr + ns) sm->partial[row * NCW + warp] = acc[0];
             }
-            acc = warp_sum(acc);
-            if (lane == 0) sm->partial[r * NCW + warp] = acc;
+            rg.advance();
         }
         consumer_sync();
         epi(rb0, nrb);
         consumer_sync();
     }
+}
+
+template <typename WT, typename Epi>
+__device__ __forceinline__ void consume_matrix(int rows, int cols, int unit, const float (&xr)[MAXIT][Chunk<WT>::EPC],
+                                               Ring &rg, const unsigned char *ring, Smem *sm, ClDevState *st, Epi epi) {
+    constexpr int EPC = Chunk<WT>::EPC;
+    int r0, r1;
+    my_rows(rows, unit, r0, r1);
+    const int nchunks = cols / EPC;
+    const int rps = rows_per_slot((size_t)nchunks * 16, unit);
+    const int nit = (nchunks + NCT - 1) / NCT;   // uniform over the grid
+    if (nit <= 2) consume_rows<WT, 2, 4>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
+    else if (nit <= 4) consume_rows<WT, 4, 2>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
+    else consume_rows<WT, 8, 1>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
 }
 
 __device__ __forceinline__ float row_sum(const Smem *sm, int r) {
@@ -395,7 +459,7 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
     constexpr int LPK = HD / EPL;               // lanes per key
     constexpr int KPW = 32 / LPK;               // keys per warp pass
     constexpr int VPL = HD / 32;                // value elements per lane
-    constexpr int PSTRIDE = HD + 2;
+    constexpr int PSTRIDE = HD + 4;              // (max, sum, pad, pad, o[HD]): o rows stay 16-byte aligned
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nkeys = pos + 1;
     const int nblk = (nkeys + 31) >> 5;
@@ -472,10 +536,12 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
         float o_acc[VPL];
 #pragma unroll
         for (int e = 0; e < VPL; ++e) o_acc[e] = 0.f;
-        for (int j = 0; j < n; ++j) {
+        // all 32 value rows are fetched at once (rows past the end repeat the last one with weight 0)
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
             const float pj = __shfl_sync(0xffffffffu, p, j);
             float vv[VPL];
-            load_vals<ST, VPL>(Vc + (size_t)(j0 + j) * d + h * HD + lane * VPL, vv);
+            load_vals<ST, VPL>(Vc + (size_t)(j0 + min(j, n - 1)) * d + h * HD + lane * VPL, vv);
 #pragma unroll
             for (int e = 0; e < VPL; ++e) o_acc[e] = fmaf(pj, vv[e], o_acc[e]);
         }
@@ -485,27 +551,55 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
             part[1] = l;
         }
 #pragma unroll
-        for (int e = 0; e < VPL; ++e) part[2 + lane * VPL + e] = o_acc[e];
+        for (int e = 0; e < VPL; ++e) part[4 + lane * VPL + e] = o_acc[e];
         __threadfence();
         __syncwarp();
         unsigned prev = 0;
         if (lane == 0) prev = atomicAdd(a.att_tickets + h, 1u);
         prev = __shfl_sync(0xffffffffu, prev, 0);
         if (prev == (unsigned)nblk - 1) {
-            // last block of this head to finish: merge all blocks in order, normalise, write the head's output
+            // last block of this head to finish: merge all blocks in a fixed order, normalise, write the head's
+            // output.  Lanes first work across blocks (maximum, weights, denominator), then each lane sums its VPL
+            // output elements over the blocks with 16 partial rows in flight at a time.
             __threadfence();
             const float *p0 = a.att_part + (size_t)h * a.max_blk * PSTRIDE;
             float M = -INFINITY;
-            for (int b = 0; b < nblk; ++b) M = fmaxf(M, ldcg_f(p0 + (size_t)b * PSTRIDE));
+            for (int b = lane; b < nblk; b += 32) M = fmaxf(M, ldcg_f(p0 + (size_t)b * PSTRIDE));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
             float Ls = 0.f, O[VPL];
 #pragma unroll
             for (int e = 0; e < VPL; ++e) O[e] = 0.f;
-            for (int b = 0; b < nblk; ++b) {
-                const float w = expf(ldcg_f(p0 + (size_t)b * PSTRIDE) - M);
-                Ls = fmaf(ldcg_f(p0 + (size_t)b * PSTRIDE + 1), w, Ls);
+            for (int b0 = 0; b0 < nblk; b0 += 32) {
+                const int b = b0 + lane;
+                const float w = (b < nblk) ? expf(ldcg_f(p0 + (size_t)b * PSTRIDE) - M) : 0.f;
+                if (b < nblk) Ls = fmaf(ldcg_f(p0 + (size_t)b * PSTRIDE + 1), w, Ls);
 #pragma unroll
-                for (int e = 0; e < VPL; ++e) O[e] = fmaf(ldcg_f(p0 + (size_t)b * PSTRIDE + 2 + lane * VPL + e), w, O[e]);
+                for (int kb0 = 0; kb0 < 32; kb0 += 16) {
+                    if (b0 + kb0 < nblk) {
+                        float pv[16][VPL];
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            const int bb = min(b0 + kb0 + k, nblk - 1);
+                            const float *src = p0 + (size_t)bb * PSTRIDE + 4 + lane * VPL;
+                            if (VPL == 4) {
+                                const float4 t = ldcg_f4(src);
+                                pv[k][0] = t.x; pv[k][1 % VPL] = t.y; pv[k][2 % VPL] = t.z; pv[k][3 % VPL] = t.w;
+                            } else {
+                                const float2 t = __ldcg((const float2 *)src);
+                                pv[k][0] = t.x; pv[k][1 % VPL] = t.y;
+                            }
+                        }
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            const float wk = __shfl_sync(0xffffffffu, w, kb0 + k);   // 0 for blocks past the end
+#pragma unroll
+                            for (int e = 0; e < VPL; ++e) O[e] = fmaf(pv[k][e], wk, O[e]);
+                        }
+                    }
+                }
             }
+            Ls = warp_sum(Ls);
 #pragma unroll
             for (int e = 0; e < VPL; ++e) a.att[h * HD + lane * VPL + e] = O[e] / Ls;
             if (lane == 0) a.att_tickets[h] = 0u;
