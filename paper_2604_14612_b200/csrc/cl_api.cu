@@ -53,10 +53,9 @@ struct cl_ctx {
     // token-step kernel (persistent single-token step)
     ClLayerDev *layers_dev;
     int *kept_dev, *kept_all_dev;
-    int n_kept, use_step, max_blk;
+    int n_kept, use_step, max_blk, att_parts, l2_ahead;
     unsigned *bar_dev;
     float *att_part2;
-    unsigned *att_tickets2;
     ClHeadPartial *head_part2;
     std::vector<ClLayer> layers;
     std::vector<uint8_t> mask;    // host copy of the skip set
@@ -181,7 +180,7 @@ static void free_all(cl_ctx *c) {
     void *ptrs[] = {c->wbuf, c->embed, c->lm_head, c->final_norm, c->norms, c->kv, c->rope_cs, c->x, c->xn, c->qkv,
                     c->att, c->hff, c->att_part, c->logits, c->tickets, c->head_part, c->st, c->prompt_dev, c->out_dev,
                     c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sel_mask, c->sel_margins, c->sel_clayers,
-                    c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->att_tickets2, c->head_part2};
+                    c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->head_part2};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->h_st) cudaFreeHost(c->h_st);
@@ -331,9 +330,14 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
             c->max_blk = (g.max_seq + 31) / 32;
             DM(c->bar_dev, 2 * sizeof(unsigned));
             CU(cudaMemsetAsync(c->bar_dev, 0, 2 * sizeof(unsigned), c->stream));
-            DM(c->att_part2, (size_t)g.n_heads * c->max_blk * (g.head_dim + 4) * 4);
-            DM(c->att_tickets2, (size_t)g.n_heads * 4);
-            CU(cudaMemsetAsync(c->att_tickets2, 0, (size_t)g.n_heads * 4, c->stream));
+            DM(c->att_part2, (size_t)g.n_heads * 8 * (g.head_dim + 4) * 4);
+            CU(cudaMemsetAsync(c->att_part2, 0, (size_t)g.n_heads * 8 * (g.head_dim + 4) * 4, c->stream));
+            c->att_parts = c->n_sm / g.n_heads;
+            if (c->att_parts > 8) c->att_parts = 8;
+            if (c->att_parts < 1) c->att_parts = 1;
+            const char *ah = getenv("CL_L2_AHEAD_KB");   // tuning knob: L2 run-ahead of the weight stream per SM
+            c->l2_ahead = (ah && ah[0]) ? atoi(ah) * 1024 : 0;   // measured on B200: any run-ahead made decoding slower
+            if (c->l2_ahead < 0) c->l2_ahead = 0;
             DM(c->head_part2, (size_t)c->n_sm * sizeof(ClHeadPartial));
             const int maxc = cl_step_max_cols(g.weight_dtype);
             int coop = 0;
@@ -425,12 +429,14 @@ static int run_steps(cl_ctx *c, int mode, int n_steps, int row0, bool full_model
     a.kept = full_model ? c->kept_all_dev : c->kept_dev;
     a.n_kept = full_model ? g.n_layers : c->n_kept;
     a.embed = c->embed; a.lm_head = c->lm_head; a.final_norm = c->final_norm;
-    a.d = g.d_model; a.F = g.d_ffn; a.V = g.vocab; a.H = g.n_heads; a.max_seq = g.max_seq; a.max_blk = c->max_blk;
+    a.d = g.d_model; a.F = g.d_ffn; a.V = g.vocab; a.H = g.n_heads; a.max_seq = g.max_seq;
+    a.att_parts = c->att_parts; a.l2_ahead = c->l2_ahead;
     a.eps = g.rms_eps; a.inv_log_v = (float)(1.0 / log((double)g.vocab));
     a.rope_cs = c->rope_cs; a.st = c->st;
-    a.x = c->x; a.qkv = c->qkv; a.att = c->att; a.hff = c->hff;
-    a.att_part = c->att_part2; a.att_tickets = c->att_tickets2; a.head_part = c->head_part2; a.bar = c->bar_dev;
+    a.x = c->x; a.qkv = c->qkv; a.hff = c->hff;
+    a.att_part = c->att_part2; a.head_part = c->head_part2; a.bar = c->bar_dev;
     a.n_steps = n_steps; a.mode = mode; a.row0 = row0; a.out_tokens = out_tokens; a.logits = logits;
+    CU(cudaMemsetAsync(c->bar_dev, 0, 2 * sizeof(unsigned), c->stream));   // the arrival counter starts at zero
     KL(cl_launch_token_steps(g.weight_dtype, g.head_dim, a, c->n_sm, c->stream));
     return CL_OK;
 }
@@ -441,7 +447,6 @@ static int check_device_err(cl_ctx *c, const char *fn) {
         const int e = c->h_st->err;
         cudaMemsetAsync(c->bar_dev, 0, 2 * sizeof(unsigned), c->stream);
         cudaMemsetAsync(&c->st->err, 0, sizeof(int), c->stream);
-        cudaMemsetAsync(c->att_tickets2, 0, (size_t)c->cfg.n_heads * 4, c->stream);
         cudaStreamSynchronize(c->stream);
         return fail(c, CL_ETIMEOUT, "%s: a bounded device-side wait expired (flags %d); results of this call are invalid", fn, e);
     }

@@ -82,15 +82,16 @@ struct ClStepArgs {
     int n_kept;
     const void *embed, *lm_head;
     const float *final_norm;
-    int d, F, V, H, max_seq, max_blk;
+    int d, F, V, H, max_seq;
+    int att_parts;                       // S: parts the cached keys of a head are cut into (1 .. 8), one CTA each
+    int l2_ahead;                        // bytes per CTA the weight prefetch into L2 runs in front of the ring
     float eps, inv_log_v;
     const float2 *rope_cs;
     ClDevState *st;
-    float *x, *qkv, *att, *hff;          // global activation vectors [d] [3d] [d] [F]
-    float *att_part;                     // [H, max_blk, hd + 4]
-    unsigned *att_tickets;               // [H]
+    float *x, *qkv, *hff;                // global activation vectors [d] [3d] [F]
+    float *att_part;                     // [H, 8, hd + 4] per-part attention records (max, sum, -, -, o[hd])
     ClHeadPartial *head_part;            // [grid]
-    unsigned *bar;                       // grid barrier: [0] arrivals, [1] generation
+    unsigned *bar;                       // grid barrier: arrival counter, zero at launch
     int n_steps, mode, row0;
     int *out_tokens;                     // vanilla mode: emitted tokens (may be null)
     float *logits;                       // optional [n_steps, V]

@@ -88,28 +88,47 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
                  : "memory");
 }
 
+// The same copy, marking the lines evict-first in L2: streamed weights are used once per token.
+__device__ __forceinline__ void bulk_g2s_stream(void *dst, const void *src, unsigned bytes, unsigned long long *bar,
+                                                unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+            smem_u32(dst)),
+        "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ unsigned long long policy_evict_first() {
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+// Ask L2 to fetch a 16-byte-aligned range (multiple of 16 bytes); nothing waits for it.
+__device__ __forceinline__ void l2_prefetch_bulk(const void *src, unsigned bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void l2_prefetch_line(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NCT) : "memory"); }
 
 __device__ __forceinline__ float ldcg_f(const float *p) { return __ldcg(p); }
 __device__ __forceinline__ float4 ldcg_f4(const float *p) { return __ldcg((const float4 *)p); }
 
-// Sense-reversing grid barrier on (count, generation) in global memory, called by every consumer
+// Grid barrier on one arrival counter in global memory that only ever grows during a launch (the host zeroes
+// it before every launch): barrier number i is passed once the counter reaches i * gridDim.x.  One release
+// increment and an acquire poll per CTA; `target` lives in thread 0's registers.  Called by every consumer
 // thread of every CTA; bounded in time.
-__device__ __forceinline__ void grid_barrier(unsigned *bar, Smem *sm, ClDevState *st) {
+__device__ __forceinline__ void grid_barrier(unsigned *bar, unsigned &target, Smem *sm, ClDevState *st) {
     consumer_sync();
     if (threadIdx.x == 0 && !*(volatile int *)&sm->abort) {
-        volatile unsigned *gen = bar + 1;
-        const unsigned my_gen = *gen;
-        __threadfence();
-        const unsigned arrived = atomicAdd(bar, 1u);
-        if (arrived == gridDim.x - 1) {
-            *(volatile unsigned *)bar = 0u;
-            __threadfence();
-            atomicAdd(bar + 1, 1u);
-        } else {
+        target += gridDim.x;
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
+        if ((int)(v - target) < 0) {
             const unsigned long long t0 = gtime();
             unsigned i = 0;
-            while (*gen == my_gen) {
+            do {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
                 if ((++i & 255u) == 0u) {
                     if (*(volatile int *)&st->err || gtime() - t0 > WAIT_NS) {
                         *(volatile int *)&sm->abort = 1;
@@ -117,9 +136,8 @@ __device__ __forceinline__ void grid_barrier(unsigned *bar, Smem *sm, ClDevState
                         break;
                     }
                 }
-            }
+            } while ((int)(v - target) < 0);
         }
-        __threadfence();
     }
     consumer_sync();
 }
@@ -270,23 +288,100 @@ __device__ __forceinline__ int rows_per_slot(size_t rowbytes, int unit) {
 }
 
 // ---- producer -------------------------------------------------------------------------------------
-// One bulk copy per slot: the next rps rows of this CTA's block, which are contiguous in memory.
+// Walks the static schedule (steps x kept layers x {QKV, O, gate/up, down} + LM head) slot by slot: each call of
+// next() yields the next rps rows of this CTA's block of the current matrix, which are contiguous in memory.
 template <typename WT>
-__device__ void produce_matrix(const char *W, int rows, int cols, int unit, Ring &rg, unsigned char *ring, Smem *sm,
-                               ClDevState *st, unsigned *last_par) {
-    int r0, r1;
-    my_rows(rows, unit, r0, r1);
-    const size_t rowbytes = (size_t)cols * sizeof(WT);
-    const int rps = rows_per_slot(rowbytes, unit);
-    for (int r = r0; r < r1; r += rps) {
-        const unsigned bytes = (unsigned)((size_t)min(rps, r1 - r) * rowbytes);
+struct SchedIter {
+    const ClStepArgs &a;
+    int step, ki, m;        // m: 0..3 = the layer's matrices; ki == n_kept: the LM head (m = 0)
+    int r, r1, rps;
+    size_t rowbytes;
+    const char *W;
+    ClLayerDev L;
+    bool done;
+    __device__ SchedIter(const ClStepArgs &args) : a(args), step(0), ki(0), m(0), done(false) {
+        if (a.n_steps <= 0) done = true;
+        else open();
+    }
+    __device__ void open() {   // set up (step, ki, m); skips matrices of which this CTA owns no row
+        for (;;) {
+            int rows, cols, unit = 1;
+            if (ki < a.n_kept) {
+                if (m == 0) L = a.layers[a.kept[ki]];
+                if (m == 0) { W = L.wqkv; rows = 3 * a.d; cols = a.d; }
+                else if (m == 1) { W = L.wo; rows = a.d; cols = a.d; }
+                else if (m == 2) { W = L.wgu; rows = 2 * a.F; cols = a.d; unit = 2; }
+                else { W = L.wd; rows = a.d; cols = a.F; }
+            } else {
+                W = (const char *)a.lm_head; rows = a.V; cols = a.d;
+            }
+            my_rows(rows, unit, r, r1);
+            rowbytes = (size_t)cols * sizeof(WT);
+            rps = rows_per_slot(rowbytes, unit);
+            if (r < r1) return;
+            if (!advance()) return;
+        }
+    }
+    __device__ bool advance() {   // to the next matrix of the schedule; false at the end
+        if (ki < a.n_kept && m < 3) { ++m; return true; }
+        m = 0;
+        if (ki < a.n_kept) { ++ki; return true; }
+        ki = 0;
+        if (++step < a.n_steps) return true;
+        done = true;
+        return false;
+    }
+    __device__ bool next(const char *&src, unsigned &bytes) {
+        if (done) return false;
+        const int n = min(rps, r1 - r);
+        src = W + (size_t)r * rowbytes;
+        bytes = (unsigned)((size_t)n * rowbytes);
+        r += n;
+        if (r >= r1 && advance()) open();
+        return true;
+    }
+};
+
+// The producer thread.  Two cursors over the same schedule: the fill cursor feeds the shared-memory ring as slots
+// come free; the prefetch cursor runs up to l2_ahead bytes in front of it and only asks L2 to fetch, so that HBM
+// keeps streaming into L2 while the consumers sit in a grid barrier or the attention phase and the ring is full.
+template <typename WT>
+__device__ void producer_loop(const ClStepArgs &a, unsigned char *ring, Smem *sm, ClDevState *st) {
+    Ring rg{0u, 0u};
+    unsigned last_par[NSLOT];
+    for (int i = 0; i < NSLOT; ++i) last_par[i] = 2u;
+    const unsigned long long policy = policy_evict_first();
+    SchedIter<WT> fill(a), pf(a);
+    unsigned long long filled = 0, fetched = 0;
+    const unsigned long long ahead = (unsigned long long)a.l2_ahead;
+    const char *src;
+    unsigned bytes;
+    while (fill.next(src, bytes)) {
+        if (ahead) {
+            const char *psrc;
+            unsigned pbytes;
+            while (fetched < filled + bytes + ahead && pf.next(psrc, pbytes)) {
+                if (fetched >= filled + bytes) l2_prefetch_bulk(psrc, pbytes);   // not what is about to be copied anyway
+                fetched += pbytes;
+            }
+        }
         mbar_wait(&sm->empty[rg.slot], rg.par ^ 1u, sm, st);
         if (!*(volatile int *)&sm->abort) {
             mbar_expect_tx(&sm->full[rg.slot], bytes);
-            bulk_g2s(ring + (size_t)rg.slot * SLOT_BYTES, W + (size_t)r * rowbytes, bytes, &sm->full[rg.slot]);
+            bulk_g2s_stream(ring + (size_t)rg.slot * SLOT_BYTES, src, bytes, &sm->full[rg.slot], policy);
             last_par[rg.slot] = rg.par;
         }
         rg.advance();
+        filled += bytes;
+    }
+    // Drain: every copy this thread issued must have landed before the CTA may exit.  In the normal path the
+    // consumers have already waited for all of them; after an abort this is the bounded wait for copies in flight.
+    for (int i = 0; i < NSLOT; ++i) {
+        if (last_par[i] < 2u) {
+            const unsigned long long t0 = gtime();
+            while (!mbar_try(&sm->full[i], last_par[i]))
+                if (gtime() - t0 > WAIT_NS) break;
+        }
     }
 }
 
@@ -419,10 +514,27 @@ __device__ __forceinline__ void load_x(const float *x, int cols, float (&xr)[MAX
     }
 }
 
-// RMSNorm in registers: xr <- x * rsqrt(mean(x^2) + eps) * g.
+// RMSNorm in registers: xr <- x * rsqrt(mean(x^2) + eps) * g.  The gains are requested together with x so that the
+// phase start costs one memory round trip, not two.
 template <int EPC>
 __device__ __forceinline__ void load_x_rmsnorm(const float *x, const float *g, int cols, float eps, float (&xr)[MAXIT][EPC],
                                                Smem *sm) {
+    const int nchunks = cols / EPC;
+    float gr[MAXIT][EPC];
+#pragma unroll
+    for (int it = 0; it < MAXIT; ++it) {
+        const int ch = it * NCT + threadIdx.x;
+        if (ch < nchunks) {
+#pragma unroll
+            for (int q = 0; q < EPC / 4; ++q) {
+                const float4 gv = __ldg((const float4 *)(g + (size_t)ch * EPC + 4 * q));
+                gr[it][4 * q] = gv.x; gr[it][4 * q + 1] = gv.y; gr[it][4 * q + 2] = gv.z; gr[it][4 * q + 3] = gv.w;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < EPC; ++e) gr[it][e] = 0.f;
+        }
+    }
     load_x<EPC>(x, cols, xr);
     float ss = 0.f;
 #pragma unroll
@@ -437,55 +549,72 @@ __device__ __forceinline__ void load_x_rmsnorm(const float *x, const float *g, i
 #pragma unroll
     for (int w = 0; w < NCW; ++w) tot += sm->red[w];
     const float sc = 1.0f / sqrtf(tot / (float)cols + eps);
-    const int nchunks = cols / EPC;
 #pragma unroll
-    for (int it = 0; it < MAXIT; ++it) {
-        const int ch = it * NCT + threadIdx.x;
-        if (ch < nchunks) {
+    for (int it = 0; it < MAXIT; ++it)
 #pragma unroll
-            for (int q = 0; q < EPC / 4; ++q) {
-                const float4 gv = __ldg((const float4 *)(g + (size_t)ch * EPC + 4 * q));
-                xr[it][4 * q] *= sc * gv.x; xr[it][4 * q + 1] *= sc * gv.y;
-                xr[it][4 * q + 2] *= sc * gv.z; xr[it][4 * q + 3] *= sc * gv.w;
-            }
-        }
+        for (int e = 0; e < EPC; ++e) xr[it][e] *= sc * gr[it][e];
+}
+
+// ---- attention phase ---------------------------------------------------------------------------------
+// Work split: (head h, part s) -> one CTA; the cached keys [0, pos) of a head are cut into S contiguous parts and a
+// part into NCW contiguous warp ranges.  A warp walks its range 32 keys at a time (one score per lane) with an
+// online softmax; the new position's key and value (this step's QKV output, rotated, rounded to the storage type
+// and appended to the cache) are one more partial, taken by the last warp of the last part.  The CTA merges its
+// warps' partials in shared memory and writes one (max, sum, unnormalised output) record per (h, s); the S records
+// of a head are merged by whoever reads the attention output (load_att_merged), so no CTA waits on another here.
+constexpr int ATT_MAX_PARTS = 8;
+
+template <typename ST, int HD>
+struct AttnGeom {
+    static constexpr int EPL = 16 / (int)sizeof(ST);   // elements per lane per key
+    static constexpr int LPK = HD / EPL;               // lanes per key
+    static constexpr int KPW = 32 / LPK;               // keys per warp pass
+    static constexpr int VPL = HD / 32;                // value elements per lane
+    static constexpr int PSTRIDE = HD + 4;             // (max, sum, pad, pad, o[HD]): o stays 16-byte aligned
+};
+
+__device__ __forceinline__ void warp_key_range(int pos, int s, int S, int warp, int &kw0, int &kw1) {
+    const int k0 = (int)((long long)pos * s / S), k1 = (int)((long long)pos * (s + 1) / S);
+    kw0 = k0 + (k1 - k0) * warp / NCW;
+    kw1 = k0 + (k1 - k0) * (warp + 1) / NCW;
+}
+
+// Ask L2 for the cache lines this CTA's warps will read in the attention phase (issued a whole matrix phase earlier).
+template <typename ST, int HD>
+__device__ __forceinline__ void attention_prefetch(const ClStepArgs &a, const ClLayerDev &L, int pos) {
+    const int S = a.att_parts, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int item = blockIdx.x;
+    if (item >= a.H * S) return;
+    const int h = item % a.H, s = item / a.H;
+    int kw0, kw1;
+    warp_key_range(pos, s, S, warp, kw0, kw1);
+    constexpr int ROWB = HD * (int)sizeof(ST);
+    constexpr int LINES = (ROWB + 127) / 128;
+    const int n = (kw1 - kw0) * LINES;
+    for (int i = lane; i < n; i += 32) {
+        const size_t off = ((size_t)(kw0 + i / LINES) * a.d + (size_t)h * HD) * sizeof(ST) + (size_t)(i % LINES) * 128;
+        l2_prefetch_line(L.kc + off);
+        l2_prefetch_line(L.vc + off);
     }
 }
 
-// ---- attention phase: one warp per (head, block of 32 keys) ------------------------------------------
 template <typename ST, int HD>
 __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int pos, Smem *sm) {
-    constexpr int EPL = 16 / (int)sizeof(ST);   // elements per lane per key
-    constexpr int LPK = HD / EPL;               // lanes per key
-    constexpr int KPW = 32 / LPK;               // keys per warp pass
-    constexpr int VPL = HD / 32;                // value elements per lane
-    constexpr int PSTRIDE = HD + 4;              // (max, sum, pad, pad, o[HD]): o rows stay 16-byte aligned
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int nkeys = pos + 1;
-    const int nblk = (nkeys + 31) >> 5;
-    const int nitems = a.H * nblk;
-    const int d = a.d;
+    using G = AttnGeom<ST, HD>;
+    constexpr int EPL = G::EPL, LPK = G::LPK, KPW = G::KPW, VPL = G::VPL, PSTRIDE = G::PSTRIDE;
+    constexpr int WSTRIDE = HD + 2;   // per-warp record in shared memory: (max, sum, o[HD])
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int S = a.att_parts, d = a.d;
     const int sub = lane / LPK, li = lane % LPK;
     const float scale = rsqrtf((float)HD);
     ST *Kc = (ST *)L.kc;
     ST *Vc = (ST *)L.vc;
-    for (int item = blockIdx.x * NCW + warp; item < nitems; item += gridDim.x * NCW) {
-        const int h = item / nblk, kb = item % nblk;
-        const int j0 = kb << 5, n = min(32, nkeys - j0);
+    float *wrec = sm->partial;   // [NCW][WSTRIDE]
+    for (int item = blockIdx.x; item < a.H * S; item += gridDim.x) {
+        const int h = item % a.H, s = item / a.H;
+        int kw0, kw1;
+        warp_key_range(pos, s, S, warp, kw0, kw1);
         const float *qraw = a.qkv + h * HD;
-        // the block that holds the new position first appends its rotated key and its value to the cache
-        if (j0 + n == nkeys) {
-            const float *kraw = a.qkv + d + h * HD, *vraw = a.qkv + 2 * d + h * HD;
-            for (int i = lane; i < HD / 2; i += 32) {
-                const float2 cs = a.rope_cs[(size_t)pos * (HD / 2) + i];
-                const float ka = ldcg_f(kraw + i), kb2 = ldcg_f(kraw + i + HD / 2);
-                Kc[(size_t)pos * d + h * HD + i] = st_from_f32<ST>(ka * cs.x - kb2 * cs.y);
-                Kc[(size_t)pos * d + h * HD + i + HD / 2] = st_from_f32<ST>(kb2 * cs.x + ka * cs.y);
-                Vc[(size_t)pos * d + h * HD + i] = st_from_f32<ST>(ldcg_f(vraw + i));
-                Vc[(size_t)pos * d + h * HD + i + HD / 2] = st_from_f32<ST>(ldcg_f(vraw + i + HD / 2));
-            }
-            __syncwarp();
-        }
         // rotated query, this lane's EPL elements
         float qr[EPL];
 #pragma unroll
@@ -496,113 +625,175 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
             const float qa = ldcg_f(qraw + i), qb = ldcg_f(qraw + i + HD / 2);
             qr[e] = idx < HD / 2 ? qa * cs.x - qb * cs.y : qb * cs.x + qa * cs.y;
         }
-        // scores of up to 32 keys; lane j ends up holding the score of key j0 + j
-        float my_score = -INFINITY;
+        float m_run = -INFINITY, l_run = 0.f, o_run[VPL];
 #pragma unroll
-        for (int jb = 0; jb < 32; jb += KPW) {
-            const int j = jb + sub;
-            float s = 0.f;
-            if (j < n) {
-                const uint4 raw = __ldcg((const uint4 *)(Kc + (size_t)(j0 + j) * d + h * HD + li * EPL));
-                if (sizeof(ST) == 2) {
-                    const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
+        for (int e = 0; e < VPL; ++e) o_run[e] = 0.f;
+        for (int j0 = kw0; j0 < kw1; j0 += 32) {
+            const int n = min(32, kw1 - j0);
+            // scores of up to 32 keys; lane j ends up holding the score of key j0 + j
+            float my_score = -INFINITY;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        s = fmaf(qr[2 * e], __uint_as_float(u[e] << 16), s);
-                        s = fmaf(qr[2 * e + 1], __uint_as_float(u[e] & 0xffff0000u), s);
+            for (int jb = 0; jb < 32; jb += KPW) {
+                const int j = jb + sub;
+                float sc = 0.f;
+                if (j < n) {
+                    const uint4 raw = __ldcg((const uint4 *)(Kc + (size_t)(j0 + j) * d + h * HD + li * EPL));
+                    if (sizeof(ST) == 2) {
+                        const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            sc = fmaf(qr[(2 * e) % EPL], __uint_as_float(u[e] << 16), sc);
+                            sc = fmaf(qr[(2 * e + 1) % EPL], __uint_as_float(u[e] & 0xffff0000u), sc);
+                        }
+                    } else {
+                        sc = fmaf(qr[0], __uint_as_float(raw.x), sc);
+                        sc = fmaf(qr[1 % EPL], __uint_as_float(raw.y), sc);
+                        sc = fmaf(qr[2 % EPL], __uint_as_float(raw.z), sc);
+                        sc = fmaf(qr[3 % EPL], __uint_as_float(raw.w), sc);
                     }
-                } else {
-                    s = fmaf(qr[0], __uint_as_float(raw.x), s);
-                    s = fmaf(qr[1], __uint_as_float(raw.y), s);
-                    s = fmaf(qr[2], __uint_as_float(raw.z), s);
-                    s = fmaf(qr[3], __uint_as_float(raw.w), s);
+                }
+#pragma unroll
+                for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                sc *= scale;
+                // key jb + k sits in lanes [k * LPK, (k + 1) * LPK): hand it to lane jb + k
+#pragma unroll
+                for (int k = 0; k < KPW; ++k) {
+                    const float v = __shfl_sync(0xffffffffu, sc, k * LPK);
+                    if (lane == jb + k && jb + k < n) my_score = v;
                 }
             }
+            float m_new = my_score;
 #pragma unroll
-            for (int o = LPK >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            s *= scale;
-            // key jb + k sits in lanes [k * LPK, (k + 1) * LPK): hand it to lane jb + k
+            for (int o = 16; o > 0; o >>= 1) m_new = fmaxf(m_new, __shfl_xor_sync(0xffffffffu, m_new, o));
+            m_new = fmaxf(m_new, m_run);
+            const float p = (lane < n) ? expf(my_score - m_new) : 0.f;
+            const float resc = (l_run > 0.f) ? expf(m_run - m_new) : 0.f;
+            l_run = fmaf(l_run, resc, warp_sum(p));
 #pragma unroll
-            for (int k = 0; k < KPW; ++k) {
-                const float v = __shfl_sync(0xffffffffu, s, k * LPK);
-                if (lane == jb + k && jb + k < n) my_score = v;
+            for (int e = 0; e < VPL; ++e) o_run[e] *= resc;
+            m_run = m_new;
+            // all 32 value rows are fetched at once (rows past the end repeat the last one with weight 0)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float pj = __shfl_sync(0xffffffffu, p, j);
+                float vv[VPL];
+                load_vals<ST, VPL>(Vc + (size_t)(j0 + min(j, n - 1)) * d + h * HD + lane * VPL, vv);
+#pragma unroll
+                for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(pj, vv[e], o_run[e]);
             }
         }
-        float m = my_score;
+        if (s == S - 1 && warp == NCW - 1) {
+            // the new position: rotate this step's key, round key and value to the storage type, append both to the
+            // cache and fold them in as one more key
+            const float *kraw = a.qkv + d + h * HD, *vraw = a.qkv + 2 * d + h * HD;
+            float sc = 0.f;
+            ST kst[EPL];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        const float p = (lane < n) ? expf(my_score - m) : 0.f;
-        const float l = warp_sum(p);
-        float o_acc[VPL];
+            for (int e = 0; e < EPL; ++e) {
+                const int idx = li * EPL + e;
+                const int i = idx < HD / 2 ? idx : idx - HD / 2;
+                const float2 cs = a.rope_cs[(size_t)pos * (HD / 2) + i];
+                const float ka = ldcg_f(kraw + i), kb = ldcg_f(kraw + i + HD / 2);
+                kst[e] = st_from_f32<ST>(idx < HD / 2 ? ka * cs.x - kb * cs.y : kb * cs.x + ka * cs.y);
+                sc = fmaf(qr[e], st_to_f32<ST>(kst[e]), sc);
+            }
 #pragma unroll
-        for (int e = 0; e < VPL; ++e) o_acc[e] = 0.f;
-        // all 32 value rows are fetched at once (rows past the end repeat the last one with weight 0)
+            for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+            sc = __shfl_sync(0xffffffffu, sc, 0) * scale;
+            if (sub == 0) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const float pj = __shfl_sync(0xffffffffu, p, j);
-            float vv[VPL];
-            load_vals<ST, VPL>(Vc + (size_t)(j0 + min(j, n - 1)) * d + h * HD + lane * VPL, vv);
+                for (int e = 0; e < EPL; ++e) Kc[(size_t)pos * d + h * HD + li * EPL + e] = kst[e];
+            }
+            float vn[VPL];
 #pragma unroll
-            for (int e = 0; e < VPL; ++e) o_acc[e] = fmaf(pj, vv[e], o_acc[e]);
+            for (int e = 0; e < VPL; ++e) {
+                const ST vs = st_from_f32<ST>(ldcg_f(vraw + lane * VPL + e));
+                Vc[(size_t)pos * d + h * HD + lane * VPL + e] = vs;
+                vn[e] = st_to_f32<ST>(vs);
+            }
+            const float m_new = fmaxf(m_run, sc);
+            const float resc = (l_run > 0.f) ? expf(m_run - m_new) : 0.f;
+            const float pn = expf(sc - m_new);
+            l_run = fmaf(l_run, resc, pn);
+#pragma unroll
+            for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(o_run[e], resc, pn * vn[e]);
+            m_run = m_new;
         }
-        float *part = a.att_part + ((size_t)h * a.max_blk + kb) * PSTRIDE;
+        // merge the warps of this CTA in shared memory (fixed order), one record per (h, s) to global memory
         if (lane == 0) {
-            part[0] = m;
-            part[1] = l;
+            wrec[warp * WSTRIDE] = m_run;
+            wrec[warp * WSTRIDE + 1] = l_run;
         }
 #pragma unroll
-        for (int e = 0; e < VPL; ++e) part[4 + lane * VPL + e] = o_acc[e];
-        __threadfence();
-        __syncwarp();
-        unsigned prev = 0;
-        if (lane == 0) prev = atomicAdd(a.att_tickets + h, 1u);
-        prev = __shfl_sync(0xffffffffu, prev, 0);
-        if (prev == (unsigned)nblk - 1) {
-            // last block of this head to finish: merge all blocks in a fixed order, normalise, write the head's
-            // output.  Lanes first work across blocks (maximum, weights, denominator), then each lane sums its VPL
-            // output elements over the blocks with 16 partial rows in flight at a time.
-            __threadfence();
-            const float *p0 = a.att_part + (size_t)h * a.max_blk * PSTRIDE;
+        for (int e = 0; e < VPL; ++e) wrec[warp * WSTRIDE + 2 + lane * VPL + e] = o_run[e];
+        consumer_sync();
+        if (tid < HD) {
             float M = -INFINITY;
-            for (int b = lane; b < nblk; b += 32) M = fmaxf(M, ldcg_f(p0 + (size_t)b * PSTRIDE));
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-            float Ls = 0.f, O[VPL];
+            for (int w = 0; w < NCW; ++w)
+                if (wrec[w * WSTRIDE + 1] > 0.f) M = fmaxf(M, wrec[w * WSTRIDE]);
+            float Ls = 0.f, O = 0.f;
 #pragma unroll
-            for (int e = 0; e < VPL; ++e) O[e] = 0.f;
-            for (int b0 = 0; b0 < nblk; b0 += 32) {
-                const int b = b0 + lane;
-                const float w = (b < nblk) ? expf(ldcg_f(p0 + (size_t)b * PSTRIDE) - M) : 0.f;
-                if (b < nblk) Ls = fmaf(ldcg_f(p0 + (size_t)b * PSTRIDE + 1), w, Ls);
-#pragma unroll
-                for (int kb0 = 0; kb0 < 32; kb0 += 16) {
-                    if (b0 + kb0 < nblk) {
-                        float pv[16][VPL];
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const int bb = min(b0 + kb0 + k, nblk - 1);
-                            const float *src = p0 + (size_t)bb * PSTRIDE + 4 + lane * VPL;
-                            if (VPL == 4) {
-                                const float4 t = ldcg_f4(src);
-                                pv[k][0] = t.x; pv[k][1 % VPL] = t.y; pv[k][2 % VPL] = t.z; pv[k][3 % VPL] = t.w;
-                            } else {
-                                const float2 t = __ldcg((const float2 *)src);
-                                pv[k][0] = t.x; pv[k][1 % VPL] = t.y;
-                            }
-                        }
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const float wk = __shfl_sync(0xffffffffu, w, kb0 + k);   // 0 for blocks past the end
-#pragma unroll
-                            for (int e = 0; e < VPL; ++e) O[e] = fmaf(pv[k][e], wk, O[e]);
-                        }
-                    }
+            for (int w = 0; w < NCW; ++w) {
+                const float lw = wrec[w * WSTRIDE + 1];
+                if (lw > 0.f) {
+                    const float f = expf(wrec[w * WSTRIDE] - M);
+                    Ls = fmaf(lw, f, Ls);
+                    O = fmaf(wrec[w * WSTRIDE + 2 + tid], f, O);
                 }
             }
-            Ls = warp_sum(Ls);
+            float *rec = a.att_part + ((size_t)h * ATT_MAX_PARTS + s) * PSTRIDE;
+            if (tid == 0) {
+                rec[0] = M;     // -inf for an empty part
+                rec[1] = Ls;    // 0 for an empty part
+            }
+            rec[4 + tid] = O;
+        }
+        consumer_sync();
+    }
+}
+
+// Attention output as the next projection's input: merges the S part records of each head on the fly.
+// xr[it][e] = att[(it * NCT + tid) * EPC + e].
+template <int EPC, int HD>
+__device__ __forceinline__ void load_att_merged(const ClStepArgs &a, float (&xr)[MAXIT][EPC]) {
+    constexpr int PSTRIDE = HD + 4;
+    const int nchunks = a.d / EPC, S = a.att_parts;
 #pragma unroll
-            for (int e = 0; e < VPL; ++e) a.att[h * HD + lane * VPL + e] = O[e] / Ls;
-            if (lane == 0) a.att_tickets[h] = 0u;
+    for (int it = 0; it < MAXIT; ++it) {
+        const int ch = it * NCT + threadIdx.x;
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) xr[it][e] = 0.f;
+        if (ch < nchunks) {
+            const int h = (ch * EPC) / HD, e0 = (ch * EPC) % HD;
+            const float *rec = a.att_part + (size_t)h * ATT_MAX_PARTS * PSTRIDE;
+            float2 ml[ATT_MAX_PARTS];
+            float o[ATT_MAX_PARTS][EPC];
+#pragma unroll
+            for (int s = 0; s < ATT_MAX_PARTS; ++s) {
+                const float *r = rec + (size_t)min(s, S - 1) * PSTRIDE;   // parts past S repeat the last one, weight 0
+                ml[s] = __ldcg((const float2 *)r);
+#pragma unroll
+                for (int q = 0; q < EPC / 4; ++q) {
+                    const float4 t = ldcg_f4(r + 4 + e0 + 4 * q);
+                    o[s][4 * q] = t.x; o[s][4 * q + 1] = t.y; o[s][4 * q + 2] = t.z; o[s][4 * q + 3] = t.w;
+                }
+            }
+            float M = -INFINITY;
+#pragma unroll
+            for (int s = 0; s < ATT_MAX_PARTS; ++s)
+                if (s < S && ml[s].y > 0.f) M = fmaxf(M, ml[s].x);
+            float Ls = 0.f;
+#pragma unroll
+            for (int s = 0; s < ATT_MAX_PARTS; ++s) {
+                const float f = (s < S && ml[s].y > 0.f) ? expf(ml[s].x - M) : 0.f;
+                Ls = fmaf(ml[s].y, f, Ls);
+#pragma unroll
+                for (int e = 0; e < EPC; ++e) xr[it][e] = fmaf(o[s][e], f, xr[it][e]);
+            }
+            const float inv = 1.f / Ls;
+#pragma unroll
+            for (int e = 0; e < EPC; ++e) xr[it][e] *= inv;
         }
     }
 }
@@ -633,36 +824,13 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
 
     if (tid >= NCT) {
         // ------------------------------ producer warp ------------------------------
-        if (tid == NCT) {
-            Ring rg{0u, 0u};
-            unsigned last_par[NSLOT];
-            for (int i = 0; i < NSLOT; ++i) last_par[i] = 2u;
-            for (int step = 0; step < a.n_steps; ++step) {
-                for (int ki = 0; ki < a.n_kept; ++ki) {
-                    const ClLayerDev L = a.layers[a.kept[ki]];
-                    produce_matrix<WT>(L.wqkv, 3 * d, d, 1, rg, ring, sm, st, last_par);
-                    produce_matrix<WT>(L.wo, d, d, 1, rg, ring, sm, st, last_par);
-                    produce_matrix<WT>(L.wgu, 2 * F, d, 2, rg, ring, sm, st, last_par);
-                    produce_matrix<WT>(L.wd, d, F, 1, rg, ring, sm, st, last_par);
-                }
-                produce_matrix<WT>((const char *)a.lm_head, V, d, 1, rg, ring, sm, st, last_par);
-            }
-            // Drain: every copy this thread issued must have landed before the CTA may exit.  In the normal
-            // path the consumers have already waited for all of them; after an abort this is the bounded wait
-            // for copies still in flight.
-            for (int i = 0; i < NSLOT; ++i) {
-                if (last_par[i] < 2u) {
-                    const unsigned long long t0 = gtime();
-                    while (!mbar_try(&sm->full[i], last_par[i]))
-                        if (gtime() - t0 > WAIT_NS) break;
-                }
-            }
-        }
+        if (tid == NCT) producer_loop<WT>(a, ring, sm, st);
         return;
     }
 
     // ------------------------------ consumer warps ------------------------------
     Ring rg{0u, 0u};
+    unsigned bar_target = 0u;   // arrivals that complete the next grid barrier (thread 0's copy is the one used)
     float xr[MAXIT][EPC];
     int tok = st->cyc_tok[a.row0];
     for (int step = 0; step < a.n_steps; ++step) {
@@ -672,23 +840,24 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             const WT *erow = (const WT *)a.embed + (size_t)tok * d;
             for (int i = blockIdx.x * NCT + tid; i < d; i += gridDim.x * NCT) a.x[i] = st_to_f32<WT>(erow[i]);
         }
-        grid_barrier(a.bar, sm, st);
+        grid_barrier(a.bar, bar_target, sm, st);
         for (int ki = 0; ki < a.n_kept; ++ki) {
             const ClLayerDev L = a.layers[a.kept[ki]];
-            // QKV projection of the normalised stream
+            // QKV projection of the normalised stream (the attention phase's cache lines are requested now)
+            attention_prefetch<WT, HD>(a, L, pos);
             load_x_rmsnorm<EPC>(a.x, L.n1, d, a.eps, xr, sm);
             consume_matrix<WT>(3 * d, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.qkv[rb0 + r] = row_sum(sm, r);
             });
-            grid_barrier(a.bar, sm, st);
+            grid_barrier(a.bar, bar_target, sm, st);
             attention_phase<WT, HD>(a, L, pos, sm);
-            grid_barrier(a.bar, sm, st);
+            grid_barrier(a.bar, bar_target, sm, st);
             // attention output projection + residual
-            load_x<EPC>(a.att, d, xr);
+            load_att_merged<EPC, HD>(a, xr);
             consume_matrix<WT>(d, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
             });
-            grid_barrier(a.bar, sm, st);
+            grid_barrier(a.bar, bar_target, sm, st);
             // gate/up projections (rows interleaved) + SiLU(gate) * up
             load_x_rmsnorm<EPC>(a.x, L.n2, d, a.eps, xr, sm);
             consume_matrix<WT>(2 * F, d, 2, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
@@ -697,13 +866,13 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
                     a.hff[rb0 / 2 + pr] = gt / (1.f + expf(-gt)) * up;
                 }
             });
-            grid_barrier(a.bar, sm, st);
+            grid_barrier(a.bar, bar_target, sm, st);
             // down projection + residual
             load_x<EPC>(a.hff, F, xr);
             consume_matrix<WT>(d, F, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
             });
-            grid_barrier(a.bar, sm, st);
+            grid_barrier(a.bar, bar_target, sm, st);
         }
         // LM head on the normalised stream, fused with clamp + online softmax / entropy / argmax
         load_x_rmsnorm<EPC>(a.x, a.final_norm, d, a.eps, xr, sm);
@@ -718,7 +887,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
         });
         run = hp_block_reduce(run, sm);
         if (tid == 0) a.head_part[blockIdx.x] = run;
-        grid_barrier(a.bar, sm, st);
+        grid_barrier(a.bar, bar_target, sm, st);
         // every CTA reduces the per-CTA partials itself (same order everywhere), so all know the token
         ClHeadPartial fin{0.f, 0.f, 0.f, 0x7fffffff};
         for (int b = tid; b < (int)gridDim.x; b += NCT) {
