@@ -343,8 +343,9 @@ struct SchedIter {
 };
 
 // The producer thread.  Two cursors over the same schedule: the fill cursor feeds the shared-memory ring as slots
-// come free; the prefetch cursor runs up to l2_ahead bytes in front of it and only asks L2 to fetch, so that HBM
-// keeps streaming into L2 while the consumers sit in a grid barrier or the attention phase and the ring is full.
+// come free; the prefetch cursor only asks L2 to fetch, and only moves while the ring is full (the consumers sit in a
+// grid barrier or the attention phase), up to l2_ahead bytes in front of the fill cursor, so that HBM keeps streaming
+// into L2 during those gaps and the ring is refilled from L2 afterwards.
 template <typename WT>
 __device__ void producer_loop(const ClStepArgs &a, unsigned char *ring, Smem *sm, ClDevState *st) {
     Ring rg{0u, 0u};
@@ -360,9 +361,13 @@ __device__ void producer_loop(const ClStepArgs &a, unsigned char *ring, Smem *sm
         if (ahead) {
             const char *psrc;
             unsigned pbytes;
-            while (fetched < filled + bytes + ahead && pf.next(psrc, pbytes)) {
-                if (fetched >= filled + bytes) l2_prefetch_bulk(psrc, pbytes);   // not what is about to be copied anyway
-                fetched += pbytes;
+            while (fetched < filled + bytes && pf.next(psrc, pbytes)) fetched += pbytes;   // never behind the fill cursor
+            if (!mbar_try(&sm->empty[rg.slot], rg.par ^ 1u)) {
+                // ring full: the consumers are held up, HBM would go idle; spend the time fetching into L2
+                while (fetched < filled + bytes + ahead && !mbar_try(&sm->empty[rg.slot], rg.par ^ 1u) && pf.next(psrc, pbytes)) {
+                    l2_prefetch_bulk(psrc, pbytes);
+                    fetched += pbytes;
+                }
             }
         }
         mbar_wait(&sm->empty[rg.slot], rg.par ^ 1u, sm, st);
@@ -419,31 +424,39 @@ template <> struct Log2<8> { static constexpr int v = 3; };
 // straight-line code: all of a group's 16-byte reads are issued before the first multiply-add, every row has
 // its own accumulation chain, and the R row sums are reduced across the warp together.
 // Calls epi(first_row_of_block, rows_in_block) once the partial table of a block of up to RB rows is ready.
+__device__ __forceinline__ uint4 lds128(unsigned addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
 template <typename WT, int NIT, int R, typename Epi>
 __device__ __forceinline__ void consume_rows(int r0, int r1, int nchunks, int rps, const float (&xr)[MAXIT][Chunk<WT>::EPC],
                                              Ring &rg, const unsigned char *ring, Smem *sm, ClDevState *st, Epi epi) {
-    constexpr int EPC = Chunk<WT>::EPC;
     constexpr int SH = 5 - Log2<R>::v;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const size_t rowbytes = (size_t)nchunks * 16;
+    const unsigned rowbytes = (unsigned)nchunks * 16u;
+    const unsigned ring_addr = smem_u32(ring);
+    // Byte offset of this thread's it-th chunk inside a row.  Chunks past the end of the row are redirected to the
+    // row's last chunk: its (finite) weights meet activation registers that hold zeros.
+    unsigned coff[NIT];
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) coff[it] = (unsigned)min(it * NCT + tid, nchunks - 1) * 16u;
     const int blockrows = max(1, RB / rps) * rps;
     for (int rb0 = r0; rb0 < r1; rb0 += blockrows) {
         const int nrb = min(blockrows, r1 - rb0);
         for (int sr = 0; sr < nrb; sr += rps) {
             const int ns = min(rps, nrb - sr);   // rows in this slot
             mbar_wait(&sm->full[rg.slot], rg.par, sm, st);
-            const unsigned char *base = ring + (size_t)rg.slot * SLOT_BYTES + (size_t)tid * 16;
+            const unsigned base = ring_addr + rg.slot * (unsigned)SLOT_BYTES;
             for (int g = 0; g < ns; g += R) {
                 uint4 w[R][NIT];
 #pragma unroll
                 for (int i = 0; i < R; ++i) {
                     // rows past the end of the slot re-read its last row (their sums are dropped below)
-                    const unsigned char *rowp = base + (size_t)min(g + i, ns - 1) * rowbytes;
+                    const unsigned rowp = base + (unsigned)min(g + i, ns - 1) * rowbytes;
 #pragma unroll
-                    for (int it = 0; it < NIT; ++it) {
-                        if (it * NCT + tid < nchunks) w[i][it] = *(const uint4 *)(rowp + (size_t)it * (NCT * 16));
-                        else w[i][it] = make_uint4(0u, 0u, 0u, 0u);
-                    }
+                    for (int it = 0; it < NIT; ++it) w[i][it] = lds128(rowp + coff[it]);
                 }
                 float acc[R];
 #pragma unroll
