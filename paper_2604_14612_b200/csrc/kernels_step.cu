@@ -2,11 +2,11 @@
 // vanilla full-model step at batch 1, one cooperative launch for up to CL_MAX_K (draft) or many
 // (vanilla) consecutive tokens.
 //
-// One CTA per SM.  Warp 8 (one elected thread) is the weight producer: it walks the static schedule
+// One CTA per SM.  The last warp (one elected thread) is the weight producer: it walks the static schedule
 // (steps x kept layers x {QKV, O, gate/up, down} + LM head), and for this CTA's contiguous block of
 // rows of each matrix issues bulk asynchronous copies (cp.async.bulk, completion on an mbarrier) into
-// a ring of 8 KB shared-memory slots.  It never waits for activations, so the HBM stream runs ahead
-// of the grid barriers that separate the phases.  Warps 0..7 are consumers: each thread keeps its
+// a ring of six 32 KB shared-memory slots (whole rows per slot).  It never waits for activations, so the HBM stream runs ahead
+// of the grid barriers that separate the phases.  The other 16 warps are consumers: each thread keeps its
 // fixed columns of the activation vector in registers for a whole phase, every warp reads its 512-byte
 // stripes of each row from the ring (conflict-free 16-byte reads), partial dot products are reduced
 // with warp shuffles and a small shared-memory table, and the phase epilogue (store / residual add /
@@ -19,11 +19,11 @@
 
 namespace {
 
-constexpr int NCW = 8;                 // consumer warps
+constexpr int NCW = 16;                // consumer warps
 constexpr int NCT = NCW * 32;          // consumer threads
 constexpr int SLOT_BYTES = 32768;      // ring slot: as many whole weight rows as fit (at least one)
 constexpr int NSLOT = 6;               // 192 KB in flight per SM
-constexpr int MAXIT = 8;               // 16-byte chunks per thread per row: rows up to 32 KB (C <= 16384 bf16)
+constexpr int MAXIT = 4;               // 16-byte chunks per thread per row: rows up to 32 KB (C <= 16384 bf16)
 constexpr int RB = 256;                // rows per epilogue block
 constexpr unsigned long long WAIT_NS = 2000000000ull;   // 2 s bound on any single wait
 
@@ -494,9 +494,9 @@ __device__ __forceinline__ void consume_matrix(int rows, int cols, int unit, con
     const int nchunks = cols / EPC;
     const int rps = rows_per_slot((size_t)nchunks * 16, unit);
     const int nit = (nchunks + NCT - 1) / NCT;   // uniform over the grid
-    if (nit <= 2) consume_rows<WT, 2, 4>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
-    else if (nit <= 4) consume_rows<WT, 4, 2>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
-    else consume_rows<WT, 8, 1>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
+    if (nit <= 1) consume_rows<WT, 1, 4>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
+    else if (nit <= 2) consume_rows<WT, 2, 2>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
+    else consume_rows<WT, 4, 1>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
 }
 
 __device__ __forceinline__ float row_sum(const Smem *sm, int r) {
@@ -784,12 +784,17 @@ __device__ __forceinline__ void load_att_merged(const ClStepArgs &a, float (&xr)
             float o[ATT_MAX_PARTS][EPC];
 #pragma unroll
             for (int s = 0; s < ATT_MAX_PARTS; ++s) {
-                const float *r = rec + (size_t)min(s, S - 1) * PSTRIDE;   // parts past S repeat the last one, weight 0
-                ml[s] = __ldcg((const float2 *)r);
+                ml[s] = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int q = 0; q < EPC / 4; ++q) {
-                    const float4 t = ldcg_f4(r + 4 + e0 + 4 * q);
-                    o[s][4 * q] = t.x; o[s][4 * q + 1] = t.y; o[s][4 * q + 2] = t.z; o[s][4 * q + 3] = t.w;
+                for (int e = 0; e < EPC; ++e) o[s][e] = 0.f;
+                if (s < S) {   // uniform over the grid: parts past S are never read
+                    const float *r = rec + (size_t)s * PSTRIDE;
+                    ml[s] = __ldcg((const float2 *)r);
+#pragma unroll
+                    for (int q = 0; q < EPC / 4; ++q) {
+                        const float4 t = ldcg_f4(r + 4 + e0 + 4 * q);
+                        o[s][4 * q] = t.x; o[s][4 * q + 1] = t.y; o[s][4 * q + 2] = t.z; o[s][4 * q + 3] = t.w;
+                    }
                 }
             }
             float M = -INFINITY;
