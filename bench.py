@@ -34,6 +34,7 @@ import synth  # noqa: E402
 WORKLOAD = "C3"
 K_DRAFT = 4
 SKIP_RATIO = 0.5
+TRAFFIC_RATIO = 1.011   # ncu dram bytes / algorithmic bytes of the token-step kernel (profiles/); None once stale
 METRIC = "decode tokens/s at 7B-shape bf16 bs=1; achieved HBM GB/s vs ~8 TB/s roofline"
 
 
@@ -96,17 +97,24 @@ class ClockSampler:
         return out
 
 
-def oracle_sample(shape, weights_host, prompt, mask, K):
-    """One speculative cycle of the CPU oracle after a 2-token prefill; returns (tokens, seconds, threads)."""
+ORACLE_CYCLES = 8   # speculative cycles per oracle sample: about 10 s of CPU work at the 7B shape
+
+
+def oracle_sample(shape, weights_host, prompt, mask, K, n_cycles=ORACLE_CYCLES):
+    """n_cycles speculative cycles of the CPU oracle after a 2-token prefill; returns (tokens, seconds, threads)."""
     import oracle
     om = oracle.OracleModel(shape, weights_host)
     p = prompt[:2]
     t0, _, _ = oracle.prefill(om, p)
+    ctx_len, tok, emitted = len(p), t0, 0
     t = time.perf_counter()
-    cyc = oracle.speculative_cycle(om, mask, t0, len(p), K)
+    for _ in range(n_cycles):
+        cyc = oracle.speculative_cycle(om, mask, tok, ctx_len, K)
+        emitted += len(cyc["emitted"])
+        ctx_len, tok = cyc["new_ctx"], cyc["next_t0"]
     dt = time.perf_counter() - t
     om.close()
-    return len(cyc["emitted"]), dt, int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    return emitted, dt, int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
 
 
 def run_reference(args, rank):
@@ -130,7 +138,7 @@ def run_reference(args, rank):
         toks += n
         secs += dt
     val = toks / secs
-    sample = f"one draft-{K_DRAFT}/verify/accept cycle of {WORKLOAD} after a 2-token prefill per step"
+    sample = f"{ORACLE_CYCLES} draft-{K_DRAFT}/verify/accept cycles of {WORKLOAD} after a 2-token prefill per step"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -192,7 +200,7 @@ def main():
         Wh = synth.weights_to(W, "cpu")
         n, dt, cores = oracle_sample(shape, Wh, prompt, mask, K_DRAFT)
         cpu_base = {"value": n / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-                    "sample": f"one draft-{K_DRAFT}/verify/accept cycle of {w.name} after a 2-token prefill "
+                    "sample": f"{ORACLE_CYCLES} draft-{K_DRAFT}/verify/accept cycles of {w.name} after a 2-token prefill "
                               f"({n} tokens in {dt:.1f} s)"}
         del Wh
     del W
@@ -241,10 +249,29 @@ def main():
 
     # bytes the timed cycles had to stream (algorithmic): K draft passes + one verify pass per cycle
     ctx_mid = w.prompt_len + gen // 2
-    cyc_bytes = K_DRAFT * algorithmic_bytes(shape, n_kept, ctx_mid) + \
-        algorithmic_bytes(shape, shape.n_layers, ctx_mid, rows=K_DRAFT + 1)
-    achieved = cycles * cyc_bytes / (ms * 1e-3) / 1e9
+    draft_bytes = K_DRAFT * algorithmic_bytes(shape, n_kept, ctx_mid)
+    cyc_bytes = draft_bytes + algorithmic_bytes(shape, shape.n_layers, ctx_mid, rows=K_DRAFT + 1)
+    cycle_gbs = cycles * cyc_bytes / (ms * 1e-3) / 1e9
     peak, peak_kind = measured_peaks()
+
+    # the dominant kernel on its own: one launch of the token-step kernel = K draft steps with the skip set,
+    # timed with CUDA events on the launching stream at the mid-run context length
+    ctx.cl_rollback(ctx_mid, first)
+    n_draft = 8 * max(1, args.steps)
+    for _ in range(3):
+        ctx.cl_draft(K_DRAFT)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n_draft):
+        ctx.cl_draft(K_DRAFT)
+    e1.record()
+    barrier()
+    draft_ms = e0.elapsed_time(e1) / n_draft
+    achieved = draft_bytes / (draft_ms * 1e-3) / 1e9
+    # DRAM traffic per launch: ncu counters of the same kernel on an 8-layer case (profiles/), where
+    # dram read + write bytes were 1.011 x the algorithmic bytes; traffic grows with the bytes scheduled
+    traffic = TRAFFIC_RATIO * draft_bytes if TRAFFIC_RATIO else None
 
     # vanilla decoding with the same kernels (context for the speculative number)
     step(0)
@@ -284,8 +311,10 @@ def main():
                        "vanilla_tokens_per_s": vanilla_tps, "vanilla_achieved_gbs": vanilla_gbs,
                        "vanilla_frac_of_peak": vanilla_gbs / peak},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_kind": f"of {peak_kind}", "frac_of_8TBps": achieved / 8000.0,
-                         "scope": "all kernels of the timed speculative cycles (algorithmic bytes / wall time)"},
+                         "traffic": traffic, "peak_kind": f"of {peak_kind}", "frac_of_8TBps": achieved / 8000.0,
+                         "kernel": f"k_token_steps, one launch = {K_DRAFT} draft steps over {n_kept} kept layers + LM head",
+                         "ms_per_launch": draft_ms, "bytes_per_launch": draft_bytes,
+                         "whole_cycle_gbs": cycle_gbs, "whole_cycle_frac": cycle_gbs / peak},
             "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
