@@ -46,6 +46,8 @@ struct cl_ctx {
     float *sc_conf, *sc_pmax, *sc_clayer;
     int *sc_arg;
     size_t sc_cap;                // rows*P capacity
+    char *sc_xn;                  // [sc_cap, d] bf16 normalised rows (tensor-core scoring)
+    ClHeadPartial *sc_part;       // per-(row, vocabulary range) softmax statistics
     uint8_t *sel_mask;            // device [iters_cap, L]
     double *sel_margins;          // device [L]
     float *sel_clayers;           // device [iters_cap, L]
@@ -179,7 +181,7 @@ extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **ou
 static void free_all(cl_ctx *c) {
     void *ptrs[] = {c->wbuf, c->embed, c->lm_head, c->final_norm, c->norms, c->kv, c->rope_cs, c->x, c->xn, c->qkv,
                     c->att, c->hff, c->att_part, c->logits, c->tickets, c->head_part, c->st, c->prompt_dev, c->out_dev,
-                    c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sel_mask, c->sel_margins, c->sel_clayers,
+                    c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sc_xn, c->sc_part, c->sel_mask, c->sel_margins, c->sel_clayers,
                     c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->head_part2};
     for (void *p : ptrs)
         if (p) cudaFree(p);
@@ -702,16 +704,34 @@ extern "C" int cl_rollback(cl_ctx *c, int ctx_len, int32_t pending_token) {
 
 static int ensure_score_cap(cl_ctx *c, size_t n) {
     if (n <= c->sc_cap) return CL_OK;
-    void *old[] = {c->sc_conf, c->sc_pmax, c->sc_arg};
+    void *old[] = {c->sc_conf, c->sc_pmax, c->sc_arg, c->sc_xn, c->sc_part};
     for (void *q : old)
         if (q) cudaFree(q);
     c->sc_conf = c->sc_pmax = nullptr;
     c->sc_arg = nullptr;
+    c->sc_xn = nullptr;
+    c->sc_part = nullptr;
     c->sc_cap = 0;
     DM(c->sc_conf, n * 4);
     DM(c->sc_pmax, n * 4);
     DM(c->sc_arg, n * 4);
+    if (c->cfg.weight_dtype == 1) {
+        DM(c->sc_xn, n * (size_t)c->cfg.d_model * 2);
+        DM(c->sc_part, cl_score_tc_partials((int)n, c->n_sm) * sizeof(ClHeadPartial));
+    }
     c->sc_cap = n;
+    return CL_OK;
+}
+
+// After a synchronisation: did a bounded wait of the scoring kernel expire?
+static int score_device_err(cl_ctx *c, const char *fn) {
+    int e = 0;
+    if (cudaMemcpy(&e, &c->st->err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return fail(c, CL_ECUDA, "%s: reading the device error flag failed", fn);
+    if (e) {
+        cudaMemset(&c->st->err, 0, sizeof(int));
+        return fail(c, CL_ETIMEOUT, "%s: a bounded device-side wait expired (flags %d); results of this call are invalid", fn, e);
+    }
     return CL_OK;
 }
 
@@ -720,6 +740,15 @@ static int score_rows(cl_ctx *c, const void *hidden, int rows, int P, float *c_l
     const size_t n = (size_t)rows * P, d = c->cfg.d_model;
     int rc = ensure_score_cap(c, n);
     if (rc) return rc;
+    if (c->cfg.weight_dtype == 1) {
+        // bf16 head: one dense contraction on the tensor cores with the softmax statistics fused into its epilogue
+        KL(cl_launch_rmsnorm_bf16(1, hidden, c->final_norm, (int)n, (int)d, c->cfg.rms_eps, c->sc_xn, c->stream));
+        KL(cl_launch_score_tc(c->sc_xn, c->lm_head, (int)n, c->cfg.vocab, (int)d, c->sc_part, c->n_sm, &c->st->err, c->sc_conf,
+                              c->sc_pmax, c->sc_arg, c->stream));
+        ++c->launches;
+        KL(cl_launch_mean_rows(c->sc_conf, rows, P, c_layer_dev, c->stream));
+        return CL_OK;
+    }
     for (size_t r0 = 0; r0 < n; r0 += 8) {
         const int T = (n - r0 < 8) ? (int)(n - r0) : 8;
         KL(cl_launch_rmsnorm_rows(c->cfg.weight_dtype, (const char *)hidden + r0 * d * c->esz, c->final_norm, T, (int)d,
@@ -756,6 +785,7 @@ extern "C" int cl_layer_confidences(cl_ctx *c, const void *hidden, int rows, int
     if (!rc) {
         const size_t n = (size_t)rows * P;
         cudaError_t e = cudaStreamSynchronize(c->stream);
+        if (e == cudaSuccess) rc = score_device_err(c, "cl_layer_confidences");
         if (e == cudaSuccess && conf_rows) e = cudaMemcpy(conf_rows, c->sc_conf, n * 4, cudaMemcpyDeviceToHost);
         if (e == cudaSuccess && p_max) e = cudaMemcpy(p_max, c->sc_pmax, n * 4, cudaMemcpyDeviceToHost);
         if (e == cudaSuccess && argmax) e = cudaMemcpy(argmax, c->sc_arg, n * 4, cudaMemcpyDeviceToHost);
@@ -820,6 +850,7 @@ extern "C" int cl_score_loop(cl_ctx *c, const cl_select_cfg *s, const void *cons
     std::vector<uint8_t> all((size_t)iters * L);
     CU(cudaMemcpyAsync(all.data(), c->sel_mask, all.size(), cudaMemcpyDeviceToHost, c->stream));
     CU(cudaStreamSynchronize(c->stream));
+    if ((rc = score_device_err(c, "cl_score_loop"))) return rc;
     if (c_layers_all) CU(cudaMemcpy(c_layers_all, c->sel_clayers, (size_t)iters * L * 4, cudaMemcpyDeviceToHost));
     int best = 0;   // round with the highest score; the earliest wins ties
     for (int it = 1; it < iters; ++it)

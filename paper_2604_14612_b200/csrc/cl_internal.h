@@ -119,6 +119,13 @@ cudaError_t cl_launch_tap(int wdtype, const float *x, int T, int row0, int d, vo
                           const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_accept(ClDevState *st, int K, int *out_tokens, cudaStream_t s);
 cudaError_t cl_launch_advance(ClDevState *st, int n, int set_pending_from_tgt, cudaStream_t s);
+// tensor-core scoring (bf16 LM head): normalise to bf16, contraction fused with the softmax statistics, finalize
+int cl_score_tc_ranges(int R, int n_sm);
+size_t cl_score_tc_partials(int R, int n_sm);
+cudaError_t cl_launch_rmsnorm_bf16(int in_dtype, const void *x, const float *g, int rows, int d, float eps, void *out,
+                                   cudaStream_t s);
+cudaError_t cl_launch_score_tc(const void *xn, const void *lm_head, int R, int V, int d, ClHeadPartial *partials, int n_sm,
+                               int *err, float *conf, float *pmax, int *arg, cudaStream_t s);
 cudaError_t cl_launch_mean_rows(const float *conf_rows, int rows, int P, float *c_layer, cudaStream_t s);
 cudaError_t cl_launch_select(const cl_select_cfg &cfg, int n_layers, const float *c_layer, uint8_t *mask, double *margins,
                              cudaStream_t s);

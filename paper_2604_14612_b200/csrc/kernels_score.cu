@@ -1,0 +1,400 @@
+// All-layer early-exit confidence scoring as one dense contraction on the 5th-generation tensor cores
+// (Section 3.1, Eq. 1-4): logits[r, v] = sum_k xn[r, k] * W_lm[v, k] for every tapped hidden row r, fused with
+// the clamp and an online softmax / entropy / top-1 / argmax reduction per row.  Logits never leave the SM.
+//
+// One persistent CTA per SM, 192 threads:
+//   warp 0   TMA producer: 128 x 64 tiles of the normalised hidden rows (A) and 256 x 64 tiles of the LM head (B),
+//            128-byte swizzled, into a 4-stage shared-memory ring (48 KB per stage), completion on mbarriers;
+//   warp 1   allocates tensor memory and issues tcgen05.mma (M 128, N 256, K 16, bf16 -> fp32) from one thread;
+//            the 128 x 256 fp32 accumulator lives in tensor memory, two of them (512 columns) so that the
+//            epilogue of one vocabulary tile overlaps the multiply-adds of the next;
+//   warps 2-5 epilogue: thread = one hidden row (one tensor-memory lane); it reads its row of the accumulator
+//            32 columns at a time (tcgen05.ld) and keeps running softmax statistics relative to the running
+//            maximum m: z = sum e^(l-m), s = sum (l-m) e^(l-m), and the argmax (lowest index on ties).
+// A CTA owns one block of 128 hidden rows and a contiguous range of vocabulary tiles; CTAs that share the
+// vocabulary range run side by side, so a tile of the LM head is fetched from HBM once and served to the other
+// row blocks from L2.  Per-(row, vocabulary range) statistics are merged in a fixed order by a second kernel,
+// which also evaluates H = log Z - S/Z, the confidence 1 - H / log V (Eq. 3-4) and the top-1 probability 1/Z.
+// Every wait is bounded in time; on expiry an error flag is raised and the kernel winds down.
+#include <cuda.h>
+#include <math.h>
+
+#include "cl_internal.h"
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int NTHREADS = 192;
+constexpr unsigned long long WAIT_NS = 2000000000ull;
+
+struct ScoreSmem {
+    unsigned long long full[STAGES], empty[STAGES], tfull[2], tempty[2];
+    unsigned tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ unsigned s_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long gtime_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void bar_init(unsigned long long *b, unsigned n) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(b)), "r"(n));
+}
+__device__ __forceinline__ void bar_arrive(unsigned long long *b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(b)) : "memory");
+}
+__device__ __forceinline__ void bar_expect(unsigned long long *b, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool bar_try(unsigned long long *b, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(s_u32(b)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; false (and the abort flags raised) if it gave up.
+__device__ __forceinline__ bool bar_wait(unsigned long long *b, unsigned parity, ScoreSmem *sm, int *err) {
+    if (bar_try(b, parity)) return true;
+    const unsigned long long t0 = gtime_ns();
+    for (unsigned i = 1;; ++i) {
+        if (bar_try(b, parity)) return true;
+        if ((i & 63u) == 0u) {
+            if (*(volatile int *)&sm->abort) return false;
+            if (gtime_ns() - t0 > WAIT_NS) {
+                *(volatile int *)&sm->abort = 1;
+                atomicOr(err, 4);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, unsigned long long *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+            s_u32(dst)),
+        "l"(map), "r"(s_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile written by TMA with the 128-byte swizzle: rows of 128
+// bytes, groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1, layout type 2 (128B swizzle).
+__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
+    unsigned long long d = 0;
+    d |= (unsigned long long)((smem_addr & 0x3ffffu) >> 4);   // start address
+    d |= (unsigned long long)1 << 16;                          // leading byte offset (unused with swizzle)
+    d |= (unsigned long long)(1024 >> 4) << 32;                // stride byte offset
+    d |= (unsigned long long)1 << 46;                          // version
+    d |= (unsigned long long)2 << 61;                          // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, both K-major, N and M of the tile.
+__device__ __forceinline__ unsigned umma_idesc(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(unsigned tmem_d, unsigned long long adesc, unsigned long long bdesc, unsigned idesc,
+                                          unsigned accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned long long *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, float (&v)[32]) {
+    unsigned r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+struct ScoreArgs {
+    int R, V, KB, MT, NCG, NT;      // hidden rows, vocabulary, K blocks of 64, row blocks, vocabulary ranges, vocabulary tiles
+    ClHeadPartial *partials;        // [MT * BM, NCG]
+    int *err;
+};
+
+__device__ __forceinline__ ClHeadPartial sc_merge(const ClHeadPartial &a, const ClHeadPartial &b) {
+    if (b.z == 0.f) return a;
+    if (a.z == 0.f) return b;
+    ClHeadPartial r;
+    r.m = fmaxf(a.m, b.m);
+    const float ea = expf(a.m - r.m), eb = expf(b.m - r.m);
+    r.z = a.z * ea + b.z * eb;
+    r.s = ea * (a.s + (a.m - r.m) * a.z) + eb * (b.s + (b.m - r.m) * b.z);
+    r.idx = (a.m > b.m) ? a.idx : (b.m > a.m) ? b.idx : min(a.idx, b.idx);
+    return r;
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_score(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, ScoreArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *tiles = (unsigned char *)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);   // swizzled tiles: 1 KB aligned
+    ScoreSmem *sm = (ScoreSmem *)(tiles + (size_t)STAGES * STAGE_BYTES);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x;
+    if (cta >= a.MT * a.NCG) return;   // whole CTA leaves before anything is set up
+    const int mt = cta % a.MT, cg = cta / a.MT;
+    const int nt0 = (int)((long long)a.NT * cg / a.NCG), nt1 = (int)((long long)a.NT * (cg + 1) / a.NCG);
+    const int ntiles = nt1 - nt0;
+
+    if (tid == 0) {
+        for (int i = 0; i < STAGES; ++i) {
+            bar_init(&sm->full[i], 1);
+            bar_init(&sm->empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            bar_init(&sm->tfull[i], 1);
+            bar_init(&sm->tempty[i], 128);
+        }
+        sm->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(s_u32(&sm->tmem_base)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem = *(volatile unsigned *)&sm->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            unsigned stage = 0, par = 0, issued[STAGES];
+            for (int i = 0; i < STAGES; ++i) issued[i] = 2u;
+            bool ok = true;
+            for (int t = 0; t < ntiles && ok; ++t) {
+                for (int kb = 0; kb < a.KB; ++kb) {
+                    if (!bar_wait(&sm->empty[stage], par ^ 1u, sm, a.err)) { ok = false; break; }
+                    unsigned char *dst = tiles + (size_t)stage * STAGE_BYTES;
+                    bar_expect(&sm->full[stage], STAGE_BYTES);
+                    tma_load_2d(dst, &mapA, kb * BK, mt * BM, &sm->full[stage]);
+                    tma_load_2d(dst + A_BYTES, &mapB, kb * BK, (nt0 + t) * BN, &sm->full[stage]);
+                    issued[stage] = par;
+                    if (++stage == STAGES) { stage = 0; par ^= 1u; }
+                }
+            }
+            if (!ok) {   // gave up: still let the copies in flight land before the CTA may exit (bounded)
+                for (int i = 0; i < STAGES; ++i) {
+                    if (issued[i] < 2u) {
+                        const unsigned long long t0 = gtime_ns();
+                        while (!bar_try(&sm->full[i], issued[i]))
+                            if (gtime_ns() - t0 > WAIT_NS) break;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const unsigned idesc = umma_idesc(BM, BN);
+            unsigned stage = 0, par = 0;
+            bool ok = true;
+            for (int t = 0; t < ntiles && ok; ++t) {
+                const int b = t & 1;
+                if (!bar_wait(&sm->tempty[b], (((unsigned)t >> 1) & 1u) ^ 1u, sm, a.err)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int kb = 0; kb < a.KB; ++kb) {
+                    if (!bar_wait(&sm->full[stage], par, sm, a.err)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const unsigned a_addr = s_u32(tiles + (size_t)stage * STAGE_BYTES), b_addr = a_addr + A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_bf16(tmem + (unsigned)b * BN, umma_desc(a_addr + k * 32), umma_desc(b_addr + k * 32), idesc,
+                                  (unsigned)(kb | k));
+                    umma_commit(&sm->empty[stage]);   // the stage is free once these multiply-adds have read it
+                    if (++stage == STAGES) { stage = 0; par ^= 1u; }
+                }
+                if (ok) umma_commit(&sm->tfull[b]);   // accumulator b is complete
+            }
+        }
+    } else {
+        // ---------------- epilogue: one thread per hidden row ----------------
+        const int q = warp & 3;                        // the tensor-memory lane quadrant this warp may read
+        const int row = q * 32 + lane;
+        ClHeadPartial run{0.f, 0.f, 0.f, 0x7fffffff};
+        for (int t = 0; t < ntiles; ++t) {
+            const int b = t & 1;
+            if (!bar_wait(&sm->tfull[b], ((unsigned)t >> 1) & 1u, sm, a.err)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int n0 = (nt0 + t) * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                float v[32];
+                tmem_ld32(tmem + ((unsigned)(q * 32) << 16) + (unsigned)(b * BN + c * 32), v);
+                const int col0 = n0 + c * 32;
+                const int nvalid = min(32, a.V - col0);   // uniform over the warp
+                if (nvalid <= 0) continue;
+                float cm = -INFINITY;
+                int ci = 0;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    if (i < nvalid) {
+                        const float l = fminf(fmaxf(v[i], -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);   // clamp of Section 3.1
+                        v[i] = l;
+                        if (l > cm) { cm = l; ci = col0 + i; }
+                    }
+                }
+                float m_new = cm;
+                if (run.z > 0.f) {
+                    m_new = fmaxf(run.m, cm);
+                    const float e = expf(run.m - m_new);
+                    run.s = e * (run.s + (run.m - m_new) * run.z);
+                    run.z *= e;
+                    if (cm > run.m) run.idx = ci;   // strictly larger only: the lowest index wins ties
+                } else {
+                    run.idx = ci;
+                }
+                run.m = m_new;
+                float z = 0.f, s = 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    if (i < nvalid) {
+                        const float d = v[i] - m_new;
+                        const float e = expf(d);
+                        z += e;
+                        s = fmaf(d, e, s);
+                    }
+                }
+                run.z += z;
+                run.s += s;
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            bar_arrive(&sm->tempty[b]);
+        }
+        a.partials[(size_t)(mt * BM + row) * a.NCG + cg] = run;
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+// Merge the per-range statistics of every row in a fixed order and evaluate Eq. 2-4.
+__global__ void k_score_finalize(const ClHeadPartial *partials, int NCG, int R, float inv_log_v, float *conf, float *pmax,
+                                 int *arg) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= R) return;
+    ClHeadPartial f{0.f, 0.f, 0.f, 0x7fffffff};
+    for (int g = 0; g < NCG; ++g) f = sc_merge(f, partials[(size_t)r * NCG + g]);
+    const float H = logf(f.z) - f.s / f.z;   // entropy of the softmax from sums relative to the maximum
+    conf[r] = 1.f - H * inv_log_v;
+    pmax[r] = 1.f / f.z;
+    arg[r] = f.idx;
+}
+
+// Final RMSNorm of hidden rows in the storage type -> bf16 rows (the A operand of the contraction).
+template <typename ST>
+__global__ void k_rmsnorm_to_bf16(const ST *x, const float *g, int d, float eps, __nv_bfloat16 *out) {
+    __shared__ float red[32];
+    const ST *xr = x + (size_t)blockIdx.x * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = (float)xr[i];
+        ss = fmaf(v, v, ss);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];   // fixed order
+    const float sc = 1.0f / sqrtf(tot / (float)d + eps);
+    for (int i = threadIdx.x; i < d; i += blockDim.x)
+        out[(size_t)blockIdx.x * d + i] = __float2bfloat16_rn((float)xr[i] * sc * g[i]);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major [rows, cols] tensor, box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap *m, const void *base, int rows, int cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int cl_score_tc_ranges(int R, int n_sm) {
+    const int MT = (R + BM - 1) / BM;
+    int ncg = n_sm / MT;
+    return ncg < 1 ? 1 : ncg;
+}
+
+size_t cl_score_tc_partials(int R, int n_sm) {
+    const int MT = (R + BM - 1) / BM;
+    return (size_t)MT * BM * cl_score_tc_ranges(R, n_sm);
+}
+
+cudaError_t cl_launch_rmsnorm_bf16(int in_dtype, const void *x, const float *g, int rows, int d, float eps, void *out,
+                                   cudaStream_t s) {
+    if (in_dtype == 1)
+        k_rmsnorm_to_bf16<__nv_bfloat16><<<rows, 256, 0, s>>>((const __nv_bfloat16 *)x, g, d, eps, (__nv_bfloat16 *)out);
+    else
+        k_rmsnorm_to_bf16<float><<<rows, 256, 0, s>>>((const float *)x, g, d, eps, (__nv_bfloat16 *)out);
+    return cudaGetLastError();
+}
+
+// xn: [R, d] bf16 normalised rows; lm_head: [V, d] bf16.  Needs d % 8 == 0 and 16-byte aligned bases.
+cudaError_t cl_launch_score_tc(const void *xn, const void *lm_head, int R, int V, int d, ClHeadPartial *partials, int n_sm,
+                               int *err, float *conf, float *pmax, int *arg, cudaStream_t s) {
+    CUtensorMap mapA, mapB;
+    if (!make_map(&mapA, xn, R, d, BM) || !make_map(&mapB, lm_head, V, d, BN)) return cudaErrorInvalidValue;
+    ScoreArgs a;
+    a.R = R; a.V = V; a.KB = (d + BK - 1) / BK;
+    a.MT = (R + BM - 1) / BM;
+    a.NCG = cl_score_tc_ranges(R, n_sm);
+    a.NT = (V + BN - 1) / BN;
+    if (a.NCG > a.NT) a.NCG = a.NT;
+    a.partials = partials; a.err = err;
+    const size_t smem = (size_t)STAGES * STAGE_BYTES + sizeof(ScoreSmem) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(k_score, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    // row blocks beyond n_sm CTAs are handled in waves of whole column ranges
+    k_score<<<a.MT * a.NCG, NTHREADS, smem, s>>>(mapA, mapB, a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    k_score_finalize<<<(R + 127) / 128, 128, 0, s>>>(partials, a.NCG, R, (float)(1.0 / log((double)V)), conf, pmax, arg);
+    return cudaGetLastError();
+}
