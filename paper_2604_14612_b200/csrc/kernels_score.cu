@@ -16,114 +16,20 @@
 // row blocks from L2.  Per-(row, vocabulary range) statistics are merged in a fixed order by a second kernel,
 // which also evaluates H = log Z - S/Z, the confidence 1 - H / log V (Eq. 3-4) and the top-1 probability 1/Z.
 // Every wait is bounded in time; on expiry an error flag is raised and the kernel winds down.
-#include <cuda.h>
 #include <math.h>
 
-#include "cl_internal.h"
+#include "tc_common.cuh"
 
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NTHREADS = 192;
-constexpr unsigned long long WAIT_NS = 2000000000ull;
-
 struct ScoreSmem {
     unsigned long long full[STAGES], empty[STAGES], tfull[2], tempty[2];
     unsigned tmem_base;
     int abort;
 };
-
-__device__ __forceinline__ unsigned s_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long gtime_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void bar_init(unsigned long long *b, unsigned n) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(b)), "r"(n));
-}
-__device__ __forceinline__ void bar_arrive(unsigned long long *b) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(b)) : "memory");
-}
-__device__ __forceinline__ void bar_expect(unsigned long long *b, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_u32(b)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool bar_try(unsigned long long *b, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(s_u32(b)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait; false (and the abort flags raised) if it gave up.
-__device__ __forceinline__ bool bar_wait(unsigned long long *b, unsigned parity, ScoreSmem *sm, int *err) {
-    if (bar_try(b, parity)) return true;
-    const unsigned long long t0 = gtime_ns();
-    for (unsigned i = 1;; ++i) {
-        if (bar_try(b, parity)) return true;
-        if ((i & 63u) == 0u) {
-            if (*(volatile int *)&sm->abort) return false;
-            if (gtime_ns() - t0 > WAIT_NS) {
-                *(volatile int *)&sm->abort = 1;
-                atomicOr(err, 4);
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, unsigned long long *bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
-            s_u32(dst)),
-        "l"(map), "r"(s_u32(bar)), "r"(c0), "r"(c1)
-        : "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major bf16 tile written by TMA with the 128-byte swizzle: rows of 128
-// bytes, groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1, layout type 2 (128B swizzle).
-__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
-    unsigned long long d = 0;
-    d |= (unsigned long long)((smem_addr & 0x3ffffu) >> 4);   // start address
-    d |= (unsigned long long)1 << 16;                          // leading byte offset (unused with swizzle)
-    d |= (unsigned long long)(1024 >> 4) << 32;                // stride byte offset
-    d |= (unsigned long long)1 << 46;                          // version
-    d |= (unsigned long long)2 << 61;                          // 128-byte swizzle
-    return d;
-}
-// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, both K-major, N and M of the tile.
-__device__ __forceinline__ unsigned umma_idesc(int m, int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(m >> 4) << 24);
-}
-__device__ __forceinline__ void umma_bf16(unsigned tmem_d, unsigned long long adesc, unsigned long long bdesc, unsigned idesc,
-                                          unsigned accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(unsigned long long *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(unsigned taddr, float (&v)[32]) {
-    unsigned r[32];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
 
 struct ScoreArgs {
     int R, V, KB, MT, NCG, NT;      // hidden rows, vocabulary, K blocks of 64, row blocks, vocabulary ranges, vocabulary tiles
@@ -184,7 +90,7 @@ k_score(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtens
             bool ok = true;
             for (int t = 0; t < ntiles && ok; ++t) {
                 for (int kb = 0; kb < a.KB; ++kb) {
-                    if (!bar_wait(&sm->empty[stage], par ^ 1u, sm, a.err)) { ok = false; break; }
+                    if (!bar_wait(&sm->empty[stage], par ^ 1u, &sm->abort, a.err)) { ok = false; break; }
                     unsigned char *dst = tiles + (size_t)stage * STAGE_BYTES;
                     bar_expect(&sm->full[stage], STAGE_BYTES);
                     tma_load_2d(dst, &mapA, kb * BK, mt * BM, &sm->full[stage]);
@@ -211,10 +117,10 @@ k_score(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtens
             bool ok = true;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int b = t & 1;
-                if (!bar_wait(&sm->tempty[b], (((unsigned)t >> 1) & 1u) ^ 1u, sm, a.err)) break;
+                if (!bar_wait(&sm->tempty[b], (((unsigned)t >> 1) & 1u) ^ 1u, &sm->abort, a.err)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 for (int kb = 0; kb < a.KB; ++kb) {
-                    if (!bar_wait(&sm->full[stage], par, sm, a.err)) { ok = false; break; }
+                    if (!bar_wait(&sm->full[stage], par, &sm->abort, a.err)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const unsigned a_addr = s_u32(tiles + (size_t)stage * STAGE_BYTES), b_addr = a_addr + A_BYTES;
 #pragma unroll
@@ -234,7 +140,7 @@ k_score(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtens
         ClHeadPartial run{0.f, 0.f, 0.f, 0x7fffffff};
         for (int t = 0; t < ntiles; ++t) {
             const int b = t & 1;
-            if (!bar_wait(&sm->tfull[b], ((unsigned)t >> 1) & 1u, sm, a.err)) break;
+            if (!bar_wait(&sm->tfull[b], ((unsigned)t >> 1) & 1u, &sm->abort, a.err)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int n0 = (nt0 + t) * BN;
 #pragma unroll 1
@@ -324,34 +230,6 @@ __global__ void k_rmsnorm_to_bf16(const ST *x, const float *g, int d, float eps,
     const float sc = 1.0f / sqrtf(tot / (float)d + eps);
     for (int i = threadIdx.x; i < d; i += blockDim.x)
         out[(size_t)blockIdx.x * d + i] = __float2bfloat16_rn((float)xr[i] * sc * g[i]);
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
-
-// 2-D bf16 row-major [rows, cols] tensor, box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
-bool make_map(CUtensorMap *m, const void *base, int rows, int cols, int box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace

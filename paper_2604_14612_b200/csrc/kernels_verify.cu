@@ -1,0 +1,416 @@
+// Skinny tensor-core GEMM for passes of T <= 9 token rows through the bf16 model: the (K+1)-row verify pass of
+// Section 3 (and the prefill, which is the same pass over chunks of the prompt).
+//
+//   acc[r, t] = sum_k W[r, k] * b[t, k]        W: [rows, K] bf16 weights, b: T activation rows
+//
+// "Swap-AB": the weight rows are the M = 128 operand of tcgen05.mma (they fill the tensor-memory lanes), the token
+// rows are N.  Activations are fp32 everywhere else; here each row enters twice, as hi = bf16(v) and
+// lo = bf16(v - hi), in N = 16 (T <= 8) or 32 columns, and the two accumulator columns are added in the epilogue,
+// so the product keeps about 16 mantissa bits of the activation while the weights stream exactly once.
+// The pass is bound by HBM weight streaming, so the work is cut for equal bytes per SM ("stream-K"): the units
+// (128-row tile, 64-column K block) are numbered tile-major and CTA c takes the contiguous range
+// [U c / G, U (c+1) / G).  A CTA that holds only part of a tile's K range writes its 128 x N partial
+// accumulator to a workspace and takes a ticket; the last one to arrive for a tile adds the partials in CTA
+// order (fixed, so results do not depend on timing) and runs the epilogue for that tile:
+//   STORE  qkv[t, r] = s_t * acc                     (s_t = RMSNorm scale of token t, see below)
+//   RESID  x[t, r] += acc; next input hi/lo(x * g_next[r]); per-tile sum of x^2 per token; optional hidden tap
+//   SILU   rows interleave gate/up: h = silu(s_t g) * (s_t u) -> hi/lo(h), the down projection's input
+//   HEAD   logits = clamp(s_t * acc) -> per-tile softmax statistics and argmax per token (Eq. 1-4)
+// RMSNorm is split around the GEMM: the input rows hold x * gain (unscaled), the producer of x leaves per-tile
+// sums of squares, and s_t = rsqrt(mean x^2 + eps) multiplies the accumulator in the epilogue (a per-token
+// scalar commutes with the contraction).
+// Warp roles as in the scoring kernel: warp 0 TMA producer (A 128 x 64 and B N x 64 tiles, 128-byte swizzle,
+// 8-stage ring), warp 1 tensor-memory allocation and MMA issue, warps 2-5 epilogue (thread = weight row).
+// All waits are bounded; nothing waits on another CTA (the ticket is taken, never polled).
+#include <math.h>
+
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int VM = 128, VSTAGES = 8;
+constexpr int VA_BYTES = VM * TC_BK * 2, VB_BYTES = 32 * TC_BK * 2, VSTAGE_BYTES = VA_BYTES + VB_BYTES;   // 20 KB
+constexpr int VTHREADS = 192;
+constexpr int WS_LD = 32;   // floats per row of a workspace partial
+
+struct VSmem {
+    unsigned long long full[VSTAGES], empty[VSTAGES], tfull[2], tempty[2];
+    unsigned tmem_base;
+    int abort, is_last;
+    float scale[CL_SLOTS];
+    float red[4][CL_SLOTS];
+    ClHeadPartial hp[4][CL_SLOTS];
+};
+
+struct Seg {
+    int m, kb0, kb1;
+};
+
+// CTA c's unit range and its idx-th segment (a maximal run of units inside one tile); false past the end.
+__device__ __forceinline__ bool segment_of(long long U, int G, int KB, int c, int idx, Seg &s) {
+    if (c >= G) return false;
+    long long u = U * c / G;
+    const long long u1 = U * (c + 1) / G;
+    for (int i = 0; u < u1; ++i) {
+        const int m = (int)(u / KB), kb0 = (int)(u % KB);
+        const int kb1 = (int)min((long long)KB, kb0 + (u1 - u));
+        if (i == idx) {
+            s.m = m; s.kb0 = kb0; s.kb1 = kb1;
+            return true;
+        }
+        u += kb1 - kb0;
+    }
+    return false;
+}
+__device__ __forceinline__ int cta_of_unit(long long U, int G, long long u) {
+    int c = (int)(u * G / U);
+    while (c + 1 < G && U * (c + 1) / G <= u) ++c;
+    while (c > 0 && U * c / G > u) --c;
+    return c;
+}
+
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier of the 128 epilogue threads that also tells every one of them whether all of them saw ok.
+__device__ __forceinline__ bool epi_all(bool ok) {
+    int r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.s32 p, %1, 0;\n\tbar.red.and.pred q, 1, 128, p;\n\tselp.s32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((int)ok)
+        : "memory");
+    return r != 0;
+}
+
+__device__ __forceinline__ ClHeadPartial v_merge(const ClHeadPartial &a, const ClHeadPartial &b) {
+    if (b.z == 0.f) return a;
+    if (a.z == 0.f) return b;
+    ClHeadPartial r;
+    r.m = fmaxf(a.m, b.m);
+    const float ea = expf(a.m - r.m), eb = expf(b.m - r.m);
+    r.z = a.z * ea + b.z * eb;
+    r.s = ea * (a.s + (a.m - r.m) * a.z) + eb * (b.s + (b.m - r.m) * b.z);
+    r.idx = (a.m > b.m) ? a.idx : (b.m > a.m) ? b.idx : min(a.idx, b.idx);
+    return r;
+}
+__device__ __forceinline__ ClHeadPartial v_shfl_xor(const ClHeadPartial &a, int o) {
+    ClHeadPartial r;
+    r.m = __shfl_xor_sync(0xffffffffu, a.m, o);
+    r.z = __shfl_xor_sync(0xffffffffu, a.z, o);
+    r.s = __shfl_xor_sync(0xffffffffu, a.s, o);
+    r.idx = __shfl_xor_sync(0xffffffffu, a.idx, o);
+    return r;
+}
+
+// v -> (hi, lo) bf16 with hi + lo = v to about 16 mantissa bits
+__device__ __forceinline__ void split_bf16(float v, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+    hi = __float2bfloat16_rn(v);
+    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+__global__ void __launch_bounds__(VTHREADS, 1)
+k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, ClSkinnyArgs a) {
+    if (a.st && a.st->done) return;   // written only between launches: uniform over the grid
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *tiles = (unsigned char *)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+    VSmem *sm = (VSmem *)(tiles + (size_t)VSTAGES * VSTAGE_BYTES);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int MT = (a.rows + VM - 1) / VM;
+    const long long U = (long long)MT * a.KB;
+    // the split runs over min(grid, U) CTAs so that every CTA of the split owns at least one unit (a tile's
+    // partials then come from a gap-free range of CTAs); CTAs beyond it have no segment
+    const int c = blockIdx.x, G = (int)min((long long)gridDim.x, U);
+    const unsigned b_bytes = (unsigned)a.N * TC_BK * 2;
+
+    if (tid == 0) {
+        for (int i = 0; i < VSTAGES; ++i) {
+            bar_init(&sm->full[i], 1);
+            bar_init(&sm->empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            bar_init(&sm->tfull[i], 1);
+            bar_init(&sm->tempty[i], 128);
+        }
+        sm->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 64;" ::"r"(s_u32(&sm->tmem_base)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem = *(volatile unsigned *)&sm->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            unsigned stage = 0, par = 0, issued[VSTAGES];
+            for (int i = 0; i < VSTAGES; ++i) issued[i] = 2u;
+            bool ok = true;
+            Seg sg;
+            for (int si = 0; ok && segment_of(U, G, a.KB, c, si, sg); ++si) {
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+                    if (!bar_wait(&sm->empty[stage], par ^ 1u, &sm->abort, a.err)) { ok = false; break; }
+                    unsigned char *dst = tiles + (size_t)stage * VSTAGE_BYTES;
+                    bar_expect(&sm->full[stage], VA_BYTES + b_bytes);
+                    tma_load_2d(dst, &mapA, kb * TC_BK, sg.m * VM, &sm->full[stage]);
+                    tma_load_2d(dst + VA_BYTES, &mapB, kb * TC_BK, 0, &sm->full[stage]);
+                    issued[stage] = par;
+                    if (++stage == VSTAGES) { stage = 0; par ^= 1u; }
+                }
+            }
+            if (!ok) {   // gave up: let the copies in flight land before the CTA may exit (bounded)
+                for (int i = 0; i < VSTAGES; ++i) {
+                    if (issued[i] < 2u) {
+                        const unsigned long long t0 = gtime_ns();
+                        while (!bar_try(&sm->full[i], issued[i]))
+                            if (gtime_ns() - t0 > WAIT_NS) break;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const unsigned idesc = umma_idesc(VM, a.N);
+            unsigned stage = 0, par = 0;
+            bool ok = true;
+            Seg sg;
+            for (int si = 0; ok && segment_of(U, G, a.KB, c, si, sg); ++si) {
+                const int b = si & 1;
+                if (!bar_wait(&sm->tempty[b], (((unsigned)si >> 1) & 1u) ^ 1u, &sm->abort, a.err)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+                    if (!bar_wait(&sm->full[stage], par, &sm->abort, a.err)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const unsigned a_addr = s_u32(tiles + (size_t)stage * VSTAGE_BYTES), b_addr = a_addr + VA_BYTES;
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k)
+                        umma_bf16(tmem + (unsigned)b * 32, umma_desc(a_addr + k * 32), umma_desc(b_addr + k * 32), idesc,
+                                  (unsigned)((kb - sg.kb0) | k));
+                    umma_commit(&sm->empty[stage]);
+                    if (++stage == VSTAGES) { stage = 0; par ^= 1u; }
+                }
+                if (ok) umma_commit(&sm->tfull[b]);
+            }
+        }
+    } else {
+        // ---------------- epilogue: thread = one weight row of the tile ----------------
+        const int et = tid - 64;                       // 0 .. 127
+        const int q = warp & 3, rloc = q * 32 + lane;  // tensor-memory lane = row inside the tile
+        const int ew = et >> 5;                        // epilogue warp 0 .. 3 (for shared tables)
+        const int T = a.T, nh = a.N >> 1;
+        // RMSNorm scale of every token row: fixed-order sum of the producer's per-tile sums of squares
+        if (et < T) {
+            float sc = 1.f;
+            if (a.ssq_in) {
+                float ss = 0.f;
+                for (int m = 0; m < a.ssq_tiles; ++m) ss += __ldcg(a.ssq_in + (size_t)m * CL_SLOTS + et);
+                sc = 1.0f / sqrtf(ss * a.inv_dim + a.eps);
+            }
+            sm->scale[et] = sc;
+        }
+        epi_sync();
+        const int pos0 = a.st ? a.st->ctx + a.row0 : a.row0;
+        Seg sg;
+        for (int si = 0; segment_of(U, G, a.KB, c, si, sg); ++si) {
+            const int b = si & 1;
+            if (!epi_all(bar_wait(&sm->tfull[b], ((unsigned)si >> 1) & 1u, &sm->abort, a.err))) break;   // uniform
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float v[32];
+            tmem_ld32(tmem + ((unsigned)(q * 32) << 16) + (unsigned)(b * 32), v);
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            bar_arrive(&sm->tempty[b]);   // the accumulator is in registers: the buffer may be reused
+            const int m = sg.m, row = m * VM + rloc;
+            if (!(sg.kb0 == 0 && sg.kb1 == a.KB)) {
+                // partial K range: publish, take a ticket; the last arrival adds all partials in CTA order
+                float4 *dst = (float4 *)(a.ws + (((size_t)c * CL_V_MAXSEG + si) * VM + rloc) * WS_LD);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (4 * i < a.N) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                __threadfence();
+                epi_sync();
+                const int c_first = cta_of_unit(U, G, (long long)m * a.KB), c_last = cta_of_unit(U, G, (long long)(m + 1) * a.KB - 1);
+                if (et == 0) {
+                    const unsigned prev = atomicAdd(a.tickets + m, 1u);
+                    const int last = (prev == (unsigned)(c_last - c_first));
+                    if (last) a.tickets[m] = 0u;
+                    sm->is_last = last;
+                }
+                epi_sync();
+                if (!sm->is_last) continue;
+                __threadfence();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = 0.f;
+                for (int cc = c_first; cc <= c_last; ++cc) {
+                    const int seg_idx = m - (int)((U * cc / G) / a.KB);   // tiles CTA cc touches are consecutive
+                    const float4 *src = (const float4 *)(a.ws + (((size_t)cc * CL_V_MAXSEG + seg_idx) * VM + rloc) * WS_LD);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (4 * i < a.N) {
+                            const float4 p = __ldcg(src + i);
+                            v[4 * i] += p.x; v[4 * i + 1] += p.y; v[4 * i + 2] += p.z; v[4 * i + 3] += p.w;
+                        }
+                    }
+                }
+            }
+            // ---- epilogue of a complete tile: tot[t] = hi column + lo column
+            const bool live = row < a.rows;
+            if (a.epi == CL_VEPI_STORE) {
+                if (live)
+                    for (int t = 0; t < T; ++t) a.out[(size_t)t * a.ld + row] = sm->scale[t] * (v[t] + v[nh + t]);
+            } else if (a.epi == CL_VEPI_RESID) {
+                const float g = live ? a.gnext[row] : 0.f;
+                for (int t = 0; t < T; ++t) {
+                    float xn = 0.f;
+                    if (live) {
+                        xn = a.out[(size_t)t * a.ld + row] + (v[t] + v[nh + t]);
+                        a.out[(size_t)t * a.ld + row] = xn;
+                        __nv_bfloat16 hi, lo;
+                        split_bf16(xn * g, hi, lo);
+                        a.bnext[(size_t)t * a.bn_ld + row] = hi;
+                        a.bnext[(size_t)(a.nh + t) * a.bn_ld + row] = lo;
+                        if (a.tap) {
+                            const size_t o = (size_t)((pos0 + t) % a.tap_P) * a.rows + row;
+                            ((__nv_bfloat16 *)a.tap)[o] = __float2bfloat16_rn(xn);
+                        }
+                    }
+                    float ss = xn * xn;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                    if (lane == 0) sm->red[ew][t] = ss;
+                }
+                epi_sync();
+                if (et < T) a.ssq_out[(size_t)m * CL_SLOTS + et] = (sm->red[0][et] + sm->red[1][et]) + (sm->red[2][et] + sm->red[3][et]);
+                epi_sync();
+            } else if (a.epi == CL_VEPI_SILU) {
+                for (int t = 0; t < T; ++t) {
+                    const float mine = sm->scale[t] * (v[t] + v[nh + t]);
+                    const float other = __shfl_xor_sync(0xffffffffu, mine, 1);   // gate (even row) / up (odd row) pair
+                    if (live && !(lane & 1)) {
+                        const float h = mine / (1.f + expf(-mine)) * other;
+                        __nv_bfloat16 hi, lo;
+                        split_bf16(h, hi, lo);
+                        a.bnext[(size_t)t * a.bn_ld + (row >> 1)] = hi;
+                        a.bnext[(size_t)(a.nh + t) * a.bn_ld + (row >> 1)] = lo;
+                    }
+                }
+            } else {
+                for (int t = 0; t < T; ++t) {
+                    ClHeadPartial p{0.f, 0.f, 0.f, 0x7fffffff};
+                    if (live) {
+                        const float l = fminf(fmaxf(sm->scale[t] * (v[t] + v[nh + t]), -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
+                        if (a.logits) a.logits[(size_t)t * a.rows + row] = l;
+                        p = ClHeadPartial{l, 1.f, 0.f, row};
+                    }
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const ClHeadPartial other = v_shfl_xor(p, o);
+                        p = ((lane & o) == 0) ? v_merge(p, other) : v_merge(other, p);
+                    }
+                    if (lane == 0) sm->hp[ew][t] = p;
+                }
+                epi_sync();
+                if (et < T) {
+                    // warps hold the tile's rows in tensor-memory quadrant order: combine in row order
+                    const int w0 = (0 + 2) & 3, w1 = (1 + 2) & 3, w2 = (2 + 2) & 3, w3 = (3 + 2) & 3;
+                    ClHeadPartial r = v_merge(v_merge(sm->hp[w0][et], sm->hp[w1][et]), v_merge(sm->hp[w2][et], sm->hp[w3][et]));
+                    a.head_part[(size_t)m * CL_SLOTS + et] = r;
+                }
+                epi_sync();
+            }
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 64;" ::"r"(tmem) : "memory");
+    }
+}
+
+// Start of a pass: x[t] = E[token t]; the first GEMM's input rows hi/lo(x * g) and the per-tile sums of squares.
+__global__ void k_pass_begin(const __nv_bfloat16 *embed, const int *tok, int T, int d, float *x, __nv_bfloat16 *bnext, int nh,
+                             const float *g, float *ssq_out, const ClDevState *st) {
+    if (st->done) return;
+    __shared__ float red[4][CL_SLOTS];
+    const int row = blockIdx.x * 128 + threadIdx.x, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int t = 0; t < T; ++t) {
+        float v = 0.f;
+        if (row < d) {
+            v = __bfloat162float(embed[(size_t)tok[t] * d + row]);
+            x[(size_t)t * d + row] = v;
+            __nv_bfloat16 hi, lo;
+            split_bf16(v * g[row], hi, lo);
+            bnext[(size_t)t * d + row] = hi;
+            bnext[(size_t)(nh + t) * d + row] = lo;
+        }
+        float ss = v * v;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) red[w][t] = ss;
+    }
+    __syncthreads();
+    if (threadIdx.x < T)
+        ssq_out[(size_t)blockIdx.x * CL_SLOTS + threadIdx.x] =
+            (red[0][threadIdx.x] + red[1][threadIdx.x]) + (red[2][threadIdx.x] + red[3][threadIdx.x]);
+}
+
+// Merge the per-tile LM-head statistics of every token row (one warp per row, fixed order) and evaluate Eq. 2-4.
+__global__ void k_head_finalize(const ClHeadPartial *part, int tiles, int T, float inv_log_v, int *out_tok, float *out_pmax,
+                                float *out_conf, const ClDevState *st) {
+    if (st && st->done) return;
+    const int t = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (t >= T) return;
+    ClHeadPartial p{0.f, 0.f, 0.f, 0x7fffffff};
+    for (int m = lane; m < tiles; m += 32) {
+        const ClHeadPartial *src = part + (size_t)m * CL_SLOTS + t;
+        ClHeadPartial q;
+        q.m = __ldcg(&src->m); q.z = __ldcg(&src->z); q.s = __ldcg(&src->s); q.idx = __ldcg(&src->idx);
+        p = v_merge(p, q);
+    }
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const ClHeadPartial other = v_shfl_xor(p, o);
+        p = ((lane & o) == 0) ? v_merge(p, other) : v_merge(other, p);
+    }
+    if (lane == 0) {
+        const float H = logf(p.z) - p.s / p.z;
+        if (out_tok) out_tok[t] = p.idx;
+        if (out_pmax) out_pmax[t] = 1.f / p.z;
+        if (out_conf) out_conf[t] = 1.f - H * inv_log_v;
+    }
+}
+
+}  // namespace
+
+bool cl_make_tensor_map(ClTensorMap *m, const void *base, int rows, int cols, int box_rows) {
+    static_assert(sizeof(ClTensorMap) >= sizeof(CUtensorMap), "tensor map storage");
+    return make_map((CUtensorMap *)m->bytes, base, rows, cols, box_rows);
+}
+
+cudaError_t cl_launch_skinny(const ClTensorMap &mapA, const ClTensorMap &mapB, const ClSkinnyArgs &a, int grid, cudaStream_t s) {
+    const size_t smem = (size_t)VSTAGES * VSTAGE_BYTES + sizeof(VSmem) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_skinny, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    k_skinny<<<grid, VTHREADS, smem, s>>>(*(const CUtensorMap *)mapA.bytes, *(const CUtensorMap *)mapB.bytes, a);
+    return cudaGetLastError();
+}
+
+cudaError_t cl_launch_pass_begin(const void *embed, const int *tok, int T, int d, float *x, __nv_bfloat16 *bnext, int nh,
+                                 const float *g, float *ssq_out, const ClDevState *st, cudaStream_t s) {
+    k_pass_begin<<<(d + 127) / 128, 128, 0, s>>>((const __nv_bfloat16 *)embed, tok, T, d, x, bnext, nh, g, ssq_out, st);
+    return cudaGetLastError();
+}
+
+cudaError_t cl_launch_head_finalize(const ClHeadPartial *part, int tiles, int T, float inv_log_v, int *out_tok, float *out_pmax,
+                                    float *out_conf, const ClDevState *st, cudaStream_t s) {
+    k_head_finalize<<<1, 32 * T, 0, s>>>(part, tiles, T, inv_log_v, out_tok, out_pmax, out_conf, st);
+    return cudaGetLastError();
+}
