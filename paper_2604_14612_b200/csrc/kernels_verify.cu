@@ -20,15 +20,16 @@
 // sums of squares, and s_t = rsqrt(mean x^2 + eps) multiplies the accumulator in the epilogue (a per-token
 // scalar commutes with the contraction).
 // Warp roles as in the scoring kernel: warp 0 TMA producer (A 128 x 64 and B N x 64 tiles, 128-byte swizzle,
-// 8-stage ring), warp 1 tensor-memory allocation and MMA issue, warps 2-5 epilogue (thread = weight row).
+// 4-stage ring, two CTAs per SM), warp 1 tensor-memory allocation and MMA issue, warps 2-5 epilogue (thread = weight row).
 // All waits are bounded; nothing waits on another CTA (the ticket is taken, never polled).
 #include <math.h>
+#include <string.h>
 
 #include "tc_common.cuh"
 
 namespace {
 
-constexpr int VM = 128, VSTAGES = 8;
+constexpr int VM = 128, VSTAGES = 4;   // 80 KB of tiles per CTA, so that the next launch's CTA fits beside this one
 constexpr int VA_BYTES = VM * TC_BK * 2, VB_BYTES = 32 * TC_BK * 2, VSTAGE_BYTES = VA_BYTES + VB_BYTES;   // 20 KB
 constexpr int VTHREADS = 192;
 constexpr int WS_LD = 32;   // floats per row of a workspace partial
@@ -107,7 +108,7 @@ __device__ __forceinline__ void split_bf16(float v, __nv_bfloat16 &hi, __nv_bflo
     lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
-__global__ void __launch_bounds__(VTHREADS, 1)
+__global__ void __launch_bounds__(VTHREADS, 2)
 k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, ClSkinnyArgs a) {
     if (a.st && a.st->done) return;   // written only between launches: uniform over the grid
     extern __shared__ unsigned char smem_dyn[];
@@ -141,24 +142,42 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem = *(volatile unsigned *)&sm->tmem_base;
+    // Programmatic dependent launch: the next launch on the stream may start beside this one as soon as an SM has
+    // room, and this one may have started while its predecessor was still finishing.  Weights never change, so the
+    // producer fills the ring with weight tiles right away; everything a predecessor writes (activation rows, sums
+    // of squares, residual stream, workspace, tickets) is only touched after griddepcontrol.wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             unsigned stage = 0, par = 0, issued[VSTAGES];
             for (int i = 0; i < VSTAGES; ++i) issued[i] = 2u;
-            bool ok = true;
+            bool ok = true, upstream_done = false;
+            int pend_kb[VSTAGES], npend = 0;   // stages whose weight tile is on its way but whose activation tile is not
             Seg sg;
             for (int si = 0; ok && segment_of(U, G, a.KB, c, si, sg); ++si) {
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+                    if (!upstream_done && npend == VSTAGES) {
+                        asm volatile("griddepcontrol.wait;" ::: "memory");
+                        upstream_done = true;
+                        for (int i = 0; i < npend; ++i)
+                            tma_load_2d(tiles + (size_t)i * VSTAGE_BYTES + VA_BYTES, &mapB, pend_kb[i] * TC_BK, 0, &sm->full[i]);
+                    }
                     if (!bar_wait(&sm->empty[stage], par ^ 1u, &sm->abort, a.err)) { ok = false; break; }
                     unsigned char *dst = tiles + (size_t)stage * VSTAGE_BYTES;
                     bar_expect(&sm->full[stage], VA_BYTES + b_bytes);
                     tma_load_2d(dst, &mapA, kb * TC_BK, sg.m * VM, &sm->full[stage]);
-                    tma_load_2d(dst + VA_BYTES, &mapB, kb * TC_BK, 0, &sm->full[stage]);
+                    if (upstream_done) tma_load_2d(dst + VA_BYTES, &mapB, kb * TC_BK, 0, &sm->full[stage]);
+                    else pend_kb[npend++] = kb;   // (the first VSTAGES loads use stages 0, 1, ... in order)
                     issued[stage] = par;
                     if (++stage == VSTAGES) { stage = 0; par ^= 1u; }
                 }
+            }
+            if (!upstream_done) {   // fewer than VSTAGES k-blocks in all
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                for (int i = 0; i < npend; ++i)
+                    tma_load_2d(tiles + (size_t)i * VSTAGE_BYTES + VA_BYTES, &mapB, pend_kb[i] * TC_BK, 0, &sm->full[i]);
             }
             if (!ok) {   // gave up: let the copies in flight land before the CTA may exit (bounded)
                 for (int i = 0; i < VSTAGES; ++i) {
@@ -201,6 +220,7 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
         const int q = warp & 3, rloc = q * 32 + lane;  // tensor-memory lane = row inside the tile
         const int ew = et >> 5;                        // epilogue warp 0 .. 3 (for shared tables)
         const int T = a.T, nh = a.N >> 1;
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // from here on this warp reads what earlier launches wrote
         // RMSNorm scale of every token row: fixed-order sum of the producer's per-tile sums of squares
         if (et < T) {
             float sc = 1.f;
@@ -243,50 +263,74 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
                 __threadfence();
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = 0.f;
-                for (int cc = c_first; cc <= c_last; ++cc) {
-                    const int seg_idx = m - (int)((U * cc / G) / a.KB);   // tiles CTA cc touches are consecutive
-                    const float4 *src = (const float4 *)(a.ws + (((size_t)cc * CL_V_MAXSEG + seg_idx) * VM + rloc) * WS_LD);
+                for (int cc0 = c_first; cc0 <= c_last; cc0 += 4) {   // four partials in flight, added in CTA order
+                    float4 p[4][8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        if (4 * i < a.N) {
-                            const float4 p = __ldcg(src + i);
-                            v[4 * i] += p.x; v[4 * i + 1] += p.y; v[4 * i + 2] += p.z; v[4 * i + 3] += p.w;
+                    for (int j = 0; j < 4; ++j) {
+                        const int cc = min(cc0 + j, c_last);
+                        const int seg_idx = m - (int)((U * cc / G) / a.KB);   // tiles CTA cc touches are consecutive
+                        const float4 *src = (const float4 *)(a.ws + (((size_t)cc * CL_V_MAXSEG + seg_idx) * VM + rloc) * WS_LD);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (4 * i < a.N) p[j][i] = __ldcg(src + i);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (cc0 + j <= c_last) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                if (4 * i < a.N) {
+                                    v[4 * i] += p[j][i].x; v[4 * i + 1] += p[j][i].y; v[4 * i + 2] += p[j][i].z; v[4 * i + 3] += p[j][i].w;
+                                }
+                            }
                         }
                     }
                 }
             }
-            // ---- epilogue of a complete tile: tot[t] = hi column + lo column
+            // ---- epilogue of a complete tile: tot[t] = hi column + lo column (loops unrolled so that the accumulator
+            // stays in registers; rows of a pass never exceed CL_MAX_T)
             const bool live = row < a.rows;
+            float tot[CL_MAX_T];
+#pragma unroll
+            for (int t = 0; t < CL_MAX_T; ++t) tot[t] = v[t] + (nh == 8 ? v[(8 + t) & 31] : v[(16 + t) & 31]);
             if (a.epi == CL_VEPI_STORE) {
-                if (live)
-                    for (int t = 0; t < T; ++t) a.out[(size_t)t * a.ld + row] = sm->scale[t] * (v[t] + v[nh + t]);
+#pragma unroll
+                for (int t = 0; t < CL_MAX_T; ++t)
+                    if (live && t < T) a.out[(size_t)t * a.ld + row] = sm->scale[t] * tot[t];
             } else if (a.epi == CL_VEPI_RESID) {
                 const float g = live ? a.gnext[row] : 0.f;
-                for (int t = 0; t < T; ++t) {
-                    float xn = 0.f;
-                    if (live) {
-                        xn = a.out[(size_t)t * a.ld + row] + (v[t] + v[nh + t]);
-                        a.out[(size_t)t * a.ld + row] = xn;
-                        __nv_bfloat16 hi, lo;
-                        split_bf16(xn * g, hi, lo);
-                        a.bnext[(size_t)t * a.bn_ld + row] = hi;
-                        a.bnext[(size_t)(a.nh + t) * a.bn_ld + row] = lo;
-                        if (a.tap) {
-                            const size_t o = (size_t)((pos0 + t) % a.tap_P) * a.rows + row;
-                            ((__nv_bfloat16 *)a.tap)[o] = __float2bfloat16_rn(xn);
-                        }
-                    }
-                    float ss = xn * xn;
+                float xo[CL_MAX_T];
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-                    if (lane == 0) sm->red[ew][t] = ss;
+                for (int t = 0; t < CL_MAX_T; ++t) xo[t] = (live && t < T) ? __ldcg(a.out + (size_t)t * a.ld + row) : 0.f;   // all reads first
+#pragma unroll
+                for (int t = 0; t < CL_MAX_T; ++t) {
+                    if (t < T) {   // uniform
+                        const float xn = (live ? xo[t] + tot[t] : 0.f);
+                        if (live) {
+                            a.out[(size_t)t * a.ld + row] = xn;
+                            __nv_bfloat16 hi, lo;
+                            split_bf16(xn * g, hi, lo);
+                            a.bnext[(size_t)t * a.bn_ld + row] = hi;
+                            a.bnext[(size_t)(a.nh + t) * a.bn_ld + row] = lo;
+                            if (a.tap) {
+                                const size_t o = (size_t)((pos0 + t) % a.tap_P) * a.rows + row;
+                                ((__nv_bfloat16 *)a.tap)[o] = __float2bfloat16_rn(xn);
+                            }
+                        }
+                        float ss = xn * xn;
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                        if (lane == 0) sm->red[ew][t] = ss;
+                    }
                 }
                 epi_sync();
                 if (et < T) a.ssq_out[(size_t)m * CL_SLOTS + et] = (sm->red[0][et] + sm->red[1][et]) + (sm->red[2][et] + sm->red[3][et]);
                 epi_sync();
             } else if (a.epi == CL_VEPI_SILU) {
-                for (int t = 0; t < T; ++t) {
-                    const float mine = sm->scale[t] * (v[t] + v[nh + t]);
+#pragma unroll
+                for (int t = 0; t < CL_MAX_T; ++t) {
+                    if (t >= T) break;   // uniform
+                    const float mine = sm->scale[t] * tot[t];
                     const float other = __shfl_xor_sync(0xffffffffu, mine, 1);   // gate (even row) / up (odd row) pair
                     if (live && !(lane & 1)) {
                         const float h = mine / (1.f + expf(-mine)) * other;
@@ -297,10 +341,12 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
                     }
                 }
             } else {
-                for (int t = 0; t < T; ++t) {
+#pragma unroll
+                for (int t = 0; t < CL_MAX_T; ++t) {
+                    if (t >= T) break;   // uniform
                     ClHeadPartial p{0.f, 0.f, 0.f, 0x7fffffff};
                     if (live) {
-                        const float l = fminf(fmaxf(sm->scale[t] * (v[t] + v[nh + t]), -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
+                        const float l = fminf(fmaxf(sm->scale[t] * tot[t], -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
                         if (a.logits) a.logits[(size_t)t * a.rows + row] = l;
                         p = ClHeadPartial{l, 1.f, 0.f, row};
                     }
@@ -399,8 +445,18 @@ cudaError_t cl_launch_skinny(const ClTensorMap &mapA, const ClTensorMap &mapB, c
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    k_skinny<<<grid, VTHREADS, smem, s>>>(*(const CUtensorMap *)mapA.bytes, *(const CUtensorMap *)mapB.bytes, a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(VTHREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_skinny, *(const CUtensorMap *)mapA.bytes, *(const CUtensorMap *)mapB.bytes, a);
 }
 
 cudaError_t cl_launch_pass_begin(const void *embed, const int *tok, int T, int d, float *x, __nv_bfloat16 *bnext, int nh,
