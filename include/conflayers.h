@@ -96,7 +96,7 @@ typedef struct {
 int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **out);
 
 /* Copy the weights into the context's own arena (concatenating Q/K/V and interleaving gate/up rows
- * for streaming), allocate the KV cache [n_layers][2][max_seq][d_model] and scratch.  Borrowed
+ * for streaming), allocate the KV cache [n_layers][2][n_heads][max_seq][head_dim] and scratch.  Borrowed
  * pointers may be released after the call returns.  CL_ENOMEM if the device cannot hold it. */
 int cl_load(cl_ctx *ctx, const cl_weights *w);
 

@@ -17,7 +17,7 @@
 struct ClLayer {
     char *wqkv, *wo, *wgu, *wd;   // [3d,d] [d,d] [2F,d] (gate/up rows interleaved) [d,F]
     float *n1, *n2;
-    char *kc, *vc;                // this layer's K and V cache [max_seq, d]
+    char *kc, *vc;                // this layer's K and V cache [n_heads, max_seq, head_dim]
 };
 
 struct cl_ctx {
@@ -65,7 +65,8 @@ struct cl_ctx {
     std::vector<ClTensorMap> map_qkv, map_o, map_gu, map_d;
     ClTensorMap map_head, map_bx[2], map_batt[2], map_bh[2];   // [0]: N = 16, [1]: N = 32
     __nv_bfloat16 *bx, *batt, *bh;       // GEMM input rows as bf16 hi/lo parts: [32, d] [32, d] [32, F]
-    float *v_ws, *v_ssq;
+    float *v_ws, *v_ssq, *v_att_part;
+    int v_att_S;                         // parts the keys of a head are cut into in the T-row attention
     unsigned *v_tickets;
     ClHeadPartial *v_head_part;
     std::vector<ClLayer> layers;
@@ -192,7 +193,7 @@ static void free_all(cl_ctx *c) {
                     c->att, c->hff, c->att_part, c->logits, c->tickets, c->head_part, c->st, c->prompt_dev, c->out_dev,
                     c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sc_xn, c->sc_part, c->sel_mask, c->sel_margins, c->sel_clayers,
                     c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->head_part2,
-                    c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_tickets, c->v_head_part};
+                    c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_att_part, c->v_tickets, c->v_head_part};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->h_st) cudaFreeHost(c->h_st);
@@ -380,6 +381,10 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 DM(c->v_tickets, max_tiles * 4);
                 CU(cudaMemsetAsync(c->v_tickets, 0, max_tiles * 4, c->stream));
                 DM(c->v_ssq, ((d + 127) / 128) * CL_SLOTS * 4);
+                c->v_att_S = c->n_sm / g.n_heads;   // one wave of CTAs
+                if (c->v_att_S < 1) c->v_att_S = 1;
+                if (c->v_att_S > 16) c->v_att_S = 16;
+                DM(c->v_att_part, cl_attn_rows_part_floats(g.n_heads, c->v_att_S, CL_MAX_T, g.head_dim) * 4);
                 DM(c->v_head_part, ((V + 127) / 128) * CL_SLOTS * sizeof(ClHeadPartial));
                 c->map_qkv.resize(L); c->map_o.resize(L); c->map_gu.resize(L); c->map_d.resize(L);
                 for (size_t l = 0; l < L && ok; ++l) {
@@ -501,7 +506,8 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
         t.q = c->qkv; t.ld_q = 3 * d; t.kcache = y.kc; t.vcache = y.vc; t.part = c->att_part; t.tickets = c->tickets + 1;
         t.out = c->att; t.out_b = c->batt; t.nh = nh; t.st = c->st; t.row0 = row0; t.n_heads = g.n_heads; t.head_dim = g.head_dim;
         t.d_model = d; t.nsplit = c->nsplit; t.per_max = c->per_max; t.max_seq = g.max_seq;
-        KL(cl_launch_attn(1, T, t, c->stream));
+        t.part = c->v_att_part;
+        KL(cl_launch_attn_rows(1, T, c->v_att_S, t, c->stream));
         a = b;
         a.rows = d; a.KB = KBd; a.epi = CL_VEPI_RESID; a.out = c->x; a.ld = d; a.bnext = c->bx; a.bn_ld = d; a.gnext = y.n2;
         a.ssq_out = c->v_ssq;

@@ -58,7 +58,7 @@ struct ClGemvArgs {
 struct ClAttnArgs {
     const float *q;       // [T, ld_q] rotary-embedded queries (fp32)
     int ld_q;
-    const void *kcache;   // this layer's K rows [max_seq, d] storage type
+    const void *kcache;   // this layer's K rows [n_heads, max_seq, head_dim] storage type
     const void *vcache;
     float *part;          // [T, H, nsplit, hd + 2] partial (m, l, o[hd])
     unsigned *tickets;    // [T, H]
@@ -117,6 +117,8 @@ cudaError_t cl_launch_rmsnorm_rows(int in_dtype, const void *x, const float *g, 
 cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H, int hd, int d, const float2 *rope_cs,
                                   void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_attn(int wdtype, int T, const ClAttnArgs &a, cudaStream_t s);
+size_t cl_attn_rows_part_floats(int H, int S, int T, int hd);
+cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s);
 cudaError_t cl_launch_tap(int wdtype, const float *x, int T, int row0, int d, void *ring_layer, int P,
                           const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_accept(ClDevState *st, int K, int *out_tokens, cudaStream_t s);

@@ -77,8 +77,8 @@ __global__ void k_rope_append(float *qkv, int row0, int hd, int d, const float2 
     const float qa = q[i], qb = q[i + half], ka = k[i], kb = k[i + half];
     q[i] = qa * cs.x - qb * cs.y;
     q[i + half] = qb * cs.x + qa * cs.y;
-    ST *kc = kcache + (size_t)pos * d + h * hd;
-    ST *vc = vcache + (size_t)pos * d + h * hd;
+    ST *kc = kcache + ((size_t)h * max_seq + pos) * hd;   // cache layout [head][position][hd]: a head's rows are contiguous
+    ST *vc = vcache + ((size_t)h * max_seq + pos) * hd;
     kc[i] = from_f32<ST>(ka * cs.x - kb * cs.y);
     kc[i + half] = from_f32<ST>(kb * cs.x + ka * cs.y);
     vc[i] = from_f32<ST>(v[i]);
@@ -105,8 +105,8 @@ __global__ void __launch_bounds__(128) k_attn(ClAttnArgs a) {
     const int j0 = min(nkeys, sp * per), j1 = min(nkeys, j0 + per);
     const int n = j1 - j0;
     const int d = a.d_model;
-    const ST *K = (const ST *)a.kcache + (size_t)h * HD;
-    const ST *V = (const ST *)a.vcache + (size_t)h * HD;
+    const ST *K = (const ST *)a.kcache + (size_t)h * a.max_seq * HD;
+    const ST *V = (const ST *)a.vcache + (size_t)h * a.max_seq * HD;
     const float scale = rsqrtf((float)HD);
 
     for (int i = tid; i < HD; i += blockDim.x) sq[i] = a.q[(size_t)t * a.ld_q + h * HD + i];
@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(128) k_attn(ClAttnArgs a) {
         const int j = jb + sub;
         float s = 0.f;
         if (j < n) {
-            const uint4 raw = *(const uint4 *)(K + (size_t)(j0 + j) * d + li * EPL);
+            const uint4 raw = *(const uint4 *)(K + (size_t)(j0 + j) * HD + li * EPL);
             if (sizeof(ST) == 2) {
                 const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(128) k_attn(ClAttnArgs a) {
     constexpr int NS = 128 / HD;   // 2 for HD 64, 1 for HD 128
     const int e = tid % HD, stripe = tid / HD;
     float acc = 0.f;
-    for (int j = stripe; j < n; j += NS) acc = fmaf(sc[j], to_f32<ST>(V[(size_t)(j0 + j) * d + e]), acc);
+    for (int j = stripe; j < n; j += NS) acc = fmaf(sc[j], to_f32<ST>(V[(size_t)(j0 + j) * HD + e]), acc);
     if (NS > 1) {
         red[tid] = acc;
         __syncthreads();

@@ -605,7 +605,7 @@ __device__ __forceinline__ void attention_prefetch(const ClStepArgs &a, const Cl
     constexpr int LINES = (ROWB + 127) / 128;
     const int n = (kw1 - kw0) * LINES;
     for (int i = lane; i < n; i += 32) {
-        const size_t off = ((size_t)(kw0 + i / LINES) * a.d + (size_t)h * HD) * sizeof(ST) + (size_t)(i % LINES) * 128;
+        const size_t off = ((size_t)h * a.max_seq + kw0 + i / LINES) * HD * sizeof(ST) + (size_t)(i % LINES) * 128;
         l2_prefetch_line(L.kc + off);
         l2_prefetch_line(L.vc + off);
     }
@@ -650,7 +650,7 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
                 const int j = jb + sub;
                 float sc = 0.f;
                 if (j < n) {
-                    const uint4 raw = __ldcg((const uint4 *)(Kc + (size_t)(j0 + j) * d + h * HD + li * EPL));
+                    const uint4 raw = __ldcg((const uint4 *)(Kc + ((size_t)h * a.max_seq + j0 + j) * HD + li * EPL));
                     if (sizeof(ST) == 2) {
                         const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -690,7 +690,7 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
             for (int j = 0; j < 32; ++j) {
                 const float pj = __shfl_sync(0xffffffffu, p, j);
                 float vv[VPL];
-                load_vals<ST, VPL>(Vc + (size_t)(j0 + min(j, n - 1)) * d + h * HD + lane * VPL, vv);
+                load_vals<ST, VPL>(Vc + ((size_t)h * a.max_seq + j0 + min(j, n - 1)) * HD + lane * VPL, vv);
 #pragma unroll
                 for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(pj, vv[e], o_run[e]);
             }
@@ -715,13 +715,13 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
             sc = __shfl_sync(0xffffffffu, sc, 0) * scale;
             if (sub == 0) {
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) Kc[(size_t)pos * d + h * HD + li * EPL + e] = kst[e];
+                for (int e = 0; e < EPL; ++e) Kc[((size_t)h * a.max_seq + pos) * HD + li * EPL + e] = kst[e];
             }
             float vn[VPL];
 #pragma unroll
             for (int e = 0; e < VPL; ++e) {
                 const ST vs = st_from_f32<ST>(ldcg_f(vraw + lane * VPL + e));
-                Vc[(size_t)pos * d + h * HD + lane * VPL + e] = vs;
+                Vc[((size_t)h * a.max_seq + pos) * HD + lane * VPL + e] = vs;
                 vn[e] = st_to_f32<ST>(vs);
             }
             const float m_new = fmaxf(m_run, sc);

@@ -470,3 +470,229 @@ cudaError_t cl_launch_head_finalize(const ClHeadPartial *part, int tiles, int T,
     k_head_finalize<<<1, 32 * T, 0, s>>>(part, tiles, T, inv_log_v, out_tok, out_pmax, out_conf, st);
     return cudaGetLastError();
 }
+
+// ---- attention of the T rows of a pass over the KV cache ----------------------------------------------------
+// grid (H, S): the keys [0, base + T) of a head (base = first row's position; the rows' own keys are already in
+// the cache, rotated) are cut into S contiguous parts, a part into 8 warp ranges.  A warp walks its range 32 keys
+// at a time: every key row is read once (16 bytes per lane) and scored against all T query rows, row t masking keys
+// beyond its own position; per row an online softmax; every value row is read once and accumulated into all rows.
+// The CTA merges its warps in shared memory; the last CTA of a head (ticket) merges the S parts in order and
+// writes the output rows as fp32 and as bf16 hi/lo parts (the next GEMM's input).
+namespace {
+
+constexpr int AR_WARPS = 8;
+
+// (Loops over keys stay rolled and the row count is a template parameter: the kernel runs its code once, so its
+// time is instruction fetch, and a fully unrolled version measured 55 us against a few us of work.)
+template <typename ST, int HD, int T>
+__global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S) {
+    if (a.st->done) return;
+    constexpr int EPL = 16 / (int)sizeof(ST), LPK = HD / EPL, KPW = 32 / LPK, VPL = HD / 32;
+    constexpr int REC = HD + 2;
+    extern __shared__ float wrec[];   // [AR_WARPS][T][REC]
+    __shared__ int is_last;
+    const int h = blockIdx.x, s = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int base = a.st->ctx + a.row0, nkeys = base + T, d = a.d_model;
+    if (nkeys > a.max_seq) return;
+    const int k0 = (int)((long long)nkeys * s / S), k1 = (int)((long long)nkeys * (s + 1) / S);
+    const int kw0 = k0 + (k1 - k0) * warp / AR_WARPS, kw1 = k0 + (k1 - k0) * (warp + 1) / AR_WARPS;
+    const int sub = lane / LPK, li = lane % LPK;
+    const float scale = rsqrtf((float)HD);
+    const ST *Kc = (const ST *)a.kcache + (size_t)h * a.max_seq * HD;   // cache layout [head][position][hd]
+    const ST *Vc = (const ST *)a.vcache + (size_t)h * a.max_seq * HD;
+
+    float qr[T][EPL];
+#pragma unroll
+    for (int t = 0; t < T; ++t)
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) qr[t][e] = (t < T) ? a.q[(size_t)t * a.ld_q + h * HD + li * EPL + e] * scale : 0.f;
+    float m_run[T], l_run[T], o_run[T][VPL];
+#pragma unroll
+    for (int t = 0; t < T; ++t) {
+        m_run[t] = -INFINITY;
+        l_run[t] = 0.f;
+#pragma unroll
+        for (int e = 0; e < VPL; ++e) o_run[t][e] = 0.f;
+    }
+    for (int j0 = kw0; j0 < kw1; j0 += 32) {
+        const int n = min(32, kw1 - j0);
+        float sc[T];   // lane j: score of key j0 + j against row t
+#pragma unroll
+        for (int t = 0; t < T; ++t) sc[t] = -INFINITY;
+#pragma unroll 1
+        for (int jb = 0; jb < 32; jb += KPW) {
+            const int j = jb + sub;
+            float kf[EPL];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) kf[e] = 0.f;
+            if (j < n) {
+                const uint4 raw = *(const uint4 *)(Kc + (size_t)(j0 + j) * HD + li * EPL);
+                if (sizeof(ST) == 2) {
+                    const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        kf[(2 * e) % EPL] = __uint_as_float(u[e] << 16);
+                        kf[(2 * e + 1) % EPL] = __uint_as_float(u[e] & 0xffff0000u);
+                    }
+                } else {
+                    kf[0] = __uint_as_float(raw.x); kf[1 % EPL] = __uint_as_float(raw.y);
+                    kf[2 % EPL] = __uint_as_float(raw.z); kf[3 % EPL] = __uint_as_float(raw.w);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                if (t < T) {   // uniform
+                    float v = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) v = fmaf(qr[t][e], kf[e], v);
+#pragma unroll
+                    for (int o = LPK >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+#pragma unroll
+                    for (int k = 0; k < KPW; ++k) {
+                        const float w = __shfl_sync(0xffffffffu, v, k * LPK);
+                        if (lane == jb + k && jb + k < n && j0 + jb + k <= base + t) sc[t] = w;   // causal mask
+                    }
+                }
+            }
+        }
+        float p[T];
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            p[t] = 0.f;
+            if (t < T) {
+                float mx = sc[t];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                const float m_new = fmaxf(mx, m_run[t]);
+                if (m_new > -INFINITY) {   // uniform over the warp
+                    p[t] = (sc[t] > -INFINITY) ? expf(sc[t] - m_new) : 0.f;
+                    const float resc = (l_run[t] > 0.f) ? expf(m_run[t] - m_new) : 0.f;
+                    float ps = p[t];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+                    l_run[t] = fmaf(l_run[t], resc, ps);
+#pragma unroll
+                    for (int e = 0; e < VPL; ++e) o_run[t][e] *= resc;
+                    m_run[t] = m_new;
+                }
+            }
+        }
+        // value rows: 8 at a time in flight (rows past the end repeat the last one; their weights are 0)
+#pragma unroll 1
+        for (int jh = 0; jh < 32; jh += 8) {
+            if (jh < n) {   // uniform
+                float vv[8][VPL];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const ST *vp = Vc + (size_t)(j0 + min(jh + j, n - 1)) * HD + lane * VPL;
+                    if (sizeof(ST) == 2 && VPL == 4) {
+                        const uint2 u = *(const uint2 *)vp;
+                        vv[j][0] = __uint_as_float(u.x << 16); vv[j][1 % VPL] = __uint_as_float(u.x & 0xffff0000u);
+                        vv[j][2 % VPL] = __uint_as_float(u.y << 16); vv[j][3 % VPL] = __uint_as_float(u.y & 0xffff0000u);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < VPL; ++e) vv[j][e] = (float)vp[e];
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+#pragma unroll
+                    for (int t = 0; t < T; ++t) {
+                        if (t < T) {
+                            const float pj = __shfl_sync(0xffffffffu, p[t], jh + j);
+#pragma unroll
+                            for (int e = 0; e < VPL; ++e) o_run[t][e] = fmaf(pj, vv[j][e], o_run[t][e]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    // merge the warps of this CTA (fixed order)
+#pragma unroll
+    for (int t = 0; t < T; ++t) {
+        {
+            float *r = wrec + ((size_t)warp * T + t) * REC;
+            if (lane == 0) { r[0] = m_run[t]; r[1] = l_run[t]; }
+#pragma unroll
+            for (int e = 0; e < VPL; ++e) r[2 + lane * VPL + e] = o_run[t][e];
+        }
+    }
+    __syncthreads();
+    float *part = a.part + ((size_t)h * S + s) * T * REC;
+    for (int i = tid; i < T * HD; i += blockDim.x) {
+        const int t = i / HD, e = i % HD;
+        float M = -INFINITY;
+        for (int w = 0; w < AR_WARPS; ++w) {
+            const float *r = wrec + ((size_t)w * T + t) * REC;
+            if (r[1] > 0.f) M = fmaxf(M, r[0]);
+        }
+        float Ls = 0.f, O = 0.f;
+        for (int w = 0; w < AR_WARPS; ++w) {
+            const float *r = wrec + ((size_t)w * T + t) * REC;
+            if (r[1] > 0.f) {
+                const float f = expf(r[0] - M);
+                Ls = fmaf(r[1], f, Ls);
+                O = fmaf(r[2 + e], f, O);
+            }
+        }
+        if (e == 0) { part[(size_t)t * REC] = M; part[(size_t)t * REC + 1] = Ls; }
+        part[(size_t)t * REC + 2 + e] = O;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned prev = atomicAdd(a.tickets + h, 1u);
+        is_last = (prev == (unsigned)S - 1);
+        if (is_last) a.tickets[h] = 0u;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int i = tid; i < T * HD; i += blockDim.x) {
+        const int t = i / HD, e = i % HD;
+        const float *p0 = a.part + (size_t)h * S * T * REC + (size_t)t * REC;
+        float M = -INFINITY;
+        for (int s2 = 0; s2 < S; ++s2)
+            if (__ldcg(p0 + (size_t)s2 * T * REC + 1) > 0.f) M = fmaxf(M, __ldcg(p0 + (size_t)s2 * T * REC));
+        float Ls = 0.f, O = 0.f;
+        for (int s2 = 0; s2 < S; ++s2) {
+            const float l2 = __ldcg(p0 + (size_t)s2 * T * REC + 1);
+            if (l2 > 0.f) {
+                const float f = expf(__ldcg(p0 + (size_t)s2 * T * REC) - M);
+                Ls = fmaf(l2, f, Ls);
+                O = fmaf(__ldcg(p0 + (size_t)s2 * T * REC + 2 + e), f, O);
+            }
+        }
+        const float o = O / Ls;
+        a.out[(size_t)t * d + h * HD + e] = o;
+        if (a.out_b) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(o);
+            a.out_b[(size_t)t * d + h * HD + e] = hi;
+            a.out_b[(size_t)(a.nh + t) * d + h * HD + e] = __float2bfloat16_rn(o - __bfloat162float(hi));
+        }
+    }
+}
+
+}  // namespace
+
+size_t cl_attn_rows_part_floats(int H, int S, int T, int hd) { return (size_t)H * S * T * (hd + 2); }
+
+// a.part must hold cl_attn_rows_part_floats(H, S, T, hd) floats, a.tickets H zeroed counters.
+cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s) {
+    dim3 grid(a.n_heads, S);
+    const size_t smem = (size_t)AR_WARPS * T * (a.head_dim + 2) * sizeof(float);
+#define AR_CASE(TT)                                                                                                   \
+    case TT:                                                                                                          \
+        if (wdtype == 1 && a.head_dim == 128) k_attn_rows<__nv_bfloat16, 128, TT><<<grid, AR_WARPS * 32, smem, s>>>(a, S);     \
+        else if (wdtype == 1 && a.head_dim == 64) k_attn_rows<__nv_bfloat16, 64, TT><<<grid, AR_WARPS * 32, smem, s>>>(a, S); \
+        else return cudaErrorInvalidValue;                                                                            \
+        break;
+    switch (T) {
+        AR_CASE(1) AR_CASE(2) AR_CASE(3) AR_CASE(4) AR_CASE(5) AR_CASE(6) AR_CASE(7) AR_CASE(8) AR_CASE(9)
+        default: return cudaErrorInvalidValue;
+    }
+#undef AR_CASE
+    return cudaGetLastError();
+}
