@@ -489,8 +489,13 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
     if (a.st->done) return;
     constexpr int EPL = 16 / (int)sizeof(ST), LPK = HD / EPL, KPW = 32 / LPK, VPL = HD / 32;
     constexpr int REC = HD + 2;
-    extern __shared__ float wrec[];   // [AR_WARPS][T][REC]
+    extern __shared__ __align__(16) float wrec[];   // [AR_WARPS][T][REC], then per warp 32 key rows and 32 value rows
     __shared__ int is_last;
+    constexpr int ROWB = HD * (int)sizeof(ST);                 // bytes of one cached row of a head
+    constexpr int CPR = ROWB / 16;                              // 16-byte chunks per row
+    constexpr size_t WREC_BYTES = ((size_t)AR_WARPS * T * REC * sizeof(float) + 15) & ~(size_t)15;
+    unsigned char *stage_k = (unsigned char *)wrec + WREC_BYTES + (size_t)(threadIdx.x >> 5) * 2 * 32 * ROWB;
+    unsigned char *stage_v = stage_k + 32 * ROWB;
     const int h = blockIdx.x, s = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int base = a.st->ctx + a.row0, nkeys = base + T, d = a.d_model;
@@ -517,6 +522,30 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
     }
     for (int j0 = kw0; j0 < kw1; j0 += 32) {
         const int n = min(32, kw1 - j0);
+        // stage this pass's key and value rows in shared memory: every 16-byte piece is requested before any is used,
+        // so the pass costs one memory round trip; the (rolled) loops below then read shared memory
+        __syncwarp();
+        {
+            const uint4 *gk = (const uint4 *)(Kc + (size_t)j0 * HD), *gv = (const uint4 *)(Vc + (size_t)j0 * HD);
+            uint4 tk[CPR], tv[CPR];
+#pragma unroll
+            for (int it = 0; it < CPR; ++it) {
+                const int cidx = it * 32 + lane;   // chunk cidx of the pass: row cidx / CPR
+                if (cidx < n * CPR) {
+                    tk[it] = gk[cidx];
+                    tv[it] = gv[cidx];
+                }
+            }
+#pragma unroll
+            for (int it = 0; it < CPR; ++it) {
+                const int cidx = it * 32 + lane;
+                if (cidx < n * CPR) {
+                    ((uint4 *)stage_k)[cidx] = tk[it];
+                    ((uint4 *)stage_v)[cidx] = tv[it];
+                }
+            }
+        }
+        __syncwarp();
         float sc[T];   // lane j: score of key j0 + j against row t
 #pragma unroll
         for (int t = 0; t < T; ++t) sc[t] = -INFINITY;
@@ -527,7 +556,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
 #pragma unroll
             for (int e = 0; e < EPL; ++e) kf[e] = 0.f;
             if (j < n) {
-                const uint4 raw = *(const uint4 *)(Kc + (size_t)(j0 + j) * HD + li * EPL);
+                const uint4 raw = *(const uint4 *)(stage_k + (size_t)j * ROWB + li * 16);
                 if (sizeof(ST) == 2) {
                     const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -585,7 +614,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
                 float vv[8][VPL];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const ST *vp = Vc + (size_t)(j0 + min(jh + j, n - 1)) * HD + lane * VPL;
+                    const ST *vp = (const ST *)(stage_v + (size_t)min(jh + j, n - 1) * ROWB) + lane * VPL;
                     if (sizeof(ST) == 2 && VPL == 4) {
                         const uint2 u = *(const uint2 *)vp;
                         vv[j][0] = __uint_as_float(u.x << 16); vv[j][1 % VPL] = __uint_as_float(u.x & 0xffff0000u);
@@ -682,17 +711,26 @@ size_t cl_attn_rows_part_floats(int H, int S, int T, int hd) { return (size_t)H 
 // a.part must hold cl_attn_rows_part_floats(H, S, T, hd) floats, a.tickets H zeroed counters.
 cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s) {
     dim3 grid(a.n_heads, S);
-    const size_t smem = (size_t)AR_WARPS * T * (a.head_dim + 2) * sizeof(float);
-#define AR_CASE(TT)                                                                                                   \
-    case TT:                                                                                                          \
-        if (wdtype == 1 && a.head_dim == 128) k_attn_rows<__nv_bfloat16, 128, TT><<<grid, AR_WARPS * 32, smem, s>>>(a, S);     \
-        else if (wdtype == 1 && a.head_dim == 64) k_attn_rows<__nv_bfloat16, 64, TT><<<grid, AR_WARPS * 32, smem, s>>>(a, S); \
-        else return cudaErrorInvalidValue;                                                                            \
+    const size_t es = wdtype == 1 ? 2 : 4;
+    const size_t smem = (((size_t)AR_WARPS * T * (a.head_dim + 2) * sizeof(float) + 15) & ~(size_t)15) + (size_t)AR_WARPS * 2 * 32 * a.head_dim * es;
+#define AR_LAUNCH(HDV, TT)                                                                                            \
+    {                                                                                                                 \
+        cudaError_t e_ = cudaFuncSetAttribute(k_attn_rows<__nv_bfloat16, HDV, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                              (int)smem);                                                             \
+        if (e_ != cudaSuccess) return e_;                                                                             \
+        k_attn_rows<__nv_bfloat16, HDV, TT><<<grid, AR_WARPS * 32, smem, s>>>(a, S);                                    \
+    }
+#define AR_CASE(TT)                                              \
+    case TT:                                                     \
+        if (wdtype == 1 && a.head_dim == 128) AR_LAUNCH(128, TT) \
+        else if (wdtype == 1 && a.head_dim == 64) AR_LAUNCH(64, TT) \
+        else return cudaErrorInvalidValue;                       \
         break;
     switch (T) {
         AR_CASE(1) AR_CASE(2) AR_CASE(3) AR_CASE(4) AR_CASE(5) AR_CASE(6) AR_CASE(7) AR_CASE(8) AR_CASE(9)
         default: return cudaErrorInvalidValue;
     }
 #undef AR_CASE
+#undef AR_LAUNCH
     return cudaGetLastError();
 }
