@@ -251,3 +251,33 @@ def test_generate_to_the_last_cache_slot():
     assert list(van[:lim - 1]) == ref["tokens"][1:lim]
     if lim == 21:
         assert list(toks) == list(van)
+
+
+def test_tensor_core_pass_matches_streaming_pass(monkeypatch):
+    """The tcgen05 pass (verify / prefill of bf16 models) against the CUDA-core T-row path on the same inputs:
+    two independent implementations of the same full-model pass, T = 5 (N = 16) and T = 9 (N = 32)."""
+    base = synth.WORKLOADS["C2"].shape
+    sh = dataclasses.replace(base, n_layers=2, max_seq=64)
+    W = synth.make_weights(sh, 5, device="cuda")
+    prompt = synth.make_prompt(5, 11, sh.vocab)                        # a full chunk of 8 and a ragged one of 3
+    out = {}
+    for tc in (0, 1):
+        monkeypatch.setenv("CL_DISABLE_TC_PASS", "0" if tc else "1")
+        ctx = cl.Context.from_shape(sh, tap_positions=16)               # longer than any pass: no two rows share a slot
+        ctx.cl_load(W)
+        first = ctx.cl_prefill(prompt, tap_hidden=True)
+        res = [first]
+        for drafts in ([11, 22, 33, 44], [5, 6, 7, 8, 9, 10, 11, 12]):
+            ctx.cl_rollback(len(prompt), first)
+            ctx.cl_force_tokens(drafts)
+            v = ctx.cl_verify(len(drafts) + 1, tap_hidden=True, want_logits=True)
+            res.append((v["targets"].copy(), v["logits"].copy()))
+        res.append(ctx.cl_read_hidden_ring().float().numpy())
+        out[tc] = res
+        ctx.close()
+    assert out[0][0] == out[1][0]
+    for i in (1, 2):
+        assert np.abs(out[0][i][1] - out[1][i][1]).max() <= 2e-3        # both far inside the 1e-2 tolerance
+        assert np.array_equal(out[0][i][0], out[1][i][0])
+    scale = max(1.0, float(np.abs(out[0][3]).max()))
+    assert np.abs(out[0][3] - out[1][3]).max() <= 2 ** -7 * scale        # taps: one bf16 ulp at the top of the range
