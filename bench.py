@@ -279,6 +279,36 @@ def main():
     vanilla_tps = gen / (ms_v * 1e-3)
     vanilla_gbs = gen * algorithmic_bytes(shape, shape.n_layers, ctx_mid) / (ms_v * 1e-3) / 1e9
 
+    # the all-layer confidence scoring workload (C5): 8 rounds of score -> select -> best, tensor-core bound
+    c5 = None
+    if rank == 0 and not args.layers:
+        cc = synth.C5
+        L5, P5, d5, V5 = cc["n_layers"], cc["positions"], cc["d_model"], cc["vocab"]
+        head5 = synth.make_lm_head(cc["seed"], V5, d5, device="cuda")
+        ctx5 = cl.Context(L5, d5, d5 // 128, 11008, V5, 8, "bf16", rms_eps=cc["rms_eps"])
+        ctx5.cl_load(dict(lm_head=head5, final_norm=torch.ones(d5, device="cuda")), head_only=True)
+        hid5 = [synth.make_hidden(cc["seed"], t, L5, P5, d5, device="cuda") for t in range(cc["iters"])]
+        sc5 = synth.make_round_scores(cc["seed"], cc["iters"])
+        sel5 = cl.SelectCfg.make(cc["lo"], cc["hi"], n_skip=cc["n_skip"])
+        for _ in range(3):
+            ctx5.cl_score_loop(sel5, hid5, sc5)
+        t5 = []
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ctx5.cl_score_loop(sel5, hid5, sc5)
+            e1.record()
+            torch.cuda.synchronize()
+            t5.append(e0.elapsed_time(e1))
+        ms5 = statistics.median(t5)
+        tf5 = cc["iters"] * 2.0 * L5 * P5 * d5 * V5 / (ms5 * 1e-3) / 1e12
+        pk = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+        sus = float(pk.get("bf16_tflops_sustained", 1400.0))
+        c5 = {"score_loop_ms": ms5, "tflops": tf5, "frac_of_bf16_sustained": tf5 / sus,
+              "peak_kind": "of measured" if pk else "of fallback"}
+        ctx5.close()
+        del head5, hid5
+
     # end to end through the public API with host buffers: prompt H2D + prefill + generate + tokens D2H
     e2e = None
     if not args.no_e2e:
@@ -309,7 +339,7 @@ def main():
                        "parallelism": "replicas only" if world > 1 else "1 GPU",
                        "alpha": accepted / drafted if drafted else None, "cycles_per_step": cycles / args.steps,
                        "vanilla_tokens_per_s": vanilla_tps, "vanilla_achieved_gbs": vanilla_gbs,
-                       "vanilla_frac_of_peak": vanilla_gbs / peak},
+                       "vanilla_frac_of_peak": vanilla_gbs / peak, "c5_scoring": c5},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_kind": f"of {peak_kind}", "frac_of_8TBps": achieved / 8000.0,
                          "kernel": f"k_token_steps, one launch = {K_DRAFT} draft steps over {n_kept} kept layers + LM head",
