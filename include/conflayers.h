@@ -174,6 +174,28 @@ int cl_select_skip_set(cl_ctx *ctx, const cl_select_cfg *cfg, const float *c_lay
 int cl_score_loop(cl_ctx *ctx, const cl_select_cfg *cfg, const void *const *hidden_iters, int iters, int P,
                   const float *scores, uint8_t *best_mask, int *best_iter, uint8_t *masks_all, float *c_layers_all);
 
+/* Interval-based periodic search (Section 3.3, Figure 2) around the generation loop.  The skip set installed
+ * when the call is made (the paper starts from uniformly skipped layers) is round 0.  Every set drafts for
+ * `interval` cycles (Opt_Interval); the round's score is the mean number of accepted candidates per cycle; the
+ * best-scoring set is remembered (the earlier one on ties).  After a round whose score reaches score_goal, or after
+ * max_rounds searched sets, the search ends and the best set drafts for the rest of the call (it stays installed).
+ * Otherwise the layers are scored on the hidden-state ring (Section 3.1), a new set is selected with *sel
+ * (Section 3.2) and installed.  Needs tap_positions > 0 and a cl_prefill with tap_hidden = 1 (which clears the
+ * ring); verify passes record the ring while the search is on.  The emitted tokens do not depend on the search.
+ * out: host [max_new].  rep (may be NULL): scores[i] of round i, i < n_scored; masks (host, may be NULL):
+ * [(max_rounds + 1), n_layers], row i = the set of round i. */
+#define CL_MAX_ROUNDS 32
+typedef struct {
+    int K, interval, max_rounds;   /* draft length, cycles per interval, searched sets after the initial one */
+    float score_goal;              /* the paper halts at 4 accepted tokens */
+} cl_search_cfg;
+typedef struct {
+    int n_scored, best_round, searching;   /* rounds scored, index of the best, 1 if the search was still on at the end */
+    float scores[CL_MAX_ROUNDS + 1];
+} cl_search_report;
+int cl_generate_search(cl_ctx *ctx, const cl_search_cfg *cfg, const cl_select_cfg *sel, int max_new, int32_t *out,
+                       int *n_out, cl_search_report *rep, uint8_t *masks);
+
 /* Copy the hidden-state ring to the host: out is [n_layers, tap_positions, d_model] in the storage
  * type, position slot = absolute position modulo tap_positions. */
 int cl_read_hidden_ring(cl_ctx *ctx, void *out);

@@ -44,6 +44,18 @@ class SelectCfg(C.Structure):
         return cls(w_base, lam, eps, flat_tol, w_max, lo, hi, n_skip, min_ratio, fixed_window)
 
 
+CL_MAX_ROUNDS = 32
+
+
+class SearchCfg(C.Structure):
+    _fields_ = [("K", C.c_int), ("interval", C.c_int), ("max_rounds", C.c_int), ("score_goal", C.c_float)]
+
+
+class SearchReport(C.Structure):
+    _fields_ = [("n_scored", C.c_int), ("best_round", C.c_int), ("searching", C.c_int),
+                ("scores", C.c_float * (CL_MAX_ROUNDS + 1))]
+
+
 class Stats(C.Structure):
     _fields_ = [("cycles", C.c_uint64), ("drafted", C.c_uint64), ("accepted", C.c_uint64), ("emitted", C.c_uint64),
                 ("ctx_len", C.c_int), ("n_skipped", C.c_int), ("kernel_launches", C.c_uint64)]
@@ -85,6 +97,8 @@ def load_library():
         "cl_accept": [vp, C.POINTER(C.c_int), vp],
         "cl_step_vanilla": [vp, ip],
         "cl_generate": [vp, C.c_int, C.c_int, vp, C.POINTER(C.c_int), C.POINTER(Stats)],
+        "cl_generate_search": [vp, C.POINTER(SearchCfg), C.POINTER(SelectCfg), C.c_int, vp, C.POINTER(C.c_int),
+                               C.POINTER(SearchReport), vp],
         "cl_rollback": [vp, C.c_int, C.c_int32],
         "cl_force_tokens": [vp, vp, C.c_int],
         "cl_layer_confidences": [vp, vp, C.c_int, C.c_int, vp, vp, vp, vp],
@@ -254,6 +268,20 @@ class Context:
         st = Stats()
         self._ck(self._L.cl_generate(self._h, K, max_new, _np_ptr(out), C.byref(n), C.byref(st)))
         return out[:n.value], st
+
+    def cl_generate_search(self, K: int, max_new: int, interval: int, score_goal: float, max_rounds: int, sel: SelectCfg):
+        out = np.zeros(max_new, np.int32)
+        n = C.c_int()
+        rep = SearchReport()
+        L = self.cfg.n_layers
+        masks = np.zeros((max_rounds + 1, L), np.uint8)
+        cfg = SearchCfg(K, interval, max_rounds, score_goal)
+        self._ck(self._L.cl_generate_search(self._h, C.byref(cfg), C.byref(sel), max_new, _np_ptr(out), C.byref(n),
+                                            C.byref(rep), _np_ptr(masks)))
+        k = rep.n_scored
+        return dict(tokens=out[:n.value], scores=[float(rep.scores[i]) for i in range(k)],
+                    sets=[[l for l in range(L) if masks[i][l]] for i in range(k)], best_round=rep.best_round,
+                    searching=bool(rep.searching), final_set=[l for l in range(L) if self.cl_get_skip_set()[l]])
 
     def cl_rollback(self, ctx_len: int, pending_token: int):
         self._ck(self._L.cl_rollback(self._h, ctx_len, pending_token))

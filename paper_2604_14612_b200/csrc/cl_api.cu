@@ -585,6 +585,8 @@ extern "C" int cl_prefill(cl_ctx *c, const int32_t *tokens, int n, int tap_hidde
     for (int i = 0; i < n; ++i)
         if (tokens[i] < 0 || tokens[i] >= c->cfg.vocab) return fail(c, CL_EINVAL, "cl_prefill: token %d out of range at %d", tokens[i], i);
     CU(cudaMemcpyAsync(c->prompt_dev, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, c->stream));
+    if (tap_hidden && c->ring)   // a tapped prefill starts the context window afresh
+        CU(cudaMemsetAsync(c->ring, 0, (size_t)c->cfg.n_layers * c->cfg.tap_positions * c->cfg.d_model * c->esz, c->stream));
     ClPoke p = poke_none();
     p.ctx = 0; p.n_drafted = 0; p.done = 0;
     if ((rc = poke(c, p))) return rc;
@@ -738,7 +740,7 @@ extern "C" int cl_step_vanilla(cl_ctx *c, int32_t *tok) {
     return CL_OK;
 }
 
-static int enqueue_cycle(cl_ctx *c, int K) {
+static int enqueue_cycle(cl_ctx *c, int K, int tap = 0) {
     int rc;
     if (c->use_step && K > 0) {
         if ((rc = run_steps(c, CL_STEP_DRAFT, K, 0, false, nullptr, nullptr))) return rc;
@@ -750,7 +752,7 @@ static int enqueue_cycle(cl_ctx *c, int K) {
             if (rc) return rc;
         }
     }
-    rc = forward_rows(c, ST_FIELD(c, int, cyc_tok), K + 1, 0, nullptr, 0, 1, ST_FIELD(c, int, tgt_tok),
+    rc = forward_rows(c, ST_FIELD(c, int, cyc_tok), K + 1, 0, nullptr, tap, 1, ST_FIELD(c, int, tgt_tok),
                       ST_FIELD(c, float, v_pmax), ST_FIELD(c, float, v_conf), nullptr);
     if (rc) return rc;
     KL(cl_launch_accept(c->st, K, c->out_dev, c->stream));
@@ -798,6 +800,89 @@ extern "C" int cl_generate(cl_ctx *c, int K, int max_new, int32_t *out, int *n_o
     c->h_ndraft = 0;
     if (n_out) *n_out = max_new;
     if (stats) cl_get_stats(c, stats);
+    return CL_OK;
+}
+
+static int check_select(cl_ctx *c, const cl_select_cfg *s);
+static int ensure_sel_iters(cl_ctx *c, int iters);
+static int score_rows(cl_ctx *c, const void *hidden, int rows, int P, float *c_layer_dev);
+static int score_device_err(cl_ctx *c, const char *fn);
+
+// Generation with the interval-based periodic search of Section 3.3.  Host logic only: the cycles of an interval
+// are enqueued back to back (no host round trip inside an interval), the search check reads the device counters
+// once per interval, and scoring / selection run in the kernels of cl_layer_confidences / cl_select_skip_set.
+extern "C" int cl_generate_search(cl_ctx *c, const cl_search_cfg *sc, const cl_select_cfg *sel, int max_new, int32_t *out,
+                                  int *n_out, cl_search_report *rep, uint8_t *masks) {
+    int rc = need_model(c, "cl_generate_search", true);
+    if (rc) return rc;
+    if (!sc || !sel || !out || max_new <= 0) return fail(c, CL_EINVAL, "cl_generate_search: null argument or nothing to generate");
+    const int K = sc->K, L = c->cfg.n_layers, P = c->cfg.tap_positions;
+    if (K < 1 || K > CL_MAX_K) return fail(c, CL_ERANGE, "cl_generate_search: K = %d outside 1..%d", K, CL_MAX_K);
+    if (sc->interval < 1 || sc->max_rounds < 0 || sc->max_rounds > CL_MAX_ROUNDS)
+        return fail(c, CL_ERANGE, "cl_generate_search: interval >= 1 and 0 <= max_rounds <= %d required", CL_MAX_ROUNDS);
+    if (!c->ring) return fail(c, CL_ESTATE, "cl_generate_search: the context has no hidden-state ring (tap_positions = 0)");
+    if (c->h_ctx + max_new + K > c->cfg.max_seq)
+        return fail(c, CL_ERANGE, "cl_generate_search: %d + %d + %d tokens exceed max_seq %d", c->h_ctx, max_new, K, c->cfg.max_seq);
+    if ((rc = check_select(c, sel))) return rc;
+    if ((rc = ensure_sel_iters(c, 1))) return rc;
+    if (max_new > c->out_cap) {
+        if (c->out_dev) cudaFree(c->out_dev);
+        c->out_dev = nullptr;
+        c->out_cap = 0;
+        DM(c->out_dev, (size_t)max_new * 4);
+        c->out_cap = max_new;
+    }
+    ClPoke p = poke_none();
+    p.n_out = 0; p.max_new = max_new; p.done = 0; p.n_drafted = 0;
+    if ((rc = poke(c, p))) return rc;
+    if ((rc = sync_state(c))) return rc;
+    cl_search_report r;
+    memset(&r, 0, sizeof(r));
+    r.searching = 1;
+    std::vector<uint8_t> best(c->mask), cur(c->mask);
+    float best_score = -INFINITY;
+    int rnd = 0;
+    while (c->h_st->n_out < max_new) {
+        const int remaining = max_new - c->h_st->n_out;
+        const unsigned long long cyc0 = c->h_st->cycles, acc0 = c->h_st->accepted;
+        // while searching: one interval; afterwards: the fewest cycles that can finish (cycles past the end exit at once)
+        const int ncyc = r.searching ? sc->interval : (remaining + K) / (K + 1);
+        for (int i = 0; i < ncyc; ++i)
+            if ((rc = enqueue_cycle(c, K, r.searching))) return rc;
+        if ((rc = sync_state(c))) return rc;
+        if ((rc = check_device_err(c, "cl_generate_search"))) return rc;
+        if (!r.searching || (int)(c->h_st->cycles - cyc0) < sc->interval) continue;   // no full interval: nothing to check
+        // ---- search check (Section 3.3)
+        const float score = (float)((double)(c->h_st->accepted - acc0) / (double)sc->interval);
+        r.scores[rnd] = score;
+        if (masks) memcpy(masks + (size_t)rnd * L, cur.data(), (size_t)L);
+        r.n_scored = rnd + 1;
+        if (score > best_score) {
+            best_score = score;
+            best = cur;
+            r.best_round = rnd;
+        }
+        if (score >= sc->score_goal || rnd >= sc->max_rounds) {
+            r.searching = 0;
+            cur = best;
+        } else {
+            if ((rc = score_rows(c, c->ring, L, P, c->sc_clayer))) return rc;
+            KL(cl_launch_select(*sel, L, c->sc_clayer, c->sel_mask, nullptr, c->stream));
+            CU(cudaMemcpyAsync(cur.data(), c->sel_mask, (size_t)L, cudaMemcpyDeviceToHost, c->stream));
+            CU(cudaStreamSynchronize(c->stream));
+            if ((rc = score_device_err(c, "cl_generate_search"))) return rc;
+            ++rnd;
+        }
+        if ((rc = cl_set_skip_set(c, cur.data()))) return rc;
+    }
+    CU(cudaMemcpy(out, c->out_dev, (size_t)max_new * 4, cudaMemcpyDeviceToHost));
+    p = poke_none();
+    p.done = 0;
+    if ((rc = poke(c, p))) return rc;
+    if ((rc = sync_state(c))) return rc;
+    c->h_ndraft = 0;
+    if (n_out) *n_out = max_new;
+    if (rep) *rep = r;
     return CL_OK;
 }
 

@@ -281,3 +281,30 @@ def test_tensor_core_pass_matches_streaming_pass(monkeypatch):
         assert np.array_equal(out[0][i][0], out[1][i][0])
     scale = max(1.0, float(np.abs(out[0][3]).max()))
     assert np.abs(out[0][3] - out[1][3]).max() <= 2 ** -7 * scale        # taps: one bf16 ulp at the top of the range
+
+
+def test_interval_search_matches_oracle_on_c1():
+    """Section 3.3 driver: same rounds, scores, sets and tokens as the oracle's loop on the fp32 model."""
+    w = synth.WORKLOADS["C1"]
+    P, K, max_new, interval, max_rounds = 8, 3, 60, 4, 3
+    sh = dataclasses.replace(w.shape, max_seq=128)
+    om, ctx, Wh = make_pair(sh, w.seed, tap_positions=P)
+    prompt = synth.make_prompt(w.seed, w.prompt_len, sh.vocab)
+    oc = SelectConfig(n_layers=sh.n_layers, lo=w.lo, hi=w.hi, n_skip=1)
+    sc = cl.SelectCfg.make(w.lo, w.hi, n_skip=1)
+    for initial, goal in (([1, 2], 10.0), ([2], 0.0), ([], 3.0)):
+        ref = oracle.generate_search(om, Wh, prompt, initial, K, max_new, interval, goal, max_rounds, oc, P)
+        van = oracle.generate_vanilla(om, prompt, max_new)
+        first = ctx.cl_prefill(prompt, tap_hidden=True)
+        ctx.cl_set_skip_set(synth.layers_to_mask(initial, sh.n_layers))
+        got = ctx.cl_generate_search(K, max_new - 1, interval, goal, max_rounds, sc)
+        toks = [first] + [int(t) for t in got["tokens"]]
+        lim = next((i for i, m in enumerate(van["margins"]) if m < 1e-4), max_new)   # fp32 both sides: only a real tie may differ
+        assert toks[:lim] == ref["tokens"][:lim]
+        if lim < max_new:
+            continue
+        # the oracle emits the prefill's token inside its count; the library's loop starts after it
+        ref2 = oracle.generate_search(om, Wh, prompt, initial, K, max_new, interval, goal, max_rounds, oc, P)
+        assert got["scores"] == pytest.approx(ref2["scores"], abs=1e-6)
+        assert got["sets"] == ref2["sets"] and got["best_round"] == ref2["best_round"]
+        assert got["final_set"] == ref2["final_set"] and got["searching"] == ref2["searching"]

@@ -241,3 +241,38 @@ def test_score_loop_keeps_best_round_earliest_on_ties():
     out = oracle.score_loop(cs, [1.0, 3.0, 3.0, 2.0, 0.5], cfg)
     assert out["best_iter"] == 1 and out["best_set"] == select_skip_set(cs[1], cfg)
     assert len(out["sets"]) == 5
+
+
+# ---------------------------------------------------------------- interval-based periodic search (Section 3.3)
+
+def _search(c1, initial, K=3, max_new=60, interval=4, goal=10.0, max_rounds=3, P=8):
+    w, W, prompt = c1
+    om = oracle.OracleModel(w.shape, W)
+    cfg = SelectConfig(n_layers=w.shape.n_layers, lo=w.lo, hi=w.hi, n_skip=1)
+    out = oracle.generate_search(om, W, prompt, initial, K, max_new, interval, goal, max_rounds, cfg, P)
+    van = oracle.generate_vanilla(om, prompt, max_new)
+    om.close()
+    return out, van
+
+
+def test_search_is_lossless_halts_and_keeps_the_best_round(c1):
+    out, van = _search(c1, [1, 2])
+    assert out["tokens"] == van["tokens"]                              # the search never changes the output
+    assert 1 <= len(out["scores"]) <= 3 + 1 and not out["searching"]   # initial set + at most max_rounds searched sets
+    best = int(np.argmax(out["scores"]))                               # first maximum: ties keep the earlier set
+    assert out["best_round"] == best and out["best_set"] == out["sets"][best]
+    assert out["final_set"] == out["best_set"]
+    assert all(0.0 <= s <= 3.0 for s in out["scores"])                 # mean accepted per cycle lies in [0, K]
+    for s in out["sets"][1:]:
+        assert len(s) == 1 and s[0] in (1, 2)                          # searched sets come from the selection rule
+
+
+def test_search_goal_and_interval_edges(c1):
+    out, _ = _search(c1, [2], goal=0.0)                                # any score reaches a goal of 0: round 0 ends it
+    assert len(out["scores"]) == 1 and out["final_set"] == [2] and not out["searching"]
+    out, _ = _search(c1, [], K=3, goal=3.0)                            # empty skip set: every draft accepted, score = K
+    assert out["scores"] == [3.0] and out["final_set"] == []
+    out, _ = _search(c1, [1], interval=1000)                           # the interval never completes: no search check
+    assert out["scores"] == [] and out["searching"] and out["final_set"] == [1]
+    out, _ = _search(c1, [1], max_rounds=0)                            # no searched set allowed: only the initial one is scored
+    assert len(out["scores"]) == 1 and out["final_set"] == [1]
