@@ -230,9 +230,9 @@ void orc_lm_head(const orc_model *m, const float *hidden, int n, float *logits) 
 }
 
 /*
- * Run n tokens, at cache positions pos0 .. pos0+n-1, through every layer whose skip_mask byte
- * is 0 (a byte of 3 leaves the residual stream and that layer's KV entries untouched; NULL
- * mask = full model).  Each row attends causally to cache positions <= its own.  Row t's
+ * Run n tokens, at cache positions pos0 .. pos0+n-1, through the layers.  skip_mask byte per layer: bit 0 skips
+ * the attention half (the stream and that layer's KV entries stay untouched), bit 1 skips the FFN half; 3 skips the
+ * whole layer; NULL mask = full model.  Each row attends causally to cache positions <= its own.  Row t's
  * arithmetic does not depend on n: running rows one at a time gives the same bits.
  *   logits_out [n,V] or NULL; hid_attn / hid_ffn [L,n,d] or NULL: the residual stream after
  *   each layer's attention add / FFN add, rounded to the storage type (skipped layers: zeros).
@@ -262,7 +262,8 @@ int orc_forward(orc_model *m, const uint8_t *skip_mask, const int32_t *tokens, i
 
     for (int l = 0; l < c->n_layers; ++l) {
         size_t tapoff = (size_t)l * nd;
-        if (skip_mask && skip_mask[l]) {
+        const int skip_attn = skip_mask && (skip_mask[l] & 1), skip_ffn = skip_mask && (skip_mask[l] & 2);
+        if (skip_attn && skip_ffn) {
             if (hid_attn) memset(hid_attn + tapoff, 0, sizeof(float) * nd);
             if (hid_ffn) memset(hid_ffn + tapoff, 0, sizeof(float) * nd);
             continue;
@@ -271,6 +272,7 @@ int orc_forward(orc_model *m, const uint8_t *skip_mask, const int32_t *tokens, i
         float *vc = m->vcache + (size_t)l * c->max_seq * d;
 
         /* attention half */
+        if (!skip_attn) {
         for (int t = 0; t < n; ++t) orc_rmsnorm(x + (size_t)t * d, m->norm1[l], d, c->rms_eps, r + (size_t)t * d);
         orc_matmul_rows(m->wq[l], dt, d, d, r, n, q);
         orc_matmul_rows(m->wk[l], dt, d, d, r, n, k);
@@ -293,16 +295,19 @@ int orc_forward(orc_model *m, const uint8_t *skip_mask, const int32_t *tokens, i
                                    a + (size_t)t * d + h * hd);
         orc_matmul_rows(m->wo[l], dt, d, d, a, n, o);
         for (size_t i = 0; i < nd; ++i) x[i] += o[i];
+        }
         if (hid_attn)
             for (size_t i = 0; i < nd; ++i) hid_attn[tapoff + i] = store_round(x[i], dt);
 
         /* FFN half */
+        if (!skip_ffn) {
         for (int t = 0; t < n; ++t) orc_rmsnorm(x + (size_t)t * d, m->norm2[l], d, c->rms_eps, r + (size_t)t * d);
         orc_matmul_rows(m->wg[l], dt, F, d, r, n, g);
         orc_matmul_rows(m->wu[l], dt, F, d, r, n, u);
         for (size_t i = 0; i < (size_t)n * F; ++i) g[i] = (float)(orc_silu((double)g[i]) * (double)u[i]);
         orc_matmul_rows(m->wd[l], dt, d, F, g, n, o);
         for (size_t i = 0; i < nd; ++i) x[i] += o[i];
+        }
         if (hid_ffn)
             for (size_t i = 0; i < nd; ++i) hid_ffn[tapoff + i] = store_round(x[i], dt);
     }

@@ -209,6 +209,33 @@ def test_skipped_layer_leaves_stream_and_cache_untouched():
     assert np.array_equal(out["logits"], lg3)
 
 
+def test_half_layer_skips_equal_zeroed_output_projections():
+    """Skipping only the attention (FFN) half of a layer gives the logits of the model whose attention output
+    (FFN down) projection in that layer is zero; the skipped attention half leaves its KV entries untouched."""
+    w = synth.WORKLOADS["C1"]
+    sh = w.shape
+    W = synth.make_weights(sh, w.seed)
+    p = synth.make_prompt(3, 7, sh.vocab)
+    for bits, key in ((1, "wo"), (2, "wd")):
+        mask = np.zeros(sh.n_layers, np.uint8)
+        mask[1] = bits
+        m = oracle.OracleModel(sh, W)
+        got = m.forward(p, 0, mask)["logits"]
+        kv_touched = bool(np.any(m.read_kv(1, 0, 2) != 0))
+        assert kv_touched == (bits == 2)
+        Wz = dict(W)
+        Wz[key] = [t if l != 1 else torch.zeros_like(t) for l, t in enumerate(W[key])]
+        want = oracle.OracleModel(sh, Wz).forward(p, 0)["logits"]
+        assert np.array_equal(got, want)
+    both = np.zeros(sh.n_layers, np.uint8)
+    both[1] = 3
+    m1 = oracle.OracleModel(sh, W).forward(p, 0, both)["logits"]
+    Wz = dict(W)
+    for key in ("wo", "wd"):
+        Wz[key] = [t if l != 1 else torch.zeros_like(t) for l, t in enumerate(W[key])]
+    assert np.array_equal(m1, oracle.OracleModel(sh, Wz).forward(p, 0)["logits"])
+
+
 def test_bf16_storage_rounds_cache_and_taps():
     import dataclasses
     sh = dataclasses.replace(synth.WORKLOADS["C1"].shape, weight_dtype="bf16")
