@@ -85,7 +85,7 @@ typedef struct {
     uint64_t accepted;   /* candidate tokens accepted (alpha = accepted / drafted, M = accepted / cycles) */
     uint64_t emitted;    /* tokens emitted by cycles (accepted + one target token per cycle) */
     int ctx_len;         /* committed KV-cache length */
-    int n_skipped;       /* |S| (beta = n_skipped / n_layers) */
+    int n_skipped;       /* |S|: layers skipped as a whole (beta = n_skipped / n_layers) */
     uint64_t kernel_launches;  /* kernels launched by this context so far */
 } cl_stats;
 
@@ -109,9 +109,9 @@ int cl_destroy(cl_ctx *ctx);
  * token of the first cycle.  tap_hidden != 0 records the hidden-state ring while doing so. */
 int cl_prefill(cl_ctx *ctx, const int32_t *tokens, int n, int tap_hidden, int32_t *first_token);
 
-/* Skip set S as a byte per layer: bit0 = skip attention, bit1 = skip FFN; only 0 (kept) and
- * 3 (whole layer skipped) are accepted.  Skipped layers stream no weights and leave their KV
- * entries untouched in draft steps. */
+/* Skip set S as a byte per layer: bit 0 = skip the attention half, bit 1 = skip the FFN half, 3 = the whole
+ * layer (Section 3.1 scores both modules of a layer; the paper's own sets are whole layers).  A skipped half
+ * streams no weights in draft steps; a skipped attention half leaves the layer's KV entries untouched. */
 int cl_set_skip_set(cl_ctx *ctx, const uint8_t *mask /* host [n_layers] */);
 int cl_get_skip_set(cl_ctx *ctx, uint8_t *mask /* host [n_layers] */);
 

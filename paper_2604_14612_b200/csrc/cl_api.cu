@@ -455,8 +455,10 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
     if (c->use_tc && !mask) return forward_rows_tc(c, tok, T, row0, tap, want_head, out_tok, out_pmax, out_conf, logits);
     KL(cl_launch_embed(wd, c->embed, tok, T, d, c->x, c->st, c->stream));
     for (int l = 0; l < g.n_layers; ++l) {
-        if (mask && mask[l]) continue;
+        const int skip_bits = mask ? mask[l] : 0;
+        if (skip_bits == 3) continue;
         const ClLayer &y = c->layers[l];
+        if (!(skip_bits & 1)) {
         // attention half: RMSNorm -> QKV -> rotary + cache append -> attention over the cache -> output projection + residual
         KL(cl_launch_rmsnorm(c->x, y.n1, T, d, g.rms_eps, c->xn, c->st, c->stream));
         if ((rc = gemv(c, T, CL_EPI_STORE, y.wqkv, 3 * d, d, c->xn, c->qkv, 3 * d))) return rc;
@@ -468,10 +470,13 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
         a.nsplit = c->nsplit; a.per_max = c->per_max; a.max_seq = g.max_seq;
         KL(cl_launch_attn(wd, T, a, c->stream));
         if ((rc = gemv(c, T, CL_EPI_RESID, y.wo, d, d, c->att, c->x, d))) return rc;
+        }
+        if (!(skip_bits & 2)) {
         // FFN half: RMSNorm -> gate/up + SiLU -> down projection + residual
         KL(cl_launch_rmsnorm(c->x, y.n2, T, d, g.rms_eps, c->xn, c->st, c->stream));
         if ((rc = gemv(c, T, CL_EPI_SILU, y.wgu, 2 * F, d, c->xn, c->hff, F))) return rc;
         if ((rc = gemv(c, T, CL_EPI_RESID, y.wd, d, F, c->hff, c->x, d))) return rc;
+        }
         if (tap && c->ring)
             KL(cl_launch_tap(wd, c->x, T, row0, d, c->ring + (size_t)l * g.tap_positions * d * c->esz, g.tap_positions, c->st,
                              c->stream));
@@ -609,13 +614,12 @@ extern "C" int cl_prefill(cl_ctx *c, const int32_t *tokens, int n, int tap_hidde
 extern "C" int cl_set_skip_set(cl_ctx *c, const uint8_t *mask) {
     if (!c || !mask) return fail(c, CL_EINVAL, "cl_set_skip_set: null argument");
     for (int l = 0; l < c->cfg.n_layers; ++l)
-        if (mask[l] != 0 && mask[l] != 3)
-            return fail(c, CL_EINVAL, "cl_set_skip_set: layer %d has mask %d; only 0 (kept) and 3 (whole layer) are supported", l, mask[l]);
+        if (mask[l] > 3) return fail(c, CL_EINVAL, "cl_set_skip_set: layer %d has mask %d; bits 0 and 1 only", l, mask[l]);
     c->mask.assign(mask, mask + c->cfg.n_layers);
     if (c->kept_dev) {
         std::vector<int> kept;
         for (int l = 0; l < c->cfg.n_layers; ++l)
-            if (!mask[l]) kept.push_back(l);
+            if (mask[l] != 3) kept.push_back(l | ((int)mask[l] << 16));
         CU(cudaStreamSynchronize(c->stream));
         if (!kept.empty()) CU(cudaMemcpy(c->kept_dev, kept.data(), kept.size() * sizeof(int), cudaMemcpyHostToDevice));
         c->n_kept = (int)kept.size();
@@ -1080,7 +1084,7 @@ extern "C" int cl_get_stats(cl_ctx *c, cl_stats *out) {
         out->emitted = c->h_st->emitted_total;
         out->ctx_len = c->h_st->ctx;
     }
-    for (uint8_t m : c->mask) out->n_skipped += (m != 0);
+    for (uint8_t m : c->mask) out->n_skipped += (m == 3);   // whole layers (half-skipped layers are not counted)
     out->kernel_launches = c->launches;
     return CL_OK;
 }

@@ -80,7 +80,8 @@ enum { CL_STEP_DRAFT = 0, CL_STEP_VANILLA = 1 };
 
 struct ClStepArgs {
     const ClLayerDev *layers;   // device [n_layers]
-    const int *kept;            // device [n_kept] indices of the layers that run
+    const int *kept;            // device [n_kept]: layer index | flags << 16 of the layers that run at least in part
+                                // (flag bit 0: attention half skipped, bit 1: FFN half skipped)
     int n_kept;
     const void *embed, *lm_head;
     const float *final_norm;

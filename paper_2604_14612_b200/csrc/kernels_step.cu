@@ -298,8 +298,9 @@ struct SchedIter {
     size_t rowbytes;
     const char *W;
     ClLayerDev L;
+    int lk;                 // kept-list position L was loaded for (-1: none)
     bool done;
-    __device__ SchedIter(const ClStepArgs &args) : a(args), step(0), ki(0), m(0), done(false) {
+    __device__ SchedIter(const ClStepArgs &args) : a(args), step(0), ki(0), m(0), lk(-1), done(false) {
         if (a.n_steps <= 0) done = true;
         else open();
     }
@@ -307,7 +308,12 @@ struct SchedIter {
         for (;;) {
             int rows, cols, unit = 1;
             if (ki < a.n_kept) {
-                if (m == 0) L = a.layers[a.kept[ki]];
+                const int ent = a.kept[ki], fl = ent >> 16;   // layer | flags << 16: bit 0 no attention half, bit 1 no FFN half
+                if ((m < 2 && (fl & 1)) || (m >= 2 && (fl & 2))) {
+                    if (!advance()) return;
+                    continue;
+                }
+                if (lk != ki) { L = a.layers[ent & 0xffff]; lk = ki; }
                 if (m == 0) { W = L.wqkv; rows = 3 * a.d; cols = a.d; }
                 else if (m == 1) { W = L.wo; rows = a.d; cols = a.d; }
                 else if (m == 2) { W = L.wgu; rows = 2 * a.F; cols = a.d; unit = 2; }
@@ -860,7 +866,9 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
         }
         grid_barrier(a.bar, bar_target, sm, st);
         for (int ki = 0; ki < a.n_kept; ++ki) {
-            const ClLayerDev L = a.layers[a.kept[ki]];
+            const int ent = a.kept[ki], fl = ent >> 16;   // bit 0: this layer's attention half is skipped, bit 1: its FFN half
+            const ClLayerDev L = a.layers[ent & 0xffff];
+            if (!(fl & 1)) {
             // QKV projection of the normalised stream (the attention phase's cache lines are requested now)
             attention_prefetch<WT, HD>(a, L, pos);
             load_x_rmsnorm<EPC>(a.x, L.n1, d, a.eps, xr, sm);
@@ -876,6 +884,8 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
                 for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
             });
             grid_barrier(a.bar, bar_target, sm, st);
+            }
+            if (!(fl & 2)) {
             // gate/up projections (rows interleaved) + SiLU(gate) * up
             load_x_rmsnorm<EPC>(a.x, L.n2, d, a.eps, xr, sm);
             consume_matrix<WT>(2 * F, d, 2, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
@@ -891,6 +901,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
                 for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
             });
             grid_barrier(a.bar, bar_target, sm, st);
+            }
         }
         // LM head on the normalised stream, fused with clamp + online softmax / entropy / argmax
         load_x_rmsnorm<EPC>(a.x, a.final_norm, d, a.eps, xr, sm);

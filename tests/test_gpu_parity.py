@@ -218,7 +218,7 @@ def test_edge_cases_and_errors():
         ctx.cl_generate(4, 30)
     assert e.value.code == 5
     with pytest.raises(cl.ConfLayersError) as e:
-        ctx.cl_set_skip_set([1, 0, 0, 0])
+        ctx.cl_set_skip_set([4, 0, 0, 0])
     assert e.value.code == 1
     with pytest.raises(cl.ConfLayersError) as e:
         ctx.cl_prefill([V])
@@ -308,3 +308,22 @@ def test_interval_search_matches_oracle_on_c1():
         assert got["scores"] == pytest.approx(ref2["scores"], abs=1e-6)
         assert got["sets"] == ref2["sets"] and got["best_round"] == ref2["best_round"]
         assert got["final_set"] == ref2["final_set"] and got["searching"] == ref2["searching"]
+
+
+@pytest.mark.parametrize("name,L,mask", [("C1", 4, [0, 1, 2, 0]), ("C1", 4, [0, 3, 1, 2]), ("C3", 4, [0, 2, 1, 0])])
+def test_half_layer_skip_sets(name, L, mask):
+    """Attention-only and FFN-only skips (mask bits 0 and 1) in draft steps, lock-step against the oracle."""
+    w0 = synth.WORKLOADS[name]
+    w = synth.reduced(w0, n_layers=L, prompt_len=min(w0.prompt_len, 24), gen_len=10)
+    om, ctx, _ = make_pair(w.shape, w.seed, gen_device="cuda" if name != "C1" else "cpu")
+    prompt = synth.make_prompt(w.seed, w.prompt_len, w.shape.vocab)
+    rep = lockstep_generate(om, ctx, prompt, np.array(mask, np.uint8), 3, w.gen_len)
+    assert rep.cycles > 0
+    # the fallback path (one launch per kernel) takes the same bits
+    import os
+    os.environ["CL_DISABLE_STEP_KERNEL"] = "1"
+    try:
+        om2, ctx2, _ = make_pair(w.shape, w.seed, gen_device="cuda" if name != "C1" else "cpu")
+        lockstep_generate(om2, ctx2, prompt, np.array(mask, np.uint8), 3, w.gen_len)
+    finally:
+        os.environ.pop("CL_DISABLE_STEP_KERNEL", None)
