@@ -33,6 +33,7 @@ typedef struct {
     int n_layers, d_model, n_heads, head_dim, d_ffn, vocab, max_seq;
     float rms_eps, rope_theta;
     int weight_dtype; /* 0 = fp32, 1 = bf16 (also the storage type of KV cache and taps) */
+    int n_kv_heads;   /* key/value heads (grouped-query attention): query head h reads key/value head h / (n_heads / n_kv_heads) */
 } orc_cfg;
 
 typedef struct {
@@ -41,7 +42,7 @@ typedef struct {
     const float *final_norm;
     const void **wq, **wk, **wv, **wo, **wg, **wu, **wd;
     const float **norm1, **norm2;
-    float *kcache, *vcache; /* [L][max_seq][d], values already rounded to the storage type */
+    float *kcache, *vcache; /* [L][max_seq][n_kv_heads * head_dim], values already rounded to the storage type */
 } orc_model;
 
 /* ---- storage-type helpers ------------------------------------------------------------ */
@@ -205,7 +206,7 @@ orc_model *orc_create(const orc_cfg *c, const void *embed, const void *lm_head, 
     m->wd = dup_ptrs(wd, L);
     m->norm1 = (const float **)dup_ptrs((const void *const *)norm1, L);
     m->norm2 = (const float **)dup_ptrs((const void *const *)norm2, L);
-    size_t kv = (size_t)L * c->max_seq * c->d_model;
+    size_t kv = (size_t)L * c->max_seq * c->n_kv_heads * c->head_dim;
     m->kcache = (float *)calloc(kv, sizeof(float));
     m->vcache = (float *)calloc(kv, sizeof(float));
     return m;
@@ -242,7 +243,9 @@ int orc_forward(orc_model *m, const uint8_t *skip_mask, const int32_t *tokens, i
                 float *logits_out, float *hid_attn, float *hid_ffn) {
     const orc_cfg *c = &m->c;
     int d = c->d_model, H = c->n_heads, hd = c->head_dim, F = c->d_ffn, dt = c->weight_dtype;
-    if (n <= 0 || pos0 < 0 || pos0 + n > c->max_seq || H * hd != d) return -1;
+    int Hkv = c->n_kv_heads, kvd = Hkv * hd;   /* keys and values have n_kv_heads heads: [n, kvd] */
+    if (n <= 0 || pos0 < 0 || pos0 + n > c->max_seq || H * hd != d || Hkv < 1 || H % Hkv) return -1;
+    int group = H / Hkv;
     for (int t = 0; t < n; ++t)
         if (tokens[t] < 0 || tokens[t] >= c->vocab) return -1;
 
@@ -268,31 +271,29 @@ int orc_forward(orc_model *m, const uint8_t *skip_mask, const int32_t *tokens, i
             if (hid_ffn) memset(hid_ffn + tapoff, 0, sizeof(float) * nd);
             continue;
         }
-        float *kc = m->kcache + (size_t)l * c->max_seq * d;
-        float *vc = m->vcache + (size_t)l * c->max_seq * d;
+        float *kc = m->kcache + (size_t)l * c->max_seq * kvd;
+        float *vc = m->vcache + (size_t)l * c->max_seq * kvd;
 
         /* attention half */
         if (!skip_attn) {
         for (int t = 0; t < n; ++t) orc_rmsnorm(x + (size_t)t * d, m->norm1[l], d, c->rms_eps, r + (size_t)t * d);
         orc_matmul_rows(m->wq[l], dt, d, d, r, n, q);
-        orc_matmul_rows(m->wk[l], dt, d, d, r, n, k);
-        orc_matmul_rows(m->wv[l], dt, d, d, r, n, v);
+        orc_matmul_rows(m->wk[l], dt, kvd, d, r, n, k);
+        orc_matmul_rows(m->wv[l], dt, kvd, d, r, n, v);
         for (int t = 0; t < n; ++t) {
             int pos = pos0 + t;
-            for (int h = 0; h < H; ++h) {
-                orc_rope(q + (size_t)t * d + h * hd, hd, pos, c->rope_theta);
-                orc_rope(k + (size_t)t * d + h * hd, hd, pos, c->rope_theta);
-            }
-            for (int i = 0; i < d; ++i) {
-                kc[(size_t)pos * d + i] = store_round(k[(size_t)t * d + i], dt);
-                vc[(size_t)pos * d + i] = store_round(v[(size_t)t * d + i], dt);
+            for (int h = 0; h < H; ++h) orc_rope(q + (size_t)t * d + h * hd, hd, pos, c->rope_theta);
+            for (int h = 0; h < Hkv; ++h) orc_rope(k + (size_t)t * kvd + h * hd, hd, pos, c->rope_theta);
+            for (int i = 0; i < kvd; ++i) {
+                kc[(size_t)pos * kvd + i] = store_round(k[(size_t)t * kvd + i], dt);
+                vc[(size_t)pos * kvd + i] = store_round(v[(size_t)t * kvd + i], dt);
             }
         }
 #pragma omp parallel for collapse(2) schedule(static)
         for (int t = 0; t < n; ++t)
             for (int h = 0; h < H; ++h)
-                orc_attention_head(q + (size_t)t * d + h * hd, kc + h * hd, vc + h * hd, pos0 + t + 1, hd, d,
-                                   a + (size_t)t * d + h * hd);
+                orc_attention_head(q + (size_t)t * d + h * hd, kc + (h / group) * hd, vc + (h / group) * hd, pos0 + t + 1, hd,
+                                   kvd, a + (size_t)t * d + h * hd);
         orc_matmul_rows(m->wo[l], dt, d, d, a, n, o);
         for (size_t i = 0; i < nd; ++i) x[i] += o[i];
         }
@@ -320,6 +321,7 @@ int orc_forward(orc_model *m, const uint8_t *skip_mask, const int32_t *tokens, i
 
 /* Read back one cached K or V row (tests of the cache contract). */
 void orc_read_kv(const orc_model *m, int layer, int which, int pos, float *out) {
-    const float *src = (which ? m->vcache : m->kcache) + ((size_t)layer * m->c.max_seq + pos) * m->c.d_model;
-    memcpy(out, src, sizeof(float) * (size_t)m->c.d_model);
+    const size_t kvd = (size_t)m->c.n_kv_heads * m->c.head_dim;
+    const float *src = (which ? m->vcache : m->kcache) + ((size_t)layer * m->c.max_seq + pos) * kvd;
+    memcpy(out, src, sizeof(float) * kvd);
 }

@@ -21,7 +21,7 @@ EPS_H = 1.0e-10    # epsilon inside the log of Eq. 2 (the paper gives no value)
 
 class _Cfg(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab", "max_seq")] + \
-               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("weight_dtype", C.c_int)]
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("weight_dtype", C.c_int), ("n_kv_heads", C.c_int)]
 
 
 def build_oracle(force: bool = False) -> str:
@@ -109,7 +109,7 @@ class OracleModel:
             return arr
 
         cfg = _Cfg(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
-                   shape.max_seq, shape.rms_eps, shape.rope_theta, wd)
+                   shape.max_seq, shape.rms_eps, shape.rope_theta, wd, getattr(shape, "kv_heads", shape.n_heads))
         lists = [ptr_list(n) for n in ("wq", "wk", "wv", "wo", "wg", "wu", "wd", "norm1", "norm2")]
         self._h = lib().orc_create(C.byref(cfg), hold("embed", weights["embed"]), hold("lm_head", weights["lm_head"]),
                                    hold("final_norm", weights["final_norm"]), *lists)
@@ -148,6 +148,6 @@ class OracleModel:
         return out
 
     def read_kv(self, layer: int, which: int, pos: int) -> np.ndarray:
-        out = np.empty(self.d, np.float32)
+        out = np.empty(getattr(self.shape, "kv_heads", self.shape.n_heads) * self.shape.head_dim, np.float32)
         lib().orc_read_kv(self._h, layer, which, pos, _ptr(out))
         return out

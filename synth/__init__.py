@@ -40,10 +40,15 @@ class ModelShape:
     rope_theta: float = 10000.0
     std: float = 0.02
     lm_head_scale: float = 1.0
+    n_kv_heads: int = 0                 # key/value heads of grouped-query attention (0: same as n_heads)
 
     @property
     def head_dim(self) -> int:
         return self.d_model // self.n_heads
+
+    @property
+    def kv_heads(self) -> int:
+        return self.n_kv_heads or self.n_heads
 
 
 @dataclasses.dataclass(frozen=True)
@@ -105,7 +110,7 @@ def make_weights(shape: ModelShape, seed: int, device="cpu") -> Dict[str, object
     """Random-init Llama-style decoder weights, every matrix stored (out, in) row-major.
 
     Returns a dict: embed [V,d], lm_head [V,d], final_norm fp32[d], and per-layer lists
-    wq, wk, wv, wo [d,d], wg, wu [F,d], wd [d,F], norm1, norm2 fp32[d] (gains = 1).
+    wq, wo [d,d], wk, wv [kv_heads*head_dim, d], wg, wu [F,d], wd [d,F], norm1, norm2 fp32[d] (gains = 1).
     """
     dt = torch_dtype(shape.weight_dtype)
     L, d, F, V = shape.n_layers, shape.d_model, shape.d_ffn, shape.vocab
@@ -114,8 +119,9 @@ def make_weights(shape: ModelShape, seed: int, device="cpu") -> Dict[str, object
         "lm_head": _normal((V, d), shape.std * shape.lm_head_scale, seed, _T_HEAD, dt, device),
         "final_norm": torch.ones(d, dtype=torch.float32, device=device),
     }
+    kvd = shape.kv_heads * shape.head_dim
     names = ("wq", "wk", "wv", "wo", "wg", "wu", "wd")
-    dims = ((d, d), (d, d), (d, d), (d, d), (F, d), (F, d), (d, F))
+    dims = ((d, d), (kvd, d), (kvd, d), (d, d), (F, d), (F, d), (d, F))
     for n in names + ("norm1", "norm2"):
         w[n] = []
     for l in range(L):

@@ -255,3 +255,24 @@ def test_bad_arguments_are_rejected():
         m.forward([w.shape.vocab], 0)
     with pytest.raises(ValueError):
         m.forward([1, 2], w.shape.max_seq - 1)
+
+
+def test_grouped_query_attention_equals_replicated_kv_heads():
+    """A model with n_kv_heads < n_heads gives the logits of the multi-head model whose K and V projections repeat
+    every key/value head for its group of query heads; n_kv_heads = n_heads is the multi-head model itself."""
+    import dataclasses
+    w = synth.WORKLOADS["C1"]
+    sh_g = dataclasses.replace(w.shape, n_kv_heads=2)          # 4 query heads, 2 key/value heads
+    Wg = synth.make_weights(sh_g, 7)
+    hd, group = sh_g.head_dim, sh_g.n_heads // 2
+    Wm = dict(Wg)
+    for key in ("wk", "wv"):
+        Wm[key] = [t.view(2, hd, -1).repeat_interleave(group, dim=0).reshape(sh_g.d_model, -1).contiguous() for t in Wg[key]]
+    p = synth.make_prompt(4, 9, sh_g.vocab)
+    mask = synth.layers_to_mask([2], sh_g.n_layers)
+    got = oracle.OracleModel(sh_g, Wg).forward(p, 0, mask)["logits"]
+    want = oracle.OracleModel(w.shape, Wm).forward(p, 0, mask)["logits"]
+    assert np.array_equal(got, want)
+    same = oracle.OracleModel(dataclasses.replace(w.shape, n_kv_heads=w.shape.n_heads), Wm).forward(p, 0, mask)["logits"]
+    assert np.array_equal(same, want)
+    assert oracle.OracleModel(sh_g, Wg).read_kv(0, 0, 0).shape[0] == 2 * hd
