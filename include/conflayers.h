@@ -20,7 +20,8 @@
  *   - Matrices are row-major (out_features, in_features), as Llama checkpoints store them.
  *     weight_dtype selects the storage type of weights, KV cache and hidden-state taps:
  *     0 = fp32, 1 = bf16.  Norm gains are always fp32.  Arithmetic accumulates in fp32.
- *   - Requirements: d_model = n_heads * head_dim, n_kv_heads = n_heads (multi-head attention),
+ *   - Requirements: d_model = n_heads * head_dim, n_kv_heads divides n_heads (n_kv_heads < n_heads: grouped-query
+ *     attention, query head h reads key/value head h / (n_heads / n_kv_heads)),
  *     head_dim in {64, 128}, d_model and d_ffn multiples of 8, 1 <= K <= CL_MAX_K.
  */
 #ifndef CONFLAYERS_H
@@ -57,7 +58,7 @@ typedef struct {
     const void *embed;                /* [vocab, d_model] */
     const void *lm_head;              /* [vocab, d_model] (shared by all early exits) */
     const float *final_norm;          /* [d_model] */
-    const void *const *wq, *const *wk, *const *wv, *const *wo;   /* n_layers pointers, each [d_model, d_model] */
+    const void *const *wq, *const *wk, *const *wv, *const *wo;   /* n_layers pointers; wq, wo [d_model, d_model], wk, wv [n_kv_heads * head_dim, d_model] */
     const void *const *wg, *const *wu;                           /* each [d_ffn, d_model] */
     const void *const *wd;                                       /* each [d_model, d_ffn] */
     const float *const *norm1, *const *norm2;                    /* each [d_model] */

@@ -153,9 +153,9 @@ class Context:
 
     def __init__(self, n_layers: int, d_model: int, n_heads: int, d_ffn: int, vocab: int, max_seq: int,
                  weight_dtype: str = "bf16", rms_eps: float = 1e-5, rope_theta: float = 10000.0,
-                 tap_positions: int = 0, stream: Optional[int] = None):
+                 tap_positions: int = 0, stream: Optional[int] = None, n_kv_heads: int = 0):
         self._L = load_library()
-        self.cfg = ModelCfg(n_layers, d_model, n_heads, n_heads, d_model // n_heads, d_ffn, vocab, max_seq, rms_eps,
+        self.cfg = ModelCfg(n_layers, d_model, n_heads, n_kv_heads or n_heads, d_model // n_heads, d_ffn, vocab, max_seq, rms_eps,
                             rope_theta, 1 if weight_dtype == "bf16" else 0, tap_positions)
         self.weight_dtype = weight_dtype
         self._h = C.c_void_p()
@@ -169,7 +169,8 @@ class Context:
     @classmethod
     def from_shape(cls, shape, tap_positions: int = 0, stream: Optional[int] = None) -> "Context":
         return cls(shape.n_layers, shape.d_model, shape.n_heads, shape.d_ffn, shape.vocab, shape.max_seq,
-                   shape.weight_dtype, shape.rms_eps, shape.rope_theta, tap_positions, stream)
+                   shape.weight_dtype, shape.rms_eps, shape.rope_theta, tap_positions, stream,
+                   getattr(shape, "kv_heads", shape.n_heads))
 
     # -- helpers
     def _ck(self, rc: int):

@@ -162,7 +162,8 @@ extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **ou
     if (cfg->n_layers < 0 || cfg->d_model <= 0 || cfg->n_heads <= 0 || cfg->vocab < 2 || cfg->max_seq <= 0)
         return fail(c, CL_EINVAL, "cl_create: non-positive dimension");
     if (cfg->n_heads * cfg->head_dim != cfg->d_model) return fail(c, CL_EINVAL, "cl_create: d_model != n_heads * head_dim");
-    if (cfg->n_kv_heads != cfg->n_heads) return fail(c, CL_EINVAL, "cl_create: only n_kv_heads == n_heads is supported");
+    if (cfg->n_kv_heads < 1 || cfg->n_heads % cfg->n_kv_heads)
+        return fail(c, CL_EINVAL, "cl_create: n_kv_heads must be at least 1 and divide n_heads");
     if (cfg->head_dim != 64 && cfg->head_dim != 128) return fail(c, CL_EINVAL, "cl_create: head_dim must be 64 or 128");
     if (cfg->d_model % 8 || (cfg->n_layers > 0 && (cfg->d_ffn <= 0 || cfg->d_ffn % 8)))
         return fail(c, CL_EINVAL, "cl_create: d_model and d_ffn must be multiples of 8");
@@ -227,6 +228,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
     if (c->loaded) return fail(c, CL_ESTATE, "cl_load: weights already loaded");
     const cl_model_cfg &g = c->cfg;
     const size_t d = g.d_model, F = g.d_ffn, V = g.vocab, L = g.n_layers, es = c->esz;
+    const size_t kvd = (size_t)g.n_kv_heads * g.head_dim, qkv_rows = d + 2 * kvd;   // [q | k | v] rows of the fused projection
     c->head_only = w->head_only ? 1 : 0;
     if (!w->lm_head || !w->final_norm) return fail(c, CL_EINVAL, "cl_load: lm_head / final_norm missing");
     if (!c->head_only) {
@@ -260,13 +262,13 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
 
     if (!c->head_only) {
         // ---- weights: per layer [Wqkv | Wo | Wgu | Wd], contiguous in execution order
-        const size_t b_qkv = 3 * d * d * es, b_o = d * d * es, b_gu = 2 * F * d * es, b_d = d * F * es;
+        const size_t b_qkv = qkv_rows * d * es, b_o = d * d * es, b_gu = 2 * F * d * es, b_d = d * F * es;
         const size_t per_layer = b_qkv + b_o + b_gu + b_d;
         DM(c->wbuf, per_layer * L);
         DM(c->norms, 2 * L * d * 4);
         DM(c->embed, V * d * es);
         CU(cudaMemcpyAsync(c->embed, w->embed, V * d * es, kind, c->stream));
-        const size_t kv_layer = (size_t)g.max_seq * d * es;
+        const size_t kv_layer = (size_t)g.max_seq * kvd * es;
         DM(c->kv, 2 * L * kv_layer);
         CU(cudaMemsetAsync(c->kv, 0, 2 * L * kv_layer, c->stream));
         char *stage_g = nullptr, *stage_u = nullptr;
@@ -286,8 +288,8 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
             y.kc = c->kv + (2 * l) * kv_layer;
             y.vc = c->kv + (2 * l + 1) * kv_layer;
             CU(cudaMemcpyAsync(y.wqkv, w->wq[l], d * d * es, kind, c->stream));
-            CU(cudaMemcpyAsync(y.wqkv + d * d * es, w->wk[l], d * d * es, kind, c->stream));
-            CU(cudaMemcpyAsync(y.wqkv + 2 * d * d * es, w->wv[l], d * d * es, kind, c->stream));
+            CU(cudaMemcpyAsync(y.wqkv + d * d * es, w->wk[l], kvd * d * es, kind, c->stream));
+            CU(cudaMemcpyAsync(y.wqkv + (d + kvd) * d * es, w->wv[l], kvd * d * es, kind, c->stream));
             CU(cudaMemcpyAsync(y.wo, w->wo[l], b_o, kind, c->stream));
             CU(cudaMemcpyAsync(y.wd, w->wd[l], b_d, kind, c->stream));
             CU(cudaMemcpyAsync(y.n1, w->norm1[l], d * 4, kind, c->stream));
@@ -313,7 +315,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
         CU(cudaMemcpyAsync(c->rope_cs, cs.data(), cs.size() * sizeof(float2), cudaMemcpyHostToDevice, c->stream));
         // ---- activations and scratch
         DM(c->x, (size_t)CL_MAX_T * d * 4);
-        DM(c->qkv, (size_t)CL_MAX_T * 3 * d * 4);
+        DM(c->qkv, (size_t)CL_MAX_T * qkv_rows * 4);
         DM(c->att, (size_t)CL_MAX_T * d * 4);
         DM(c->hff, (size_t)CL_MAX_T * F * 4);
         c->nsplit = 4;
@@ -367,7 +369,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 const size_t MT = (rows + 127) / 128, KB = (K + 63) / 64, U = MT * KB, upc = (U + G - 1) / G;
                 return (upc + KB - 1) / KB + 1 <= (size_t)CL_V_MAXSEG;
             };
-            bool ok = !(off && off[0] == '1') && segs_ok(3 * d, d) && segs_ok(d, d) && segs_ok(2 * F, d) && segs_ok(d, F) &&
+            bool ok = !(off && off[0] == '1') && segs_ok(qkv_rows, d) && segs_ok(d, d) && segs_ok(2 * F, d) && segs_ok(d, F) &&
                       segs_ok(V, d);
             if (ok) {
                 DM(c->bx, 32 * d * 2);
@@ -377,7 +379,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 CU(cudaMemsetAsync(c->batt, 0, 32 * d * 2, c->stream));
                 CU(cudaMemsetAsync(c->bh, 0, 32 * F * 2, c->stream));
                 DM(c->v_ws, (size_t)G * CL_V_MAXSEG * 128 * 32 * 4);
-                const size_t max_tiles = (std::max(std::max(3 * d, 2 * F), V) + 127) / 128;
+                const size_t max_tiles = (std::max(std::max(qkv_rows, 2 * F), V) + 127) / 128;
                 DM(c->v_tickets, max_tiles * 4);
                 CU(cudaMemsetAsync(c->v_tickets, 0, max_tiles * 4, c->stream));
                 DM(c->v_ssq, ((d + 127) / 128) * CL_SLOTS * 4);
@@ -389,7 +391,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 c->map_qkv.resize(L); c->map_o.resize(L); c->map_gu.resize(L); c->map_d.resize(L);
                 for (size_t l = 0; l < L && ok; ++l) {
                     const ClLayer &y = c->layers[l];
-                    ok = cl_make_tensor_map(&c->map_qkv[l], y.wqkv, (int)(3 * d), (int)d, 128) &&
+                    ok = cl_make_tensor_map(&c->map_qkv[l], y.wqkv, (int)qkv_rows, (int)d, 128) &&
                          cl_make_tensor_map(&c->map_o[l], y.wo, (int)d, (int)d, 128) &&
                          cl_make_tensor_map(&c->map_gu[l], y.wgu, (int)(2 * F), (int)d, 128) &&
                          cl_make_tensor_map(&c->map_d[l], y.wd, (int)d, (int)F, 128);
@@ -450,7 +452,7 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
 static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_t *mask, int tap, int want_head,
                         int *out_tok, float *out_pmax, float *out_conf, float *logits) {
     const cl_model_cfg &g = c->cfg;
-    const int d = g.d_model, F = g.d_ffn, wd = g.weight_dtype;
+    const int d = g.d_model, F = g.d_ffn, wd = g.weight_dtype, qkv_rows = d + 2 * g.n_kv_heads * g.head_dim;
     int rc;
     if (c->use_tc && !mask) return forward_rows_tc(c, tok, T, row0, tap, want_head, out_tok, out_pmax, out_conf, logits);
     KL(cl_launch_embed(wd, c->embed, tok, T, d, c->x, c->st, c->stream));
@@ -461,11 +463,11 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
         if (!(skip_bits & 1)) {
         // attention half: RMSNorm -> QKV -> rotary + cache append -> attention over the cache -> output projection + residual
         KL(cl_launch_rmsnorm(c->x, y.n1, T, d, g.rms_eps, c->xn, c->st, c->stream));
-        if ((rc = gemv(c, T, CL_EPI_STORE, y.wqkv, 3 * d, d, c->xn, c->qkv, 3 * d))) return rc;
-        KL(cl_launch_rope_append(wd, c->qkv, T, row0, g.n_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq, c->st,
+        if ((rc = gemv(c, T, CL_EPI_STORE, y.wqkv, qkv_rows, d, c->xn, c->qkv, qkv_rows))) return rc;
+        KL(cl_launch_rope_append(wd, c->qkv, T, row0, g.n_heads, g.n_kv_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq, c->st,
                                  c->stream));
         ClAttnArgs a;
-        a.q = c->qkv; a.ld_q = 3 * d; a.kcache = y.kc; a.vcache = y.vc; a.part = c->att_part; a.tickets = c->tickets + 1;
+        a.q = c->qkv; a.ld_q = qkv_rows; a.n_kv_heads = g.n_kv_heads; a.kcache = y.kc; a.vcache = y.vc; a.part = c->att_part; a.tickets = c->tickets + 1;
         a.out = c->att; a.out_b = nullptr; a.nh = 0; a.st = c->st; a.row0 = row0; a.n_heads = g.n_heads; a.head_dim = g.head_dim; a.d_model = d;
         a.nsplit = c->nsplit; a.per_max = c->per_max; a.max_seq = g.max_seq;
         KL(cl_launch_attn(wd, T, a, c->stream));
@@ -493,7 +495,7 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
 static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, int want_head, int *out_tok, float *out_pmax,
                            float *out_conf, float *logits) {
     const cl_model_cfg &g = c->cfg;
-    const int d = g.d_model, F = g.d_ffn, V = g.vocab, L = g.n_layers, G = c->n_sm;
+    const int d = g.d_model, F = g.d_ffn, V = g.vocab, L = g.n_layers, G = c->n_sm, qkv_rows = d + 2 * g.n_kv_heads * g.head_dim;
     const int N = T <= 8 ? 16 : 32, nh = N / 2, sel = N == 16 ? 0 : 1;
     const int KBd = (d + 63) / 64, KBf = (F + 63) / 64, dtiles = (d + 127) / 128;
     ClSkinnyArgs b;
@@ -504,11 +506,11 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
     for (int l = 0; l < L; ++l) {
         const ClLayer &y = c->layers[l];
         ClSkinnyArgs a = b;
-        a.rows = 3 * d; a.KB = KBd; a.epi = CL_VEPI_STORE; a.ssq_in = c->v_ssq; a.out = c->qkv; a.ld = 3 * d;
+        a.rows = qkv_rows; a.KB = KBd; a.epi = CL_VEPI_STORE; a.ssq_in = c->v_ssq; a.out = c->qkv; a.ld = qkv_rows;
         KL(cl_launch_skinny(c->map_qkv[l], c->map_bx[sel], a, G, c->stream));
-        KL(cl_launch_rope_append(1, c->qkv, T, row0, g.n_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq, c->st, c->stream));
+        KL(cl_launch_rope_append(1, c->qkv, T, row0, g.n_heads, g.n_kv_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq, c->st, c->stream));
         ClAttnArgs t;
-        t.q = c->qkv; t.ld_q = 3 * d; t.kcache = y.kc; t.vcache = y.vc; t.part = c->att_part; t.tickets = c->tickets + 1;
+        t.q = c->qkv; t.ld_q = qkv_rows; t.n_kv_heads = g.n_kv_heads; t.kcache = y.kc; t.vcache = y.vc; t.part = c->att_part; t.tickets = c->tickets + 1;
         t.out = c->att; t.out_b = c->batt; t.nh = nh; t.st = c->st; t.row0 = row0; t.n_heads = g.n_heads; t.head_dim = g.head_dim;
         t.d_model = d; t.nsplit = c->nsplit; t.per_max = c->per_max; t.max_seq = g.max_seq;
         t.part = c->v_att_part;
@@ -550,7 +552,7 @@ static int run_steps(cl_ctx *c, int mode, int n_steps, int row0, bool full_model
     a.kept = full_model ? c->kept_all_dev : c->kept_dev;
     a.n_kept = full_model ? g.n_layers : c->n_kept;
     a.embed = c->embed; a.lm_head = c->lm_head; a.final_norm = c->final_norm;
-    a.d = g.d_model; a.F = g.d_ffn; a.V = g.vocab; a.H = g.n_heads; a.max_seq = g.max_seq;
+    a.d = g.d_model; a.F = g.d_ffn; a.V = g.vocab; a.H = g.n_heads; a.Hkv = g.n_kv_heads; a.max_seq = g.max_seq;
     a.att_parts = c->att_parts; a.l2_ahead = c->l2_ahead;
     a.eps = g.rms_eps; a.inv_log_v = (float)(1.0 / log((double)g.vocab));
     a.rope_cs = c->rope_cs; a.st = c->st;

@@ -66,7 +66,7 @@ struct ClAttnArgs {
     __nv_bfloat16 *out_b; // optional [2 * nh, d]: the output again as bf16 hi (row t) and lo (row nh + t) parts
     int nh;
     const ClDevState *st;
-    int row0, n_heads, head_dim, d_model, nsplit, per_max, max_seq;
+    int row0, n_heads, n_kv_heads, head_dim, d_model, nsplit, per_max, max_seq;
 };
 
 // Per-layer device pointers as the token-step kernel sees them.
@@ -85,13 +85,13 @@ struct ClStepArgs {
     int n_kept;
     const void *embed, *lm_head;
     const float *final_norm;
-    int d, F, V, H, max_seq;
+    int d, F, V, H, Hkv, max_seq;        // Hkv: key/value heads (grouped-query attention), H % Hkv == 0
     int att_parts;                       // S: parts the cached keys of a head are cut into (1 .. 8), one CTA each
     int l2_ahead;                        // bytes per CTA the weight prefetch into L2 runs in front of the ring
     float eps, inv_log_v;
     const float2 *rope_cs;
     ClDevState *st;
-    float *x, *qkv, *hff;                // global activation vectors [d] [3d] [F]
+    float *x, *qkv, *hff;                // global activation vectors [d] [d + 2 Hkv hd] [F]
     float *att_part;                     // [H, 8, hd + 4] per-part attention records (max, sum, -, -, o[hd])
     ClHeadPartial *head_part;            // [grid]
     unsigned *bar;                       // grid barrier: arrival counter, zero at launch
@@ -115,7 +115,7 @@ cudaError_t cl_launch_rmsnorm(const float *x, const float *g, int T, int d, floa
                               cudaStream_t s);
 cudaError_t cl_launch_rmsnorm_rows(int in_dtype, const void *x, const float *g, int T, int d, float eps, float *out,
                                    cudaStream_t s);
-cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H, int hd, int d, const float2 *rope_cs,
+cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H, int Hkv, int hd, int d, const float2 *rope_cs,
                                   void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_attn(int wdtype, int T, const ClAttnArgs &a, cudaStream_t s);
 size_t cl_attn_rows_part_floats(int H, int S, int T, int hd);

@@ -61,22 +61,26 @@ __global__ void k_rmsnorm(const ST *x, const float *g, int d, float eps, float *
 }
 
 // ---- rotary embedding of q and k (pairs (i, i + hd/2)), append k, v to the cache -----------
-// qkv: [T, 3d] fp32 = [q | k | v]; q is rotated in place; k (rotated) and v go to the cache rows
-// of positions ctx + row0 + t, rounded to the storage type.
+// qkv: [T, d + 2 kvd] fp32 = [q (H heads) | k (Hkv heads) | v (Hkv heads)]; q is rotated in place; k (rotated) and
+// v go to the cache rows of positions ctx + row0 + t, rounded to the storage type.  grid (T, H): block h rotates
+// query head h and, if h < Hkv, appends key/value head h.
 template <typename ST>
-__global__ void k_rope_append(float *qkv, int row0, int hd, int d, const float2 *rope_cs, ST *kcache, ST *vcache,
+__global__ void k_rope_append(float *qkv, int row0, int hd, int d, int Hkv, const float2 *rope_cs, ST *kcache, ST *vcache,
                               int max_seq, const ClDevState *st) {
     if (st->done) return;
     const int t = blockIdx.x, h = blockIdx.y, i = threadIdx.x, half = hd >> 1;
     const int pos = st->ctx + row0 + t;
     if (pos >= max_seq) return;
-    float *q = qkv + (size_t)t * 3 * d + h * hd;
-    float *k = q + d;
-    const float *v = q + 2 * d;
+    const int kvd = Hkv * hd;
+    float *row = qkv + (size_t)t * (d + 2 * kvd);
+    float *q = row + h * hd;
     const float2 cs = rope_cs[(size_t)pos * half + i];
-    const float qa = q[i], qb = q[i + half], ka = k[i], kb = k[i + half];
+    const float qa = q[i], qb = q[i + half];
     q[i] = qa * cs.x - qb * cs.y;
     q[i + half] = qb * cs.x + qa * cs.y;
+    if (h >= Hkv) return;
+    const float *k = row + d + h * hd, *v = row + d + kvd + h * hd;
+    const float ka = k[i], kb = k[i + half];
     ST *kc = kcache + ((size_t)h * max_seq + pos) * hd;   // cache layout [head][position][hd]: a head's rows are contiguous
     ST *vc = vcache + ((size_t)h * max_seq + pos) * hd;
     kc[i] = from_f32<ST>(ka * cs.x - kb * cs.y);
@@ -105,8 +109,9 @@ __global__ void __launch_bounds__(128) k_attn(ClAttnArgs a) {
     const int j0 = min(nkeys, sp * per), j1 = min(nkeys, j0 + per);
     const int n = j1 - j0;
     const int d = a.d_model;
-    const ST *K = (const ST *)a.kcache + (size_t)h * a.max_seq * HD;
-    const ST *V = (const ST *)a.vcache + (size_t)h * a.max_seq * HD;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);   // grouped-query attention: the key/value head of this query head
+    const ST *K = (const ST *)a.kcache + (size_t)kvh * a.max_seq * HD;
+    const ST *V = (const ST *)a.vcache + (size_t)kvh * a.max_seq * HD;
     const float scale = rsqrtf((float)HD);
 
     for (int i = tid; i < HD; i += blockDim.x) sq[i] = a.q[(size_t)t * a.ld_q + h * HD + i];
@@ -412,13 +417,13 @@ cudaError_t cl_launch_rmsnorm_rows(int in_dtype, const void *x, const float *g, 
     return cudaGetLastError();
 }
 
-cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H, int hd, int d, const float2 *rope_cs,
+cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H, int Hkv, int hd, int d, const float2 *rope_cs,
                                   void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s) {
     dim3 grid(T, H);
     CL_DISPATCH_ST(wdtype,
-                   (k_rope_append<__nv_bfloat16><<<grid, hd / 2, 0, s>>>(qkv, row0, hd, d, rope_cs, (__nv_bfloat16 *)kcache,
+                   (k_rope_append<__nv_bfloat16><<<grid, hd / 2, 0, s>>>(qkv, row0, hd, d, Hkv, rope_cs, (__nv_bfloat16 *)kcache,
                                                                          (__nv_bfloat16 *)vcache, max_seq, st)),
-                   (k_rope_append<float><<<grid, hd / 2, 0, s>>>(qkv, row0, hd, d, rope_cs, (float *)kcache,
+                   (k_rope_append<float><<<grid, hd / 2, 0, s>>>(qkv, row0, hd, d, Hkv, rope_cs, (float *)kcache,
                                                                  (float *)vcache, max_seq, st)));
     return cudaGetLastError();
 }

@@ -314,7 +314,7 @@ struct SchedIter {
                     continue;
                 }
                 if (lk != ki) { L = a.layers[ent & 0xffff]; lk = ki; }
-                if (m == 0) { W = L.wqkv; rows = 3 * a.d; cols = a.d; }
+                if (m == 0) { W = L.wqkv; rows = a.d + 2 * a.Hkv * (a.d / a.H); cols = a.d; }
                 else if (m == 1) { W = L.wo; rows = a.d; cols = a.d; }
                 else if (m == 2) { W = L.wgu; rows = 2 * a.F; cols = a.d; unit = 2; }
                 else { W = L.wd; rows = a.d; cols = a.F; }
@@ -611,7 +611,7 @@ __device__ __forceinline__ void attention_prefetch(const ClStepArgs &a, const Cl
     constexpr int LINES = (ROWB + 127) / 128;
     const int n = (kw1 - kw0) * LINES;
     for (int i = lane; i < n; i += 32) {
-        const size_t off = ((size_t)h * a.max_seq + kw0 + i / LINES) * HD * sizeof(ST) + (size_t)(i % LINES) * 128;
+        const size_t off = ((size_t)(h / (a.H / a.Hkv)) * a.max_seq + kw0 + i / LINES) * HD * sizeof(ST) + (size_t)(i % LINES) * 128;
         l2_prefetch_line(L.kc + off);
         l2_prefetch_line(L.vc + off);
     }
@@ -628,9 +628,10 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
     const float scale = rsqrtf((float)HD);
     ST *Kc = (ST *)L.kc;
     ST *Vc = (ST *)L.vc;
+    const int group = a.H / a.Hkv, kvd = a.Hkv * HD;   // grouped-query attention: `group` query heads share a key/value head
     float *wrec = sm->partial;   // [NCW][WSTRIDE]
     for (int item = blockIdx.x; item < a.H * S; item += gridDim.x) {
-        const int h = item % a.H, s = item / a.H;
+        const int h = item % a.H, s = item / a.H, kvh = h / group;
         int kw0, kw1;
         warp_key_range(pos, s, S, warp, kw0, kw1);
         const float *qraw = a.qkv + h * HD;
@@ -656,7 +657,7 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
                 const int j = jb + sub;
                 float sc = 0.f;
                 if (j < n) {
-                    const uint4 raw = __ldcg((const uint4 *)(Kc + ((size_t)h * a.max_seq + j0 + j) * HD + li * EPL));
+                    const uint4 raw = __ldcg((const uint4 *)(Kc + ((size_t)kvh * a.max_seq + j0 + j) * HD + li * EPL));
                     if (sizeof(ST) == 2) {
                         const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -696,7 +697,7 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
             for (int j = 0; j < 32; ++j) {
                 const float pj = __shfl_sync(0xffffffffu, p, j);
                 float vv[VPL];
-                load_vals<ST, VPL>(Vc + ((size_t)h * a.max_seq + j0 + min(j, n - 1)) * HD + lane * VPL, vv);
+                load_vals<ST, VPL>(Vc + ((size_t)kvh * a.max_seq + j0 + min(j, n - 1)) * HD + lane * VPL, vv);
 #pragma unroll
                 for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(pj, vv[e], o_run[e]);
             }
@@ -704,7 +705,8 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
         if (s == S - 1 && warp == NCW - 1) {
             // the new position: rotate this step's key, round key and value to the storage type, append both to the
             // cache and fold them in as one more key
-            const float *kraw = a.qkv + d + h * HD, *vraw = a.qkv + 2 * d + h * HD;
+            const float *kraw = a.qkv + d + kvh * HD, *vraw = a.qkv + d + kvd + kvh * HD;
+            const bool owner = (h % group) == 0;   // one query head of the group appends the shared key/value head
             float sc = 0.f;
             ST kst[EPL];
 #pragma unroll
@@ -719,15 +721,15 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
 #pragma unroll
             for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
             sc = __shfl_sync(0xffffffffu, sc, 0) * scale;
-            if (sub == 0) {
+            if (sub == 0 && owner) {
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) Kc[((size_t)h * a.max_seq + pos) * HD + li * EPL + e] = kst[e];
+                for (int e = 0; e < EPL; ++e) Kc[((size_t)kvh * a.max_seq + pos) * HD + li * EPL + e] = kst[e];
             }
             float vn[VPL];
 #pragma unroll
             for (int e = 0; e < VPL; ++e) {
                 const ST vs = st_from_f32<ST>(ldcg_f(vraw + lane * VPL + e));
-                Vc[((size_t)h * a.max_seq + pos) * HD + lane * VPL + e] = vs;
+                if (owner) Vc[((size_t)kvh * a.max_seq + pos) * HD + lane * VPL + e] = vs;
                 vn[e] = st_to_f32<ST>(vs);
             }
             const float m_new = fmaxf(m_run, sc);
@@ -872,7 +874,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             // QKV projection of the normalised stream (the attention phase's cache lines are requested now)
             attention_prefetch<WT, HD>(a, L, pos);
             load_x_rmsnorm<EPC>(a.x, L.n1, d, a.eps, xr, sm);
-            consume_matrix<WT>(3 * d, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
+            consume_matrix<WT>(d + 2 * a.Hkv * HD, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.qkv[rb0 + r] = row_sum(sm, r);
             });
             grid_barrier(a.bar, bar_target, sm, st);

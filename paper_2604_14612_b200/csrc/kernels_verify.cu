@@ -504,8 +504,9 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
     const int kw0 = k0 + (k1 - k0) * warp / AR_WARPS, kw1 = k0 + (k1 - k0) * (warp + 1) / AR_WARPS;
     const int sub = lane / LPK, li = lane % LPK;
     const float scale = rsqrtf((float)HD);
-    const ST *Kc = (const ST *)a.kcache + (size_t)h * a.max_seq * HD;   // cache layout [head][position][hd]
-    const ST *Vc = (const ST *)a.vcache + (size_t)h * a.max_seq * HD;
+    const int kvh = h / (a.n_heads / a.n_kv_heads);                       // grouped-query attention
+    const ST *Kc = (const ST *)a.kcache + (size_t)kvh * a.max_seq * HD;   // cache layout [kv head][position][hd]
+    const ST *Vc = (const ST *)a.vcache + (size_t)kvh * a.max_seq * HD;
 
     float qr[T][EPL];
 #pragma unroll

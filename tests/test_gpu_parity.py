@@ -398,3 +398,30 @@ def test_c3_full_depth_against_oracle():
     mask = synth.layers_to_mask(synth.uniform_skip_layers(w.lo, w.hi, n_skip), 32)
     rep = lockstep_generate(om, ctx, prompt, mask, 4, w.gen_len, tol=4e-2, near_tie=4e-2)
     print("C3 full depth", rep)
+
+
+@pytest.mark.parametrize("name,L,kv,K", [("C1", 4, 2, 3), ("C1", 4, 1, 4), ("C2", 3, 4, 4), ("C3", 3, 8, 8)])
+def test_grouped_query_attention(name, L, kv, K):
+    """n_kv_heads < n_heads (LLaMA-3 / 70B style): draft steps, verify pass, prefill and taps against the oracle."""
+    w0 = synth.WORKLOADS[name]
+    w = synth.reduced(w0, n_layers=L, prompt_len=min(w0.prompt_len, 21), gen_len=9)
+    sh = dataclasses.replace(w.shape, n_kv_heads=kv)
+    P = 8
+    om, ctx, _ = make_pair(sh, w.seed + 11, tap_positions=P, gen_device="cuda" if name == "C3" else "cpu")
+    prompt = synth.make_prompt(w.seed, w.prompt_len, sh.vocab)
+    mask = synth.layers_to_mask([1], L)
+    rep = lockstep_generate(om, ctx, prompt, mask, K, w.gen_len, tap=True)
+    assert rep.cycles > 0
+    got = ring_in_position_order(ctx.cl_read_hidden_ring(), ctx.cl_get_stats().ctx_len - 1)
+    assert np.isfinite(got).all()
+    # free-running generation on the device is lossless with grouped heads too
+    first = ctx.cl_prefill(prompt)
+    van, _ = ctx.cl_generate(0, 12)
+    ctx.cl_prefill(prompt)
+    ctx.cl_set_skip_set(mask)
+    spec, _ = ctx.cl_generate(K, 12)
+    ref = oracle.generate_vanilla(om, prompt, 13)
+    lim = next((i for i, m in enumerate(ref["margins"]) if m < NEAR_TIE), 13)
+    if lim >= 1:
+        assert [first] + list(van[:lim - 1]) == ref["tokens"][:lim]
+        assert list(spec[:lim - 1]) == list(van[:lim - 1])
