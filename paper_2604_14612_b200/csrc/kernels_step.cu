@@ -81,14 +81,9 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
     }
 }
 
-__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
 
-// The same copy, marking the lines evict-first in L2: streamed weights are used once per token.
+// Bulk asynchronous copy global -> shared (completion counted in bytes on an mbarrier), marking the lines
+// evict-first in L2: streamed weights are used once per token.
 __device__ __forceinline__ void bulk_g2s_stream(void *dst, const void *src, unsigned bytes, unsigned long long *bar,
                                                 unsigned long long policy) {
     asm volatile(
