@@ -52,6 +52,8 @@ typedef struct {
     float rms_eps, rope_theta;
     int weight_dtype;    /* 0 fp32, 1 bf16 */
     int tap_positions;   /* P: ring of the last P positions' per-layer hidden states (0 = no ring) */
+    int tap_modules;     /* 0 or 1: record each layer's output (after the FFN add); 2: also the stream after the attention add
+                            (Section 3.1 scores "FFNN and Attention" hidden states); a layer's confidence = mean over its taps */
 } cl_model_cfg;
 
 typedef struct {
@@ -157,7 +159,7 @@ int cl_force_tokens(cl_ctx *ctx, const int32_t *toks, int n);
  * RMSNorm and the shared LM head; logits are clamped in fp32; per row the entropy confidence
  * 1 - H/log(vocab), the top-1 probability and the greedy token are reduced on the fly (logits are
  * never stored).  hidden: DEVICE pointer [rows, P, d_model] in the model's storage type, or NULL to
- * score the context's own ring (rows = n_layers, P = tap_positions, most recent positions).
+ * score the context's own ring (rows = n_layers, P = taps * tap_positions with taps = 1 or 2, see tap_modules).
  * Outputs (host, may be NULL): conf_rows, p_max, argmax [rows, P]; c_layer [rows] = mean over P. */
 int cl_layer_confidences(cl_ctx *ctx, const void *hidden, int rows, int P, float *conf_rows, float *p_max,
                          int32_t *argmax, float *c_layer);
@@ -197,8 +199,9 @@ typedef struct {
 int cl_generate_search(cl_ctx *ctx, const cl_search_cfg *cfg, const cl_select_cfg *sel, int max_new, int32_t *out,
                        int *n_out, cl_search_report *rep, uint8_t *masks);
 
-/* Copy the hidden-state ring to the host: out is [n_layers, tap_positions, d_model] in the storage
- * type, position slot = absolute position modulo tap_positions. */
+/* Copy the hidden-state ring to the host: out is [n_layers, taps, tap_positions, d_model] in the storage type
+ * (taps = 2: index 0 after the attention add, 1 after the FFN add), position slot = absolute position modulo
+ * tap_positions. */
 int cl_read_hidden_ring(cl_ctx *ctx, void *out);
 
 /* Confidence scoring for callers that cannot allocate device memory.  The paper has no counterpart of

@@ -33,23 +33,26 @@ def _mask_of(layers: Sequence[int], n_layers: int) -> np.ndarray:
 
 def generate_search(model, weights: Dict[str, object], prompt: Sequence[int], initial_set: Sequence[int], K: int,
                     max_new: int, interval: int, score_goal: float, max_rounds: int, select_cfg: SelectConfig,
-                    P: int, storage_dtype=None) -> Dict[str, object]:
+                    P: int, storage_dtype=None, taps: int = 1) -> Dict[str, object]:
     """Returns tokens (max_new of them, the first being the prefill's), per-round scores and sets, the best round
     and the set in use at the end.  `weights` supplies lm_head and final_norm for the confidence scoring;
-    `storage_dtype` (a torch dtype or None) is the type the ring rounds hidden states to."""
+    `storage_dtype` (a torch dtype or None) is the type the ring rounds hidden states to.  taps = 2 also records the
+    stream after each layer's attention add (Section 3.1 names both modules); a layer's confidence is then the mean
+    over both taps and all positions."""
     import torch
     L, d = model.L, model.d
     t0, _, pre = prefill(model, prompt, want_hidden=True)
-    ring = np.zeros((L, P, d), np.float32)
+    ring = np.zeros((L, taps, P, d), np.float32)
 
-    def store(hid, pos0):   # hid [L, n, d]: rows at positions pos0 ..
-        h = torch.tensor(hid)
-        if storage_dtype is not None:
-            h = h.to(storage_dtype).float()
-        for i in range(hid.shape[1]):
-            ring[:, (pos0 + i) % P, :] = h[:, i, :].numpy()
+    def store(fwd, pos0):   # fwd: forward dict with hid_attn / hid_ffn [L, n, d]: rows at positions pos0 ..
+        for ti, key in enumerate(("hid_attn", "hid_ffn") if taps == 2 else ("hid_ffn",)):
+            h = torch.tensor(fwd[key])
+            if storage_dtype is not None:
+                h = h.to(storage_dtype).float()
+            for i in range(h.shape[1]):
+                ring[:, ti, (pos0 + i) % P, :] = h[:, i, :].numpy()
 
-    store(pre["hid_ffn"], 0)
+    store(pre, 0)
     out = [t0]
     ctx = len(prompt)
     cur = sorted(int(l) for l in initial_set)
@@ -61,7 +64,7 @@ def generate_search(model, weights: Dict[str, object], prompt: Sequence[int], in
     while len(out) < max_new:
         cyc = speculative_cycle(model, _mask_of(cur, L), out[-1], ctx, K, want_hidden=searching)
         if searching:
-            store(cyc["hid_ffn"], ctx)
+            store(cyc, ctx)
         out.extend(cyc["emitted"])
         ctx = cyc["new_ctx"]
         if not searching:
@@ -79,7 +82,7 @@ def generate_search(model, weights: Dict[str, object], prompt: Sequence[int], in
             searching = False
             cur = list(best_set)
         else:
-            h = torch.tensor(ring)
+            h = torch.tensor(ring.reshape(L, taps * P, d))
             if storage_dtype is not None:
                 h = h.to(storage_dtype)
             c = layer_confidences(h, weights["lm_head"], weights["final_norm"], model.shape.rms_eps)["c_layer"]

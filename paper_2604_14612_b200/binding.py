@@ -24,7 +24,8 @@ class ConfLayersError(RuntimeError):
 class ModelCfg(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab",
                                        "max_seq")] + \
-               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("weight_dtype", C.c_int), ("tap_positions", C.c_int)]
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("weight_dtype", C.c_int), ("tap_positions", C.c_int),
+                ("tap_modules", C.c_int)]
 
 
 class Weights(C.Structure):
@@ -153,10 +154,11 @@ class Context:
 
     def __init__(self, n_layers: int, d_model: int, n_heads: int, d_ffn: int, vocab: int, max_seq: int,
                  weight_dtype: str = "bf16", rms_eps: float = 1e-5, rope_theta: float = 10000.0,
-                 tap_positions: int = 0, stream: Optional[int] = None, n_kv_heads: int = 0):
+                 tap_positions: int = 0, stream: Optional[int] = None, n_kv_heads: int = 0, tap_modules: int = 1):
         self._L = load_library()
         self.cfg = ModelCfg(n_layers, d_model, n_heads, n_kv_heads or n_heads, d_model // n_heads, d_ffn, vocab, max_seq, rms_eps,
-                            rope_theta, 1 if weight_dtype == "bf16" else 0, tap_positions)
+                            rope_theta, 1 if weight_dtype == "bf16" else 0, tap_positions, tap_modules)
+        self.taps = 2 if tap_modules == 2 else 1
         self.weight_dtype = weight_dtype
         self._h = C.c_void_p()
         if stream is None:
@@ -167,10 +169,10 @@ class Context:
             raise ConfLayersError(rc, self._L.cl_last_error(None).decode())
 
     @classmethod
-    def from_shape(cls, shape, tap_positions: int = 0, stream: Optional[int] = None) -> "Context":
+    def from_shape(cls, shape, tap_positions: int = 0, stream: Optional[int] = None, tap_modules: int = 1) -> "Context":
         return cls(shape.n_layers, shape.d_model, shape.n_heads, shape.d_ffn, shape.vocab, shape.max_seq,
                    shape.weight_dtype, shape.rms_eps, shape.rope_theta, tap_positions, stream,
-                   getattr(shape, "kv_heads", shape.n_heads))
+                   getattr(shape, "kv_heads", shape.n_heads), tap_modules)
 
     # -- helpers
     def _ck(self, rc: int):
@@ -290,7 +292,7 @@ class Context:
     def cl_layer_confidences(self, hidden=None, rows: int = 0, P: int = 0):
         """hidden: CUDA tensor [rows, P, d] in the storage type, or None for the context's ring."""
         if hidden is None:
-            rows, P = self.cfg.n_layers, self.cfg.tap_positions
+            rows, P = self.cfg.n_layers, self.taps * self.cfg.tap_positions
             hp = None
         else:
             assert hidden.is_cuda and hidden.is_contiguous()
@@ -331,9 +333,9 @@ class Context:
         import torch
         L, P, d = self.cfg.n_layers, self.cfg.tap_positions, self.cfg.d_model
         dt = torch.bfloat16 if self.cfg.weight_dtype == 1 else torch.float32
-        out = torch.empty((L, P, d), dtype=dt)
+        out = torch.empty((L, self.taps, P, d), dtype=dt)
         self._ck(self._L.cl_read_hidden_ring(self._h, out.data_ptr()))
-        return out
+        return out if self.taps == 2 else out[:, 0]
 
     def cl_get_stats(self) -> Stats:
         st = Stats()

@@ -26,6 +26,7 @@ struct cl_ctx {
     int device, n_sm;
     char err[512];
     size_t esz;                   // bytes per stored element (weights, KV, taps)
+    int taps;                     // hidden states recorded per layer: 1 = after the FFN add, 2 = after the attention add and after the FFN add
     int loaded, head_only, prefilled;
     // device memory
     char *wbuf;                   // all layer matrices, one allocation, in execution order
@@ -169,6 +170,7 @@ extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **ou
         return fail(c, CL_EINVAL, "cl_create: d_model and d_ffn must be multiples of 8");
     if (cfg->weight_dtype != 0 && cfg->weight_dtype != 1) return fail(c, CL_EINVAL, "cl_create: weight_dtype must be 0 or 1");
     if (cfg->tap_positions < 0) return fail(c, CL_EINVAL, "cl_create: tap_positions < 0");
+    if (cfg->tap_modules < 0 || cfg->tap_modules > 2) return fail(c, CL_EINVAL, "cl_create: tap_modules must be 0, 1 or 2");
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(c, CL_ECUDA, "cl_create: no CUDA device: %s", cudaGetErrorString(e));
@@ -183,6 +185,7 @@ extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **ou
     c->device = dev;
     c->n_sm = prop.multiProcessorCount;
     c->esz = cfg->weight_dtype == 1 ? 2 : 4;
+    c->taps = cfg->tap_modules == 2 ? 2 : 1;
     c->err[0] = 0;
     c->mask.assign((size_t)cfg->n_layers, 0);
     *out = c;
@@ -323,8 +326,8 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
         DM(c->att_part, (size_t)CL_MAX_T * g.n_heads * c->nsplit * (g.head_dim + 2) * 4);
         DM(c->prompt_dev, (size_t)g.max_seq * 4);
         if (g.tap_positions > 0) {
-            DM(c->ring, L * (size_t)g.tap_positions * d * es);
-            CU(cudaMemsetAsync(c->ring, 0, L * (size_t)g.tap_positions * d * es, c->stream));
+            DM(c->ring, L * (size_t)c->taps * g.tap_positions * d * es);
+            CU(cudaMemsetAsync(c->ring, 0, L * (size_t)c->taps * g.tap_positions * d * es, c->stream));
         }
         // ---- token-step kernel: per-layer pointer table, kept-layer lists, barrier, attention / head partials
         {
@@ -417,6 +420,14 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
     return CL_OK;
 }
 
+// Ring [L][taps][P][d]: where layer l's tap after the attention add (which = 0) or after the FFN add (which = 1) goes;
+// null if that tap is not recorded.
+static char *ring_slot(cl_ctx *c, int l, int which) {
+    if (!c->ring || (c->taps == 1 && which == 0)) return nullptr;
+    const size_t idx = (size_t)l * c->taps + (c->taps == 2 ? which : 0);
+    return c->ring + idx * c->cfg.tap_positions * c->cfg.d_model * c->esz;
+}
+
 // ---- one pass of T rows through the kept layers ------------------------------------------------
 
 static int gemv(cl_ctx *c, int T, int epi, const void *W, int rows, int cols, const float *xin, float *out, int ld) {
@@ -473,15 +484,16 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
         KL(cl_launch_attn(wd, T, a, c->stream));
         if ((rc = gemv(c, T, CL_EPI_RESID, y.wo, d, d, c->att, c->x, d))) return rc;
         }
+        if (tap && ring_slot(c, l, 0))
+            KL(cl_launch_tap(wd, c->x, T, row0, d, ring_slot(c, l, 0), g.tap_positions, c->st, c->stream));
         if (!(skip_bits & 2)) {
         // FFN half: RMSNorm -> gate/up + SiLU -> down projection + residual
         KL(cl_launch_rmsnorm(c->x, y.n2, T, d, g.rms_eps, c->xn, c->st, c->stream));
         if ((rc = gemv(c, T, CL_EPI_SILU, y.wgu, 2 * F, d, c->xn, c->hff, F))) return rc;
         if ((rc = gemv(c, T, CL_EPI_RESID, y.wd, d, F, c->hff, c->x, d))) return rc;
         }
-        if (tap && c->ring)
-            KL(cl_launch_tap(wd, c->x, T, row0, d, c->ring + (size_t)l * g.tap_positions * d * c->esz, g.tap_positions, c->st,
-                             c->stream));
+        if (tap && ring_slot(c, l, 1))
+            KL(cl_launch_tap(wd, c->x, T, row0, d, ring_slot(c, l, 1), g.tap_positions, c->st, c->stream));
     }
     if (want_head) {
         KL(cl_launch_rmsnorm(c->x, c->final_norm, T, d, g.rms_eps, c->xn, c->st, c->stream));
@@ -518,6 +530,10 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
         a = b;
         a.rows = d; a.KB = KBd; a.epi = CL_VEPI_RESID; a.out = c->x; a.ld = d; a.bnext = c->bx; a.bn_ld = d; a.gnext = y.n2;
         a.ssq_out = c->v_ssq;
+        if (tap && ring_slot(c, l, 0)) {
+            a.tap = ring_slot(c, l, 0);
+            a.tap_P = g.tap_positions;
+        }
         KL(cl_launch_skinny(c->map_o[l], c->map_batt[sel], a, G, c->stream));
         a = b;
         a.rows = 2 * F; a.KB = KBd; a.epi = CL_VEPI_SILU; a.ssq_in = c->v_ssq; a.bnext = c->bh; a.bn_ld = F;
@@ -526,8 +542,8 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
         a.rows = d; a.KB = KBf; a.epi = CL_VEPI_RESID; a.out = c->x; a.ld = d; a.bnext = c->bx; a.bn_ld = d;
         a.gnext = (l + 1 < L) ? c->layers[l + 1].n1 : c->final_norm;
         a.ssq_out = c->v_ssq;
-        if (tap && c->ring) {
-            a.tap = c->ring + (size_t)l * g.tap_positions * d * c->esz;
+        if (tap && ring_slot(c, l, 1)) {
+            a.tap = ring_slot(c, l, 1);
             a.tap_P = g.tap_positions;
         }
         KL(cl_launch_skinny(c->map_d[l], c->map_bh[sel], a, G, c->stream));
@@ -593,7 +609,7 @@ extern "C" int cl_prefill(cl_ctx *c, const int32_t *tokens, int n, int tap_hidde
         if (tokens[i] < 0 || tokens[i] >= c->cfg.vocab) return fail(c, CL_EINVAL, "cl_prefill: token %d out of range at %d", tokens[i], i);
     CU(cudaMemcpyAsync(c->prompt_dev, tokens, (size_t)n * 4, cudaMemcpyHostToDevice, c->stream));
     if (tap_hidden && c->ring)   // a tapped prefill starts the context window afresh
-        CU(cudaMemsetAsync(c->ring, 0, (size_t)c->cfg.n_layers * c->cfg.tap_positions * c->cfg.d_model * c->esz, c->stream));
+        CU(cudaMemsetAsync(c->ring, 0, (size_t)c->cfg.n_layers * c->taps * c->cfg.tap_positions * c->cfg.d_model * c->esz, c->stream));
     ClPoke p = poke_none();
     p.ctx = 0; p.n_drafted = 0; p.done = 0;
     if ((rc = poke(c, p))) return rc;
@@ -872,7 +888,7 @@ extern "C" int cl_generate_search(cl_ctx *c, const cl_search_cfg *sc, const cl_s
             r.searching = 0;
             cur = best;
         } else {
-            if ((rc = score_rows(c, c->ring, L, P, c->sc_clayer))) return rc;
+            if ((rc = score_rows(c, c->ring, L, c->taps * P, c->sc_clayer))) return rc;
             KL(cl_launch_select(*sel, L, c->sc_clayer, c->sel_mask, nullptr, c->stream));
             CU(cudaMemcpyAsync(cur.data(), c->sel_mask, (size_t)L, cudaMemcpyDeviceToHost, c->stream));
             CU(cudaStreamSynchronize(c->stream));
@@ -974,7 +990,7 @@ extern "C" int cl_layer_confidences(cl_ctx *c, const void *hidden, int rows, int
             return fail(c, CL_ESTATE, "cl_layer_confidences: ring holds %d of %d positions", c->tapped, c->cfg.tap_positions);
         hidden = c->ring;
         rows = c->cfg.n_layers;
-        P = c->cfg.tap_positions;
+        P = c->taps * c->cfg.tap_positions;   // a layer's taps are contiguous: its confidence is the mean over taps and positions
     }
     if (rows <= 0 || P <= 0) return fail(c, CL_EINVAL, "cl_layer_confidences: rows and P must be positive");
     if (rows > c->cfg.n_layers && c->cfg.n_layers > 0) {
@@ -1070,7 +1086,7 @@ extern "C" int cl_read_hidden_ring(cl_ctx *c, void *out) {
     if (!c || !out) return fail(c, CL_EINVAL, "cl_read_hidden_ring: null argument");
     if (!c->ring) return fail(c, CL_ESTATE, "cl_read_hidden_ring: no ring (tap_positions = 0 or head-only context)");
     CU(cudaStreamSynchronize(c->stream));
-    CU(cudaMemcpy(out, c->ring, (size_t)c->cfg.n_layers * c->cfg.tap_positions * c->cfg.d_model * c->esz, cudaMemcpyDeviceToHost));
+    CU(cudaMemcpy(out, c->ring, (size_t)c->cfg.n_layers * c->taps * c->cfg.tap_positions * c->cfg.d_model * c->esz, cudaMemcpyDeviceToHost));
     return CL_OK;
 }
 

@@ -425,3 +425,44 @@ def test_grouped_query_attention(name, L, kv, K):
     if lim >= 1:
         assert [first] + list(van[:lim - 1]) == ref["tokens"][:lim]
         assert list(spec[:lim - 1]) == list(van[:lim - 1])
+
+
+@pytest.mark.parametrize("name,L", [("C1", 4), ("C2", 3)])
+def test_two_tap_confidences(name, L):
+    """tap_modules = 2: the stream after the attention add and after the FFN add of every layer is recorded (prefill
+    and verify passes) and a layer's confidence is the mean over both taps and all positions."""
+    w0 = synth.WORKLOADS[name]
+    w = synth.reduced(w0, n_layers=L, prompt_len=19, gen_len=8)
+    P = 8
+    W = synth.make_weights(w.shape, w.seed)
+    om = oracle.OracleModel(w.shape, W)
+    ctx = cl.Context.from_shape(w.shape, tap_positions=P, tap_modules=2)
+    ctx.cl_load(synth.weights_to(W, "cuda"))
+    prompt = synth.make_prompt(w.seed, w.prompt_len, w.shape.vocab)
+    first = ctx.cl_prefill(prompt, tap_hidden=True)
+    out = om.forward(prompt, 0, None, want_hidden=True, want_logits=False)
+    ring = ctx.cl_read_hidden_ring()                                  # [L, 2, P, d]
+    assert ring.shape[1] == 2
+    order = [(p % P) for p in range(len(prompt) - P, len(prompt))]
+    for ti, key in enumerate(("hid_attn", "hid_ffn")):
+        want = out[key][:, -P:, :]
+        got = ring[:, ti].float().numpy()[:, order, :]
+        scale = max(1.0, float(np.abs(want).max()))
+        assert np.abs(got - want).max() <= 2 ** -7 * scale, key
+    g = ctx.cl_layer_confidences()
+    dt = synth.torch_dtype(w.shape.weight_dtype)
+    both = np.concatenate([out["hid_attn"][:, -P:, :], out["hid_ffn"][:, -P:, :]], axis=1)    # [L, 2P, d]
+    o = oracle.layer_confidences(torch.tensor(both).to(dt), W["lm_head"], W["final_norm"], w.shape.rms_eps)
+    assert g["conf"].shape == (L, 2 * P)
+    assert np.abs(g["c_layer"] - o["c_layer"]).max() <= TOL
+    # a verify pass records both taps too
+    ctx.cl_set_skip_set(np.zeros(L, np.uint8))
+    ctx.cl_force_tokens([3, 4])
+    ctx.cl_verify(3, tap_hidden=True)
+    v = om.forward([first, 3, 4], len(prompt), None, want_hidden=True, want_logits=False)
+    ring = ctx.cl_read_hidden_ring()
+    for i in range(3):
+        slot = (len(prompt) + i) % P
+        for ti, key in enumerate(("hid_attn", "hid_ffn")):
+            want = v[key][:, i, :]
+            assert np.abs(ring[:, ti, slot].float().numpy() - want).max() <= 2 ** -7 * max(1.0, float(np.abs(want).max()))

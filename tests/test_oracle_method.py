@@ -245,11 +245,11 @@ def test_score_loop_keeps_best_round_earliest_on_ties():
 
 # ---------------------------------------------------------------- interval-based periodic search (Section 3.3)
 
-def _search(c1, initial, K=3, max_new=60, interval=4, goal=10.0, max_rounds=3, P=8):
+def _search(c1, initial, K=3, max_new=60, interval=4, goal=10.0, max_rounds=3, P=8, taps=1):
     w, W, prompt = c1
     om = oracle.OracleModel(w.shape, W)
     cfg = SelectConfig(n_layers=w.shape.n_layers, lo=w.lo, hi=w.hi, n_skip=1)
-    out = oracle.generate_search(om, W, prompt, initial, K, max_new, interval, goal, max_rounds, cfg, P)
+    out = oracle.generate_search(om, W, prompt, initial, K, max_new, interval, goal, max_rounds, cfg, P, taps=taps)
     van = oracle.generate_vanilla(om, prompt, max_new)
     om.close()
     return out, van
@@ -274,5 +274,7 @@ def test_search_goal_and_interval_edges(c1):
     assert out["scores"] == [3.0] and out["final_set"] == []
     out, _ = _search(c1, [1], interval=1000)                           # the interval never completes: no search check
     assert out["scores"] == [] and out["searching"] and out["final_set"] == [1]
+    out, van = _search(c1, [1, 2], taps=2)                             # two taps per layer: still lossless, still halts
+    assert out["tokens"] == van["tokens"] and not out["searching"]
     out, _ = _search(c1, [1], max_rounds=0)                            # no searched set allowed: only the initial one is scored
     assert len(out["scores"]) == 1 and out["final_set"] == [1]
