@@ -55,9 +55,11 @@ struct cl_ctx {
     float *sel_clayers;           // device [iters_cap, L]
     int sel_iters_cap;
     // token-step kernel (persistent single-token step)
+    float *cum_w_dev;             // [n_sm + 1] cumulative row shares of the token-step kernel's CTAs (null until calibrated)
+    unsigned long long *busy_dev; // [n_sm] calibration timings
     ClLayerDev *layers_dev;
     int *kept_dev, *kept_all_dev;
-    int n_kept, use_step, max_blk, att_parts, l2_ahead;
+    int n_kept, use_step, max_blk, att_parts, l2_ahead, cum_w_ready, calibrating;
     unsigned *bar_dev;
     float *att_part2;
     ClHeadPartial *head_part2;
@@ -197,7 +199,7 @@ static void free_all(cl_ctx *c) {
                     c->att, c->hff, c->att_part, c->logits, c->tickets, c->head_part, c->st, c->prompt_dev, c->out_dev,
                     c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sc_xn, c->sc_part, c->sel_mask, c->sel_margins, c->sel_clayers,
                     c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->head_part2,
-                    c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_att_part, c->v_tickets, c->v_head_part};
+                    c->cum_w_dev, c->busy_dev, c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_att_part, c->v_tickets, c->v_head_part};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->h_st) cudaFreeHost(c->h_st);
@@ -225,6 +227,8 @@ static cudaError_t dmalloc(T **p, size_t bytes) {
                         (size_t)(bytes), #ptr, cudaGetErrorString(e_));                                         \
         }                                                                                                       \
     } while (0)
+
+static int calibrate_row_shares(cl_ctx *c);
 
 extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
     if (!c || !w) return fail(c, CL_EINVAL, "cl_load: null argument");
@@ -413,6 +417,15 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
         CU(cudaStreamSynchronize(c->stream));   // host staging vector and borrowed pointers are released after this
         if (stage_g) cudaFree(stage_g);
         if (stage_u) cudaFree(stage_u);
+        {
+            const char *nb = getenv("CL_DISABLE_ROW_SHARES");
+            if (c->use_step && L > 0 && g.max_seq >= 2 && !(nb && nb[0] == '1')) {
+                DM(c->cum_w_dev, ((size_t)c->n_sm + 1) * sizeof(float));
+                DM(c->busy_dev, (size_t)c->n_sm * sizeof(unsigned long long));
+                int rc = calibrate_row_shares(c);
+                if (rc) return rc;
+            }
+        }
     } else {
         CU(cudaStreamSynchronize(c->stream));
     }
@@ -575,6 +588,8 @@ static int run_steps(cl_ctx *c, int mode, int n_steps, int row0, bool full_model
     a.x = c->x; a.qkv = c->qkv; a.hff = c->hff;
     a.att_part = c->att_part2; a.head_part = c->head_part2; a.bar = c->bar_dev;
     a.n_steps = n_steps; a.mode = mode; a.row0 = row0; a.out_tokens = out_tokens; a.logits = logits;
+    a.cum_w = c->cum_w_ready ? c->cum_w_dev : nullptr;
+    a.busy_ns = c->calibrating ? c->busy_dev : nullptr;
     CU(cudaMemsetAsync(c->bar_dev, 0, 2 * sizeof(unsigned), c->stream));   // the arrival counter starts at zero
     KL(cl_launch_token_steps(g.weight_dtype, g.head_dim, a, c->n_sm, c->stream));
     return CL_OK;
@@ -598,6 +613,54 @@ static int need_model(cl_ctx *c, const char *fn, bool need_prefill) {
     if (c->head_only) return fail(c, CL_ESTATE, "%s: context was loaded head-only", fn);
     if (need_prefill && !c->prefilled) return fail(c, CL_ESTATE, "%s: call cl_prefill first", fn);
     return CL_OK;
+}
+
+// One-time measurement of how fast each CTA of the token-step kernel streams (its SM's path to HBM): two full-model
+// steps from an empty cache are timed per CTA, the row shares are set in proportion to rows / time, and the measurement
+// is repeated once with the new shares.  The shares stay fixed afterwards, so results do not depend on timing.
+static int calibrate_row_shares(cl_ctx *c) {
+    const int G = c->n_sm;
+    std::vector<float> w((size_t)G, 1.0f / (float)G), cum((size_t)G + 1);
+    std::vector<unsigned long long> busy((size_t)G);
+    auto upload = [&]() -> cudaError_t {
+        double acc = 0.0, tot = 0.0;
+        for (float v : w) tot += v;
+        cum[0] = 0.f;
+        for (int b = 0; b < G; ++b) {
+            acc += w[b] / tot;
+            cum[b + 1] = (float)acc;
+        }
+        cum[G] = 1.0f;
+        return cudaMemcpy(c->cum_w_dev, cum.data(), cum.size() * sizeof(float), cudaMemcpyHostToDevice);
+    };
+    CU(upload());
+    c->cum_w_ready = 1;
+    int rc = CL_OK;
+    for (int pass = 0; pass < 3 && !rc; ++pass) {
+        CU(cudaMemsetAsync(c->st, 0, sizeof(ClDevState), c->stream));
+        CU(cudaMemsetAsync(c->busy_dev, 0, (size_t)G * sizeof(unsigned long long), c->stream));
+        c->calibrating = pass > 0;   // pass 0 warms up
+        rc = run_steps(c, CL_STEP_VANILLA, 2, 0, true, nullptr, nullptr);
+        c->calibrating = 0;
+        if (rc) break;
+        CU(cudaStreamSynchronize(c->stream));
+        if (pass == 0) continue;
+        CU(cudaMemcpy(busy.data(), c->busy_dev, busy.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+        double mean = 0.0;
+        for (unsigned long long t : busy) mean += (double)t;
+        mean /= G;
+        if (mean <= 0.0) break;
+        for (int b = 0; b < G; ++b) {
+            double f = busy[b] > 0 ? mean / (double)busy[b] : 1.0;   // faster CTA (less time for its share) -> larger share
+            if (f < 0.8) f = 0.8;
+            if (f > 1.25) f = 1.25;
+            w[b] = (float)(w[b] * f);
+        }
+        CU(upload());
+    }
+    CU(cudaMemsetAsync(c->st, 0, sizeof(ClDevState), c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    return rc;
 }
 
 extern "C" int cl_prefill(cl_ctx *c, const int32_t *tokens, int n, int tap_hidden, int32_t *first_token) {

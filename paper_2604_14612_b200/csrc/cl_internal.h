@@ -95,6 +95,8 @@ struct ClStepArgs {
     float *att_part;                     // [H, 8, hd + 4] per-part attention records (max, sum, -, -, o[hd])
     ClHeadPartial *head_part;            // [grid]
     unsigned *bar;                       // grid barrier: arrival counter, zero at launch
+    const float *cum_w;                  // [grid + 1] cumulative row shares of the CTAs (null: equal shares)
+    unsigned long long *busy_ns;         // [grid], calibration launches only: time each CTA spent in the matrix phases
     int n_steps, mode, row0;
     int *out_tokens;                     // vanilla mode: emitted tokens (may be null)
     float *logits;                       // optional [n_steps, V]

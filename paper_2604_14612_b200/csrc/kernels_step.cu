@@ -266,11 +266,19 @@ struct Ring {
     }
 };
 
-// This CTA's share of `units` row units (a unit is `unit` consecutive rows).
-__device__ __forceinline__ void my_rows(int rows, int unit, int &r0, int &r1) {
+// This CTA's share of `units` row units (a unit is `unit` consecutive rows): an equal share, or -- with a table of
+// cumulative shares cum_w[0 .. grid] (0 ... 1), measured once per context -- a share in proportion to the rate at which
+// this CTA's SM streams from HBM (SMs differ by several percent; equal rows would make every phase wait for the
+// slowest).  Which CTA computes a row never changes the row's arithmetic.
+__device__ __forceinline__ void my_rows(int rows, int unit, const float *cum_w, int &r0, int &r1) {
     const long long units = rows / unit;
-    r0 = (int)(units * blockIdx.x / gridDim.x) * unit;
-    r1 = (int)(units * (blockIdx.x + 1) / gridDim.x) * unit;
+    if (cum_w) {
+        r0 = (int)((double)units * (double)cum_w[blockIdx.x] + 0.5) * unit;
+        r1 = (int)((double)units * (double)cum_w[blockIdx.x + 1] + 0.5) * unit;
+    } else {
+        r0 = (int)(units * blockIdx.x / gridDim.x) * unit;
+        r1 = (int)(units * (blockIdx.x + 1) / gridDim.x) * unit;
+    }
 }
 
 // Rows per ring slot for a matrix with `rowbytes` bytes per row.  Phases whose epilogue pairs rows (unit 2) keep
@@ -316,7 +324,7 @@ struct SchedIter {
             } else {
                 W = (const char *)a.lm_head; rows = a.V; cols = a.d;
             }
-            my_rows(rows, unit, r, r1);
+            my_rows(rows, unit, a.cum_w, r, r1);
             rowbytes = (size_t)cols * sizeof(WT);
             rps = rows_per_slot(rowbytes, unit);
             if (r < r1) return;
@@ -488,16 +496,19 @@ __device__ __forceinline__ void consume_rows(int r0, int r1, int nchunks, int rp
 
 template <typename WT, typename Epi>
 __device__ __forceinline__ void consume_matrix(int rows, int cols, int unit, const float (&xr)[MAXIT][Chunk<WT>::EPC],
-                                               Ring &rg, const unsigned char *ring, Smem *sm, ClDevState *st, Epi epi) {
+                                               Ring &rg, const unsigned char *ring, Smem *sm, ClDevState *st, Epi epi,
+                                               const float *cum_w, unsigned long long *busy) {
     constexpr int EPC = Chunk<WT>::EPC;
     int r0, r1;
-    my_rows(rows, unit, r0, r1);
+    my_rows(rows, unit, cum_w, r0, r1);
+    const unsigned long long t_start = busy ? gtime() : 0ull;   // calibration launches only
     const int nchunks = cols / EPC;
     const int rps = rows_per_slot((size_t)nchunks * 16, unit);
     const int nit = (nchunks + NCT - 1) / NCT;   // uniform over the grid
     if (nit <= 1) consume_rows<WT, 1, 4>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
     else if (nit <= 2) consume_rows<WT, 2, 2>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
     else consume_rows<WT, 4, 1>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
+    if (busy) *busy += gtime() - t_start;
 }
 
 __device__ __forceinline__ float row_sum(const Smem *sm, int r) {
@@ -852,6 +863,8 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
     // ------------------------------ consumer warps ------------------------------
     Ring rg{0u, 0u};
     unsigned bar_target = 0u;   // arrivals that complete the next grid barrier (thread 0's copy is the one used)
+    unsigned long long busy = 0ull;   // calibration: time this CTA spent in the matrix phases
+    unsigned long long *busy_p = (a.busy_ns && tid == 0) ? &busy : nullptr;
     float xr[MAXIT][EPC];
     int tok = st->cyc_tok[a.row0];
     for (int step = 0; step < a.n_steps; ++step) {
@@ -871,7 +884,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             load_x_rmsnorm<EPC>(a.x, L.n1, d, a.eps, xr, sm);
             consume_matrix<WT>(d + 2 * a.Hkv * HD, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.qkv[rb0 + r] = row_sum(sm, r);
-            });
+            }, a.cum_w, busy_p);
             grid_barrier(a.bar, bar_target, sm, st);
             attention_phase<WT, HD>(a, L, pos, sm);
             grid_barrier(a.bar, bar_target, sm, st);
@@ -879,7 +892,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             load_att_merged<EPC, HD>(a, xr);
             consume_matrix<WT>(d, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
-            });
+            }, a.cum_w, busy_p);
             grid_barrier(a.bar, bar_target, sm, st);
             }
             if (!(fl & 2)) {
@@ -890,13 +903,13 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
                     const float gt = row_sum(sm, 2 * pr), up = row_sum(sm, 2 * pr + 1);
                     a.hff[rb0 / 2 + pr] = gt / (1.f + expf(-gt)) * up;
                 }
-            });
+            }, a.cum_w, busy_p);
             grid_barrier(a.bar, bar_target, sm, st);
             // down projection + residual
             load_x<EPC>(a.hff, F, xr);
             consume_matrix<WT>(d, F, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
-            });
+            }, a.cum_w, busy_p);
             grid_barrier(a.bar, bar_target, sm, st);
             }
         }
@@ -910,7 +923,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
                 if (lg) lg[rb0 + r] = l;
                 run = hp_merge(run, ClHeadPartial{l, 1.f, 0.f, rb0 + r});
             }
-        });
+        }, a.cum_w, busy_p);
         run = hp_block_reduce(run, sm);
         if (tid == 0) a.head_part[blockIdx.x] = run;
         grid_barrier(a.bar, bar_target, sm, st);
@@ -950,6 +963,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
         // the next step's phase 0 writes x, which nobody reads any more in this step: no barrier needed here,
         // and head_part is rewritten only after the next step's grid barriers
     }
+    if (busy_p) a.busy_ns[blockIdx.x] = busy;
 }
 
 }  // namespace
