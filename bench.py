@@ -54,6 +54,21 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def reduce_over_ranks(ms_local, dist=None, device=None):
+    """A timed region costs what its slowest rank took: MAX over ranks (one rank: the value itself)."""
+    if dist is None:
+        return float(ms_local)
+    import torch
+    t = torch.tensor([float(ms_local)], device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank, world, ms):
+    """Replicas only: every rank runs the same job, the aggregate is world x units over the slowest rank's time."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -227,11 +242,7 @@ def main():
             toks, st = step(K)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = reduce_over_ranks(e0.elapsed_time(e1), dist, "cuda")
         s1 = ctx.cl_get_stats()
         return ms, s0, s1
 
@@ -245,7 +256,7 @@ def main():
     accepted = int(s1.accepted - s0.accepted)
     drafted = int(s1.drafted - s0.drafted)
     tokens = args.steps * gen
-    value = world * tokens / (ms * 1e-3)
+    value = whole_job_value(tokens, world, ms)
 
     # bytes the timed cycles had to stream (algorithmic): K draft passes + one verify pass per cycle
     ctx_mid = w.prompt_len + gen // 2
@@ -319,11 +330,7 @@ def main():
             ctx.cl_prefill(prompt)
             toks, _ = ctx.cl_generate(K_DRAFT, gen)
         barrier()
-        dt = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([dt], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = reduce_over_ranks(time.perf_counter() - t0, dist, "cuda")
         e2e = {"value": world * n_e2e * gen / dt, "unit": "tokens/s (prefill of the 512-token prompt included)",
                "h2d_bytes_per_step": int(4 * w.prompt_len), "d2h_bytes_per_step": int(4 * gen)}
 
