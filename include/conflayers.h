@@ -23,6 +23,11 @@
  *   - Requirements: d_model = n_heads * head_dim, n_kv_heads divides n_heads (n_kv_heads < n_heads: grouped-query
  *     attention, query head h reads key/value head h / (n_heads / n_kv_heads)),
  *     head_dim in {64, 128}, d_model and d_ffn multiples of 8, 1 <= K <= CL_MAX_K.
+ *   - Which kernels run: single-token steps (draft, vanilla) run in one persistent cooperative kernel when d_model and
+ *     d_ffn are at most 16384 (bf16) / 8192 (fp32); passes of several rows (verify, prefill) and the confidence scoring
+ *     of bf16 models run on the tensor cores (tcgen05); fp32 models and the cases above use per-matrix CUDA-core kernels.
+ *     Environment switches read by cl_load (diagnostics): CL_DISABLE_STEP_KERNEL=1, CL_DISABLE_TC_PASS=1,
+ *     CL_DISABLE_ROW_SHARES=1, CL_L2_AHEAD_KB=<n>.
  */
 #ifndef CONFLAYERS_H
 #define CONFLAYERS_H
@@ -99,8 +104,10 @@ typedef struct {
 int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **out);
 
 /* Copy the weights into the context's own arena (concatenating Q/K/V and interleaving gate/up rows
- * for streaming), allocate the KV cache [n_layers][2][n_heads][max_seq][head_dim] and scratch.  Borrowed
- * pointers may be released after the call returns.  CL_ENOMEM if the device cannot hold it. */
+ * for streaming; one copy, in execution order), allocate the KV cache [n_layers][2][n_heads][max_seq][head_dim] and scratch.  Borrowed
+ * pointers may be released after the call returns.  CL_ENOMEM if the device cannot hold it.  With the persistent
+ * step kernel the call also runs a few token steps on an empty cache to measure each SM's streaming rate (fixed row
+ * shares afterwards); it synchronises the stream. */
 int cl_load(cl_ctx *ctx, const cl_weights *w);
 
 int cl_destroy(cl_ctx *ctx);
