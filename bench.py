@@ -156,7 +156,7 @@ def run_reference(args, rank):
     sample = f"{ORACLE_CYCLES} draft-{K_DRAFT}/verify/accept cycles of {WORKLOAD} after a 2-token prefill per step"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 (f64 reductions)", "data": "synthetic",
             "config": {"workload": f"{WORKLOAD}: 7B-shape Llama decoder, bf16 weights, K={K_DRAFT}, "
                                    f"uniform {int(SKIP_RATIO * 100)}% skip set"},
             "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},

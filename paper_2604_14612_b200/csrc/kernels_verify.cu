@@ -551,7 +551,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
 #pragma unroll
         for (int t = 0; t < T; ++t) sc[t] = -INFINITY;
 #pragma unroll 1
-        for (int jb = 0; jb < 32; jb += KPW) {
+        for (int jb = 0; jb < n; jb += KPW) {   // (uniform bound: keys past n have no score)
             const int j = jb + sub;
             float kf[EPL];
 #pragma unroll
