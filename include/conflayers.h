@@ -26,8 +26,10 @@
  *   - Which kernels run: single-token steps (draft, vanilla) run in one persistent cooperative kernel when d_model and
  *     d_ffn are at most 16384 (bf16) / 8192 (fp32); passes of several rows (verify, prefill) and the confidence scoring
  *     of bf16 models run on the tensor cores (tcgen05); fp32 models and the cases above use per-matrix CUDA-core kernels.
+ *     A prompt of more than 16 tokens (bf16 models) runs all rows but the last through wide tensor-core GEMMs, up to
+ *     512 rows at a time, and the last row through the pass of several rows, which has the LM head.
  *     Environment switches read by cl_load (diagnostics): CL_DISABLE_STEP_KERNEL=1, CL_DISABLE_TC_PASS=1,
- *     CL_DISABLE_ROW_SHARES=1, CL_L2_AHEAD_KB=<n>.
+ *     CL_DISABLE_WIDE_PREFILL=1, CL_DISABLE_ROW_SHARES=1, CL_L2_AHEAD_KB=<n>.
  */
 #ifndef CONFLAYERS_H
 #define CONFLAYERS_H

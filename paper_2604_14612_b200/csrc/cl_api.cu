@@ -72,6 +72,13 @@ struct cl_ctx {
     int v_att_S;                         // parts the keys of a head are cut into in the T-row attention
     unsigned *v_tickets;
     ClHeadPartial *v_head_part;
+    // wide tensor-core GEMM path of the prompt pass (bf16 models)
+    int use_wide;
+    ClTensorMap map_wx, map_watt, map_wh;  // activation rows as bf16 hi/lo parts, boxes of 128 rows
+    __nv_bfloat16 *w_ax, *w_aatt, *w_ah;   // [2 * CL_WIDE_MAX_M, d] [.., d] [.., F]
+    float *w_x, *w_P, *w_att_part;         // residual stream [CL_WIDE_MAX_M, d], product parts, attention parts
+    size_t w_P_floats;
+    unsigned *w_tickets;
     std::vector<ClLayer> layers;
     std::vector<uint8_t> mask;    // host copy of the skip set
     int nsplit, per_max;
@@ -199,7 +206,8 @@ static void free_all(cl_ctx *c) {
                     c->att, c->hff, c->att_part, c->logits, c->tickets, c->head_part, c->st, c->prompt_dev, c->out_dev,
                     c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sc_xn, c->sc_part, c->sel_mask, c->sel_margins, c->sel_clayers,
                     c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->head_part2,
-                    c->cum_w_dev, c->busy_dev, c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_att_part, c->v_tickets, c->v_head_part};
+                    c->cum_w_dev, c->busy_dev, c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_att_part, c->v_tickets, c->v_head_part,
+                    c->w_ax, c->w_aatt, c->w_ah, c->w_x, c->w_P, c->w_att_part, c->w_tickets};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->h_st) cudaFreeHost(c->h_st);
@@ -412,6 +420,29 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 }
                 if (!ok) return fail(c, CL_ECUDA, "cl_load: encoding a TMA tensor map failed");
                 c->use_tc = 1;
+                // ---- wide GEMM path of the prompt pass: hi/lo activation rows, residual stream, product parts
+                const char *woff = getenv("CL_DISABLE_WIDE_PREFILL");
+                if (!(woff && woff[0] == '1') && g.max_seq > 17) {
+                    const size_t Mw = CL_WIDE_MAX_M, widest = std::max(qkv_rows, 2 * F);
+                    DM(c->w_ax, 2 * Mw * d * 2);
+                    DM(c->w_aatt, 2 * Mw * d * 2);
+                    DM(c->w_ah, 2 * Mw * F * 2);
+                    CU(cudaMemsetAsync(c->w_ax, 0, 2 * Mw * d * 2, c->stream));
+                    CU(cudaMemsetAsync(c->w_aatt, 0, 2 * Mw * d * 2, c->stream));
+                    CU(cudaMemsetAsync(c->w_ah, 0, 2 * Mw * F * 2, c->stream));
+                    DM(c->w_x, Mw * d * 4);
+                    c->w_P_floats = 2 * Mw * widest;
+                    DM(c->w_P, c->w_P_floats * 4);
+                    const size_t groups = Mw / 8;
+                    DM(c->w_att_part, groups * cl_attn_rows_part_floats(g.n_heads, 4, 8, g.head_dim) * 4);
+                    DM(c->w_tickets, groups * g.n_heads * 4);
+                    CU(cudaMemsetAsync(c->w_tickets, 0, groups * g.n_heads * 4, c->stream));
+                    if (!(cl_make_tensor_map(&c->map_wx, c->w_ax, (int)(2 * Mw), (int)d, 128) &&
+                          cl_make_tensor_map(&c->map_watt, c->w_aatt, (int)(2 * Mw), (int)d, 128) &&
+                          cl_make_tensor_map(&c->map_wh, c->w_ah, (int)(2 * Mw), (int)F, 128)))
+                        return fail(c, CL_ECUDA, "cl_load: encoding a TMA tensor map failed");
+                    c->use_wide = 1;
+                }
             }
         }
         CU(cudaStreamSynchronize(c->stream));   // host staging vector and borrowed pointers are released after this
@@ -571,6 +602,69 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
     return CL_OK;
 }
 
+// The prompt pass over M <= CL_WIDE_MAX_M rows at positions ctx .. ctx + M - 1 (bf16 models): every matrix is one wide
+// tensor-core GEMM whose product a small kernel consumes (rotary + cache append, residual add + RMSNorm, SiLU).
+// Fills the KV cache and, when asked, the hidden taps; computes no logits (the caller runs the last prompt token
+// through the T-row pass for those).
+static int forward_wide(cl_ctx *c, const int *tok, int M, int tap) {
+    const cl_model_cfg &g = c->cfg;
+    const int d = g.d_model, F = g.d_ffn, L = g.n_layers, qkv_rows = d + 2 * g.n_kv_heads * g.head_dim;
+    const int KBd = (d + 63) / 64, KBf = (F + 63) / 64, MT = (M + 127) / 128, lo0 = CL_WIDE_MAX_M;
+    auto gemm = [&](const ClTensorMap &mapA, const ClTensorMap &mapB, int rows, int KB, int *splits) -> int {
+        ClWideArgs a;
+        a.M = M; a.rows = rows; a.KB = KB; a.MT = MT; a.NT = (rows + 255) / 256;
+        a.splits = *splits = cl_wide_splits(M, rows, KB, c->n_sm, c->w_P_floats);
+        a.lo_row0 = lo0; a.P = c->w_P; a.err = &c->st->err;
+        KL(cl_launch_wide(mapA, mapB, a, c->stream));
+        return CL_OK;
+    };
+    ClWideNormArgs nb;
+    memset(&nb, 0, sizeof(nb));
+    nb.x = c->w_x; nb.M = M; nb.d = d; nb.eps = g.rms_eps; nb.A = c->w_ax; nb.lo_row0 = lo0; nb.st = c->st;
+    nb.tap_P = g.tap_positions;
+    {
+        ClWideNormArgs n = nb;
+        n.embed = c->embed; n.tok = tok; n.g = L ? c->layers[0].n1 : nullptr;
+        KL(cl_launch_wide_norm(n, c->stream));
+    }
+    const int full = M / 8, tail = M % 8;
+    int S = (2 * c->n_sm + full * g.n_heads - 1) / (full * g.n_heads > 0 ? full * g.n_heads : 1);
+    if (S > 4) S = 4;
+    if (S < 1) S = 1;
+    int rc, sp;
+    for (int l = 0; l < L; ++l) {
+        const ClLayer &y = c->layers[l];
+        if ((rc = gemm(c->map_wx, c->map_qkv[l], qkv_rows, KBd, &sp))) return rc;
+        KL(cl_launch_wide_rope_append(c->w_P, sp, M, g.n_heads, g.n_kv_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq,
+                                      c->st, c->stream));
+        ClAttnArgs t;
+        memset(&t, 0, sizeof(t));
+        t.q = c->w_P; t.ld_q = qkv_rows; t.n_kv_heads = g.n_kv_heads; t.kcache = y.kc; t.vcache = y.vc;
+        t.part = c->w_att_part; t.tickets = c->w_tickets; t.out = nullptr; t.out_b = c->w_aatt; t.nh = lo0; t.st = c->st;
+        t.row0 = 0; t.n_heads = g.n_heads; t.head_dim = g.head_dim; t.d_model = d; t.max_seq = g.max_seq;
+        if (full) KL(cl_launch_attn_rows(1, 8, S, t, c->stream, full));
+        if (tail) {   // the last, shorter block of rows
+            t.row0 = full * 8;
+            t.q = c->w_P + (size_t)full * 8 * qkv_rows;
+            t.out_b = c->w_aatt + (size_t)full * 8 * d;
+            KL(cl_launch_attn_rows(1, tail, 4, t, c->stream, 1));
+        }
+        if ((rc = gemm(c->map_watt, c->map_o[l], d, KBd, &sp))) return rc;
+        ClWideNormArgs n = nb;
+        n.P = c->w_P; n.splits = sp; n.g = y.n2;
+        if (tap) n.tap = ring_slot(c, l, 0);
+        KL(cl_launch_wide_norm(n, c->stream));
+        if ((rc = gemm(c->map_wx, c->map_gu[l], 2 * F, KBd, &sp))) return rc;
+        KL(cl_launch_wide_silu(c->w_P, sp, M, F, c->w_ah, lo0, c->stream));
+        if ((rc = gemm(c->map_wh, c->map_d[l], d, KBf, &sp))) return rc;
+        n = nb;
+        n.P = c->w_P; n.splits = sp; n.g = (l + 1 < L) ? c->layers[l + 1].n1 : nullptr;
+        if (tap) n.tap = ring_slot(c, l, 1);
+        KL(cl_launch_wide_norm(n, c->stream));
+    }
+    return CL_OK;
+}
+
 // n_steps consecutive single-token steps in one persistent launch (draft steps with the skip set, or
 // vanilla full-model steps that emit and advance on the device).
 static int run_steps(cl_ctx *c, int mode, int n_steps, int row0, bool full_model, float *logits, int *out_tokens) {
@@ -676,7 +770,17 @@ extern "C" int cl_prefill(cl_ctx *c, const int32_t *tokens, int n, int tap_hidde
     ClPoke p = poke_none();
     p.ctx = 0; p.n_drafted = 0; p.done = 0;
     if ((rc = poke(c, p))) return rc;
-    for (int c0 = 0; c0 < n; c0 += CL_PREFILL_CHUNK) {
+    int c0 = 0;
+    if (c->use_wide && n > 2 * CL_PREFILL_CHUNK) {
+        // all prompt rows but the last go through the wide GEMMs; the last one takes the T-row pass, which has the LM head
+        while (c0 < n - 1) {
+            const int M = (n - 1 - c0 < CL_WIDE_MAX_M) ? n - 1 - c0 : CL_WIDE_MAX_M;
+            if ((rc = forward_wide(c, c->prompt_dev + c0, M, tap_hidden))) return rc;
+            KL(cl_launch_advance(c->st, M, 0, c->stream));
+            c0 += M;
+        }
+    }
+    for (; c0 < n; c0 += CL_PREFILL_CHUNK) {
         const int T = (n - c0 < CL_PREFILL_CHUNK) ? n - c0 : CL_PREFILL_CHUNK;
         const bool last = c0 + T >= n;
         rc = forward_rows(c, c->prompt_dev + c0, T, 0, nullptr, tap_hidden, last, ST_FIELD(c, int, tgt_tok),

@@ -121,7 +121,8 @@ cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H
                                   void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_attn(int wdtype, int T, const ClAttnArgs &a, cudaStream_t s);
 size_t cl_attn_rows_part_floats(int H, int S, int T, int hd);
-cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s);
+// groups > 1: `groups` consecutive blocks of T rows in one launch (part: groups times the floats above, tickets: groups * H)
+cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s, int groups = 1);
 cudaError_t cl_launch_tap(int wdtype, const float *x, int T, int row0, int d, void *ring_layer, int P,
                           const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_accept(ClDevState *st, int K, int *out_tokens, cudaStream_t s);
@@ -161,6 +162,36 @@ cudaError_t cl_launch_pass_begin(const void *embed, const int *tok, int T, int d
                                  const float *g, float *ssq_out, const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_head_finalize(const ClHeadPartial *part, int tiles, int T, float inv_log_v, int *out_tok, float *out_pmax,
                                     float *out_conf, const ClDevState *st, cudaStream_t s);
+
+// ---- wide tensor-core GEMM of the prompt pass (bf16 models): up to CL_WIDE_MAX_M prompt rows at a time ----
+#define CL_WIDE_MAX_M 512
+struct ClWideArgs {
+    int M, rows, KB;                  // token rows of the pass, weight rows, K blocks of 64
+    int MT, NT, splits;               // 128-row token tiles, 256-row weight tiles, parts the K range is cut into
+    int lo_row0;                      // first row of the lo parts in the activation buffer (hi parts start at row 0)
+    float *P;                         // [splits, M, rows] partial products (a later kernel adds the splits in order)
+    int *err;
+};
+struct ClWideNormArgs {
+    float *x;                         // [M, d] residual stream of the pass
+    int M, d, splits;
+    const float *P;                   // [splits, M, d] products to add to x, or null
+    const void *embed;                // with tok: x = E[tok[t]] instead (start of the pass)
+    const int *tok;
+    const float *g;                   // gain of the RMSNorm that follows, or null (no normalised rows are written)
+    float eps;
+    __nv_bfloat16 *A;                 // [2 * lo_row0, d]: normalised rows as bf16 hi (row t) and lo (row lo_row0 + t)
+    int lo_row0;
+    void *tap;                        // optional: this layer's hidden-state ring [tap_P, d] (bf16)
+    int tap_P;
+    const ClDevState *st;
+};
+int cl_wide_splits(int M, int rows, int KB, int n_sm, size_t ws_floats);
+cudaError_t cl_launch_wide(const ClTensorMap &mapA, const ClTensorMap &mapB, const ClWideArgs &a, cudaStream_t s);
+cudaError_t cl_launch_wide_norm(const ClWideNormArgs &a, cudaStream_t s);
+cudaError_t cl_launch_wide_rope_append(float *P, int splits, int M, int H, int Hkv, int hd, int d, const float2 *rope_cs,
+                                       void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
+cudaError_t cl_launch_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, cudaStream_t s);
 
 // tensor-core scoring (bf16 LM head): normalise to bf16, contraction fused with the softmax statistics, finalize
 int cl_score_tc_ranges(int R, int n_sm);

@@ -1,0 +1,290 @@
+// Wide tensor-core GEMM for the prompt pass of the bf16 model: the full-model pass of Section 3 over up to 512
+// prompt rows at a time, so that the weights stream from HBM once per 512 tokens instead of once per 8.
+//
+//   P[ks, t, r] = sum_{k in part ks} a[t, k] * W[r, k]        a: M activation rows, W: [rows, K] bf16 weights
+//
+// Here the token rows are the M = 128 operand of tcgen05.mma (one tensor-memory lane per token) and 256 weight rows
+// are N.  Activations are fp32 everywhere else; each row enters as hi = bf16(v) and lo = bf16(v - hi) and both
+// products accumulate into the same fp32 accumulator, so the product keeps about 16 mantissa bits of the activation.
+// One CTA computes one (token tile, weight tile, K part): the K range is cut into `splits` parts only to fill the
+// 148 SMs when a matrix has few output tiles (4096 outputs are 16 tiles), and the parts are added in a fixed order
+// by the small kernel that consumes the product:
+//   k_wide_rope_append   q, k, v: rotary embedding at the row's position, cache append, q left in place
+//   k_wide_norm          x += product (or x = E[token]); hidden tap; RMSNorm -> hi/lo rows of the next GEMM
+//   k_wide_silu          h = silu(gate) * up on the interleaved gate/up product -> hi/lo rows of the down projection
+// Warp roles: warp 0 TMA producer (A hi 128 x 64, A lo 128 x 64, B 256 x 64 as two 128-row boxes, 128-byte swizzle,
+// 3-stage ring of 64 KB), warp 1 tensor-memory allocation and MMA issue, warps 2-5 store the accumulator (thread =
+// token row, 256 consecutive outputs).  CTAs that share a weight tile are neighbours in the grid, so the tile comes
+// from HBM once and from L2 for the other token tiles.  Every wait is bounded in time.
+#include <math.h>
+
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int WM = 128, WN = 256, WSTAGES = 3;
+constexpr int WA_BYTES = WM * TC_BK * 2, WB_BYTES = WN * TC_BK * 2, WSTAGE_BYTES = 2 * WA_BYTES + WB_BYTES;   // 64 KB
+constexpr int WTHREADS = 192;
+
+struct WSmem {
+    unsigned long long full[WSTAGES], empty[WSTAGES], tfull;
+    unsigned tmem_base;
+    int abort;
+};
+
+__global__ void __launch_bounds__(WTHREADS, 1)
+k_wide(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, ClWideArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *tiles = (unsigned char *)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+    WSmem *sm = (WSmem *)(tiles + (size_t)WSTAGES * WSTAGE_BYTES);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x;
+    if (cta >= a.MT * a.NT * a.splits) return;   // whole CTA leaves before anything is set up
+    const int mt = cta % a.MT, nt = (cta / a.MT) % a.NT, ks = cta / (a.MT * a.NT);
+    const int kb0 = (int)((long long)a.KB * ks / a.splits), kb1 = (int)((long long)a.KB * (ks + 1) / a.splits);
+
+    if (tid == 0) {
+        for (int i = 0; i < WSTAGES; ++i) {
+            bar_init(&sm->full[i], 1);
+            bar_init(&sm->empty[i], 1);
+        }
+        bar_init(&sm->tfull, 1);
+        sm->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(s_u32(&sm->tmem_base)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem = *(volatile unsigned *)&sm->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            unsigned stage = 0, par = 0, issued[WSTAGES];
+            for (int i = 0; i < WSTAGES; ++i) issued[i] = 2u;
+            bool ok = true;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!bar_wait(&sm->empty[stage], par ^ 1u, &sm->abort, a.err)) { ok = false; break; }
+                unsigned char *dst = tiles + (size_t)stage * WSTAGE_BYTES;
+                bar_expect(&sm->full[stage], WSTAGE_BYTES);
+                tma_load_2d(dst, &mapA, kb * TC_BK, mt * WM, &sm->full[stage]);
+                tma_load_2d(dst + WA_BYTES, &mapA, kb * TC_BK, a.lo_row0 + mt * WM, &sm->full[stage]);
+                tma_load_2d(dst + 2 * WA_BYTES, &mapB, kb * TC_BK, nt * WN, &sm->full[stage]);
+                tma_load_2d(dst + 2 * WA_BYTES + WB_BYTES / 2, &mapB, kb * TC_BK, nt * WN + WN / 2, &sm->full[stage]);
+                issued[stage] = par;
+                if (++stage == WSTAGES) { stage = 0; par ^= 1u; }
+            }
+            if (!ok) {   // gave up: still let the copies in flight land before the CTA may exit (bounded)
+                for (int i = 0; i < WSTAGES; ++i) {
+                    if (issued[i] < 2u) {
+                        const unsigned long long t0 = gtime_ns();
+                        while (!bar_try(&sm->full[i], issued[i]))
+                            if (gtime_ns() - t0 > WAIT_NS) break;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const unsigned idesc = umma_idesc(WM, WN);
+            unsigned stage = 0, par = 0;
+            bool ok = true;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!bar_wait(&sm->full[stage], par, &sm->abort, a.err)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const unsigned hi_addr = s_u32(tiles + (size_t)stage * WSTAGE_BYTES), lo_addr = hi_addr + WA_BYTES,
+                               b_addr = hi_addr + 2 * WA_BYTES;
+#pragma unroll
+                for (int k = 0; k < TC_BK / 16; ++k) {
+                    umma_bf16(tmem, umma_desc(hi_addr + k * 32), umma_desc(b_addr + k * 32), idesc, (unsigned)((kb - kb0) | k));
+                    umma_bf16(tmem, umma_desc(lo_addr + k * 32), umma_desc(b_addr + k * 32), idesc, 1u);
+                }
+                umma_commit(&sm->empty[stage]);   // the stage is free once these multiply-adds have read it
+                if (++stage == WSTAGES) { stage = 0; par ^= 1u; }
+            }
+            if (ok) umma_commit(&sm->tfull);
+        }
+    } else {
+        // ---------------- store: one thread per token row ----------------
+        const int q = warp & 3;                        // the tensor-memory lane quadrant this warp may read
+        const int t = mt * WM + q * 32 + lane;
+        if (bar_wait(&sm->tfull, 0u, &sm->abort, a.err)) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float *dst = a.P + ((size_t)ks * a.M + (size_t)min(t, a.M - 1)) * a.rows;
+#pragma unroll 1
+            for (int cb = 0; cb < WN / 32; ++cb) {
+                float v[32];
+                tmem_ld32(tmem + ((unsigned)(q * 32) << 16) + (unsigned)(cb * 32), v);   // (whole warp, also for rows past M)
+                const int col0 = nt * WN + cb * 32;
+                if (t < a.M) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (col0 + 4 * i + 4 <= a.rows)
+                            *(float4 *)(dst + col0 + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
+    }
+}
+
+__device__ __forceinline__ void w_split(float v, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+    hi = __float2bfloat16_rn(v);
+    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+// One CTA per token row: x[t] = E[token] or x[t] += product parts (added in part order); the optional hidden tap;
+// then the rows of the next GEMM: hi/lo(x * rsqrt(mean x^2 + eps) * g).
+__global__ void __launch_bounds__(256) k_wide_norm(ClWideNormArgs a) {
+    __shared__ float red[8];
+    const int t = blockIdx.x, tid = threadIdx.x, d = a.d;
+    float *xr = a.x + (size_t)t * d;
+    const __nv_bfloat16 *er = a.tok ? (const __nv_bfloat16 *)a.embed + (size_t)a.tok[t] * d : nullptr;
+    // only the last tap_P rows of the pass reach the ring: an earlier row of the same slot would be overwritten anyway
+    __nv_bfloat16 *tap = nullptr;
+    if (a.tap && t >= a.M - a.tap_P) tap = (__nv_bfloat16 *)a.tap + (size_t)((a.st->ctx + t) % a.tap_P) * d;
+    float ss = 0.f;
+    for (int i = tid * 4; i < d; i += 1024) {
+        float4 v;
+        if (er) {
+            const uint2 u = *(const uint2 *)(er + i);
+            v = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                            __uint_as_float(u.y & 0xffff0000u));
+        } else {
+            v = *(const float4 *)(xr + i);
+            for (int s = 0; s < a.splits; ++s) {
+                const float4 p = __ldcg((const float4 *)(a.P + ((size_t)s * a.M + t) * d + i));
+                v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+            }
+        }
+        *(float4 *)(xr + i) = v;
+        if (tap) {
+            tap[i] = __float2bfloat16_rn(v.x); tap[i + 1] = __float2bfloat16_rn(v.y);
+            tap[i + 2] = __float2bfloat16_rn(v.z); tap[i + 3] = __float2bfloat16_rn(v.w);
+        }
+        ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+    }
+    if (!a.g) return;   // uniform
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((tid & 31) == 0) red[tid >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+    for (int w = 0; w < 8; ++w) tot += red[w];   // fixed order
+    const float sc = 1.0f / sqrtf(tot / (float)d + a.eps);
+    __nv_bfloat16 *hi = a.A + (size_t)t * d, *lo = a.A + (size_t)(a.lo_row0 + t) * d;
+    for (int i = tid * 4; i < d; i += 1024) {
+        const float4 v = *(const float4 *)(xr + i);   // this thread's own writes
+        const float4 g = *(const float4 *)(a.g + i);
+        w_split(v.x * sc * g.x, hi[i], lo[i]);
+        w_split(v.y * sc * g.y, hi[i + 1], lo[i + 1]);
+        w_split(v.z * sc * g.z, hi[i + 2], lo[i + 2]);
+        w_split(v.w * sc * g.w, hi[i + 3], lo[i + 3]);
+    }
+}
+
+// grid (M, H), hd / 2 threads: q, k, v of row t and head h from the QKV product parts; rotary embedding at position
+// ctx + t; q goes back in place (part 0), k and v (the first Hkv heads) go to the cache [kv head][position][hd].
+__global__ void k_wide_rope_append(float *P, int splits, int M, int hd, int d, int Hkv, const float2 *rope_cs,
+                                   __nv_bfloat16 *kcache, __nv_bfloat16 *vcache, int max_seq, const ClDevState *st) {
+    const int t = blockIdx.x, h = blockIdx.y, i = threadIdx.x, half = hd >> 1;
+    const int pos = st->ctx + t;
+    if (pos >= max_seq) return;
+    const int kvd = Hkv * hd, ld = d + 2 * kvd;
+    const size_t part = (size_t)M * ld;
+    float *row = P + (size_t)t * ld;
+    auto total = [&](int col) {
+        float v = row[col];
+        for (int s = 1; s < splits; ++s) v += __ldcg(row + (size_t)s * part + col);
+        return v;
+    };
+    const float2 cs = rope_cs[(size_t)pos * half + i];
+    const float qa = total(h * hd + i), qb = total(h * hd + i + half);
+    row[h * hd + i] = qa * cs.x - qb * cs.y;
+    row[h * hd + i + half] = qb * cs.x + qa * cs.y;
+    if (h >= Hkv) return;
+    const float ka = total(d + h * hd + i), kb = total(d + h * hd + i + half);
+    __nv_bfloat16 *kc = kcache + ((size_t)h * max_seq + pos) * hd, *vc = vcache + ((size_t)h * max_seq + pos) * hd;
+    kc[i] = __float2bfloat16_rn(ka * cs.x - kb * cs.y);
+    kc[i + half] = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
+    vc[i] = __float2bfloat16_rn(total(d + kvd + h * hd + i));
+    vc[i + half] = __float2bfloat16_rn(total(d + kvd + h * hd + i + half));
+}
+
+// grid (M, ceil(F / 256)): the gate/up product has rows interleaved (2 i = gate_i, 2 i + 1 = up_i).
+__global__ void __launch_bounds__(256) k_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0) {
+    const int t = blockIdx.x, i = blockIdx.y * 256 + threadIdx.x;
+    if (i >= F) return;
+    float g = 0.f, u = 0.f;
+    for (int s = 0; s < splits; ++s) {
+        const float2 p = __ldcg((const float2 *)(P + ((size_t)s * M + t) * 2 * F) + i);
+        g += p.x;
+        u += p.y;
+    }
+    const float h = g / (1.f + expf(-g)) * u;
+    w_split(h, A[(size_t)t * F + i], A[(size_t)(lo_row0 + t) * F + i]);
+}
+
+}  // namespace
+
+// Parts to cut the K range into: the fewest that fill at least 90 % of the last wave of CTAs (else the best found),
+// with at least 8 K blocks per part and the partial products inside the workspace.
+int cl_wide_splits(int M, int rows, int KB, int n_sm, size_t ws_floats) {
+    const long long tiles = (long long)((M + WM - 1) / WM) * ((rows + WN - 1) / WN);
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= 16; ++s) {
+        if (s > 1 && (KB / s < 8 || (size_t)s * M * rows > ws_floats)) break;
+        const long long n = tiles * s, waves = (n + n_sm - 1) / n_sm;
+        const double eff = (double)n / (double)(waves * n_sm);
+        if (eff > best_eff + 1e-9) {
+            best_eff = eff;
+            best = s;
+        }
+        if (eff >= 0.9) break;
+    }
+    return best;
+}
+
+cudaError_t cl_launch_wide(const ClTensorMap &mapA, const ClTensorMap &mapB, const ClWideArgs &a, cudaStream_t s) {
+    const size_t smem = (size_t)WSTAGES * WSTAGE_BYTES + sizeof(WSmem) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    if (a.rows % 4 || a.M < 1 || a.M > CL_WIDE_MAX_M) return cudaErrorInvalidValue;
+    k_wide<<<a.MT * a.NT * a.splits, WTHREADS, smem, s>>>(*(const CUtensorMap *)mapA.bytes, *(const CUtensorMap *)mapB.bytes, a);
+    return cudaGetLastError();
+}
+
+cudaError_t cl_launch_wide_norm(const ClWideNormArgs &a, cudaStream_t s) {
+    if (a.d % 4) return cudaErrorInvalidValue;
+    k_wide_norm<<<a.M, 256, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t cl_launch_wide_rope_append(float *P, int splits, int M, int H, int Hkv, int hd, int d, const float2 *rope_cs,
+                                       void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s) {
+    k_wide_rope_append<<<dim3(M, H), hd / 2, 0, s>>>(P, splits, M, hd, d, Hkv, rope_cs, (__nv_bfloat16 *)kcache,
+                                                     (__nv_bfloat16 *)vcache, max_seq, st);
+    return cudaGetLastError();
+}
+
+cudaError_t cl_launch_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, cudaStream_t s) {
+    k_wide_silu<<<dim3(M, (F + 255) / 256), 256, 0, s>>>(P, splits, M, F, A, lo_row0);
+    return cudaGetLastError();
+}

@@ -283,6 +283,35 @@ def test_tensor_core_pass_matches_streaming_pass(monkeypatch):
     assert np.abs(out[0][3] - out[1][3]).max() <= 2 ** -7 * scale        # taps: one bf16 ulp at the top of the range
 
 
+def test_wide_prompt_pass_matches_chunked_prompt_pass(monkeypatch):
+    """The wide tcgen05 GEMMs of the prompt pass (up to 512 rows at a time) against the 8-row passes on the same
+    prompt: the same KV cache (seen through the logits of a verify pass that follows), first token and hidden taps.
+    700 prompt tokens = one full pass of 512 rows and a ragged one of 187 (a partial token tile, 3 rows left over
+    for the attention) before the last token."""
+    base = synth.WORKLOADS["C2"].shape
+    sh = dataclasses.replace(base, n_layers=2, max_seq=768)
+    W = synth.make_weights(sh, 6, device="cuda")
+    prompt = synth.make_prompt(6, 700, sh.vocab)
+    out = {}
+    for wide in (0, 1):
+        monkeypatch.setenv("CL_DISABLE_WIDE_PREFILL", "0" if wide else "1")
+        ctx = cl.Context.from_shape(sh, tap_positions=64)
+        ctx.cl_load(W)
+        first = ctx.cl_prefill(prompt, tap_hidden=True)
+        ring = ctx.cl_read_hidden_ring().float().numpy()
+        ctx.cl_force_tokens([11, 22, 33, 44])
+        v = ctx.cl_verify(5, want_logits=True)
+        out[wide] = (first, ring, v["targets"].copy(), v["logits"].copy())
+        ctx.close()
+    assert out[0][0] == out[1][0]
+    scale = max(1.0, float(np.abs(out[0][1]).max()))
+    assert np.abs(out[0][1] - out[1][1]).max() <= 2 ** -7 * scale        # taps: one bf16 ulp at the top of the range
+    assert np.abs(out[0][3] - out[1][3]).max() <= 2e-3                   # both far inside the 1e-2 tolerance
+    top2 = np.sort(out[0][3], axis=1)[:, -2:]
+    clear = (top2[:, 1] - top2[:, 0]) >= NEAR_TIE                        # rows whose greedy token is not a near tie
+    assert np.array_equal(out[0][2][clear], out[1][2][clear])
+
+
 def test_interval_search_matches_oracle_on_c1():
     """Section 3.3 driver: same rounds, scores, sets and tokens as the oracle's loop on the fp32 model."""
     w = synth.WORKLOADS["C1"]
