@@ -76,9 +76,8 @@ struct cl_ctx {
     int use_wide;
     ClTensorMap map_wx, map_watt, map_wh;  // activation rows as bf16 hi/lo parts, boxes of 128 rows
     __nv_bfloat16 *w_ax, *w_aatt, *w_ah;   // [2 * CL_WIDE_MAX_M, d] [.., d] [.., F]
-    float *w_x, *w_P, *w_att_part;         // residual stream [CL_WIDE_MAX_M, d], product parts, attention parts
+    float *w_x, *w_P;                      // residual stream [CL_WIDE_MAX_M, d], product parts
     size_t w_P_floats;
-    unsigned *w_tickets;
     std::vector<ClLayer> layers;
     std::vector<uint8_t> mask;    // host copy of the skip set
     int nsplit, per_max;
@@ -207,7 +206,7 @@ static void free_all(cl_ctx *c) {
                     c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sc_xn, c->sc_part, c->sel_mask, c->sel_margins, c->sel_clayers,
                     c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->head_part2,
                     c->cum_w_dev, c->busy_dev, c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_att_part, c->v_tickets, c->v_head_part,
-                    c->w_ax, c->w_aatt, c->w_ah, c->w_x, c->w_P, c->w_att_part, c->w_tickets};
+                    c->w_ax, c->w_aatt, c->w_ah, c->w_x, c->w_P};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->h_st) cudaFreeHost(c->h_st);
@@ -433,10 +432,6 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                     DM(c->w_x, Mw * d * 4);
                     c->w_P_floats = 2 * Mw * widest;
                     DM(c->w_P, c->w_P_floats * 4);
-                    const size_t groups = Mw / 8;
-                    DM(c->w_att_part, groups * cl_attn_rows_part_floats(g.n_heads, 4, 8, g.head_dim) * 4);
-                    DM(c->w_tickets, groups * g.n_heads * 4);
-                    CU(cudaMemsetAsync(c->w_tickets, 0, groups * g.n_heads * 4, c->stream));
                     if (!(cl_make_tensor_map(&c->map_wx, c->w_ax, (int)(2 * Mw), (int)d, 128) &&
                           cl_make_tensor_map(&c->map_watt, c->w_aatt, (int)(2 * Mw), (int)d, 128) &&
                           cl_make_tensor_map(&c->map_wh, c->w_ah, (int)(2 * Mw), (int)F, 128)))
@@ -627,28 +622,14 @@ static int forward_wide(cl_ctx *c, const int *tok, int M, int tap) {
         n.embed = c->embed; n.tok = tok; n.g = L ? c->layers[0].n1 : nullptr;
         KL(cl_launch_wide_norm(n, c->stream));
     }
-    const int full = M / 8, tail = M % 8;
-    int S = (2 * c->n_sm + full * g.n_heads - 1) / (full * g.n_heads > 0 ? full * g.n_heads : 1);
-    if (S > 4) S = 4;
-    if (S < 1) S = 1;
     int rc, sp;
     for (int l = 0; l < L; ++l) {
         const ClLayer &y = c->layers[l];
         if ((rc = gemm(c->map_wx, c->map_qkv[l], qkv_rows, KBd, &sp))) return rc;
         KL(cl_launch_wide_rope_append(c->w_P, sp, M, g.n_heads, g.n_kv_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq,
                                       c->st, c->stream));
-        ClAttnArgs t;
-        memset(&t, 0, sizeof(t));
-        t.q = c->w_P; t.ld_q = qkv_rows; t.n_kv_heads = g.n_kv_heads; t.kcache = y.kc; t.vcache = y.vc;
-        t.part = c->w_att_part; t.tickets = c->w_tickets; t.out = nullptr; t.out_b = c->w_aatt; t.nh = lo0; t.st = c->st;
-        t.row0 = 0; t.n_heads = g.n_heads; t.head_dim = g.head_dim; t.d_model = d; t.max_seq = g.max_seq;
-        if (full) KL(cl_launch_attn_rows(1, 8, S, t, c->stream, full));
-        if (tail) {   // the last, shorter block of rows
-            t.row0 = full * 8;
-            t.q = c->w_P + (size_t)full * 8 * qkv_rows;
-            t.out_b = c->w_aatt + (size_t)full * 8 * d;
-            KL(cl_launch_attn_rows(1, tail, 4, t, c->stream, 1));
-        }
+        KL(cl_launch_attn_wide(c->w_P, qkv_rows, y.kc, y.vc, c->w_aatt, lo0, M, d, g.n_heads, g.n_kv_heads, g.head_dim,
+                               g.max_seq, c->st, c->stream));
         if ((rc = gemm(c->map_watt, c->map_o[l], d, KBd, &sp))) return rc;
         ClWideNormArgs n = nb;
         n.P = c->w_P; n.splits = sp; n.g = y.n2;

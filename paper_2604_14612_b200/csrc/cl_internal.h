@@ -121,8 +121,7 @@ cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H
                                   void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_attn(int wdtype, int T, const ClAttnArgs &a, cudaStream_t s);
 size_t cl_attn_rows_part_floats(int H, int S, int T, int hd);
-// groups > 1: `groups` consecutive blocks of T rows in one launch (part: groups times the floats above, tickets: groups * H)
-cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s, int groups = 1);
+cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s);
 cudaError_t cl_launch_tap(int wdtype, const float *x, int T, int row0, int d, void *ring_layer, int P,
                           const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_accept(ClDevState *st, int K, int *out_tokens, cudaStream_t s);
@@ -191,6 +190,11 @@ cudaError_t cl_launch_wide(const ClTensorMap &mapA, const ClTensorMap &mapB, con
 cudaError_t cl_launch_wide_norm(const ClWideNormArgs &a, cudaStream_t s);
 cudaError_t cl_launch_wide_rope_append(float *P, int splits, int M, int H, int Hkv, int hd, int d, const float2 *rope_cs,
                                        void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
+// causal attention of the M rows of the pass (positions ctx ..) over the cache; q: fp32 rows [M, ld_q], rotary applied;
+// the output goes out as bf16 hi (row t) and lo (row lo_row0 + t) parts [.., d]
+cudaError_t cl_launch_attn_wide(const float *q, int ld_q, const void *kcache, const void *vcache, __nv_bfloat16 *out_b,
+                                int lo_row0, int M, int d, int H, int Hkv, int hd, int max_seq, const ClDevState *st,
+                                cudaStream_t s);
 cudaError_t cl_launch_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, cudaStream_t s);
 
 // tensor-core scoring (bf16 LM head): normalise to bf16, contraction fused with the softmax statistics, finalize

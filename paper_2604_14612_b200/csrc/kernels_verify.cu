@@ -472,7 +472,7 @@ cudaError_t cl_launch_head_finalize(const ClHeadPartial *part, int tiles, int T,
 }
 
 // ---- attention of the T rows of a pass over the KV cache ----------------------------------------------------
-// grid (H, S, blocks of T rows; one block except in the prompt pass): the keys [0, base + T) of a head (base = first row's position; the rows' own keys are already in
+// grid (H, S): the keys [0, base + T) of a head (base = first row's position; the rows' own keys are already in
 // the cache, rotated) are cut into S contiguous parts, a part into 8 warp ranges.  A warp walks its range 32 keys
 // at a time: every key row is read once (16 bytes per lane) and scored against all T query rows, row t masking keys
 // beyond its own position; per row an online softmax; every value row is read once and accumulated into all rows.
@@ -496,10 +496,9 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
     constexpr size_t WREC_BYTES = ((size_t)AR_WARPS * T * REC * sizeof(float) + 15) & ~(size_t)15;
     unsigned char *stage_k = (unsigned char *)wrec + WREC_BYTES + (size_t)(threadIdx.x >> 5) * 2 * 32 * ROWB;
     unsigned char *stage_v = stage_k + 32 * ROWB;
-    const int h = blockIdx.x, s = blockIdx.y, H = gridDim.x;
-    const int rg = blockIdx.z * T;   // first row of this block of T rows (several blocks per launch in the prompt pass)
+    const int h = blockIdx.x, s = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int base = a.st->ctx + a.row0 + rg, nkeys = base + T, d = a.d_model;
+    const int base = a.st->ctx + a.row0, nkeys = base + T, d = a.d_model;
     if (nkeys > a.max_seq) return;
     const int k0 = (int)((long long)nkeys * s / S), k1 = (int)((long long)nkeys * (s + 1) / S);
     const int kw0 = k0 + (k1 - k0) * warp / AR_WARPS, kw1 = k0 + (k1 - k0) * (warp + 1) / AR_WARPS;
@@ -513,7 +512,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
 #pragma unroll
     for (int t = 0; t < T; ++t)
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) qr[t][e] = (t < T) ? a.q[(size_t)(rg + t) * a.ld_q + h * HD + li * EPL + e] * scale : 0.f;
+        for (int e = 0; e < EPL; ++e) qr[t][e] = (t < T) ? a.q[(size_t)t * a.ld_q + h * HD + li * EPL + e] * scale : 0.f;
     float m_run[T], l_run[T], o_run[T][VPL];
 #pragma unroll
     for (int t = 0; t < T; ++t) {
@@ -651,7 +650,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
         }
     }
     __syncthreads();
-    float *part = a.part + (((size_t)blockIdx.z * H + h) * S + s) * T * REC;
+    float *part = a.part + ((size_t)h * S + s) * T * REC;
     for (int i = tid; i < T * HD; i += blockDim.x) {
         const int t = i / HD, e = i % HD;
         float M = -INFINITY;
@@ -674,17 +673,16 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        unsigned *ticket = a.tickets + (size_t)blockIdx.z * H + h;
-        const unsigned prev = atomicAdd(ticket, 1u);
+        const unsigned prev = atomicAdd(a.tickets + h, 1u);
         is_last = (prev == (unsigned)S - 1);
-        if (is_last) *ticket = 0u;
+        if (is_last) a.tickets[h] = 0u;
     }
     __syncthreads();
     if (!is_last) return;
     __threadfence();
     for (int i = tid; i < T * HD; i += blockDim.x) {
         const int t = i / HD, e = i % HD;
-        const float *p0 = a.part + ((size_t)blockIdx.z * H + h) * S * T * REC + (size_t)t * REC;
+        const float *p0 = a.part + (size_t)h * S * T * REC + (size_t)t * REC;
         float M = -INFINITY;
         for (int s2 = 0; s2 < S; ++s2)
             if (__ldcg(p0 + (size_t)s2 * T * REC + 1) > 0.f) M = fmaxf(M, __ldcg(p0 + (size_t)s2 * T * REC));
@@ -698,11 +696,11 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
             }
         }
         const float o = O / Ls;
-        if (a.out) a.out[(size_t)(rg + t) * d + h * HD + e] = o;
+        a.out[(size_t)t * d + h * HD + e] = o;
         if (a.out_b) {
             const __nv_bfloat16 hi = __float2bfloat16_rn(o);
-            a.out_b[(size_t)(rg + t) * d + h * HD + e] = hi;
-            a.out_b[(size_t)(a.nh + rg + t) * d + h * HD + e] = __float2bfloat16_rn(o - __bfloat162float(hi));
+            a.out_b[(size_t)t * d + h * HD + e] = hi;
+            a.out_b[(size_t)(a.nh + t) * d + h * HD + e] = __float2bfloat16_rn(o - __bfloat162float(hi));
         }
     }
 }
@@ -711,9 +709,9 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
 
 size_t cl_attn_rows_part_floats(int H, int S, int T, int hd) { return (size_t)H * S * T * (hd + 2); }
 
-// a.part must hold groups * cl_attn_rows_part_floats(H, S, T, hd) floats, a.tickets groups * H zeroed counters.
-cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s, int groups) {
-    dim3 grid(a.n_heads, S, groups);
+// a.part must hold cl_attn_rows_part_floats(H, S, T, hd) floats, a.tickets H zeroed counters.
+cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s) {
+    dim3 grid(a.n_heads, S);
     const size_t es = wdtype == 1 ? 2 : 4;
     const size_t smem = (((size_t)AR_WARPS * T * (a.head_dim + 2) * sizeof(float) + 15) & ~(size_t)15) + (size_t)AR_WARPS * 2 * 32 * a.head_dim * es;
 #define AR_LAUNCH(HDV, TT)                                                                                            \

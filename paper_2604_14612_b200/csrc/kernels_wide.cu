@@ -10,6 +10,7 @@
 // 148 SMs when a matrix has few output tiles (4096 outputs are 16 tiles), and the parts are added in a fixed order
 // by the small kernel that consumes the product:
 //   k_wide_rope_append   q, k, v: rotary embedding at the row's position, cache append, q left in place
+//   k_attn_wide          causal attention of the pass's rows over the cache -> hi/lo rows of the output projection
 //   k_wide_norm          x += product (or x = E[token]); hidden tap; RMSNorm -> hi/lo rows of the next GEMM
 //   k_wide_silu          h = silu(gate) * up on the interleaved gate/up product -> hi/lo rows of the down projection
 // Warp roles: warp 0 TMA producer (A hi 128 x 64, A lo 128 x 64, B 256 x 64 as two 128-row boxes, 128-byte swizzle,
@@ -223,6 +224,175 @@ __global__ void k_wide_rope_append(float *P, int splits, int M, int hd, int d, i
     vc[i + half] = __float2bfloat16_rn(total(d + kvd + h * hd + i + half));
 }
 
+// ---- causal attention of the rows of the pass over the cache -------------------------------------------------
+// grid (H, blocks of 64 rows), 256 threads.  Row t sits at position ctx + t and attends to the keys 0 .. ctx + t
+// (its own key is already in the cache).  The keys are walked 64 at a time; per tile the 64 x 64 scores
+// S = Q K^T and the update O += P V are register-tiled fp32 products out of shared memory (thread (ty, tx): rows
+// 4 ty .. 4 ty + 3; keys 4 tx .. 4 tx + 3 of S; columns tx * 4 + 64 v .. of O), with the usual running maximum and
+// sum per row.  The 16 threads of a row group are half a warp, so row reductions are four shuffles.  Blocks of
+// late rows see the most keys and are scheduled first.
+constexpr int AQ = 64, AK = 64, APS = 68;   // rows per CTA, keys per tile, row stride of the probability tile
+
+template <int HD>
+__global__ void __launch_bounds__(256, 2)
+k_attn_wide(const float *q, int ld_q, const __nv_bfloat16 *kcache, const __nv_bfloat16 *vcache, __nv_bfloat16 *out_b,
+            int lo_row0, int M, int d, int H, int Hkv, int max_seq, const ClDevState *st) {
+    constexpr int NV = HD / 64;                       // float4 column groups of O per thread
+    constexpr int KP = (HD * AK > AQ * APS) ? HD * AK : AQ * APS;
+    extern __shared__ __align__(16) float asm_[];
+    float *Qt = asm_;              // [HD][AQ]   queries, transposed, scaled by 1 / sqrt(hd)
+    float *Kt = Qt + HD * AQ;      // [HD][AK]   keys of the tile, transposed; reused as Ps [AQ][APS] (probabilities)
+    float *Vs = Kt + KP;           // [AK][HD]   values of the tile
+    float *Ps = Kt;
+    const int h = blockIdx.x, qb = (int)gridDim.y - 1 - (int)blockIdx.y;
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int ctx = st->ctx, r0 = qb * AQ;
+    const int rlast = min(r0 + AQ, M) - 1;            // last live row of this block
+    const int nkeys = min(ctx + rlast + 1, max_seq);
+    const int kvh = h / (H / Hkv);
+    const __nv_bfloat16 *Kc = kcache + (size_t)kvh * max_seq * HD, *Vc = vcache + (size_t)kvh * max_seq * HD;
+    const float scale = rsqrtf((float)HD);
+
+    for (int i = tid; i < AQ * HD / 4; i += 256) {
+        const int row = i % AQ, c4 = i / AQ;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r0 + row < M) v = *(const float4 *)(q + (size_t)(r0 + row) * ld_q + h * HD + c4 * 4);
+        Qt[(c4 * 4 + 0) * AQ + row] = v.x * scale;
+        Qt[(c4 * 4 + 1) * AQ + row] = v.y * scale;
+        Qt[(c4 * 4 + 2) * AQ + row] = v.z * scale;
+        Qt[(c4 * 4 + 3) * AQ + row] = v.w * scale;
+    }
+    float m_run[4], l_run[4], o[4][NV][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        m_run[i] = -INFINITY;
+        l_run[i] = 0.f;
+#pragma unroll
+        for (int v = 0; v < NV; ++v)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) o[i][v][e] = 0.f;
+    }
+
+    for (int k0 = 0; k0 < nkeys; k0 += AK) {
+        __syncthreads();   // the previous tile's reads of Ps and Vs are over (and Qt is written, first time round)
+        // keys: thread -> (key, 8 head-dim elements); transposed to Kt.  values: natural layout.
+        for (int i = tid; i < AK * HD / 8; i += 256) {
+            const int key = i % AK, c8 = i / AK;
+            uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+            if (k0 + key < nkeys) raw = *(const uint4 *)(Kc + (size_t)(k0 + key) * HD + c8 * 8);
+            const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                Kt[(c8 * 8 + 2 * e) * AK + key] = __uint_as_float(u[e] << 16);
+                Kt[(c8 * 8 + 2 * e + 1) * AK + key] = __uint_as_float(u[e] & 0xffff0000u);
+            }
+        }
+        for (int i = tid; i < AK * HD / 8; i += 256) {
+            const int key = i / (HD / 8), c8 = i % (HD / 8);
+            uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+            if (k0 + key < nkeys) raw = *(const uint4 *)(Vc + (size_t)(k0 + key) * HD + c8 * 8);
+            float4 *dst = (float4 *)(Vs + key * HD + c8 * 8);
+            dst[0] = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u), __uint_as_float(raw.y << 16),
+                                 __uint_as_float(raw.y & 0xffff0000u));
+            dst[1] = make_float4(__uint_as_float(raw.z << 16), __uint_as_float(raw.z & 0xffff0000u), __uint_as_float(raw.w << 16),
+                                 __uint_as_float(raw.w & 0xffff0000u));
+        }
+        __syncthreads();
+        float sc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) sc[i][j] = 0.f;
+#pragma unroll 8
+        for (int k = 0; k < HD; ++k) {
+            const float4 qv = *(const float4 *)(Qt + k * AQ + 4 * ty);
+            const float4 kv = *(const float4 *)(Kt + k * AK + 4 * tx);
+            const float qa[4] = {qv.x, qv.y, qv.z, qv.w}, ka[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) sc[i][j] = fmaf(qa[i], ka[j], sc[i][j]);
+        }
+        __syncthreads();   // everyone is done with Kt: it becomes Ps
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int pos = ctx + r0 + 4 * ty + i;   // causal limit of this row
+            const bool live = r0 + 4 * ty + i < M;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (!(live && k0 + 4 * tx + j <= pos)) sc[i][j] = -INFINITY;
+                mx = fmaxf(mx, sc[i][j]);
+            }
+#pragma unroll
+            for (int w = 8; w > 0; w >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, w));
+            const float m_new = fmaxf(m_run[i], mx);
+            float p[4] = {0.f, 0.f, 0.f, 0.f}, ps = 0.f, resc = 1.f;
+            if (m_new > -INFINITY) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    p[j] = (sc[i][j] > -INFINITY) ? expf(sc[i][j] - m_new) : 0.f;
+                    ps += p[j];
+                }
+                resc = (m_run[i] > -INFINITY) ? expf(m_run[i] - m_new) : 0.f;
+                m_run[i] = m_new;
+            }
+#pragma unroll
+            for (int w = 8; w > 0; w >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, w);
+            l_run[i] = fmaf(l_run[i], resc, ps);
+#pragma unroll
+            for (int v = 0; v < NV; ++v)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o[i][v][e] *= resc;
+            *(float4 *)(Ps + (4 * ty + i) * APS + 4 * tx) = make_float4(p[0], p[1], p[2], p[3]);
+        }
+        __syncthreads();
+#pragma unroll 2
+        for (int kk = 0; kk < AK; kk += 4) {
+            float pr[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 t4 = *(const float4 *)(Ps + (4 * ty + i) * APS + kk);
+                pr[i][0] = t4.x; pr[i][1] = t4.y; pr[i][2] = t4.z; pr[i][3] = t4.w;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const float4 vv = *(const float4 *)(Vs + (kk + j) * HD + v * 64 + tx * 4);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        o[i][v][0] = fmaf(pr[i][j], vv.x, o[i][v][0]);
+                        o[i][v][1] = fmaf(pr[i][j], vv.y, o[i][v][1]);
+                        o[i][v][2] = fmaf(pr[i][j], vv.z, o[i][v][2]);
+                        o[i][v][3] = fmaf(pr[i][j], vv.w, o[i][v][3]);
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = r0 + 4 * ty + i;
+        if (row >= M || !(l_run[i] > 0.f)) continue;
+        const float inv = 1.f / l_run[i];
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const size_t col = (size_t)h * HD + v * 64 + tx * 4;
+            unsigned hi[4], lo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                __nv_bfloat16 bh, bl;
+                w_split(o[i][v][e] * inv, bh, bl);
+                hi[e] = __bfloat16_as_ushort(bh);
+                lo[e] = __bfloat16_as_ushort(bl);
+            }
+            *(uint2 *)(out_b + (size_t)row * d + col) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+            *(uint2 *)(out_b + (size_t)(lo_row0 + row) * d + col) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+        }
+    }
+}
+
 // grid (M, ceil(F / 256)): the gate/up product has rows interleaved (2 i = gate_i, 2 i + 1 = up_i).
 __global__ void __launch_bounds__(256) k_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0) {
     const int t = blockIdx.x, i = blockIdx.y * 256 + threadIdx.x;
@@ -286,5 +456,35 @@ cudaError_t cl_launch_wide_rope_append(float *P, int splits, int M, int H, int H
 
 cudaError_t cl_launch_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, cudaStream_t s) {
     k_wide_silu<<<dim3(M, (F + 255) / 256), 256, 0, s>>>(P, splits, M, F, A, lo_row0);
+    return cudaGetLastError();
+}
+
+cudaError_t cl_launch_attn_wide(const float *q, int ld_q, const void *kcache, const void *vcache, __nv_bfloat16 *out_b,
+                                int lo_row0, int M, int d, int H, int Hkv, int hd, int max_seq, const ClDevState *st,
+                                cudaStream_t s) {
+    const dim3 grid(H, (M + AQ - 1) / AQ);
+    const int kp = (hd * AK > AQ * APS) ? hd * AK : AQ * APS;
+    const size_t smem = (size_t)(hd * AQ + kp + AK * hd) * sizeof(float);
+    if (hd == 128) {
+        static bool set128 = false;
+        if (!set128) {
+            cudaError_t e = cudaFuncSetAttribute(k_attn_wide<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            set128 = true;
+        }
+        k_attn_wide<128><<<grid, 256, smem, s>>>(q, ld_q, (const __nv_bfloat16 *)kcache, (const __nv_bfloat16 *)vcache, out_b,
+                                                 lo_row0, M, d, H, Hkv, max_seq, st);
+    } else if (hd == 64) {
+        static bool set64 = false;
+        if (!set64) {
+            cudaError_t e = cudaFuncSetAttribute(k_attn_wide<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            set64 = true;
+        }
+        k_attn_wide<64><<<grid, 256, smem, s>>>(q, ld_q, (const __nv_bfloat16 *)kcache, (const __nv_bfloat16 *)vcache, out_b,
+                                                lo_row0, M, d, H, Hkv, max_seq, st);
+    } else {
+        return cudaErrorInvalidValue;
+    }
     return cudaGetLastError();
 }
