@@ -495,3 +495,46 @@ def test_two_tap_confidences(name, L):
         for ti, key in enumerate(("hid_attn", "hid_ffn")):
             want = v[key][:, i, :]
             assert np.abs(ring[:, ti, slot].float().numpy() - want).max() <= 2 ** -7 * max(1.0, float(np.abs(want).max()))
+
+
+def test_llama3_vocabulary_head():
+    """V = 128256 (the LLaMA-3 vocabulary, 501 head tiles of 256 rows) on a small bf16 model: draft head, verify head,
+    prompt pass and the all-layer scoring against the oracle."""
+    base = synth.WORKLOADS["C2"].shape
+    sh = dataclasses.replace(base, n_layers=2, d_model=256, n_heads=4, n_kv_heads=4, d_ffn=688, vocab=128256, max_seq=96)
+    P = 16
+    om, ctx, _ = make_pair(sh, 21, tap_positions=P, gen_device="cuda")
+    prompt = synth.make_prompt(21, 24, sh.vocab)
+    rep = lockstep_generate(om, ctx, prompt, synth.layers_to_mask([1], 2), 4, 8, tap=True)
+    print("V128256", rep)
+    assert rep.cycles > 0
+    ctx.cl_prefill(prompt, tap_hidden=True)
+    g = ctx.cl_layer_confidences()
+    want_h = oracle_prefill_hidden(om, prompt, P)
+    hid = torch.tensor(want_h).to(torch.bfloat16)
+    o = oracle.layer_confidences(hid, om._keep["lm_head"], om._keep["final_norm"], sh.rms_eps)
+    order = [(p % P) for p in range(len(prompt) - P, len(prompt))]
+    assert np.abs(g["conf"][:, order] - o["conf"]).max() <= TOL
+    assert np.abs(g["c_layer"] - o["c_layer"]).max() <= TOL
+
+
+def test_second_prompt_reuses_the_searched_skip_set():
+    """Section 3: the set found on one input keeps drafting for later inputs.  After an interval search on prompt A the
+    best set stays installed; a new cl_prefill (prompt B) leaves it in place, and generation on B with it is lossless
+    (equal to vanilla decoding of B up to the first near tie)."""
+    w = synth.WORKLOADS["C1"]
+    sh = dataclasses.replace(w.shape, max_seq=160)
+    om, ctx, _ = make_pair(sh, w.seed, tap_positions=8)
+    a = synth.make_prompt(w.seed, w.prompt_len, sh.vocab)
+    b = synth.make_prompt(w.seed + 77, 23, sh.vocab)
+    ctx.cl_prefill(a, tap_hidden=True)
+    ctx.cl_set_skip_set(synth.layers_to_mask([1, 2], sh.n_layers))
+    got = ctx.cl_generate_search(3, 40, 4, 10.0, 2, cl.SelectCfg.make(w.lo, w.hi, n_skip=1))
+    installed = [l for l, m in enumerate(ctx.cl_get_skip_set()) if m]
+    assert installed == got["final_set"] and not got["searching"]
+    first = ctx.cl_prefill(b)
+    assert [l for l, m in enumerate(ctx.cl_get_skip_set()) if m] == installed
+    spec, _ = ctx.cl_generate(3, 30)
+    ref = oracle.generate_vanilla(om, b, 31)
+    lim = next((i for i, m in enumerate(ref["margins"]) if m < 1e-4), 31)
+    assert ([first] + [int(t) for t in spec])[:lim] == ref["tokens"][:lim]
