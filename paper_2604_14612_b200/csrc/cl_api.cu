@@ -399,7 +399,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 DM(c->v_ssq, ((d + 127) / 128) * CL_SLOTS * 4);
                 c->v_att_S = c->n_sm / g.n_heads;   // one wave of CTAs
                 if (c->v_att_S < 1) c->v_att_S = 1;
-                if (c->v_att_S > 16) c->v_att_S = 16;
+                if (c->v_att_S > 8) c->v_att_S = 8;
                 DM(c->v_att_part, cl_attn_rows_part_floats(g.n_heads, c->v_att_S, CL_MAX_T, g.head_dim) * 4);
                 DM(c->v_head_part, ((V + 127) / 128) * CL_SLOTS * sizeof(ClHeadPartial));
                 c->map_qkv.resize(L); c->map_o.resize(L); c->map_gu.resize(L); c->map_d.resize(L);
@@ -517,6 +517,7 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
         KL(cl_launch_rope_append(wd, c->qkv, T, row0, g.n_heads, g.n_kv_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq, c->st,
                                  c->stream));
         ClAttnArgs a;
+        a.rope_cs = nullptr;
         a.q = c->qkv; a.ld_q = qkv_rows; a.n_kv_heads = g.n_kv_heads; a.kcache = y.kc; a.vcache = y.vc; a.part = c->att_part; a.tickets = c->tickets + 1;
         a.out = c->att; a.out_b = nullptr; a.nh = 0; a.st = c->st; a.row0 = row0; a.n_heads = g.n_heads; a.head_dim = g.head_dim; a.d_model = d;
         a.nsplit = c->nsplit; a.per_max = c->per_max; a.max_seq = g.max_seq;
@@ -559,8 +560,8 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
         ClSkinnyArgs a = b;
         a.rows = qkv_rows; a.KB = KBd; a.epi = CL_VEPI_STORE; a.ssq_in = c->v_ssq; a.out = c->qkv; a.ld = qkv_rows;
         KL(cl_launch_skinny(c->map_qkv[l], c->map_bx[sel], a, G, c->stream));
-        KL(cl_launch_rope_append(1, c->qkv, T, row0, g.n_heads, g.n_kv_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq, c->st, c->stream));
-        ClAttnArgs t;
+        ClAttnArgs t;   // (rotary embedding and cache append of the rows happen inside the attention kernel)
+        t.rope_cs = c->rope_cs;
         t.q = c->qkv; t.ld_q = qkv_rows; t.n_kv_heads = g.n_kv_heads; t.kcache = y.kc; t.vcache = y.vc; t.part = c->att_part; t.tickets = c->tickets + 1;
         t.out = c->att; t.out_b = c->batt; t.nh = nh; t.st = c->st; t.row0 = row0; t.n_heads = g.n_heads; t.head_dim = g.head_dim;
         t.d_model = d; t.nsplit = c->nsplit; t.per_max = c->per_max; t.max_seq = g.max_seq;

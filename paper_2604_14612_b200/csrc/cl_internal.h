@@ -67,6 +67,8 @@ struct ClAttnArgs {
     int nh;
     const ClDevState *st;
     int row0, n_heads, n_kv_heads, head_dim, d_model, nsplit, per_max, max_seq;
+    const float2 *rope_cs;  // k_attn_rows only, optional: q and the rows' own k, v are still raw in the [q | k | v] rows;
+                            // the kernel applies the rotary embedding itself and appends k, v to the cache
 };
 
 // Per-layer device pointers as the token-step kernel sees them.

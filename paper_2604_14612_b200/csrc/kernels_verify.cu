@@ -108,6 +108,34 @@ __device__ __forceinline__ void split_bf16(float v, __nv_bfloat16 &hi, __nv_bflo
     lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
+// Adds the partial accumulators of tile m (from CTAs c_first .. c_last, in that order) into v: PB partials are in
+// flight at a time, NQ float4 each (N = 4 NQ columns).  (Eight in flight measured slower: tiles cut over two or three
+// CTAs are the common case and the extra requests only load L2.)
+template <int NQ, int PB>
+__device__ __forceinline__ void add_partials(float (&v)[32], const ClSkinnyArgs &a, long long U, int G, int m, int c_first,
+                                             int c_last, int rloc) {
+    for (int cc0 = c_first; cc0 <= c_last; cc0 += PB) {
+        float4 p[PB][NQ];
+#pragma unroll
+        for (int j = 0; j < PB; ++j) {
+            const int cc = min(cc0 + j, c_last);
+            const int seg_idx = m - (int)((U * cc / G) / a.KB);   // tiles CTA cc touches are consecutive
+            const float4 *src = (const float4 *)(a.ws + (((size_t)cc * CL_V_MAXSEG + seg_idx) * VM + rloc) * WS_LD);
+#pragma unroll
+            for (int i = 0; i < NQ; ++i) p[j][i] = __ldcg(src + i);
+        }
+#pragma unroll
+        for (int j = 0; j < PB; ++j) {
+            if (cc0 + j <= c_last) {
+#pragma unroll
+                for (int i = 0; i < NQ; ++i) {
+                    v[4 * i] += p[j][i].x; v[4 * i + 1] += p[j][i].y; v[4 * i + 2] += p[j][i].z; v[4 * i + 3] += p[j][i].w;
+                }
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(VTHREADS, 2)
 k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, ClSkinnyArgs a) {
     if (a.st && a.st->done) return;   // written only between launches: uniform over the grid
@@ -263,29 +291,8 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
                 __threadfence();
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = 0.f;
-                for (int cc0 = c_first; cc0 <= c_last; cc0 += 4) {   // four partials in flight, added in CTA order
-                    float4 p[4][8];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int cc = min(cc0 + j, c_last);
-                        const int seg_idx = m - (int)((U * cc / G) / a.KB);   // tiles CTA cc touches are consecutive
-                        const float4 *src = (const float4 *)(a.ws + (((size_t)cc * CL_V_MAXSEG + seg_idx) * VM + rloc) * WS_LD);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (4 * i < a.N) p[j][i] = __ldcg(src + i);
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (cc0 + j <= c_last) {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                if (4 * i < a.N) {
-                                    v[4 * i] += p[j][i].x; v[4 * i + 1] += p[j][i].y; v[4 * i + 2] += p[j][i].z; v[4 * i + 3] += p[j][i].w;
-                                }
-                            }
-                        }
-                    }
-                }
+                if (a.N == 16) add_partials<4, 4>(v, a, U, G, m, c_first, c_last, rloc);
+                else add_partials<8, 4>(v, a, U, G, m, c_first, c_last, rloc);
             }
             // ---- epilogue of a complete tile: tot[t] = hi column + lo column (loops unrolled so that the accumulator
             // stays in registers; rows of a pass never exceed CL_MAX_T)
@@ -481,12 +488,18 @@ cudaError_t cl_launch_head_finalize(const ClHeadPartial *part, int tiles, int T,
 namespace {
 
 constexpr int AR_WARPS = 8;
+constexpr int AR_MAXS = 8;   // most parts the keys of a head are cut into
 
 // (Loops over keys stay rolled and the row count is a template parameter: the kernel runs its code once, so its
 // time is instruction fetch, and a fully unrolled version measured 55 us against a few us of work.)
 template <typename ST, int HD, int T>
 __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S) {
-    if (a.st->done) return;
+    // programmatic dependent launch: the next launch (the output projection) may set itself up beside this one;
+    // everything an earlier launch wrote is read after the wait
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int2 ctx_done = *(const int2 *)a.st;   // (ctx, done): one load
+    if (ctx_done.y) return;
     constexpr int EPL = 16 / (int)sizeof(ST), LPK = HD / EPL, KPW = 32 / LPK, VPL = HD / 32;
     constexpr int REC = HD + 2;
     extern __shared__ __align__(16) float wrec[];   // [AR_WARPS][T][REC], then per warp 32 key rows and 32 value rows
@@ -498,21 +511,49 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
     unsigned char *stage_v = stage_k + 32 * ROWB;
     const int h = blockIdx.x, s = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int base = a.st->ctx + a.row0, nkeys = base + T, d = a.d_model;
+    const int base = ctx_done.x + a.row0, nkeys = base + T, d = a.d_model;
     if (nkeys > a.max_seq) return;
     const int k0 = (int)((long long)nkeys * s / S), k1 = (int)((long long)nkeys * (s + 1) / S);
     const int kw0 = k0 + (k1 - k0) * warp / AR_WARPS, kw1 = k0 + (k1 - k0) * (warp + 1) / AR_WARPS;
     const int sub = lane / LPK, li = lane % LPK;
     const float scale = rsqrtf((float)HD);
     const int kvh = h / (a.n_heads / a.n_kv_heads);                       // grouped-query attention
-    const ST *Kc = (const ST *)a.kcache + (size_t)kvh * a.max_seq * HD;   // cache layout [kv head][position][hd]
-    const ST *Vc = (const ST *)a.vcache + (size_t)kvh * a.max_seq * HD;
+    ST *Kc = (ST *)a.kcache + (size_t)kvh * a.max_seq * HD;   // cache layout [kv head][position][hd]
+    ST *Vc = (ST *)a.vcache + (size_t)kvh * a.max_seq * HD;
 
+    constexpr int HALF = HD / 2;
+    const int kvd = a.n_kv_heads * HD;
     float qr[T][EPL];
+    {
+        // vector loads, all requested before any is used; rotary embedding at the row's position (pairs i, i + hd / 2)
+        const int i0 = li * EPL, ip = (i0 + HALF) % HD;
+        float4 own[T][EPL / 4], par[T][EPL / 4], cs[T][EPL / 2];
 #pragma unroll
-    for (int t = 0; t < T; ++t)
+        for (int t = 0; t < T; ++t) {
+            const float *qrow = a.q + (size_t)t * a.ld_q + h * HD;
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) qr[t][e] = (t < T) ? a.q[(size_t)t * a.ld_q + h * HD + li * EPL + e] * scale : 0.f;
+            for (int v = 0; v < EPL / 4; ++v) {
+                own[t][v] = *(const float4 *)(qrow + i0 + 4 * v);
+                if (a.rope_cs) par[t][v] = *(const float4 *)(qrow + ip + 4 * v);
+            }
+            if (a.rope_cs) {
+                const float4 *c4 = (const float4 *)(a.rope_cs + (size_t)(base + t) * HALF + (i0 % HALF));
+#pragma unroll
+                for (int v = 0; v < EPL / 2; ++v) cs[t][v] = c4[v];
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < T; ++t)
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                float v = ((const float *)own[t])[e];
+                if (a.rope_cs) {
+                    const float p = ((const float *)par[t])[e], c = ((const float *)cs[t])[2 * e], sn = ((const float *)cs[t])[2 * e + 1];
+                    v = (i0 < HALF) ? v * c - p * sn : v * c + p * sn;
+                }
+                qr[t][e] = v * scale;
+            }
+    }
     float m_run[T], l_run[T], o_run[T][VPL];
 #pragma unroll
     for (int t = 0; t < T; ++t) {
@@ -523,6 +564,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
     }
     for (int j0 = kw0; j0 < kw1; j0 += 32) {
         const int n = min(32, kw1 - j0);
+        const int n_old = a.rope_cs ? max(0, min(n, base - j0)) : n;   // rows of this pass that are in the cache already
         // stage this pass's key and value rows in shared memory: every 16-byte piece is requested before any is used,
         // so the pass costs one memory round trip; the (rolled) loops below then read shared memory
         __syncwarp();
@@ -532,7 +574,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
 #pragma unroll
             for (int it = 0; it < CPR; ++it) {
                 const int cidx = it * 32 + lane;   // chunk cidx of the pass: row cidx / CPR
-                if (cidx < n * CPR) {
+                if (cidx < n_old * CPR) {
                     tk[it] = gk[cidx];
                     tv[it] = gv[cidx];
                 }
@@ -540,9 +582,29 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
 #pragma unroll
             for (int it = 0; it < CPR; ++it) {
                 const int cidx = it * 32 + lane;
-                if (cidx < n * CPR) {
+                if (cidx < n_old * CPR) {
                     ((uint4 *)stage_k)[cidx] = tk[it];
                     ((uint4 *)stage_v)[cidx] = tv[it];
+                }
+            }
+        }
+        if (n_old < n && sizeof(ST) == 2) {
+            // the pass's own rows: k and v come raw from the projection; rotate k at its position, round both to the
+            // storage type, stage them, and (one query head per key/value head) append them to the cache
+            const bool writer = h % (a.n_heads / a.n_kv_heads) == 0;
+#pragma unroll 4
+            for (int idx = lane; idx < (n - n_old) * HALF; idx += 32) {
+                const int r = n_old + idx / HALF, i = idx % HALF, j = j0 + r;
+                const float *krow = a.q + (size_t)(j - base) * a.ld_q + d + kvh * HD, *vrow = krow + kvd;
+                const float2 cs = a.rope_cs[(size_t)j * HALF + i];
+                const float ka = krow[i], kb = krow[i + HALF];
+                const __nv_bfloat16 k0 = __float2bfloat16_rn(ka * cs.x - kb * cs.y), k1 = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
+                const __nv_bfloat16 v0 = __float2bfloat16_rn(vrow[i]), v1 = __float2bfloat16_rn(vrow[i + HALF]);
+                __nv_bfloat16 *sk = (__nv_bfloat16 *)(stage_k + (size_t)r * ROWB), *sv = (__nv_bfloat16 *)(stage_v + (size_t)r * ROWB);
+                sk[i] = k0; sk[i + HALF] = k1; sv[i] = v0; sv[i + HALF] = v1;
+                if (writer) {
+                    __nv_bfloat16 *ck = (__nv_bfloat16 *)(Kc + (size_t)j * HD), *cv = (__nv_bfloat16 *)(Vc + (size_t)j * HD);
+                    ck[i] = k0; ck[i + HALF] = k1; cv[i] = v0; cv[i + HALF] = v1;
                 }
             }
         }
@@ -680,19 +742,38 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    for (int i = tid; i < T * HD; i += blockDim.x) {
-        const int t = i / HD, e = i % HD;
+    // every part's (max, sum, output element) of every output of this thread is requested before any is used:
+    // one round trip in all, not one per part and output
+    constexpr int NOUT = (T * HD + AR_WARPS * 32 - 1) / (AR_WARPS * 32);
+    float pm[NOUT][AR_MAXS], pl[NOUT][AR_MAXS], po[NOUT][AR_MAXS];
+#pragma unroll
+    for (int it = 0; it < NOUT; ++it) {
+        const int i = min(it * AR_WARPS * 32 + tid, T * HD - 1), t = i / HD, e = i % HD;
         const float *p0 = a.part + (size_t)h * S * T * REC + (size_t)t * REC;
+#pragma unroll
+        for (int s2 = 0; s2 < AR_MAXS; ++s2) {
+            const float *ps = p0 + (size_t)min(s2, S - 1) * T * REC;
+            pm[it][s2] = __ldcg(ps);
+            pl[it][s2] = (s2 < S) ? __ldcg(ps + 1) : 0.f;
+            po[it][s2] = __ldcg(ps + 2 + e);
+        }
+    }
+#pragma unroll
+    for (int it = 0; it < NOUT; ++it) {
+        const int i = it * AR_WARPS * 32 + tid;
+        if (i >= T * HD) break;
+        const int t = i / HD, e = i % HD;
         float M = -INFINITY;
-        for (int s2 = 0; s2 < S; ++s2)
-            if (__ldcg(p0 + (size_t)s2 * T * REC + 1) > 0.f) M = fmaxf(M, __ldcg(p0 + (size_t)s2 * T * REC));
+#pragma unroll
+        for (int s2 = 0; s2 < AR_MAXS; ++s2)
+            if (pl[it][s2] > 0.f) M = fmaxf(M, pm[it][s2]);
         float Ls = 0.f, O = 0.f;
-        for (int s2 = 0; s2 < S; ++s2) {
-            const float l2 = __ldcg(p0 + (size_t)s2 * T * REC + 1);
-            if (l2 > 0.f) {
-                const float f = expf(__ldcg(p0 + (size_t)s2 * T * REC) - M);
-                Ls = fmaf(l2, f, Ls);
-                O = fmaf(__ldcg(p0 + (size_t)s2 * T * REC + 2 + e), f, O);
+#pragma unroll
+        for (int s2 = 0; s2 < AR_MAXS; ++s2) {   // part order
+            if (pl[it][s2] > 0.f) {
+                const float f = expf(pm[it][s2] - M);
+                Ls = fmaf(pl[it][s2], f, Ls);
+                O = fmaf(po[it][s2], f, O);
             }
         }
         const float o = O / Ls;
@@ -711,6 +792,7 @@ size_t cl_attn_rows_part_floats(int H, int S, int T, int hd) { return (size_t)H 
 
 // a.part must hold cl_attn_rows_part_floats(H, S, T, hd) floats, a.tickets H zeroed counters.
 cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s) {
+    if (S < 1 || S > AR_MAXS) return cudaErrorInvalidValue;
     dim3 grid(a.n_heads, S);
     const size_t es = wdtype == 1 ? 2 : 4;
     const size_t smem = (((size_t)AR_WARPS * T * (a.head_dim + 2) * sizeof(float) + 15) & ~(size_t)15) + (size_t)AR_WARPS * 2 * 32 * a.head_dim * es;
@@ -719,7 +801,18 @@ cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, c
         cudaError_t e_ = cudaFuncSetAttribute(k_attn_rows<__nv_bfloat16, HDV, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                               (int)smem);                                                             \
         if (e_ != cudaSuccess) return e_;                                                                             \
-        k_attn_rows<__nv_bfloat16, HDV, TT><<<grid, AR_WARPS * 32, smem, s>>>(a, S);                                    \
+        cudaLaunchConfig_t cfg_;                                                                                      \
+        memset(&cfg_, 0, sizeof(cfg_));                                                                               \
+        cfg_.gridDim = grid;                                                                                          \
+        cfg_.blockDim = dim3(AR_WARPS * 32);                                                                          \
+        cfg_.dynamicSmemBytes = smem;                                                                                 \
+        cfg_.stream = s;                                                                                              \
+        cudaLaunchAttribute attr_[1];                                                                                 \
+        attr_[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                             \
+        attr_[0].val.programmaticStreamSerializationAllowed = 1;                                                      \
+        cfg_.attrs = attr_;                                                                                           \
+        cfg_.numAttrs = 1;                                                                                            \
+        return cudaLaunchKernelEx(&cfg_, k_attn_rows<__nv_bfloat16, HDV, TT>, a, S);                                  \
     }
 #define AR_CASE(TT)                                              \
     case TT:                                                     \
