@@ -15,7 +15,7 @@
  * Only tests, the smoke check and the benchmark's CPU-baseline leg may call this; it shares
  * no code with the CUDA library and the CUDA library never calls it.
  *
- * Arithmetic: weights are read in their storage type (fp32, or bf16 bit patterns widened
+ * Arithmetic: weights are read in their storage type (fp32, or bf16 / fp16 bit patterns widened
  * exactly); activations are kept as fp32 values; every dot product, norm, softmax and entropy
  * sum is accumulated in double.  There is no blocking, fusion or reordering: each output
  * element is one straight loop over its inputs.  OpenMP only spreads independent output rows
@@ -32,7 +32,7 @@
 typedef struct {
     int n_layers, d_model, n_heads, head_dim, d_ffn, vocab, max_seq;
     float rms_eps, rope_theta;
-    int weight_dtype; /* 0 = fp32, 1 = bf16 (also the storage type of KV cache and taps) */
+    int weight_dtype; /* 0 = fp32, 1 = bf16, 2 = fp16 (also the storage type of KV cache and taps) */
     int n_kv_heads;   /* key/value heads (grouped-query attention): query head h reads key/value head h / (n_heads / n_kv_heads) */
 } orc_cfg;
 
@@ -65,10 +65,40 @@ float orc_round_bf16(float f) {
     return f;
 }
 
-static inline float store_round(float f, int dtype) { return dtype == 1 ? orc_round_bf16(f) : f; }
+/* IEEE 754 binary16 (1 sign, 5 exponent, 10 fraction bits) -> fp32, exact */
+float orc_fp16_bits_to_f32(uint16_t b) {
+    const int sign = b >> 15, e = (b >> 10) & 31, frac = b & 1023;
+    double v;
+    if (e == 31) v = frac ? NAN : INFINITY;
+    else if (e == 0) v = ldexp((double)frac, -24);            /* subnormal: frac * 2^-24 */
+    else v = ldexp(1.0 + (double)frac / 1024.0, e - 15);
+    return (float)(sign ? -v : v);
+}
+
+/* round-to-nearest-even fp32 -> fp16 -> fp32, from the definition: the representable neighbours of |f| are
+ * multiples of the spacing 2^(E-10) with E = max(floor(log2 |f|), -14); ties go to the even multiple; what rounds to
+ * 2^16 or beyond is infinity. */
+float orc_round_fp16(float f) {
+    if (isnan(f) || isinf(f) || f == 0.0f) return f;
+    const double a = fabs((double)f);
+    int E;
+    frexp(a, &E);      /* a = m * 2^E with m in [0.5, 1): floor(log2 a) = E - 1 */
+    E -= 1;
+    if (E < -14) E = -14;
+    const double ulp = ldexp(1.0, E - 10);
+    double q = a / ulp, fl = floor(q), r = q - fl;
+    if (r > 0.5 || (r == 0.5 && fmod(fl, 2.0) == 1.0)) fl += 1.0;
+    double v = fl * ulp;
+    if (v >= 65520.0) v = INFINITY;   /* beyond the largest finite value 65504 plus half a spacing */
+    return (float)(f < 0 ? -v : v);
+}
+
+static inline float store_round(float f, int dtype) { return dtype == 1 ? orc_round_bf16(f) : dtype == 2 ? orc_round_fp16(f) : f; }
 
 static inline float wload(const void *w, size_t i, int dtype) {
-    return dtype == 1 ? bf16_bits_to_f32(((const uint16_t *)w)[i]) : ((const float *)w)[i];
+    return dtype == 1   ? bf16_bits_to_f32(((const uint16_t *)w)[i])
+           : dtype == 2 ? orc_fp16_bits_to_f32(((const uint16_t *)w)[i])
+                        : ((const float *)w)[i];
 }
 
 /* ---- elementary steps (exported so tests can pin each against its closed form) --------- */
@@ -81,6 +111,9 @@ double orc_dot_row(const void *W, int dtype, size_t row, int cols, const float *
         const uint16_t *w = (const uint16_t *)W + base;
 #pragma omp simd reduction(+ : acc)
         for (int c = 0; c < cols; ++c) acc += (double)bf16_bits_to_f32(w[c]) * (double)x[c];
+    } else if (dtype == 2) {
+        const uint16_t *w = (const uint16_t *)W + base;
+        for (int c = 0; c < cols; ++c) acc += (double)orc_fp16_bits_to_f32(w[c]) * (double)x[c];
     } else {
         const float *w = (const float *)W + base;
 #pragma omp simd reduction(+ : acc)

@@ -59,13 +59,18 @@ def lib():
         L.orc_matmul_rows.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp, C.c_int, vp]
         L.orc_round_bf16.restype = C.c_float
         L.orc_round_bf16.argtypes = [C.c_float]
+        L.orc_round_fp16.restype = C.c_float
+        L.orc_round_fp16.argtypes = [C.c_float]
+        L.orc_fp16_bits_to_f32.restype = C.c_float
+        L.orc_fp16_bits_to_f32.argtypes = [C.c_uint16]
         L.orc_read_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp]
         _LIB = L
     return _LIB
 
 
 def _as_host_array(t):
-    """torch tensor (cpu; bf16 or fp32) or ndarray -> contiguous ndarray viewing the storage bits."""
+    """torch tensor (cpu; bf16, fp16 or fp32) or ndarray -> contiguous ndarray viewing the storage bits (bf16 as
+    uint16, fp16 as float16)."""
     if isinstance(t, np.ndarray):
         return np.ascontiguousarray(t)
     import torch
@@ -94,11 +99,11 @@ class OracleModel:
         self.shape = shape
         self.L, self.d, self.V = shape.n_layers, shape.d_model, shape.vocab
         self._keep = {}
-        wd = 1 if shape.weight_dtype == "bf16" else 0
+        wd = {"fp32": 0, "bf16": 1, "fp16": 2}[shape.weight_dtype]
 
         def hold(name, t):
             a = _as_host_array(t)
-            exp = np.uint16 if (wd == 1 and not name.startswith(("norm", "final"))) else np.float32
+            exp = np.float32 if (wd == 0 or name.startswith(("norm", "final"))) else (np.uint16 if wd == 1 else np.float16)
             assert a.dtype == exp, (name, a.dtype)
             self._keep[name] = a
             return _ptr(a)

@@ -25,7 +25,7 @@ def _to_f32(hidden) -> np.ndarray:
 def layer_confidences(hidden, lm_head, final_norm, rms_eps: float = 1e-5,
                       rows: Optional[Sequence[int]] = None, positions: Optional[Sequence[int]] = None
                       ) -> Dict[str, np.ndarray]:
-    """hidden [R, P, d] (bf16 tensor or fp32 array); lm_head [V, d] (bf16 tensor / fp32); final_norm fp32 [d].
+    """hidden [R, P, d] (bf16 tensor or fp32 array); lm_head [V, d] (bf16 / fp16 tensor or fp32); final_norm fp32 [d].
 
     Returns conf, p_max (float64 [R', P']), argmax (int32), margin (top-2 logit gap) and
     c_layer (float64 [R'] = mean of conf over positions), restricted to the requested rows /
@@ -34,7 +34,7 @@ def layer_confidences(hidden, lm_head, final_norm, rms_eps: float = 1e-5,
     h = _to_f32(hidden)
     R, P, d = h.shape
     W = _as_host_array(lm_head)
-    wd = 1 if W.dtype == np.uint16 else 0
+    wd = 1 if W.dtype == np.uint16 else 2 if W.dtype == np.float16 else 0
     V = W.shape[0]
     g = np.ascontiguousarray(_to_f32(final_norm))
     rows = list(range(R)) if rows is None else list(rows)

@@ -35,7 +35,7 @@ class ModelShape:
     d_ffn: int
     vocab: int
     max_seq: int
-    weight_dtype: str = "bf16"          # "bf16" | "fp32": storage type of weights, KV cache and taps
+    weight_dtype: str = "bf16"          # "bf16" | "fp16" | "fp32": storage type of weights, KV cache and taps
     rms_eps: float = 1e-5
     rope_theta: float = 10000.0
     std: float = 0.02
@@ -103,7 +103,7 @@ def _normal(shape, std, seed, tid, dtype, device) -> torch.Tensor:
 
 
 def torch_dtype(weight_dtype: str) -> torch.dtype:
-    return {"bf16": torch.bfloat16, "fp32": torch.float32}[weight_dtype]
+    return {"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}[weight_dtype]
 
 
 def make_weights(shape: ModelShape, seed: int, device="cpu") -> Dict[str, object]:

@@ -248,6 +248,49 @@ def test_bf16_storage_rounds_cache_and_taps():
     assert np.array_equal(h, torch.tensor(h).to(torch.bfloat16).float().numpy())
 
 
+def test_round_fp16_and_widening_match_numpy_float16():
+    """The oracle's binary16 rounding and widening are written from the format's definition; numpy's float16 is an
+    independent implementation of the same format: random values over the whole range (subnormals, overflow), every
+    one of the 65536 bit patterns, and the tie cases."""
+    g = torch.Generator().manual_seed(6)
+    x = (torch.randn(8192, generator=g) * torch.logspace(-9, 6, 8192)).numpy().astype(np.float32)
+    with np.errstate(over="ignore"):
+        want = x.astype(np.float16).astype(np.float32)
+    got = np.array([lib().orc_round_fp16(float(v)) for v in x], np.float32)
+    assert np.array_equal(want, got)
+    bits = np.arange(65536, dtype=np.uint16)
+    wide = bits.view(np.float16).astype(np.float32)
+    mine = np.array([lib().orc_fp16_bits_to_f32(int(b)) for b in bits], np.float32)
+    ok = np.isfinite(wide)
+    assert np.array_equal(wide[ok], mine[ok]) and np.array_equal(np.isnan(wide), np.isnan(mine))
+    assert np.array_equal(np.isinf(wide), np.isinf(mine))
+    # ties to even: 1 + 2^-11 is halfway between 1 and 1 + 2^-10; 2^-25 is halfway between 0 and the smallest subnormal
+    assert lib().orc_round_fp16(1.0 + 2.0 ** -11) == 1.0
+    assert lib().orc_round_fp16(1.0 + 3 * 2.0 ** -11) == 1.0 + 2.0 ** -9
+    assert lib().orc_round_fp16(2.0 ** -25) == 0.0 and lib().orc_round_fp16(3 * 2.0 ** -25) == 2.0 ** -23
+    assert lib().orc_round_fp16(65519.0) == 65504.0 and np.isinf(lib().orc_round_fp16(65520.0))
+
+
+def test_fp16_storage_rounds_cache_and_taps_and_reads_weights_exactly():
+    import dataclasses
+    sh = dataclasses.replace(synth.WORKLOADS["C1"].shape, weight_dtype="fp16")
+    W = synth.make_weights(sh, 7)
+    m = oracle.OracleModel(sh, W)
+    out = m.forward(synth.make_prompt(7, 5, sh.vocab), 0, want_hidden=True)
+    k = m.read_kv(1, 0, 2)
+    assert np.array_equal(k, torch.tensor(k).to(torch.float16).float().numpy()) and np.any(k != 0)
+    h = out["hid_ffn"]
+    assert np.array_equal(h, torch.tensor(h).to(torch.float16).float().numpy())
+    # the same model with its fp16 weights widened to fp32 differs only by the storage rounding of the cache
+    # (relative 2^-11 per cached value): the weights are read exactly
+    sh32 = dataclasses.replace(sh, weight_dtype="fp32")
+    W32 = {n: ([t.float() for t in v] if isinstance(v, list) else v.float()) for n, v in W.items()}
+    one = synth.make_prompt(7, 1, sh.vocab)
+    a = oracle.OracleModel(sh, W).forward(one, 0)["logits"]
+    b = oracle.OracleModel(sh32, W32).forward(one, 0)["logits"]
+    assert np.abs(a - b).max() < 1e-3 and not np.array_equal(a, b)
+
+
 def test_bad_arguments_are_rejected():
     w = synth.WORKLOADS["C1"]
     m = oracle.OracleModel(w.shape, synth.make_weights(w.shape, w.seed))
