@@ -19,13 +19,15 @@
  *   - There is no CPU fallback: without a CUDA device every compute call fails with CL_ECUDA.
  *   - Matrices are row-major (out_features, in_features), as Llama checkpoints store them.
  *     weight_dtype selects the storage type of weights, KV cache and hidden-state taps:
- *     0 = fp32, 1 = bf16.  Norm gains are always fp32.  Arithmetic accumulates in fp32.
+ *     0 = fp32, 1 = bf16, 2 = fp16 (the type the paper's models run in, Section 4.1.1).  Norm gains are always
+ *     fp32.  Arithmetic accumulates in fp32.
  *   - Requirements: d_model = n_heads * head_dim, n_kv_heads divides n_heads (n_kv_heads < n_heads: grouped-query
  *     attention, query head h reads key/value head h / (n_heads / n_kv_heads)),
  *     head_dim in {64, 128}, d_model and d_ffn multiples of 8, 1 <= K <= CL_MAX_K.
  *   - Which kernels run: single-token steps (draft, vanilla) run in one persistent cooperative kernel when d_model and
  *     d_ffn are at most 16384 (bf16) / 8192 (fp32); passes of several rows (verify, prefill) and the confidence scoring
- *     of bf16 models run on the tensor cores (tcgen05); fp32 models and the cases above use per-matrix CUDA-core kernels.
+ *     of bf16 models run on the tensor cores (tcgen05); fp32 and fp16 models and the cases above use per-matrix
+ *     CUDA-core kernels.
  *     A prompt of more than 16 tokens (bf16 models) runs all rows but the last through wide tensor-core GEMMs, up to
  *     512 rows at a time, and the last row through the pass of several rows, which has the LM head.
  *     Environment switches read by cl_load (diagnostics): CL_DISABLE_STEP_KERNEL=1, CL_DISABLE_TC_PASS=1,
@@ -57,7 +59,7 @@ typedef struct cl_ctx cl_ctx;
 typedef struct {
     int n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab, max_seq;
     float rms_eps, rope_theta;
-    int weight_dtype;    /* 0 fp32, 1 bf16 */
+    int weight_dtype;    /* 0 fp32, 1 bf16, 2 fp16 */
     int tap_positions;   /* P: ring of the last P positions' per-layer hidden states (0 = no ring) */
     int tap_modules;     /* 0 or 1: record each layer's output (after the FFN add); 2: also the stream after the attention add
                             (Section 3.1 scores "FFNN and Attention" hidden states); a layer's confidence = mean over its taps */

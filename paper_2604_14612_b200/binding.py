@@ -157,7 +157,7 @@ class Context:
                  tap_positions: int = 0, stream: Optional[int] = None, n_kv_heads: int = 0, tap_modules: int = 1):
         self._L = load_library()
         self.cfg = ModelCfg(n_layers, d_model, n_heads, n_kv_heads or n_heads, d_model // n_heads, d_ffn, vocab, max_seq, rms_eps,
-                            rope_theta, 1 if weight_dtype == "bf16" else 0, tap_positions, tap_modules)
+                            rope_theta, {"fp32": 0, "bf16": 1, "fp16": 2}[weight_dtype], tap_positions, tap_modules)
         self.taps = 2 if tap_modules == 2 else 1
         self.weight_dtype = weight_dtype
         self._h = C.c_void_p()
@@ -332,7 +332,7 @@ class Context:
     def cl_read_hidden_ring(self):
         import torch
         L, P, d = self.cfg.n_layers, self.cfg.tap_positions, self.cfg.d_model
-        dt = torch.bfloat16 if self.cfg.weight_dtype == 1 else torch.float32
+        dt = {0: torch.float32, 1: torch.bfloat16, 2: torch.float16}[self.cfg.weight_dtype]
         out = torch.empty((L, self.taps, P, d), dtype=dt)
         self._ck(self._L.cl_read_hidden_ring(self._h, out.data_ptr()))
         return out if self.taps == 2 else out[:, 0]

@@ -176,7 +176,7 @@ extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **ou
     if (cfg->head_dim != 64 && cfg->head_dim != 128) return fail(c, CL_EINVAL, "cl_create: head_dim must be 64 or 128");
     if (cfg->d_model % 8 || (cfg->n_layers > 0 && (cfg->d_ffn <= 0 || cfg->d_ffn % 8)))
         return fail(c, CL_EINVAL, "cl_create: d_model and d_ffn must be multiples of 8");
-    if (cfg->weight_dtype != 0 && cfg->weight_dtype != 1) return fail(c, CL_EINVAL, "cl_create: weight_dtype must be 0 or 1");
+    if (cfg->weight_dtype < 0 || cfg->weight_dtype > 2) return fail(c, CL_EINVAL, "cl_create: weight_dtype must be 0, 1 or 2");
     if (cfg->tap_positions < 0) return fail(c, CL_EINVAL, "cl_create: tap_positions < 0");
     if (cfg->tap_modules < 0 || cfg->tap_modules > 2) return fail(c, CL_EINVAL, "cl_create: tap_modules must be 0, 1 or 2");
     int dev = 0;
@@ -192,7 +192,7 @@ extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **ou
     c->stream = (cudaStream_t)cuda_stream;
     c->device = dev;
     c->n_sm = prop.multiProcessorCount;
-    c->esz = cfg->weight_dtype == 1 ? 2 : 4;
+    c->esz = cfg->weight_dtype == 0 ? 4 : 2;
     c->taps = cfg->tap_modules == 2 ? 2 : 1;
     c->err[0] = 0;
     c->mask.assign((size_t)cfg->n_layers, 0);

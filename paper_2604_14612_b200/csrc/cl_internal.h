@@ -1,10 +1,36 @@
 // Internal declarations shared by the CUDA translation units of libconflayers.so.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 #include "conflayers.h"
+
+#ifdef __CUDACC__
+// Two stored 16-bit elements in one 32-bit word (the lower address in the low half) widened to fp32.
+template <typename ST>
+struct ClPair16;
+template <>
+struct ClPair16<__nv_bfloat16> {
+    static __device__ __forceinline__ void get(unsigned u, float &a, float &b) {
+        a = __uint_as_float(u << 16);
+        b = __uint_as_float(u & 0xffff0000u);
+    }
+};
+template <>
+struct ClPair16<__half> {
+    static __device__ __forceinline__ void get(unsigned u, float &a, float &b) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&u));
+        a = f.x;
+        b = f.y;
+    }
+};
+template <>
+struct ClPair16<float> {   // never used: fp32 storage has no packed pairs
+    static __device__ __forceinline__ void get(unsigned, float &a, float &b) { a = b = 0.f; }
+};
+#endif
 
 #define CL_MAX_T (CL_MAX_K + 1)   // rows of the widest pass (verify)
 #define CL_PREFILL_CHUNK 8        // prompt tokens per prefill pass

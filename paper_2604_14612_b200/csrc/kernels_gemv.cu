@@ -39,6 +39,16 @@ struct W8<__nv_bfloat16> {
     }
 };
 template <>
+struct W8<__half> {
+    static __device__ __forceinline__ void load(const __half *p, float (&w)[8]) {
+        uint4 v = ld_stream16(p);
+        ClPair16<__half>::get(v.x, w[0], w[1]);
+        ClPair16<__half>::get(v.y, w[2], w[3]);
+        ClPair16<__half>::get(v.z, w[4], w[5]);
+        ClPair16<__half>::get(v.w, w[6], w[7]);
+    }
+};
+template <>
 struct W8<float> {
     static __device__ __forceinline__ void load(const float *p, float (&w)[8]) {
         uint4 a = ld_stream16(p), b = ld_stream16(p + 4);
@@ -223,6 +233,7 @@ cudaError_t launch_w(int T, int epi, const ClGemvArgs &a, int grid, cudaStream_t
 
 cudaError_t cl_launch_gemv(int wdtype, int T, int epi, const ClGemvArgs &a, int grid, cudaStream_t s) {
     if (wdtype == 1) return launch_w<__nv_bfloat16>(T, epi, a, grid, s);
+    if (wdtype == 2) return launch_w<__half>(T, epi, a, grid, s);
     return launch_w<float>(T, epi, a, grid, s);
 }
 

@@ -14,8 +14,12 @@ __device__ __forceinline__ float to_f32<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
+template <>
+__device__ __forceinline__ float to_f32<__half>(__half v) { return __half2float(v); }
 template <typename ST>
 __device__ __forceinline__ ST from_f32(float v);
+template <>
+__device__ __forceinline__ __half from_f32<__half>(float v) { return __float2half_rn(v); }
 template <>
 __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <>
@@ -135,8 +139,10 @@ __global__ void __launch_bounds__(128) k_attn(ClAttnArgs a) {
                 const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    s = fmaf(qr[2 * e], __uint_as_float(u[e] << 16), s);
-                    s = fmaf(qr[2 * e + 1], __uint_as_float(u[e] & 0xffff0000u), s);
+                    float k0, k1;
+                    ClPair16<ST>::get(u[e], k0, k1);
+                    s = fmaf(qr[2 * e], k0, s);
+                    s = fmaf(qr[2 * e + 1], k1, s);
                 }
             } else {
                 s = fmaf(qr[0], __uint_as_float(raw.x), s);
@@ -392,15 +398,17 @@ __global__ void k_select(cl_select_cfg cfg, int L, const float *c_layer, uint8_t
 
 }  // namespace
 
-#define CL_DISPATCH_ST(wdtype, EXPR_BF16, EXPR_F32) \
-    do {                                            \
-        if ((wdtype) == 1) { EXPR_BF16; } else { EXPR_F32; } \
+// Runs CALL with ST = the storage type that wdtype names (0 fp32, 1 bf16, 2 fp16).
+#define CL_DISPATCH_ST(wdtype, CALL)                                \
+    do {                                                            \
+        if ((wdtype) == 1) { using ST = __nv_bfloat16; CALL; }      \
+        else if ((wdtype) == 2) { using ST = __half; CALL; }        \
+        else { using ST = float; CALL; }                            \
     } while (0)
 
 cudaError_t cl_launch_embed(int wdtype, const void *embed, const int *tok, int T, int d, float *x, const ClDevState *st,
                             cudaStream_t s) {
-    CL_DISPATCH_ST(wdtype, (k_embed<__nv_bfloat16><<<T, 256, 0, s>>>((const __nv_bfloat16 *)embed, tok, d, x, st)),
-                   (k_embed<float><<<T, 256, 0, s>>>((const float *)embed, tok, d, x, st)));
+    CL_DISPATCH_ST(wdtype, (k_embed<ST><<<T, 256, 0, s>>>((const ST *)embed, tok, d, x, st)));
     return cudaGetLastError();
 }
 
@@ -412,19 +420,15 @@ cudaError_t cl_launch_rmsnorm(const float *x, const float *g, int T, int d, floa
 
 cudaError_t cl_launch_rmsnorm_rows(int in_dtype, const void *x, const float *g, int T, int d, float eps, float *out,
                                    cudaStream_t s) {
-    CL_DISPATCH_ST(in_dtype, (k_rmsnorm<__nv_bfloat16><<<T, 256, 0, s>>>((const __nv_bfloat16 *)x, g, d, eps, out, nullptr)),
-                   (k_rmsnorm<float><<<T, 256, 0, s>>>((const float *)x, g, d, eps, out, nullptr)));
+    CL_DISPATCH_ST(in_dtype, (k_rmsnorm<ST><<<T, 256, 0, s>>>((const ST *)x, g, d, eps, out, nullptr)));
     return cudaGetLastError();
 }
 
 cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H, int Hkv, int hd, int d, const float2 *rope_cs,
                                   void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s) {
     dim3 grid(T, H);
-    CL_DISPATCH_ST(wdtype,
-                   (k_rope_append<__nv_bfloat16><<<grid, hd / 2, 0, s>>>(qkv, row0, hd, d, Hkv, rope_cs, (__nv_bfloat16 *)kcache,
-                                                                         (__nv_bfloat16 *)vcache, max_seq, st)),
-                   (k_rope_append<float><<<grid, hd / 2, 0, s>>>(qkv, row0, hd, d, Hkv, rope_cs, (float *)kcache,
-                                                                 (float *)vcache, max_seq, st)));
+    CL_DISPATCH_ST(wdtype, (k_rope_append<ST><<<grid, hd / 2, 0, s>>>(qkv, row0, hd, d, Hkv, rope_cs, (ST *)kcache, (ST *)vcache,
+                                                                      max_seq, st)));
     return cudaGetLastError();
 }
 
@@ -432,11 +436,9 @@ cudaError_t cl_launch_attn(int wdtype, int T, const ClAttnArgs &a, cudaStream_t 
     dim3 grid(a.n_heads, T, a.nsplit);
     const size_t smem = (size_t)(3 * a.head_dim + 32 + a.per_max) * sizeof(float);
     if (a.head_dim == 64) {
-        CL_DISPATCH_ST(wdtype, (k_attn<__nv_bfloat16, 64><<<grid, 128, smem, s>>>(a)),
-                       (k_attn<float, 64><<<grid, 128, smem, s>>>(a)));
+        CL_DISPATCH_ST(wdtype, (k_attn<ST, 64><<<grid, 128, smem, s>>>(a)));
     } else if (a.head_dim == 128) {
-        CL_DISPATCH_ST(wdtype, (k_attn<__nv_bfloat16, 128><<<grid, 128, smem, s>>>(a)),
-                       (k_attn<float, 128><<<grid, 128, smem, s>>>(a)));
+        CL_DISPATCH_ST(wdtype, (k_attn<ST, 128><<<grid, 128, smem, s>>>(a)));
     } else {
         return cudaErrorInvalidValue;
     }
@@ -445,8 +447,7 @@ cudaError_t cl_launch_attn(int wdtype, int T, const ClAttnArgs &a, cudaStream_t 
 
 cudaError_t cl_launch_tap(int wdtype, const float *x, int T, int row0, int d, void *ring_layer, int P,
                           const ClDevState *st, cudaStream_t s) {
-    CL_DISPATCH_ST(wdtype, (k_tap<__nv_bfloat16><<<T, 256, 0, s>>>(x, row0, d, (__nv_bfloat16 *)ring_layer, P, st)),
-                   (k_tap<float><<<T, 256, 0, s>>>(x, row0, d, (float *)ring_layer, P, st)));
+    CL_DISPATCH_ST(wdtype, (k_tap<ST><<<T, 256, 0, s>>>(x, row0, d, (ST *)ring_layer, P, st)));
     return cudaGetLastError();
 }
 
@@ -473,9 +474,6 @@ cudaError_t cl_launch_select(const cl_select_cfg &cfg, int n_layers, const float
 }
 
 cudaError_t cl_launch_interleave(int wdtype, const void *wg, const void *wu, void *dst, int F, int d, cudaStream_t s) {
-    CL_DISPATCH_ST(wdtype,
-                   (k_interleave<__nv_bfloat16><<<1184, 256, 0, s>>>((const __nv_bfloat16 *)wg, (const __nv_bfloat16 *)wu,
-                                                                     (__nv_bfloat16 *)dst, F, d)),
-                   (k_interleave<float><<<1184, 256, 0, s>>>((const float *)wg, (const float *)wu, (float *)dst, F, d)));
+    CL_DISPATCH_ST(wdtype, (k_interleave<ST><<<1184, 256, 0, s>>>((const ST *)wg, (const ST *)wu, (ST *)dst, F, d)));
     return cudaGetLastError();
 }

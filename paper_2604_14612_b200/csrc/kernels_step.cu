@@ -200,6 +200,21 @@ struct Chunk<__nv_bfloat16> {
     }
 };
 template <>
+struct Chunk<__half> {
+    static constexpr int EPC = 8;
+    static __device__ __forceinline__ float dot(const uint4 &w, const float (&x)[8], float acc) {
+        const unsigned u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float lo, hi;
+            ClPair16<__half>::get(u[e], lo, hi);
+            acc = fmaf(lo, x[2 * e], acc);
+            acc = fmaf(hi, x[2 * e + 1], acc);
+        }
+        return acc;
+    }
+};
+template <>
 struct Chunk<float> {
     static constexpr int EPC = 4;
     static __device__ __forceinline__ float dot(const uint4 &w, const float (&x)[4], float acc) {
@@ -217,8 +232,12 @@ template <>
 __device__ __forceinline__ float st_to_f32<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ float st_to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <>
+__device__ __forceinline__ float st_to_f32<__half>(__half v) { return __half2float(v); }
 template <typename ST>
 __device__ __forceinline__ ST st_from_f32(float v);
+template <>
+__device__ __forceinline__ __half st_from_f32<__half>(float v) { return __float2half_rn(v); }
 template <>
 __device__ __forceinline__ float st_from_f32<float>(float v) { return v; }
 template <>
@@ -231,18 +250,15 @@ __device__ __forceinline__ void load_vals(const ST *p, float (&o)[VPL]) {
     if (BYTES == 4) {
         const unsigned u = __ldcg((const unsigned *)p);
         if (sizeof(ST) == 2) {
-            o[0] = __uint_as_float(u << 16);
-            o[VPL - 1] = __uint_as_float(u & 0xffff0000u);
+            ClPair16<ST>::get(u, o[0], o[VPL - 1]);
         } else {
             o[0] = __uint_as_float(u);
         }
     } else if (BYTES == 8) {
         const uint2 u = __ldcg((const uint2 *)p);
         if (sizeof(ST) == 2) {
-            o[0] = __uint_as_float(u.x << 16);
-            o[1 % VPL] = __uint_as_float(u.x & 0xffff0000u);
-            o[2 % VPL] = __uint_as_float(u.y << 16);
-            o[3 % VPL] = __uint_as_float(u.y & 0xffff0000u);
+            ClPair16<ST>::get(u.x, o[0], o[1 % VPL]);
+            ClPair16<ST>::get(u.y, o[2 % VPL], o[3 % VPL]);
         } else {
             o[0] = __uint_as_float(u.x);
             o[1 % VPL] = __uint_as_float(u.y);
@@ -668,8 +684,10 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
                         const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            sc = fmaf(qr[(2 * e) % EPL], __uint_as_float(u[e] << 16), sc);
-                            sc = fmaf(qr[(2 * e + 1) % EPL], __uint_as_float(u[e] & 0xffff0000u), sc);
+                            float k0, k1;
+                            ClPair16<ST>::get(u[e], k0, k1);
+                            sc = fmaf(qr[(2 * e) % EPL], k0, sc);
+                            sc = fmaf(qr[(2 * e + 1) % EPL], k1, sc);
                         }
                     } else {
                         sc = fmaf(qr[0], __uint_as_float(raw.x), sc);
@@ -970,12 +988,14 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
 
 size_t cl_step_smem_bytes() { return (size_t)NSLOT * SLOT_BYTES + sizeof(Smem); }
 
-int cl_step_max_cols(int wdtype) { return MAXIT * NCT * (wdtype == 1 ? 8 : 4); }
+int cl_step_max_cols(int wdtype) { return MAXIT * NCT * (wdtype != 0 ? 8 : 4); }
 
 cudaError_t cl_launch_token_steps(int wdtype, int head_dim, const ClStepArgs &a, int grid, cudaStream_t s) {
     const void *fn = nullptr;
     if (wdtype == 1 && head_dim == 64) fn = (const void *)k_token_steps<__nv_bfloat16, 64>;
     else if (wdtype == 1 && head_dim == 128) fn = (const void *)k_token_steps<__nv_bfloat16, 128>;
+    else if (wdtype == 2 && head_dim == 64) fn = (const void *)k_token_steps<__half, 64>;
+    else if (wdtype == 2 && head_dim == 128) fn = (const void *)k_token_steps<__half, 128>;
     else if (wdtype == 0 && head_dim == 64) fn = (const void *)k_token_steps<float, 64>;
     else if (wdtype == 0 && head_dim == 128) fn = (const void *)k_token_steps<float, 128>;
     else return cudaErrorInvalidValue;

@@ -27,7 +27,7 @@ def test_create_rejects_bad_shapes_before_any_device_work(lib):
     h = C.c_void_p()
     good = dict(n_layers=2, d_model=128, n_heads=2, n_kv_heads=2, head_dim=64, d_ffn=256, vocab=100, max_seq=32,
                 rms_eps=1e-5, rope_theta=1e4, weight_dtype=1, tap_positions=0)
-    for bad in (dict(head_dim=32, d_model=64), dict(n_kv_heads=3), dict(d_ffn=100), dict(weight_dtype=2), dict(vocab=1),
+    for bad in (dict(head_dim=32, d_model=64), dict(n_kv_heads=3), dict(d_ffn=100), dict(weight_dtype=3), dict(vocab=1),
                 dict(max_seq=0), dict(n_heads=3)):
         cfg = ModelCfg(**{**good, **bad})
         rc = lib.cl_create(C.byref(cfg), None, C.byref(h))

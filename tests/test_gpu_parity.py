@@ -538,3 +538,41 @@ def test_second_prompt_reuses_the_searched_skip_set():
     ref = oracle.generate_vanilla(om, b, 31)
     lim = next((i for i, m in enumerate(ref["margins"]) if m < 1e-4), 31)
     assert ([first] + [int(t) for t in spec])[:lim] == ref["tokens"][:lim]
+
+
+@pytest.mark.parametrize("name,L,K", [("C2", 3, 4), ("C3", 2, 8)])
+def test_fp16_storage_model(name, L, K):
+    """weight_dtype = fp16 (the type the paper's models run in): weights, KV cache and taps in binary16, every step on
+    the CUDA-core kernels; draft steps, verify pass, prefill, taps and the layer confidences against the oracle."""
+    w0 = synth.WORKLOADS[name]
+    w = synth.reduced(w0, n_layers=L, prompt_len=21, gen_len=9)
+    sh = dataclasses.replace(w.shape, weight_dtype="fp16")
+    P = 8
+    om, ctx, _ = make_pair(sh, w.seed + 5, tap_positions=P, gen_device="cuda" if name == "C3" else "cpu")
+    prompt = synth.make_prompt(w.seed, w.prompt_len, sh.vocab)
+    rep = lockstep_generate(om, ctx, prompt, synth.layers_to_mask([1], L), K, w.gen_len, tap=True)
+    print("fp16", name, rep)
+    assert rep.cycles > 0
+    ctx.cl_prefill(prompt, tap_hidden=True)
+    ring = ctx.cl_read_hidden_ring()
+    assert ring.dtype == torch.float16
+    want_h = oracle_prefill_hidden(om, prompt, P)
+    got_h = ring_in_position_order(ring, len(prompt) - 1)
+    scale = max(1.0, float(np.abs(want_h).max()))
+    assert np.abs(got_h - want_h).max() <= 2 ** -10 * scale               # one binary16 ulp at the top of the range
+    g = ctx.cl_layer_confidences()
+    o = oracle.layer_confidences(torch.tensor(want_h).to(torch.float16), om._keep["lm_head"], om._keep["final_norm"], sh.rms_eps)
+    order = [(p % P) for p in range(len(prompt) - P, len(prompt))]
+    assert np.abs(g["conf"][:, order] - o["conf"]).max() <= TOL
+    assert np.abs(g["c_layer"] - o["c_layer"]).max() <= TOL
+    # lossless on the device with fp16 storage too
+    first = ctx.cl_prefill(prompt)
+    van, _ = ctx.cl_generate(0, 12)
+    ctx.cl_prefill(prompt)
+    ctx.cl_set_skip_set(synth.layers_to_mask([1], L))
+    spec, _ = ctx.cl_generate(K, 12)
+    ref = oracle.generate_vanilla(om, prompt, 13)
+    lim = next((i for i, m in enumerate(ref["margins"]) if m < NEAR_TIE), 13)
+    if lim >= 1:
+        assert [first] + list(van[:lim - 1]) == ref["tokens"][:lim]
+        assert list(spec[:lim - 1]) == list(van[:lim - 1])
