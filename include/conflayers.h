@@ -26,9 +26,9 @@
  *     head_dim in {64, 128}, d_model and d_ffn multiples of 8, 1 <= K <= CL_MAX_K.
  *   - Which kernels run: single-token steps (draft, vanilla) run in one persistent cooperative kernel when d_model and
  *     d_ffn are at most 16384 (bf16) / 8192 (fp32); passes of several rows (verify, prefill) and the confidence scoring
- *     of bf16 models run on the tensor cores (tcgen05); fp32 and fp16 models and the cases above use per-matrix
- *     CUDA-core kernels.
- *     A prompt of more than 16 tokens (bf16 models) runs all rows but the last through wide tensor-core GEMMs, up to
+ *     of bf16 and fp16 models run on the tensor cores (tcgen05, both operands in the model's 16-bit type); fp32 models
+ *     and the cases above use per-matrix CUDA-core kernels.
+ *     A prompt of more than 16 tokens (bf16 / fp16 models) runs all rows but the last through wide tensor-core GEMMs, up to
  *     512 rows at a time, and the last row through the pass of several rows, which has the LM head.
  *     Environment switches read by cl_load (diagnostics): CL_DISABLE_STEP_KERNEL=1, CL_DISABLE_TC_PASS=1,
  *     CL_DISABLE_WIDE_PREFILL=1, CL_DISABLE_ROW_SHARES=1, CL_L2_AHEAD_KB=<n>.

@@ -376,7 +376,8 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
         }
         // ---- skinny tensor-core GEMM path (bf16): tensor maps of every matrix, hi/lo input rows, workspace
         c->use_tc = 0;
-        if (g.weight_dtype == 1) {
+        if (g.weight_dtype != 0) {
+            const int f16 = g.weight_dtype == 2;
             const char *off = getenv("CL_DISABLE_TC_PASS");
             const int G = c->n_sm;
             auto segs_ok = [&](size_t rows, size_t K) {
@@ -405,17 +406,17 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 c->map_qkv.resize(L); c->map_o.resize(L); c->map_gu.resize(L); c->map_d.resize(L);
                 for (size_t l = 0; l < L && ok; ++l) {
                     const ClLayer &y = c->layers[l];
-                    ok = cl_make_tensor_map(&c->map_qkv[l], y.wqkv, (int)qkv_rows, (int)d, 128) &&
-                         cl_make_tensor_map(&c->map_o[l], y.wo, (int)d, (int)d, 128) &&
-                         cl_make_tensor_map(&c->map_gu[l], y.wgu, (int)(2 * F), (int)d, 128) &&
-                         cl_make_tensor_map(&c->map_d[l], y.wd, (int)d, (int)F, 128);
+                    ok = cl_make_tensor_map(&c->map_qkv[l], y.wqkv, (int)qkv_rows, (int)d, 128, f16) &&
+                         cl_make_tensor_map(&c->map_o[l], y.wo, (int)d, (int)d, 128, f16) &&
+                         cl_make_tensor_map(&c->map_gu[l], y.wgu, (int)(2 * F), (int)d, 128, f16) &&
+                         cl_make_tensor_map(&c->map_d[l], y.wd, (int)d, (int)F, 128, f16);
                 }
-                ok = ok && cl_make_tensor_map(&c->map_head, c->lm_head, (int)V, (int)d, 128);
+                ok = ok && cl_make_tensor_map(&c->map_head, c->lm_head, (int)V, (int)d, 128, f16);
                 for (int i = 0; i < 2 && ok; ++i) {
                     const int N = i ? 32 : 16;
-                    ok = cl_make_tensor_map(&c->map_bx[i], c->bx, N, (int)d, N) &&
-                         cl_make_tensor_map(&c->map_batt[i], c->batt, N, (int)d, N) &&
-                         cl_make_tensor_map(&c->map_bh[i], c->bh, N, (int)F, N);
+                    ok = cl_make_tensor_map(&c->map_bx[i], c->bx, N, (int)d, N, f16) &&
+                         cl_make_tensor_map(&c->map_batt[i], c->batt, N, (int)d, N, f16) &&
+                         cl_make_tensor_map(&c->map_bh[i], c->bh, N, (int)F, N, f16);
                 }
                 if (!ok) return fail(c, CL_ECUDA, "cl_load: encoding a TMA tensor map failed");
                 c->use_tc = 1;
@@ -432,9 +433,9 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                     DM(c->w_x, Mw * d * 4);
                     c->w_P_floats = 2 * Mw * widest;
                     DM(c->w_P, c->w_P_floats * 4);
-                    if (!(cl_make_tensor_map(&c->map_wx, c->w_ax, (int)(2 * Mw), (int)d, 128) &&
-                          cl_make_tensor_map(&c->map_watt, c->w_aatt, (int)(2 * Mw), (int)d, 128) &&
-                          cl_make_tensor_map(&c->map_wh, c->w_ah, (int)(2 * Mw), (int)F, 128)))
+                    if (!(cl_make_tensor_map(&c->map_wx, c->w_ax, (int)(2 * Mw), (int)d, 128, f16) &&
+                          cl_make_tensor_map(&c->map_watt, c->w_aatt, (int)(2 * Mw), (int)d, 128, f16) &&
+                          cl_make_tensor_map(&c->map_wh, c->w_ah, (int)(2 * Mw), (int)F, 128, f16)))
                         return fail(c, CL_ECUDA, "cl_load: encoding a TMA tensor map failed");
                     c->use_wide = 1;
                 }
@@ -554,7 +555,9 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
     memset(&b, 0, sizeof(b));
     b.T = T; b.N = N; b.st = c->st; b.ws = c->v_ws; b.tickets = c->v_tickets; b.ssq_tiles = dtiles;
     b.inv_dim = 1.0f / (float)d; b.eps = g.rms_eps; b.nh = nh; b.row0 = row0; b.err = &c->st->err;
-    KL(cl_launch_pass_begin(c->embed, tok, T, d, c->x, c->bx, nh, L ? c->layers[0].n1 : c->final_norm, c->v_ssq, c->st, c->stream));
+    b.f16 = g.weight_dtype == 2;
+    KL(cl_launch_pass_begin(c->embed, tok, T, d, c->x, c->bx, nh, L ? c->layers[0].n1 : c->final_norm, c->v_ssq, c->st, b.f16,
+                            c->stream));
     for (int l = 0; l < L; ++l) {
         const ClLayer &y = c->layers[l];
         ClSkinnyArgs a = b;
@@ -566,7 +569,7 @@ static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, 
         t.out = c->att; t.out_b = c->batt; t.nh = nh; t.st = c->st; t.row0 = row0; t.n_heads = g.n_heads; t.head_dim = g.head_dim;
         t.d_model = d; t.nsplit = c->nsplit; t.per_max = c->per_max; t.max_seq = g.max_seq;
         t.part = c->v_att_part;
-        KL(cl_launch_attn_rows(1, T, c->v_att_S, t, c->stream));
+        KL(cl_launch_attn_rows(g.weight_dtype, T, c->v_att_S, t, c->stream));
         a = b;
         a.rows = d; a.KB = KBd; a.epi = CL_VEPI_RESID; a.out = c->x; a.ld = d; a.bnext = c->bx; a.bn_ld = d; a.gnext = y.n2;
         a.ssq_out = c->v_ssq;
@@ -606,18 +609,19 @@ static int forward_wide(cl_ctx *c, const int *tok, int M, int tap) {
     const cl_model_cfg &g = c->cfg;
     const int d = g.d_model, F = g.d_ffn, L = g.n_layers, qkv_rows = d + 2 * g.n_kv_heads * g.head_dim;
     const int KBd = (d + 63) / 64, KBf = (F + 63) / 64, MT = (M + 127) / 128, lo0 = CL_WIDE_MAX_M;
+    const int f16 = g.weight_dtype == 2;
     auto gemm = [&](const ClTensorMap &mapA, const ClTensorMap &mapB, int rows, int KB, int *splits) -> int {
         ClWideArgs a;
         a.M = M; a.rows = rows; a.KB = KB; a.MT = MT; a.NT = (rows + 255) / 256;
         a.splits = *splits = cl_wide_splits(M, rows, KB, c->n_sm, c->w_P_floats);
-        a.lo_row0 = lo0; a.P = c->w_P; a.err = &c->st->err;
+        a.lo_row0 = lo0; a.P = c->w_P; a.err = &c->st->err; a.f16 = f16;
         KL(cl_launch_wide(mapA, mapB, a, c->stream));
         return CL_OK;
     };
     ClWideNormArgs nb;
     memset(&nb, 0, sizeof(nb));
     nb.x = c->w_x; nb.M = M; nb.d = d; nb.eps = g.rms_eps; nb.A = c->w_ax; nb.lo_row0 = lo0; nb.st = c->st;
-    nb.tap_P = g.tap_positions;
+    nb.tap_P = g.tap_positions; nb.f16 = f16;
     {
         ClWideNormArgs n = nb;
         n.embed = c->embed; n.tok = tok; n.g = L ? c->layers[0].n1 : nullptr;
@@ -628,16 +632,16 @@ static int forward_wide(cl_ctx *c, const int *tok, int M, int tap) {
         const ClLayer &y = c->layers[l];
         if ((rc = gemm(c->map_wx, c->map_qkv[l], qkv_rows, KBd, &sp))) return rc;
         KL(cl_launch_wide_rope_append(c->w_P, sp, M, g.n_heads, g.n_kv_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq,
-                                      c->st, c->stream));
+                                      c->st, f16, c->stream));
         KL(cl_launch_attn_wide(c->w_P, qkv_rows, y.kc, y.vc, c->w_aatt, lo0, M, d, g.n_heads, g.n_kv_heads, g.head_dim,
-                               g.max_seq, c->st, c->stream));
+                               g.max_seq, c->st, f16, c->stream));
         if ((rc = gemm(c->map_watt, c->map_o[l], d, KBd, &sp))) return rc;
         ClWideNormArgs n = nb;
         n.P = c->w_P; n.splits = sp; n.g = y.n2;
         if (tap) n.tap = ring_slot(c, l, 0);
         KL(cl_launch_wide_norm(n, c->stream));
         if ((rc = gemm(c->map_wx, c->map_gu[l], 2 * F, KBd, &sp))) return rc;
-        KL(cl_launch_wide_silu(c->w_P, sp, M, F, c->w_ah, lo0, c->stream));
+        KL(cl_launch_wide_silu(c->w_P, sp, M, F, c->w_ah, lo0, f16, c->stream));
         if ((rc = gemm(c->map_wh, c->map_d[l], d, KBf, &sp))) return rc;
         n = nb;
         n.P = c->w_P; n.splits = sp; n.g = (l + 1 < L) ? c->layers[l + 1].n1 : nullptr;
@@ -1085,7 +1089,7 @@ static int ensure_score_cap(cl_ctx *c, size_t n) {
     DM(c->sc_conf, n * 4);
     DM(c->sc_pmax, n * 4);
     DM(c->sc_arg, n * 4);
-    if (c->cfg.weight_dtype == 1) {
+    if (c->cfg.weight_dtype != 0) {
         DM(c->sc_xn, n * (size_t)c->cfg.d_model * 2);
         DM(c->sc_part, cl_score_tc_partials((int)n, c->n_sm) * sizeof(ClHeadPartial));
     }
@@ -1110,11 +1114,12 @@ static int score_rows(cl_ctx *c, const void *hidden, int rows, int P, float *c_l
     const size_t n = (size_t)rows * P, d = c->cfg.d_model;
     int rc = ensure_score_cap(c, n);
     if (rc) return rc;
-    if (c->cfg.weight_dtype == 1) {
-        // bf16 head: one dense contraction on the tensor cores with the softmax statistics fused into its epilogue
-        KL(cl_launch_rmsnorm_bf16(1, hidden, c->final_norm, (int)n, (int)d, c->cfg.rms_eps, c->sc_xn, c->stream));
+    if (c->cfg.weight_dtype != 0) {
+        // 16-bit head: one dense contraction on the tensor cores with the softmax statistics fused into its epilogue
+        const int f16 = c->cfg.weight_dtype == 2;
+        KL(cl_launch_rmsnorm_bf16(c->cfg.weight_dtype, hidden, c->final_norm, (int)n, (int)d, c->cfg.rms_eps, c->sc_xn, f16, c->stream));
         KL(cl_launch_score_tc(c->sc_xn, c->lm_head, (int)n, c->cfg.vocab, (int)d, c->sc_part, c->n_sm, &c->st->err, c->sc_conf,
-                              c->sc_pmax, c->sc_arg, c->stream));
+                              c->sc_pmax, c->sc_arg, f16, c->stream));
         ++c->launches;
         KL(cl_launch_mean_rows(c->sc_conf, rows, P, c_layer_dev, c->stream));
         return CL_OK;

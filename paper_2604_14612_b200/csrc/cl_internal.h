@@ -177,16 +177,17 @@ struct ClSkinnyArgs {
     float *logits;                    // HEAD, optional [T, rows]
     ClHeadPartial *head_part;         // HEAD: [tiles, CL_SLOTS]
     int *err;
+    int f16;                          // the model's 16-bit type: 0 bf16, 1 fp16 (weights, activation parts, taps)
 };
 
 struct ClTensorMap {                  // opaque 128-byte TMA descriptor (CUtensorMap)
     alignas(64) unsigned char bytes[128];
 };
 
-bool cl_make_tensor_map(ClTensorMap *m, const void *base, int rows, int cols, int box_rows);
+bool cl_make_tensor_map(ClTensorMap *m, const void *base, int rows, int cols, int box_rows, int f16 = 0);
 cudaError_t cl_launch_skinny(const ClTensorMap &mapA, const ClTensorMap &mapB, const ClSkinnyArgs &a, int grid, cudaStream_t s);
 cudaError_t cl_launch_pass_begin(const void *embed, const int *tok, int T, int d, float *x, __nv_bfloat16 *bnext, int nh,
-                                 const float *g, float *ssq_out, const ClDevState *st, cudaStream_t s);
+                                 const float *g, float *ssq_out, const ClDevState *st, int f16, cudaStream_t s);
 cudaError_t cl_launch_head_finalize(const ClHeadPartial *part, int tiles, int T, float inv_log_v, int *out_tok, float *out_pmax,
                                     float *out_conf, const ClDevState *st, cudaStream_t s);
 
@@ -198,6 +199,7 @@ struct ClWideArgs {
     int lo_row0;                      // first row of the lo parts in the activation buffer (hi parts start at row 0)
     float *P;                         // [splits, M, rows] partial products (a later kernel adds the splits in order)
     int *err;
+    int f16;                          // the model's 16-bit type: 0 bf16, 1 fp16
 };
 struct ClWideNormArgs {
     float *x;                         // [M, d] residual stream of the pass
@@ -212,26 +214,27 @@ struct ClWideNormArgs {
     void *tap;                        // optional: this layer's hidden-state ring [tap_P, d] (bf16)
     int tap_P;
     const ClDevState *st;
+    int f16;                          // the model's 16-bit type: 0 bf16, 1 fp16 (embedding, taps, normalised rows)
 };
 int cl_wide_splits(int M, int rows, int KB, int n_sm, size_t ws_floats);
 cudaError_t cl_launch_wide(const ClTensorMap &mapA, const ClTensorMap &mapB, const ClWideArgs &a, cudaStream_t s);
 cudaError_t cl_launch_wide_norm(const ClWideNormArgs &a, cudaStream_t s);
 cudaError_t cl_launch_wide_rope_append(float *P, int splits, int M, int H, int Hkv, int hd, int d, const float2 *rope_cs,
-                                       void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
+                                       void *kcache, void *vcache, int max_seq, const ClDevState *st, int f16, cudaStream_t s);
 // causal attention of the M rows of the pass (positions ctx ..) over the cache; q: fp32 rows [M, ld_q], rotary applied;
 // the output goes out as bf16 hi (row t) and lo (row lo_row0 + t) parts [.., d]
 cudaError_t cl_launch_attn_wide(const float *q, int ld_q, const void *kcache, const void *vcache, __nv_bfloat16 *out_b,
                                 int lo_row0, int M, int d, int H, int Hkv, int hd, int max_seq, const ClDevState *st,
-                                cudaStream_t s);
-cudaError_t cl_launch_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, cudaStream_t s);
+                                int f16, cudaStream_t s);
+cudaError_t cl_launch_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, int f16, cudaStream_t s);
 
-// tensor-core scoring (bf16 LM head): normalise to bf16, contraction fused with the softmax statistics, finalize
+// tensor-core scoring (bf16 / fp16 LM head): normalise to the 16-bit type, contraction fused with the softmax statistics, finalize
 int cl_score_tc_ranges(int R, int n_sm);
 size_t cl_score_tc_partials(int R, int n_sm);
 cudaError_t cl_launch_rmsnorm_bf16(int in_dtype, const void *x, const float *g, int rows, int d, float eps, void *out,
-                                   cudaStream_t s);
+                                   int f16, cudaStream_t s);
 cudaError_t cl_launch_score_tc(const void *xn, const void *lm_head, int R, int V, int d, ClHeadPartial *partials, int n_sm,
-                               int *err, float *conf, float *pmax, int *arg, cudaStream_t s);
+                               int *err, float *conf, float *pmax, int *arg, int f16, cudaStream_t s);
 cudaError_t cl_launch_mean_rows(const float *conf_rows, int rows, int P, float *c_layer, cudaStream_t s);
 cudaError_t cl_launch_select(const cl_select_cfg &cfg, int n_layers, const float *c_layer, uint8_t *mask, double *margins,
                              cudaStream_t s);

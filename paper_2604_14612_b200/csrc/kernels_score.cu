@@ -35,6 +35,7 @@ struct ScoreArgs {
     int R, V, KB, MT, NCG, NT;      // hidden rows, vocabulary, K blocks of 64, row blocks, vocabulary ranges, vocabulary tiles
     ClHeadPartial *partials;        // [MT * BM, NCG]
     int *err;
+    int f16;                        // 16-bit type of both operands: 0 bf16, 1 fp16
 };
 
 __device__ __forceinline__ ClHeadPartial sc_merge(const ClHeadPartial &a, const ClHeadPartial &b) {
@@ -112,7 +113,7 @@ k_score(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtens
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const unsigned idesc = umma_idesc(BM, BN);
+            const unsigned idesc = umma_idesc(BM, BN, a.f16);
             unsigned stage = 0, par = 0;
             bool ok = true;
             for (int t = 0; t < ntiles && ok; ++t) {
@@ -211,9 +212,10 @@ __global__ void k_score_finalize(const ClHeadPartial *partials, int NCG, int R, 
     arg[r] = f.idx;
 }
 
-// Final RMSNorm of hidden rows in the storage type -> bf16 rows (the A operand of the contraction).
+// Final RMSNorm of hidden rows in the storage type -> rows in the 16-bit type of the LM head (the A operand of the
+// contraction).
 template <typename ST>
-__global__ void k_rmsnorm_to_bf16(const ST *x, const float *g, int d, float eps, __nv_bfloat16 *out) {
+__global__ void k_rmsnorm_to_bf16(const ST *x, const float *g, int d, float eps, unsigned short *out, int f16) {
     __shared__ float red[32];
     const ST *xr = x + (size_t)blockIdx.x * d;
     float ss = 0.f;
@@ -229,7 +231,7 @@ __global__ void k_rmsnorm_to_bf16(const ST *x, const float *g, int d, float eps,
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];   // fixed order
     const float sc = 1.0f / sqrtf(tot / (float)d + eps);
     for (int i = threadIdx.x; i < d; i += blockDim.x)
-        out[(size_t)blockIdx.x * d + i] = __float2bfloat16_rn((float)xr[i] * sc * g[i]);
+        out[(size_t)blockIdx.x * d + i] = f32_to_b16((float)xr[i] * sc * g[i], f16);
 }
 
 }  // namespace
@@ -246,20 +248,23 @@ size_t cl_score_tc_partials(int R, int n_sm) {
 }
 
 cudaError_t cl_launch_rmsnorm_bf16(int in_dtype, const void *x, const float *g, int rows, int d, float eps, void *out,
-                                   cudaStream_t s) {
+                                   int f16, cudaStream_t s) {
     if (in_dtype == 1)
-        k_rmsnorm_to_bf16<__nv_bfloat16><<<rows, 256, 0, s>>>((const __nv_bfloat16 *)x, g, d, eps, (__nv_bfloat16 *)out);
+        k_rmsnorm_to_bf16<__nv_bfloat16><<<rows, 256, 0, s>>>((const __nv_bfloat16 *)x, g, d, eps, (unsigned short *)out, f16);
+    else if (in_dtype == 2)
+        k_rmsnorm_to_bf16<__half><<<rows, 256, 0, s>>>((const __half *)x, g, d, eps, (unsigned short *)out, f16);
     else
-        k_rmsnorm_to_bf16<float><<<rows, 256, 0, s>>>((const float *)x, g, d, eps, (__nv_bfloat16 *)out);
+        k_rmsnorm_to_bf16<float><<<rows, 256, 0, s>>>((const float *)x, g, d, eps, (unsigned short *)out, f16);
     return cudaGetLastError();
 }
 
 // xn: [R, d] bf16 normalised rows; lm_head: [V, d] bf16.  Needs d % 8 == 0 and 16-byte aligned bases.
 cudaError_t cl_launch_score_tc(const void *xn, const void *lm_head, int R, int V, int d, ClHeadPartial *partials, int n_sm,
-                               int *err, float *conf, float *pmax, int *arg, cudaStream_t s) {
+                               int *err, float *conf, float *pmax, int *arg, int f16, cudaStream_t s) {
     CUtensorMap mapA, mapB;
-    if (!make_map(&mapA, xn, R, d, BM) || !make_map(&mapB, lm_head, V, d, BN)) return cudaErrorInvalidValue;
+    if (!make_map(&mapA, xn, R, d, BM, f16) || !make_map(&mapB, lm_head, V, d, BN, f16)) return cudaErrorInvalidValue;
     ScoreArgs a;
+    a.f16 = f16;
     a.R = R; a.V = V; a.KB = (d + BK - 1) / BK;
     a.MT = (R + BM - 1) / BM;
     a.NCG = cl_score_tc_ranges(R, n_sm);

@@ -1,12 +1,14 @@
-// Skinny tensor-core GEMM for passes of T <= 9 token rows through the bf16 model: the (K+1)-row verify pass of
-// Section 3 (and the prefill, which is the same pass over chunks of the prompt).
+// Skinny tensor-core GEMM for passes of T <= 9 token rows through a model stored in a 16-bit type (bf16, or fp16:
+// both operands of a tcgen05.mma are of that one type): the (K+1)-row verify pass of Section 3 (and short prompts,
+// which are the same pass over chunks of the prompt).
 //
-//   acc[r, t] = sum_k W[r, k] * b[t, k]        W: [rows, K] bf16 weights, b: T activation rows
+//   acc[r, t] = sum_k W[r, k] * b[t, k]        W: [rows, K] 16-bit weights, b: T activation rows
 //
 // "Swap-AB": the weight rows are the M = 128 operand of tcgen05.mma (they fill the tensor-memory lanes), the token
-// rows are N.  Activations are fp32 everywhere else; here each row enters twice, as hi = bf16(v) and
-// lo = bf16(v - hi), in N = 16 (T <= 8) or 32 columns, and the two accumulator columns are added in the epilogue,
-// so the product keeps about 16 mantissa bits of the activation while the weights stream exactly once.
+// rows are N.  Activations are fp32 everywhere else; here each row enters twice, as hi = round16(v) and
+// lo = round16(v - hi), in N = 16 (T <= 8) or 32 columns, and the two accumulator columns are added in the epilogue,
+// so the product keeps about 16 (bf16) or 22 (fp16) mantissa bits of the activation while the weights stream exactly
+// once.
 // The pass is bound by HBM weight streaming, so the work is cut for equal bytes per SM ("stream-K"): the units
 // (128-row tile, 64-column K block) are numbered tile-major and CTA c takes the contiguous range
 // [U c / G, U (c+1) / G).  A CTA that holds only part of a tile's K range writes its 128 x N partial
@@ -100,12 +102,6 @@ __device__ __forceinline__ ClHeadPartial v_shfl_xor(const ClHeadPartial &a, int 
     r.s = __shfl_xor_sync(0xffffffffu, a.s, o);
     r.idx = __shfl_xor_sync(0xffffffffu, a.idx, o);
     return r;
-}
-
-// v -> (hi, lo) bf16 with hi + lo = v to about 16 mantissa bits
-__device__ __forceinline__ void split_bf16(float v, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
-    hi = __float2bfloat16_rn(v);
-    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
 // Adds the partial accumulators of tile m (from CTAs c_first .. c_last, in that order) into v: PB partials are in
@@ -220,7 +216,7 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const unsigned idesc = umma_idesc(VM, a.N);
+            const unsigned idesc = umma_idesc(VM, a.N, a.f16);
             unsigned stage = 0, par = 0;
             bool ok = true;
             Seg sg;
@@ -315,13 +311,10 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
                         const float xn = (live ? xo[t] + tot[t] : 0.f);
                         if (live) {
                             a.out[(size_t)t * a.ld + row] = xn;
-                            __nv_bfloat16 hi, lo;
-                            split_bf16(xn * g, hi, lo);
-                            a.bnext[(size_t)t * a.bn_ld + row] = hi;
-                            a.bnext[(size_t)(a.nh + t) * a.bn_ld + row] = lo;
+                            store_split(a.bnext + (size_t)t * a.bn_ld + row, a.bnext + (size_t)(a.nh + t) * a.bn_ld + row, xn * g, a.f16);
                             if (a.tap) {
                                 const size_t o = (size_t)((pos0 + t) % a.tap_P) * a.rows + row;
-                                ((__nv_bfloat16 *)a.tap)[o] = __float2bfloat16_rn(xn);
+                                ((unsigned short *)a.tap)[o] = f32_to_b16(xn, a.f16);
                             }
                         }
                         float ss = xn * xn;
@@ -341,10 +334,7 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
                     const float other = __shfl_xor_sync(0xffffffffu, mine, 1);   // gate (even row) / up (odd row) pair
                     if (live && !(lane & 1)) {
                         const float h = mine / (1.f + expf(-mine)) * other;
-                        __nv_bfloat16 hi, lo;
-                        split_bf16(h, hi, lo);
-                        a.bnext[(size_t)t * a.bn_ld + (row >> 1)] = hi;
-                        a.bnext[(size_t)(a.nh + t) * a.bn_ld + (row >> 1)] = lo;
+                        store_split(a.bnext + (size_t)t * a.bn_ld + (row >> 1), a.bnext + (size_t)(a.nh + t) * a.bn_ld + (row >> 1), h, a.f16);
                     }
                 }
             } else {
@@ -385,20 +375,17 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
 }
 
 // Start of a pass: x[t] = E[token t]; the first GEMM's input rows hi/lo(x * g) and the per-tile sums of squares.
-__global__ void k_pass_begin(const __nv_bfloat16 *embed, const int *tok, int T, int d, float *x, __nv_bfloat16 *bnext, int nh,
-                             const float *g, float *ssq_out, const ClDevState *st) {
+__global__ void k_pass_begin(const unsigned short *embed, const int *tok, int T, int d, float *x, __nv_bfloat16 *bnext, int nh,
+                             const float *g, float *ssq_out, const ClDevState *st, int f16) {
     if (st->done) return;
     __shared__ float red[4][CL_SLOTS];
     const int row = blockIdx.x * 128 + threadIdx.x, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     for (int t = 0; t < T; ++t) {
         float v = 0.f;
         if (row < d) {
-            v = __bfloat162float(embed[(size_t)tok[t] * d + row]);
+            v = b16_to_f32(embed[(size_t)tok[t] * d + row], f16);
             x[(size_t)t * d + row] = v;
-            __nv_bfloat16 hi, lo;
-            split_bf16(v * g[row], hi, lo);
-            bnext[(size_t)t * d + row] = hi;
-            bnext[(size_t)(nh + t) * d + row] = lo;
+            store_split(bnext + (size_t)t * d + row, bnext + (size_t)(nh + t) * d + row, v * g[row], f16);
         }
         float ss = v * v;
 #pragma unroll
@@ -439,9 +426,9 @@ __global__ void k_head_finalize(const ClHeadPartial *part, int tiles, int T, flo
 
 }  // namespace
 
-bool cl_make_tensor_map(ClTensorMap *m, const void *base, int rows, int cols, int box_rows) {
+bool cl_make_tensor_map(ClTensorMap *m, const void *base, int rows, int cols, int box_rows, int f16) {
     static_assert(sizeof(ClTensorMap) >= sizeof(CUtensorMap), "tensor map storage");
-    return make_map((CUtensorMap *)m->bytes, base, rows, cols, box_rows);
+    return make_map((CUtensorMap *)m->bytes, base, rows, cols, box_rows, f16);
 }
 
 cudaError_t cl_launch_skinny(const ClTensorMap &mapA, const ClTensorMap &mapB, const ClSkinnyArgs &a, int grid, cudaStream_t s) {
@@ -467,8 +454,8 @@ cudaError_t cl_launch_skinny(const ClTensorMap &mapA, const ClTensorMap &mapB, c
 }
 
 cudaError_t cl_launch_pass_begin(const void *embed, const int *tok, int T, int d, float *x, __nv_bfloat16 *bnext, int nh,
-                                 const float *g, float *ssq_out, const ClDevState *st, cudaStream_t s) {
-    k_pass_begin<<<(d + 127) / 128, 128, 0, s>>>((const __nv_bfloat16 *)embed, tok, T, d, x, bnext, nh, g, ssq_out, st);
+                                 const float *g, float *ssq_out, const ClDevState *st, int f16, cudaStream_t s) {
+    k_pass_begin<<<(d + 127) / 128, 128, 0, s>>>((const unsigned short *)embed, tok, T, d, x, bnext, nh, g, ssq_out, st, f16);
     return cudaGetLastError();
 }
 
@@ -489,6 +476,17 @@ namespace {
 
 constexpr int AR_WARPS = 8;
 constexpr int AR_MAXS = 8;   // most parts the keys of a head are cut into
+
+template <typename ST>
+__device__ __forceinline__ ST ar_from_f32(float v);
+template <>
+__device__ __forceinline__ __nv_bfloat16 ar_from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+template <>
+__device__ __forceinline__ __half ar_from_f32<__half>(float v) { return __float2half_rn(v); }
+template <typename ST>
+__device__ __forceinline__ constexpr int ar_is_f16() { return 0; }
+template <>
+__device__ __forceinline__ constexpr int ar_is_f16<__half>() { return 1; }
 
 // (Loops over keys stay rolled and the row count is a template parameter: the kernel runs its code once, so its
 // time is instruction fetch, and a fully unrolled version measured 55 us against a few us of work.)
@@ -598,12 +596,12 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
                 const float *krow = a.q + (size_t)(j - base) * a.ld_q + d + kvh * HD, *vrow = krow + kvd;
                 const float2 cs = a.rope_cs[(size_t)j * HALF + i];
                 const float ka = krow[i], kb = krow[i + HALF];
-                const __nv_bfloat16 k0 = __float2bfloat16_rn(ka * cs.x - kb * cs.y), k1 = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
-                const __nv_bfloat16 v0 = __float2bfloat16_rn(vrow[i]), v1 = __float2bfloat16_rn(vrow[i + HALF]);
-                __nv_bfloat16 *sk = (__nv_bfloat16 *)(stage_k + (size_t)r * ROWB), *sv = (__nv_bfloat16 *)(stage_v + (size_t)r * ROWB);
+                const ST k0 = ar_from_f32<ST>(ka * cs.x - kb * cs.y), k1 = ar_from_f32<ST>(kb * cs.x + ka * cs.y);
+                const ST v0 = ar_from_f32<ST>(vrow[i]), v1 = ar_from_f32<ST>(vrow[i + HALF]);
+                ST *sk = (ST *)(stage_k + (size_t)r * ROWB), *sv = (ST *)(stage_v + (size_t)r * ROWB);
                 sk[i] = k0; sk[i + HALF] = k1; sv[i] = v0; sv[i + HALF] = v1;
                 if (writer) {
-                    __nv_bfloat16 *ck = (__nv_bfloat16 *)(Kc + (size_t)j * HD), *cv = (__nv_bfloat16 *)(Vc + (size_t)j * HD);
+                    ST *ck = Kc + (size_t)j * HD, *cv = Vc + (size_t)j * HD;
                     ck[i] = k0; ck[i + HALF] = k1; cv[i] = v0; cv[i + HALF] = v1;
                 }
             }
@@ -624,8 +622,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
                     const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        kf[(2 * e) % EPL] = __uint_as_float(u[e] << 16);
-                        kf[(2 * e + 1) % EPL] = __uint_as_float(u[e] & 0xffff0000u);
+                        ClPair16<ST>::get(u[e], kf[(2 * e) % EPL], kf[(2 * e + 1) % EPL]);
                     }
                 } else {
                     kf[0] = __uint_as_float(raw.x); kf[1 % EPL] = __uint_as_float(raw.y);
@@ -680,8 +677,8 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
                     const ST *vp = (const ST *)(stage_v + (size_t)min(jh + j, n - 1) * ROWB) + lane * VPL;
                     if (sizeof(ST) == 2 && VPL == 4) {
                         const uint2 u = *(const uint2 *)vp;
-                        vv[j][0] = __uint_as_float(u.x << 16); vv[j][1 % VPL] = __uint_as_float(u.x & 0xffff0000u);
-                        vv[j][2 % VPL] = __uint_as_float(u.y << 16); vv[j][3 % VPL] = __uint_as_float(u.y & 0xffff0000u);
+                        ClPair16<ST>::get(u.x, vv[j][0], vv[j][1 % VPL]);
+                        ClPair16<ST>::get(u.y, vv[j][2 % VPL], vv[j][3 % VPL]);
                     } else {
 #pragma unroll
                         for (int e = 0; e < VPL; ++e) vv[j][e] = (float)vp[e];
@@ -779,9 +776,7 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
         const float o = O / Ls;
         a.out[(size_t)t * d + h * HD + e] = o;
         if (a.out_b) {
-            const __nv_bfloat16 hi = __float2bfloat16_rn(o);
-            a.out_b[(size_t)t * d + h * HD + e] = hi;
-            a.out_b[(size_t)(a.nh + t) * d + h * HD + e] = __float2bfloat16_rn(o - __bfloat162float(hi));
+            store_split(a.out_b + (size_t)t * d + h * HD + e, a.out_b + (size_t)(a.nh + t) * d + h * HD + e, o, sizeof(ST) == 2 && ar_is_f16<ST>());
         }
     }
 }
@@ -794,11 +789,11 @@ size_t cl_attn_rows_part_floats(int H, int S, int T, int hd) { return (size_t)H 
 cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s) {
     if (S < 1 || S > AR_MAXS) return cudaErrorInvalidValue;
     dim3 grid(a.n_heads, S);
-    const size_t es = wdtype == 1 ? 2 : 4;
+    const size_t es = wdtype != 0 ? 2 : 4;
     const size_t smem = (((size_t)AR_WARPS * T * (a.head_dim + 2) * sizeof(float) + 15) & ~(size_t)15) + (size_t)AR_WARPS * 2 * 32 * a.head_dim * es;
-#define AR_LAUNCH(HDV, TT)                                                                                            \
+#define AR_LAUNCH(STT, HDV, TT)                                                                                          \
     {                                                                                                                 \
-        cudaError_t e_ = cudaFuncSetAttribute(k_attn_rows<__nv_bfloat16, HDV, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+        cudaError_t e_ = cudaFuncSetAttribute(k_attn_rows<STT, HDV, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                               (int)smem);                                                             \
         if (e_ != cudaSuccess) return e_;                                                                             \
         cudaLaunchConfig_t cfg_;                                                                                      \
@@ -812,12 +807,14 @@ cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, c
         attr_[0].val.programmaticStreamSerializationAllowed = 1;                                                      \
         cfg_.attrs = attr_;                                                                                           \
         cfg_.numAttrs = 1;                                                                                            \
-        return cudaLaunchKernelEx(&cfg_, k_attn_rows<__nv_bfloat16, HDV, TT>, a, S);                                  \
+        return cudaLaunchKernelEx(&cfg_, k_attn_rows<STT, HDV, TT>, a, S);                                  \
     }
 #define AR_CASE(TT)                                              \
     case TT:                                                     \
-        if (wdtype == 1 && a.head_dim == 128) AR_LAUNCH(128, TT) \
-        else if (wdtype == 1 && a.head_dim == 64) AR_LAUNCH(64, TT) \
+        if (wdtype == 1 && a.head_dim == 128) AR_LAUNCH(__nv_bfloat16, 128, TT) \
+        else if (wdtype == 1 && a.head_dim == 64) AR_LAUNCH(__nv_bfloat16, 64, TT) \
+        else if (wdtype == 2 && a.head_dim == 128) AR_LAUNCH(__half, 128, TT) \
+        else if (wdtype == 2 && a.head_dim == 64) AR_LAUNCH(__half, 64, TT) \
         else return cudaErrorInvalidValue;                       \
         break;
     switch (T) {

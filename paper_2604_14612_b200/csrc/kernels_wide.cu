@@ -1,11 +1,13 @@
-// Wide tensor-core GEMM for the prompt pass of the bf16 model: the full-model pass of Section 3 over up to 512
-// prompt rows at a time, so that the weights stream from HBM once per 512 tokens instead of once per 8.
+// Wide tensor-core GEMM for the prompt pass of a model stored in a 16-bit type (bf16 or fp16): the full-model pass of
+// Section 3 over up to 512 prompt rows at a time, so that the weights stream from HBM once per 512 tokens instead
+// of once per 8.
 //
-//   P[ks, t, r] = sum_{k in part ks} a[t, k] * W[r, k]        a: M activation rows, W: [rows, K] bf16 weights
+//   P[ks, t, r] = sum_{k in part ks} a[t, k] * W[r, k]        a: M activation rows, W: [rows, K] 16-bit weights
 //
 // Here the token rows are the M = 128 operand of tcgen05.mma (one tensor-memory lane per token) and 256 weight rows
-// are N.  Activations are fp32 everywhere else; each row enters as hi = bf16(v) and lo = bf16(v - hi) and both
-// products accumulate into the same fp32 accumulator, so the product keeps about 16 mantissa bits of the activation.
+// are N.  Activations are fp32 everywhere else; each row enters as hi = round16(v) and lo = round16(v - hi) in the
+// weights' type and both products accumulate into the same fp32 accumulator, so the product keeps about 16 (bf16)
+// or 22 (fp16) mantissa bits of the activation.
 // One CTA computes one (token tile, weight tile, K part): the K range is cut into `splits` parts only to fill the
 // 148 SMs when a matrix has few output tiles (4096 outputs are 16 tiles), and the parts are added in a fixed order
 // by the small kernel that consumes the product:
@@ -92,7 +94,7 @@ k_wide(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtenso
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const unsigned idesc = umma_idesc(WM, WN);
+            const unsigned idesc = umma_idesc(WM, WN, a.f16);
             unsigned stage = 0, par = 0;
             bool ok = true;
             for (int kb = kb0; kb < kb1; ++kb) {
@@ -141,28 +143,23 @@ k_wide(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtenso
     }
 }
 
-__device__ __forceinline__ void w_split(float v, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
-    hi = __float2bfloat16_rn(v);
-    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-}
-
 // One CTA per token row: x[t] = E[token] or x[t] += product parts (added in part order); the optional hidden tap;
 // then the rows of the next GEMM: hi/lo(x * rsqrt(mean x^2 + eps) * g).
 __global__ void __launch_bounds__(256) k_wide_norm(ClWideNormArgs a) {
     __shared__ float red[8];
     const int t = blockIdx.x, tid = threadIdx.x, d = a.d;
     float *xr = a.x + (size_t)t * d;
-    const __nv_bfloat16 *er = a.tok ? (const __nv_bfloat16 *)a.embed + (size_t)a.tok[t] * d : nullptr;
+    const unsigned short *er = a.tok ? (const unsigned short *)a.embed + (size_t)a.tok[t] * d : nullptr;
     // only the last tap_P rows of the pass reach the ring: an earlier row of the same slot would be overwritten anyway
-    __nv_bfloat16 *tap = nullptr;
-    if (a.tap && t >= a.M - a.tap_P) tap = (__nv_bfloat16 *)a.tap + (size_t)((a.st->ctx + t) % a.tap_P) * d;
+    unsigned short *tap = nullptr;
+    if (a.tap && t >= a.M - a.tap_P) tap = (unsigned short *)a.tap + (size_t)((a.st->ctx + t) % a.tap_P) * d;
     float ss = 0.f;
     for (int i = tid * 4; i < d; i += 1024) {
         float4 v;
         if (er) {
             const uint2 u = *(const uint2 *)(er + i);
-            v = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
-                            __uint_as_float(u.y & 0xffff0000u));
+            pair16_to_f32(u.x, a.f16, v.x, v.y);
+            pair16_to_f32(u.y, a.f16, v.z, v.w);
         } else {
             v = *(const float4 *)(xr + i);
             for (int s = 0; s < a.splits; ++s) {
@@ -172,8 +169,8 @@ __global__ void __launch_bounds__(256) k_wide_norm(ClWideNormArgs a) {
         }
         *(float4 *)(xr + i) = v;
         if (tap) {
-            tap[i] = __float2bfloat16_rn(v.x); tap[i + 1] = __float2bfloat16_rn(v.y);
-            tap[i + 2] = __float2bfloat16_rn(v.z); tap[i + 3] = __float2bfloat16_rn(v.w);
+            tap[i] = f32_to_b16(v.x, a.f16); tap[i + 1] = f32_to_b16(v.y, a.f16);
+            tap[i + 2] = f32_to_b16(v.z, a.f16); tap[i + 3] = f32_to_b16(v.w, a.f16);
         }
         ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
     }
@@ -189,17 +186,17 @@ __global__ void __launch_bounds__(256) k_wide_norm(ClWideNormArgs a) {
     for (int i = tid * 4; i < d; i += 1024) {
         const float4 v = *(const float4 *)(xr + i);   // this thread's own writes
         const float4 g = *(const float4 *)(a.g + i);
-        w_split(v.x * sc * g.x, hi[i], lo[i]);
-        w_split(v.y * sc * g.y, hi[i + 1], lo[i + 1]);
-        w_split(v.z * sc * g.z, hi[i + 2], lo[i + 2]);
-        w_split(v.w * sc * g.w, hi[i + 3], lo[i + 3]);
+        store_split(hi + i, lo + i, v.x * sc * g.x, a.f16);
+        store_split(hi + i + 1, lo + i + 1, v.y * sc * g.y, a.f16);
+        store_split(hi + i + 2, lo + i + 2, v.z * sc * g.z, a.f16);
+        store_split(hi + i + 3, lo + i + 3, v.w * sc * g.w, a.f16);
     }
 }
 
 // grid (M, H), hd / 2 threads: q, k, v of row t and head h from the QKV product parts; rotary embedding at position
 // ctx + t; q goes back in place (part 0), k and v (the first Hkv heads) go to the cache [kv head][position][hd].
 __global__ void k_wide_rope_append(float *P, int splits, int M, int hd, int d, int Hkv, const float2 *rope_cs,
-                                   __nv_bfloat16 *kcache, __nv_bfloat16 *vcache, int max_seq, const ClDevState *st) {
+                                   unsigned short *kcache, unsigned short *vcache, int max_seq, const ClDevState *st, int f16) {
     const int t = blockIdx.x, h = blockIdx.y, i = threadIdx.x, half = hd >> 1;
     const int pos = st->ctx + t;
     if (pos >= max_seq) return;
@@ -217,11 +214,11 @@ __global__ void k_wide_rope_append(float *P, int splits, int M, int hd, int d, i
     row[h * hd + i + half] = qb * cs.x + qa * cs.y;
     if (h >= Hkv) return;
     const float ka = total(d + h * hd + i), kb = total(d + h * hd + i + half);
-    __nv_bfloat16 *kc = kcache + ((size_t)h * max_seq + pos) * hd, *vc = vcache + ((size_t)h * max_seq + pos) * hd;
-    kc[i] = __float2bfloat16_rn(ka * cs.x - kb * cs.y);
-    kc[i + half] = __float2bfloat16_rn(kb * cs.x + ka * cs.y);
-    vc[i] = __float2bfloat16_rn(total(d + kvd + h * hd + i));
-    vc[i + half] = __float2bfloat16_rn(total(d + kvd + h * hd + i + half));
+    unsigned short *kc = kcache + ((size_t)h * max_seq + pos) * hd, *vc = vcache + ((size_t)h * max_seq + pos) * hd;
+    kc[i] = f32_to_b16(ka * cs.x - kb * cs.y, f16);
+    kc[i + half] = f32_to_b16(kb * cs.x + ka * cs.y, f16);
+    vc[i] = f32_to_b16(total(d + kvd + h * hd + i), f16);
+    vc[i + half] = f32_to_b16(total(d + kvd + h * hd + i + half), f16);
 }
 
 // ---- causal attention of the rows of the pass over the cache -------------------------------------------------
@@ -235,8 +232,8 @@ constexpr int AQ = 64, AK = 64, APS = 68;   // rows per CTA, keys per tile, row 
 
 template <int HD>
 __global__ void __launch_bounds__(256, 2)
-k_attn_wide(const float *q, int ld_q, const __nv_bfloat16 *kcache, const __nv_bfloat16 *vcache, __nv_bfloat16 *out_b,
-            int lo_row0, int M, int d, int H, int Hkv, int max_seq, const ClDevState *st) {
+k_attn_wide(const float *q, int ld_q, const unsigned short *kcache, const unsigned short *vcache, __nv_bfloat16 *out_b,
+            int lo_row0, int M, int d, int H, int Hkv, int max_seq, const ClDevState *st, int f16) {
     constexpr int NV = HD / 64;                       // float4 column groups of O per thread
     constexpr int KP = (HD * AK > AQ * APS) ? HD * AK : AQ * APS;
     extern __shared__ __align__(16) float asm_[];
@@ -250,7 +247,7 @@ k_attn_wide(const float *q, int ld_q, const __nv_bfloat16 *kcache, const __nv_bf
     const int rlast = min(r0 + AQ, M) - 1;            // last live row of this block
     const int nkeys = min(ctx + rlast + 1, max_seq);
     const int kvh = h / (H / Hkv);
-    const __nv_bfloat16 *Kc = kcache + (size_t)kvh * max_seq * HD, *Vc = vcache + (size_t)kvh * max_seq * HD;
+    const unsigned short *Kc = kcache + (size_t)kvh * max_seq * HD, *Vc = vcache + (size_t)kvh * max_seq * HD;
     const float scale = rsqrtf((float)HD);
 
     for (int i = tid; i < AQ * HD / 4; i += 256) {
@@ -283,8 +280,7 @@ k_attn_wide(const float *q, int ld_q, const __nv_bfloat16 *kcache, const __nv_bf
             const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                Kt[(c8 * 8 + 2 * e) * AK + key] = __uint_as_float(u[e] << 16);
-                Kt[(c8 * 8 + 2 * e + 1) * AK + key] = __uint_as_float(u[e] & 0xffff0000u);
+                pair16_to_f32(u[e], f16, Kt[(c8 * 8 + 2 * e) * AK + key], Kt[(c8 * 8 + 2 * e + 1) * AK + key]);
             }
         }
         for (int i = tid; i < AK * HD / 8; i += 256) {
@@ -292,10 +288,13 @@ k_attn_wide(const float *q, int ld_q, const __nv_bfloat16 *kcache, const __nv_bf
             uint4 raw = make_uint4(0u, 0u, 0u, 0u);
             if (k0 + key < nkeys) raw = *(const uint4 *)(Vc + (size_t)(k0 + key) * HD + c8 * 8);
             float4 *dst = (float4 *)(Vs + key * HD + c8 * 8);
-            dst[0] = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u), __uint_as_float(raw.y << 16),
-                                 __uint_as_float(raw.y & 0xffff0000u));
-            dst[1] = make_float4(__uint_as_float(raw.z << 16), __uint_as_float(raw.z & 0xffff0000u), __uint_as_float(raw.w << 16),
-                                 __uint_as_float(raw.w & 0xffff0000u));
+            float4 lo4, hi4;
+            pair16_to_f32(raw.x, f16, lo4.x, lo4.y);
+            pair16_to_f32(raw.y, f16, lo4.z, lo4.w);
+            pair16_to_f32(raw.z, f16, hi4.x, hi4.y);
+            pair16_to_f32(raw.w, f16, hi4.z, hi4.w);
+            dst[0] = lo4;
+            dst[1] = hi4;
         }
         __syncthreads();
         float sc[4][4];
@@ -382,10 +381,10 @@ k_attn_wide(const float *q, int ld_q, const __nv_bfloat16 *kcache, const __nv_bf
             unsigned hi[4], lo[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                __nv_bfloat16 bh, bl;
-                w_split(o[i][v][e] * inv, bh, bl);
-                hi[e] = __bfloat16_as_ushort(bh);
-                lo[e] = __bfloat16_as_ushort(bl);
+                unsigned short bh, bl;
+                split_b16(o[i][v][e] * inv, f16, bh, bl);
+                hi[e] = bh;
+                lo[e] = bl;
             }
             *(uint2 *)(out_b + (size_t)row * d + col) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
             *(uint2 *)(out_b + (size_t)(lo_row0 + row) * d + col) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
@@ -394,7 +393,7 @@ k_attn_wide(const float *q, int ld_q, const __nv_bfloat16 *kcache, const __nv_bf
 }
 
 // grid (M, ceil(F / 256)): the gate/up product has rows interleaved (2 i = gate_i, 2 i + 1 = up_i).
-__global__ void __launch_bounds__(256) k_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0) {
+__global__ void __launch_bounds__(256) k_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, int f16) {
     const int t = blockIdx.x, i = blockIdx.y * 256 + threadIdx.x;
     if (i >= F) return;
     float g = 0.f, u = 0.f;
@@ -404,7 +403,7 @@ __global__ void __launch_bounds__(256) k_wide_silu(const float *P, int splits, i
         u += p.y;
     }
     const float h = g / (1.f + expf(-g)) * u;
-    w_split(h, A[(size_t)t * F + i], A[(size_t)(lo_row0 + t) * F + i]);
+    store_split(A + (size_t)t * F + i, A + (size_t)(lo_row0 + t) * F + i, h, f16);
 }
 
 }  // namespace
@@ -448,20 +447,20 @@ cudaError_t cl_launch_wide_norm(const ClWideNormArgs &a, cudaStream_t s) {
 }
 
 cudaError_t cl_launch_wide_rope_append(float *P, int splits, int M, int H, int Hkv, int hd, int d, const float2 *rope_cs,
-                                       void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s) {
-    k_wide_rope_append<<<dim3(M, H), hd / 2, 0, s>>>(P, splits, M, hd, d, Hkv, rope_cs, (__nv_bfloat16 *)kcache,
-                                                     (__nv_bfloat16 *)vcache, max_seq, st);
+                                       void *kcache, void *vcache, int max_seq, const ClDevState *st, int f16, cudaStream_t s) {
+    k_wide_rope_append<<<dim3(M, H), hd / 2, 0, s>>>(P, splits, M, hd, d, Hkv, rope_cs, (unsigned short *)kcache,
+                                                     (unsigned short *)vcache, max_seq, st, f16);
     return cudaGetLastError();
 }
 
-cudaError_t cl_launch_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, cudaStream_t s) {
-    k_wide_silu<<<dim3(M, (F + 255) / 256), 256, 0, s>>>(P, splits, M, F, A, lo_row0);
+cudaError_t cl_launch_wide_silu(const float *P, int splits, int M, int F, __nv_bfloat16 *A, int lo_row0, int f16, cudaStream_t s) {
+    k_wide_silu<<<dim3(M, (F + 255) / 256), 256, 0, s>>>(P, splits, M, F, A, lo_row0, f16);
     return cudaGetLastError();
 }
 
 cudaError_t cl_launch_attn_wide(const float *q, int ld_q, const void *kcache, const void *vcache, __nv_bfloat16 *out_b,
                                 int lo_row0, int M, int d, int H, int Hkv, int hd, int max_seq, const ClDevState *st,
-                                cudaStream_t s) {
+                                int f16, cudaStream_t s) {
     const dim3 grid(H, (M + AQ - 1) / AQ);
     const int kp = (hd * AK > AQ * APS) ? hd * AK : AQ * APS;
     const size_t smem = (size_t)(hd * AQ + kp + AK * hd) * sizeof(float);
@@ -472,8 +471,8 @@ cudaError_t cl_launch_attn_wide(const float *q, int ld_q, const void *kcache, co
             if (e != cudaSuccess) return e;
             set128 = true;
         }
-        k_attn_wide<128><<<grid, 256, smem, s>>>(q, ld_q, (const __nv_bfloat16 *)kcache, (const __nv_bfloat16 *)vcache, out_b,
-                                                 lo_row0, M, d, H, Hkv, max_seq, st);
+        k_attn_wide<128><<<grid, 256, smem, s>>>(q, ld_q, (const unsigned short *)kcache, (const unsigned short *)vcache, out_b,
+                                                 lo_row0, M, d, H, Hkv, max_seq, st, f16);
     } else if (hd == 64) {
         static bool set64 = false;
         if (!set64) {
@@ -481,8 +480,8 @@ cudaError_t cl_launch_attn_wide(const float *q, int ld_q, const void *kcache, co
             if (e != cudaSuccess) return e;
             set64 = true;
         }
-        k_attn_wide<64><<<grid, 256, smem, s>>>(q, ld_q, (const __nv_bfloat16 *)kcache, (const __nv_bfloat16 *)vcache, out_b,
-                                                lo_row0, M, d, H, Hkv, max_seq, st);
+        k_attn_wide<64><<<grid, 256, smem, s>>>(q, ld_q, (const unsigned short *)kcache, (const unsigned short *)vcache, out_b,
+                                                lo_row0, M, d, H, Hkv, max_seq, st, f16);
     } else {
         return cudaErrorInvalidValue;
     }

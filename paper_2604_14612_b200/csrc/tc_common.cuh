@@ -7,7 +7,7 @@
 
 namespace {
 
-constexpr int TC_BK = 64;   // K extent of one shared-memory tile: 64 bf16 = one 128-byte swizzle row
+constexpr int TC_BK = 64;   // K extent of one shared-memory tile: 64 16-bit elements = one 128-byte swizzle row
 constexpr unsigned long long WAIT_NS = 2000000000ull;
 
 __device__ __forceinline__ unsigned s_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -70,9 +70,35 @@ __device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
     d |= (unsigned long long)2 << 61;                          // 128-byte swizzle
     return d;
 }
-// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, both K-major, N and M of the tile.
-__device__ __forceinline__ unsigned umma_idesc(int m, int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(m >> 4) << 24);
+// Instruction descriptor of kind::f16: fp32 accumulator, A and B of the same 16-bit type (format 1 = bf16, 0 = fp16),
+// both K-major, N and M of the tile.
+__device__ __forceinline__ unsigned umma_idesc(int m, int n, int f16 = 0) {
+    const unsigned fmt = f16 ? 0u : 1u;
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(m >> 4) << 24);
+}
+
+// The 16-bit type of a model (storage and tensor-core operands) chosen at run time: f16 != 0 is IEEE binary16,
+// else bfloat16.  Values travel as raw 16-bit patterns.
+__device__ __forceinline__ unsigned short f32_to_b16(float v, int f16) {
+    return f16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+__device__ __forceinline__ float b16_to_f32(unsigned short b, int f16) {
+    return f16 ? __half2float(__ushort_as_half(b)) : __uint_as_float((unsigned)b << 16);
+}
+__device__ __forceinline__ void pair16_to_f32(unsigned u, int f16, float &a, float &b) {
+    if (f16) ClPair16<__half>::get(u, a, b);
+    else ClPair16<__nv_bfloat16>::get(u, a, b);
+}
+// v -> (hi, lo) with hi + lo = v to about 16 (bf16) or 22 (fp16) mantissa bits
+__device__ __forceinline__ void split_b16(float v, int f16, unsigned short &hi, unsigned short &lo) {
+    hi = f32_to_b16(v, f16);
+    lo = f32_to_b16(v - b16_to_f32(hi, f16), f16);
+}
+__device__ __forceinline__ void store_split(__nv_bfloat16 *hi_p, __nv_bfloat16 *lo_p, float v, int f16) {
+    unsigned short hi, lo;
+    split_b16(v, f16, hi, lo);
+    *reinterpret_cast<unsigned short *>(hi_p) = hi;
+    *reinterpret_cast<unsigned short *>(lo_p) = lo;
 }
 __device__ __forceinline__ void umma_bf16(unsigned tmem_d, unsigned long long adesc, unsigned long long bdesc, unsigned idesc,
                                           unsigned accumulate) {
@@ -117,15 +143,16 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 2-D bf16 row-major [rows, cols] tensor, box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
-bool make_map(CUtensorMap *m, const void *base, int rows, int cols, int box_rows) {
+// 2-D row-major [rows, cols] tensor of 16-bit elements (bf16, or fp16 with f16 != 0), box = 64 columns x box_rows
+// rows, 128-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap *m, const void *base, int rows, int cols, int box_rows, int f16 = 0) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
     cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return fn(m, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

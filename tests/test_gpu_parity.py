@@ -253,11 +253,12 @@ def test_generate_to_the_last_cache_slot():
         assert list(toks) == list(van)
 
 
-def test_tensor_core_pass_matches_streaming_pass(monkeypatch):
-    """The tcgen05 pass (verify / prefill of bf16 models) against the CUDA-core T-row path on the same inputs:
+@pytest.mark.parametrize("wd", ["bf16", "fp16"])
+def test_tensor_core_pass_matches_streaming_pass(monkeypatch, wd):
+    """The tcgen05 pass (verify / prefill of 16-bit models) against the CUDA-core T-row path on the same inputs:
     two independent implementations of the same full-model pass, T = 5 (N = 16) and T = 9 (N = 32)."""
     base = synth.WORKLOADS["C2"].shape
-    sh = dataclasses.replace(base, n_layers=2, max_seq=64)
+    sh = dataclasses.replace(base, n_layers=2, max_seq=64, weight_dtype=wd)
     W = synth.make_weights(sh, 5, device="cuda")
     prompt = synth.make_prompt(5, 11, sh.vocab)                        # a full chunk of 8 and a ragged one of 3
     out = {}
@@ -283,13 +284,14 @@ def test_tensor_core_pass_matches_streaming_pass(monkeypatch):
     assert np.abs(out[0][3] - out[1][3]).max() <= 2 ** -7 * scale        # taps: one bf16 ulp at the top of the range
 
 
-def test_wide_prompt_pass_matches_chunked_prompt_pass(monkeypatch):
+@pytest.mark.parametrize("wd", ["bf16", "fp16"])
+def test_wide_prompt_pass_matches_chunked_prompt_pass(monkeypatch, wd):
     """The wide tcgen05 GEMMs of the prompt pass (up to 512 rows at a time) against the 8-row passes on the same
     prompt: the same KV cache (seen through the logits of a verify pass that follows), first token and hidden taps.
     700 prompt tokens = one full pass of 512 rows and a ragged one of 187 (a partial token tile, 3 rows left over
     for the attention) before the last token."""
     base = synth.WORKLOADS["C2"].shape
-    sh = dataclasses.replace(base, n_layers=2, max_seq=768)
+    sh = dataclasses.replace(base, n_layers=2, max_seq=768, weight_dtype=wd)
     W = synth.make_weights(sh, 6, device="cuda")
     prompt = synth.make_prompt(6, 700, sh.vocab)
     out = {}
