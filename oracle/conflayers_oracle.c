@@ -75,6 +75,17 @@ float orc_fp16_bits_to_f32(uint16_t b) {
     return (float)(sign ? -v : v);
 }
 
+/* all 65536 widenings, filled once (by whichever thread gets there first; every thread writes the same values) */
+static const float *fp16_table(void) {
+    static float table[65536];
+    static volatile int ready = 0;
+    if (!ready) {
+        for (int b = 0; b < 65536; ++b) table[b] = orc_fp16_bits_to_f32((uint16_t)b);
+        ready = 1;
+    }
+    return table;
+}
+
 /* round-to-nearest-even fp32 -> fp16 -> fp32, from the definition: the representable neighbours of |f| are
  * multiples of the spacing 2^(E-10) with E = max(floor(log2 |f|), -14); ties go to the even multiple; what rounds to
  * 2^16 or beyond is infinity. */
@@ -113,7 +124,9 @@ double orc_dot_row(const void *W, int dtype, size_t row, int cols, const float *
         for (int c = 0; c < cols; ++c) acc += (double)bf16_bits_to_f32(w[c]) * (double)x[c];
     } else if (dtype == 2) {
         const uint16_t *w = (const uint16_t *)W + base;
-        for (int c = 0; c < cols; ++c) acc += (double)orc_fp16_bits_to_f32(w[c]) * (double)x[c];
+        const float *wide = fp16_table();
+#pragma omp simd reduction(+ : acc)
+        for (int c = 0; c < cols; ++c) acc += (double)wide[w[c]] * (double)x[c];
     } else {
         const float *w = (const float *)W + base;
 #pragma omp simd reduction(+ : acc)
