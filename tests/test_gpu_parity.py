@@ -376,12 +376,14 @@ def _first_difference_is_a_near_tie(ctx, w, toks_a, toks_b, first):
     return diff
 
 
-@pytest.mark.parametrize("name,K,ratio,gen", [("C3", 4, 0.5, 48), ("C3", 8, 0.25, 32), ("C4", 6, 0.4, 24)])
-def test_full_size_properties_in_the_bench_configuration(name, K, ratio, gen):
+@pytest.mark.parametrize("name,K,ratio,gen,wd", [("C3", 4, 0.5, 48, "bf16"), ("C3", 8, 0.25, 32, "bf16"),
+                                                 ("C4", 6, 0.4, 24, "bf16"), ("C3", 4, 0.5, 24, "fp16")])
+def test_full_size_properties_in_the_bench_configuration(name, K, ratio, gen, wd):
     """Full 7B / 13B shapes, full depth, full prompt (the launch configuration the benchmark times): properties that
     hold at any size -- speculative decoding emits the vanilla greedy tokens (lossless), the counters add up, an
     empty skip set accepts every draft."""
     w = synth.WORKLOADS[name]
+    w = dataclasses.replace(w, shape=dataclasses.replace(w.shape, weight_dtype=wd))
     W = synth.make_weights(w.shape, w.seed, device="cuda")
     ctx = cl.Context.from_shape(w.shape)
     ctx.cl_load(W)
