@@ -101,7 +101,6 @@ __device__ __forceinline__ unsigned long long policy_evict_first() {
 __device__ __forceinline__ void l2_prefetch_bulk(const void *src, unsigned bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void l2_prefetch_line(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NCT) : "memory"); }
 
@@ -616,27 +615,11 @@ struct AttnGeom {
 
 __device__ __forceinline__ void warp_key_range(int pos, int s, int S, int warp, int &kw0, int &kw1) {
     const int k0 = (int)((long long)pos * s / S), k1 = (int)((long long)pos * (s + 1) / S);
-    kw0 = k0 + (k1 - k0) * warp / NCW;
-    kw1 = k0 + (k1 - k0) * (warp + 1) / NCW;
-}
-
-// Ask L2 for the cache lines this CTA's warps will read in the attention phase (issued a whole matrix phase earlier).
-template <typename ST, int HD>
-__device__ __forceinline__ void attention_prefetch(const ClStepArgs &a, const ClLayerDev &L, int pos) {
-    const int S = a.att_parts, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int item = blockIdx.x;
-    if (item >= a.H * S) return;
-    const int h = item % a.H, s = item / a.H;
-    int kw0, kw1;
-    warp_key_range(pos, s, S, warp, kw0, kw1);
-    constexpr int ROWB = HD * (int)sizeof(ST);
-    constexpr int LINES = (ROWB + 127) / 128;
-    const int n = (kw1 - kw0) * LINES;
-    for (int i = lane; i < n; i += 32) {
-        const size_t off = ((size_t)(h / (a.H / a.Hkv)) * a.max_seq + kw0 + i / LINES) * HD * sizeof(ST) + (size_t)(i % LINES) * 128;
-        l2_prefetch_line(L.kc + off);
-        l2_prefetch_line(L.vc + off);
-    }
+    // the last warp of the last part takes the new position, so it gets no cached keys (its CTA would otherwise
+    // finish last and hold up the barrier that follows)
+    const int nw = (s == S - 1) ? NCW - 1 : NCW;
+    kw0 = k0 + (k1 - k0) * min(warp, nw) / nw;
+    kw1 = k0 + (k1 - k0) * min(warp + 1, nw) / nw;
 }
 
 template <typename ST, int HD>
@@ -897,8 +880,9 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             const int ent = a.kept[ki], fl = ent >> 16;   // bit 0: this layer's attention half is skipped, bit 1: its FFN half
             const ClLayerDev L = a.layers[ent & 0xffff];
             if (!(fl & 1)) {
-            // QKV projection of the normalised stream (the attention phase's cache lines are requested now)
-            attention_prefetch<WT, HD>(a, L, pos);
+            // QKV projection of the normalised stream.  (Asking L2 for the attention phase's keys and values from here,
+            // a matrix phase early, measured slower: whichever thread issues the request, consumer warp or producer,
+            // stalls about 1.5 us on it, more than the attention phase gains.)
             load_x_rmsnorm<EPC>(a.x, L.n1, d, a.eps, xr, sm);
             consume_matrix<WT>(d + 2 * a.Hkv * HD, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.qkv[rb0 + r] = row_sum(sm, r);
