@@ -556,29 +556,34 @@ __device__ __forceinline__ void load_x(const float *x, int cols, float (&xr)[MAX
 
 // RMSNorm in registers: xr <- x * rsqrt(mean(x^2) + eps) * g.  The gains are requested together with x so that the
 // phase start costs one memory round trip, not two.
-template <int EPC>
-__device__ __forceinline__ void load_x_rmsnorm(const float *x, const float *g, int cols, float eps, float (&xr)[MAXIT][EPC],
-                                               Smem *sm) {
+template <int EPC, int NI>
+__device__ __forceinline__ void load_x_rmsnorm_n(const float *x, const float *g, int cols, float eps, float (&xr)[MAXIT][EPC],
+                                                 Smem *sm) {
     const int nchunks = cols / EPC;
-    float gr[MAXIT][EPC];
+    float gr[NI][EPC];
 #pragma unroll
-    for (int it = 0; it < MAXIT; ++it) {
+    for (int it = 0; it < NI; ++it) {
         const int ch = it * NCT + threadIdx.x;
         if (ch < nchunks) {
 #pragma unroll
             for (int q = 0; q < EPC / 4; ++q) {
                 const float4 gv = __ldg((const float4 *)(g + (size_t)ch * EPC + 4 * q));
+                const float4 xv = ldcg_f4(x + (size_t)ch * EPC + 4 * q);
                 gr[it][4 * q] = gv.x; gr[it][4 * q + 1] = gv.y; gr[it][4 * q + 2] = gv.z; gr[it][4 * q + 3] = gv.w;
+                xr[it][4 * q] = xv.x; xr[it][4 * q + 1] = xv.y; xr[it][4 * q + 2] = xv.z; xr[it][4 * q + 3] = xv.w;
             }
         } else {
 #pragma unroll
-            for (int e = 0; e < EPC; ++e) gr[it][e] = 0.f;
+            for (int e = 0; e < EPC; ++e) gr[it][e] = xr[it][e] = 0.f;
         }
     }
-    load_x<EPC>(x, cols, xr);
+#pragma unroll
+    for (int it = NI; it < MAXIT; ++it)
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) xr[it][e] = 0.f;
     float ss = 0.f;
 #pragma unroll
-    for (int it = 0; it < MAXIT; ++it)
+    for (int it = 0; it < NI; ++it)
 #pragma unroll
         for (int e = 0; e < EPC; ++e) ss = fmaf(xr[it][e], xr[it][e], ss);
     ss = warp_sum(ss);
@@ -590,9 +595,20 @@ __device__ __forceinline__ void load_x_rmsnorm(const float *x, const float *g, i
     for (int w = 0; w < NCW; ++w) tot += sm->red[w];
     const float sc = 1.0f / sqrtf(tot / (float)cols + eps);
 #pragma unroll
-    for (int it = 0; it < MAXIT; ++it)
+    for (int it = 0; it < NI; ++it)
 #pragma unroll
         for (int e = 0; e < EPC; ++e) xr[it][e] *= sc * gr[it][e];
+}
+
+// The vector's length decides how many chunks a thread holds (one for d_model = 4096 in 16-bit storage): the short
+// cases keep fewer gains in registers.
+template <int EPC>
+__device__ __forceinline__ void load_x_rmsnorm(const float *x, const float *g, int cols, float eps, float (&xr)[MAXIT][EPC],
+                                               Smem *sm) {
+    const int nchunks = cols / EPC;
+    if (nchunks <= NCT) load_x_rmsnorm_n<EPC, 1>(x, g, cols, eps, xr, sm);
+    else if (nchunks <= 2 * NCT) load_x_rmsnorm_n<EPC, 2>(x, g, cols, eps, xr, sm);
+    else load_x_rmsnorm_n<EPC, MAXIT>(x, g, cols, eps, xr, sm);
 }
 
 // ---- attention phase ---------------------------------------------------------------------------------
@@ -614,7 +630,7 @@ struct AttnGeom {
 };
 
 __device__ __forceinline__ void warp_key_range(int pos, int s, int S, int warp, int &kw0, int &kw1) {
-    const int k0 = (int)((long long)pos * s / S), k1 = (int)((long long)pos * (s + 1) / S);
+    const int k0 = (int)((unsigned)(pos * s) / (unsigned)S), k1 = (int)((unsigned)(pos * (s + 1)) / (unsigned)S);   // (pos * 8 fits easily)
     // the last warp of the last part takes the new position, so it gets no cached keys (its CTA would otherwise
     // finish last and hold up the barrier that follows)
     const int nw = (s == S - 1) ? NCW - 1 : NCW;
@@ -657,36 +673,49 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
             const int n = min(32, kw1 - j0);
             // scores of up to 32 keys; lane j ends up holding the score of key j0 + j
             float my_score = -INFINITY;
+            // KPW keys per pass; the key rows of up to PB passes are requested together (one memory round trip), then
+            // scored; passes past the last key are skipped (a warp usually holds far fewer than 32 keys)
+            constexpr int NPASS = 32 / KPW, PB = NPASS < 8 ? NPASS : 8;
 #pragma unroll
-            for (int jb = 0; jb < 32; jb += KPW) {
-                const int j = jb + sub;
-                float sc = 0.f;
-                if (j < n) {
-                    const uint4 raw = __ldcg((const uint4 *)(Kc + ((size_t)kvh * a.max_seq + j0 + j) * HD + li * EPL));
-                    if (sizeof(ST) == 2) {
-                        const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
+            for (int b0 = 0; b0 < NPASS; b0 += PB) {
+                if (b0 * KPW >= n) break;   // uniform
+                uint4 raw[PB];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float k0, k1;
-                            ClPair16<ST>::get(u[e], k0, k1);
-                            sc = fmaf(qr[(2 * e) % EPL], k0, sc);
-                            sc = fmaf(qr[(2 * e + 1) % EPL], k1, sc);
-                        }
-                    } else {
-                        sc = fmaf(qr[0], __uint_as_float(raw.x), sc);
-                        sc = fmaf(qr[1 % EPL], __uint_as_float(raw.y), sc);
-                        sc = fmaf(qr[2 % EPL], __uint_as_float(raw.z), sc);
-                        sc = fmaf(qr[3 % EPL], __uint_as_float(raw.w), sc);
-                    }
+                for (int p = 0; p < PB; ++p) {
+                    const int j = (b0 + p) * KPW + sub;
+                    raw[p] = make_uint4(0u, 0u, 0u, 0u);
+                    if (j < n) raw[p] = __ldcg((const uint4 *)(Kc + ((size_t)kvh * a.max_seq + j0 + j) * HD + li * EPL));
                 }
 #pragma unroll
-                for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
-                sc *= scale;
-                // key jb + k sits in lanes [k * LPK, (k + 1) * LPK): hand it to lane jb + k
+                for (int p = 0; p < PB; ++p) {
+                    const int jb = (b0 + p) * KPW;
+                    if (jb < n) {   // uniform
+                        float sc = 0.f;
+                        if (sizeof(ST) == 2) {
+                            const unsigned u[4] = {raw[p].x, raw[p].y, raw[p].z, raw[p].w};
 #pragma unroll
-                for (int k = 0; k < KPW; ++k) {
-                    const float v = __shfl_sync(0xffffffffu, sc, k * LPK);
-                    if (lane == jb + k && jb + k < n) my_score = v;
+                            for (int e = 0; e < 4; ++e) {
+                                float k0, k1;
+                                ClPair16<ST>::get(u[e], k0, k1);
+                                sc = fmaf(qr[(2 * e) % EPL], k0, sc);
+                                sc = fmaf(qr[(2 * e + 1) % EPL], k1, sc);
+                            }
+                        } else {
+                            sc = fmaf(qr[0], __uint_as_float(raw[p].x), sc);
+                            sc = fmaf(qr[1 % EPL], __uint_as_float(raw[p].y), sc);
+                            sc = fmaf(qr[2 % EPL], __uint_as_float(raw[p].z), sc);
+                            sc = fmaf(qr[3 % EPL], __uint_as_float(raw[p].w), sc);
+                        }
+#pragma unroll
+                        for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                        sc *= scale;
+                        // key jb + k sits in lanes [k * LPK, (k + 1) * LPK): hand it to lane jb + k
+#pragma unroll
+                        for (int k = 0; k < KPW; ++k) {
+                            const float v = __shfl_sync(0xffffffffu, sc, k * LPK);
+                            if (lane == jb + k && jb + k < n) my_score = v;
+                        }
+                    }
                 }
             }
             float m_new = my_score;
@@ -699,14 +728,21 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
 #pragma unroll
             for (int e = 0; e < VPL; ++e) o_run[e] *= resc;
             m_run = m_new;
-            // all 32 value rows are fetched at once (rows past the end repeat the last one with weight 0)
+            // value rows, eight requested at a time (rows past the end repeat the last one with weight 0); groups past
+            // the last key are skipped
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float pj = __shfl_sync(0xffffffffu, p, j);
-                float vv[VPL];
-                load_vals<ST, VPL>(Vc + ((size_t)kvh * a.max_seq + j0 + min(j, n - 1)) * HD + lane * VPL, vv);
+            for (int jg = 0; jg < 32; jg += 8) {
+                if (jg >= n) break;   // uniform
+                float vv[8][VPL];
 #pragma unroll
-                for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(pj, vv[e], o_run[e]);
+                for (int j = 0; j < 8; ++j)
+                    load_vals<ST, VPL>(Vc + ((size_t)kvh * a.max_seq + j0 + min(jg + j, n - 1)) * HD + lane * VPL, vv[j]);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float pj = __shfl_sync(0xffffffffu, p, jg + j);
+#pragma unroll
+                    for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(pj, vv[j][e], o_run[e]);
+                }
             }
         }
         if (s == S - 1 && warp == NCW - 1) {
@@ -795,34 +831,46 @@ __device__ __forceinline__ void load_att_merged(const ClStepArgs &a, float (&xr)
         if (ch < nchunks) {
             const int h = (ch * EPC) / HD, e0 = (ch * EPC) % HD;
             const float *rec = a.att_part + (size_t)h * ATT_MAX_PARTS * PSTRIDE;
+            // (max, sum) of every part and the outputs of the first four parts are requested together: one memory
+            // round trip for S <= 4.  (Holding all eight parts' outputs at once spilled registers.)
             float2 ml[ATT_MAX_PARTS];
-            float o[ATT_MAX_PARTS][EPC];
+            float o[4][EPC];
 #pragma unroll
             for (int s = 0; s < ATT_MAX_PARTS; ++s) {
                 ml[s] = make_float2(0.f, 0.f);
+                if (s < S) ml[s] = __ldcg((const float2 *)(rec + (size_t)s * PSTRIDE));   // uniform over the grid
+            }
+            float M = -INFINITY, Ls = 0.f, f[ATT_MAX_PARTS];
 #pragma unroll
-                for (int e = 0; e < EPC; ++e) o[s][e] = 0.f;
-                if (s < S) {   // uniform over the grid: parts past S are never read
-                    const float *r = rec + (size_t)s * PSTRIDE;
-                    ml[s] = __ldcg((const float2 *)r);
+            for (int b = 0; b < ATT_MAX_PARTS; b += 4) {
+                if (b >= S) break;   // uniform
 #pragma unroll
-                    for (int q = 0; q < EPC / 4; ++q) {
-                        const float4 t = ldcg_f4(r + 4 + e0 + 4 * q);
-                        o[s][4 * q] = t.x; o[s][4 * q + 1] = t.y; o[s][4 * q + 2] = t.z; o[s][4 * q + 3] = t.w;
+                for (int s = 0; s < 4; ++s) {
+#pragma unroll
+                    for (int e = 0; e < EPC; ++e) o[s][e] = 0.f;
+                    if (b + s < S) {
+                        const float *r = rec + (size_t)(b + s) * PSTRIDE;
+#pragma unroll
+                        for (int q = 0; q < EPC / 4; ++q) {
+                            const float4 t = ldcg_f4(r + 4 + e0 + 4 * q);
+                            o[s][4 * q] = t.x; o[s][4 * q + 1] = t.y; o[s][4 * q + 2] = t.z; o[s][4 * q + 3] = t.w;
+                        }
                     }
                 }
-            }
-            float M = -INFINITY;
+                if (b == 0) {
 #pragma unroll
-            for (int s = 0; s < ATT_MAX_PARTS; ++s)
-                if (s < S && ml[s].y > 0.f) M = fmaxf(M, ml[s].x);
-            float Ls = 0.f;
+                    for (int s = 0; s < ATT_MAX_PARTS; ++s)
+                        if (s < S && ml[s].y > 0.f) M = fmaxf(M, ml[s].x);
 #pragma unroll
-            for (int s = 0; s < ATT_MAX_PARTS; ++s) {
-                const float f = (s < S && ml[s].y > 0.f) ? expf(ml[s].x - M) : 0.f;
-                Ls = fmaf(ml[s].y, f, Ls);
+                    for (int s = 0; s < ATT_MAX_PARTS; ++s) {   // part order
+                        f[s] = (s < S && ml[s].y > 0.f) ? expf(ml[s].x - M) : 0.f;
+                        Ls = fmaf(ml[s].y, f[s], Ls);
+                    }
+                }
 #pragma unroll
-                for (int e = 0; e < EPC; ++e) xr[it][e] = fmaf(o[s][e], f, xr[it][e]);
+                for (int s = 0; s < 4; ++s)
+#pragma unroll
+                    for (int e = 0; e < EPC; ++e) xr[it][e] = fmaf(o[s][e], f[b + s], xr[it][e]);
             }
             const float inv = 1.f / Ls;
 #pragma unroll
