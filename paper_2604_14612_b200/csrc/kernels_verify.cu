@@ -273,18 +273,16 @@ k_skinny(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUten
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if (4 * i < a.N) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                __threadfence();
                 epi_sync();
                 const int c_first = cta_of_unit(U, G, (long long)m * a.KB), c_last = cta_of_unit(U, G, (long long)(m + 1) * a.KB - 1);
                 if (et == 0) {
-                    const unsigned prev = atomicAdd(a.tickets + m, 1u);
+                    const unsigned prev = ticket_acq_rel(a.tickets + m);
                     const int last = (prev == (unsigned)(c_last - c_first));
                     if (last) a.tickets[m] = 0u;
                     sm->is_last = last;
                 }
                 epi_sync();
                 if (!sm->is_last) continue;
-                __threadfence();
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = 0.f;
                 if (a.N == 16) add_partials<4, 4>(v, a, U, G, m, c_first, c_last, rloc);
@@ -729,16 +727,14 @@ __global__ void __launch_bounds__(AR_WARPS * 32) k_attn_rows(ClAttnArgs a, int S
         if (e == 0) { part[(size_t)t * REC] = M; part[(size_t)t * REC + 1] = Ls; }
         part[(size_t)t * REC + 2 + e] = O;
     }
-    __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const unsigned prev = atomicAdd(a.tickets + h, 1u);
+        const unsigned prev = ticket_acq_rel(a.tickets + h);
         is_last = (prev == (unsigned)S - 1);
         if (is_last) a.tickets[h] = 0u;
     }
     __syncthreads();
     if (!is_last) return;
-    __threadfence();
     // every part's (max, sum, output element) of every output of this thread is requested before any is used:
     // one round trip in all, not one per part and output
     constexpr int NOUT = (T * HD + AR_WARPS * 32 - 1) / (AR_WARPS * 32);

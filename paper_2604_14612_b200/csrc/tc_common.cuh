@@ -51,6 +51,16 @@ __device__ __forceinline__ bool bar_wait(unsigned long long *b, unsigned parity,
     }
 }
 
+// Ticket of a "last arrival finishes the job" protocol, taken by ONE thread after a barrier of the threads that wrote
+// the data and before the barrier after which they read other CTAs' data: the release half orders the CTA's earlier
+// writes (made visible to this thread by the barrier) before the increment, the acquire half orders the later reads
+// after it.  Replaces a __threadfence() by every thread on each side of a plain atomicAdd.
+__device__ __forceinline__ unsigned ticket_acq_rel(unsigned *p) {
+    unsigned old;
+    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(p) : "memory");
+    return old;
+}
+
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, unsigned long long *bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
