@@ -638,8 +638,21 @@ __device__ __forceinline__ void warp_key_range(int pos, int s, int S, int warp, 
     kw1 = k0 + (k1 - k0) * min(warp + 1, nw) / nw;
 }
 
+// This CTA's first (usually only) work item of the attention phase: it depends on the position alone, so it is
+// worked out once per step, not once per layer (a dozen integer divisions at the head of a latency-bound phase).
+struct AttnItem {
+    int h, s, kw0, kw1;
+};
+__device__ __forceinline__ AttnItem attn_item(const ClStepArgs &a, int item, int pos, int warp) {
+    AttnItem it;
+    it.h = item % a.H;
+    it.s = item / a.H;
+    warp_key_range(pos, it.s, a.att_parts, warp, it.kw0, it.kw1);
+    return it;
+}
+
 template <typename ST, int HD>
-__device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int pos, Smem *sm) {
+__device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int pos, Smem *sm, const AttnItem &first) {
     using G = AttnGeom<ST, HD>;
     constexpr int EPL = G::EPL, LPK = G::LPK, KPW = G::KPW, VPL = G::VPL, PSTRIDE = G::PSTRIDE;
     constexpr int WSTRIDE = HD + 2;   // per-warp record in shared memory: (max, sum, o[HD])
@@ -652,9 +665,8 @@ __device__ void attention_phase(const ClStepArgs &a, const ClLayerDev &L, int po
     const int group = a.H / a.Hkv, kvd = a.Hkv * HD;   // grouped-query attention: `group` query heads share a key/value head
     float *wrec = sm->partial;   // [NCW][WSTRIDE]
     for (int item = blockIdx.x; item < a.H * S; item += gridDim.x) {
-        const int h = item % a.H, s = item / a.H, kvh = h / group;
-        int kw0, kw1;
-        warp_key_range(pos, s, S, warp, kw0, kw1);
+        const AttnItem cur = (item == (int)blockIdx.x) ? first : attn_item(a, item, pos, warp);
+        const int h = cur.h, s = cur.s, kvh = h / group, kw0 = cur.kw0, kw1 = cur.kw1;
         const float *qraw = a.qkv + h * HD;
         // rotated query, this lane's EPL elements
         float qr[EPL];
@@ -918,6 +930,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
     int tok = st->cyc_tok[a.row0];
     for (int step = 0; step < a.n_steps; ++step) {
         const int pos = ctx0 + a.row0 + step;
+        const AttnItem att_first = attn_item(a, blockIdx.x, pos, tid >> 5);
         // phase 0: embedding row -> residual stream (each CTA writes its slice)
         {
             const WT *erow = (const WT *)a.embed + (size_t)tok * d;
@@ -936,7 +949,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
                 for (int r = tid; r < nrb; r += NCT) a.qkv[rb0 + r] = row_sum(sm, r);
             }, a.cum_w, busy_p);
             grid_barrier(a.bar, bar_target, sm, st);
-            attention_phase<WT, HD>(a, L, pos, sm);
+            attention_phase<WT, HD>(a, L, pos, sm, att_first);
             grid_barrier(a.bar, bar_target, sm, st);
             // attention output projection + residual
             load_att_merged<EPC, HD>(a, xr);
