@@ -314,6 +314,30 @@ def test_wide_prompt_pass_matches_chunked_prompt_pass(monkeypatch, wd):
     assert np.array_equal(out[0][2][clear], out[1][2][clear])
 
 
+@pytest.mark.parametrize("n", [17, 513, 529])
+def test_wide_prompt_pass_boundaries(monkeypatch, n):
+    """Prompt lengths at the edges of the wide pass: the shortest prompt that takes it (16 rows + the last token), one
+    full pass of 512 rows + the last token, and a second pass of 16 rows."""
+    base = synth.WORKLOADS["C2"].shape
+    sh = dataclasses.replace(base, n_layers=2, max_seq=544)
+    W = synth.make_weights(sh, 8, device="cuda")
+    prompt = synth.make_prompt(8, n, sh.vocab)
+    out = {}
+    for wide in (0, 1):
+        monkeypatch.setenv("CL_DISABLE_WIDE_PREFILL", "0" if wide else "1")
+        ctx = cl.Context.from_shape(sh, tap_positions=8)
+        ctx.cl_load(W)
+        first = ctx.cl_prefill(prompt, tap_hidden=True)
+        ring = ctx.cl_read_hidden_ring().float().numpy()
+        d = ctx.cl_draft(3, want_logits=True)
+        out[wide] = (first, ring, d["logits"].copy())
+        ctx.close()
+    scale = max(1.0, float(np.abs(out[0][1]).max()))
+    assert np.abs(out[0][1] - out[1][1]).max() <= 2 ** -7 * scale
+    assert np.abs(out[0][2][0] - out[1][2][0]).max() <= 5e-3              # first draft step: same cache, same logits to half the tolerance
+    assert out[0][0] == out[1][0] or np.sort(out[0][2][0])[-1] - np.sort(out[0][2][0])[-2] < NEAR_TIE
+
+
 def test_interval_search_matches_oracle_on_c1():
     """Section 3.3 driver: same rounds, scores, sets and tokens as the oracle's loop on the fp32 model."""
     w = synth.WORKLOADS["C1"]
