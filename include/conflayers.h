@@ -158,7 +158,8 @@ int cl_step_vanilla(cl_ctx *ctx, int32_t *tok);
 int cl_generate(cl_ctx *ctx, int K, int max_new, int32_t *out, int *n_out, cl_stats *stats);
 
 /* Set the committed cache length and the pending token (rollback after a rejected run, or
- * re-synchronisation of a parity harness).  0 <= ctx_len <= current filled length. */
+ * re-synchronisation of a parity harness).  0 <= ctx_len <= the number of positions full-model passes (prefill,
+ * verify, vanilla steps) have written so far; CL_ERANGE beyond that. */
 int cl_rollback(cl_ctx *ctx, int ctx_len, int32_t pending_token);
 
 /* Overwrite this cycle's drafted tokens (host int32[n], n <= CL_MAX_K) before cl_verify. */
@@ -228,6 +229,8 @@ int cl_read_hidden_ring(cl_ctx *ctx, void *out);
  *   lm_head    DEVICE [vocab, d_model] row-major, weight_dtype 0 = fp32 / 1 = bf16
  *   final_norm DEVICE float[d_model]
  *   hidden     DEVICE [n_rows, d_model] in the same storage type as lm_head
+ *   (all three 16-byte aligned: the kernels read them with vector loads; CL_EINVAL otherwise.  fp16 is not
+ *   supported by this call: weight_dtype 2 is rejected with CL_EINVAL.)
  *   conf, p_max, argmax   HOST [n_rows], caller-owned, each may be NULL
  * The call enqueues on cuda_stream (a cudaStream_t or NULL) and synchronises it before returning.
  * The first call on each device looks up the array's device address; make that first call outside any
@@ -241,6 +244,20 @@ int cl_read_hidden_ring(cl_ctx *ctx, void *out);
 int cl_layer_confidences_static(const void *lm_head, const float *final_norm, int vocab, int d_model, int weight_dtype,
                                 float rms_eps, const void *hidden, int n_rows, void *cuda_stream, float *conf,
                                 float *p_max, int32_t *argmax);
+
+/* ---- diagnostics ------------------------------------------------------------------------------ */
+
+/* Every device-side wait in the kernels (a shared-memory barrier, a grid barrier of a persistent kernel) is bounded:
+ * when the bound runs out the kernel raises a flag, lets its remaining waits fall through, drains its copies in
+ * flight and returns; the host call that finds the flag returns CL_ETIMEOUT, clears it, commits nothing of the
+ * call, and the context stays usable (re-run cl_prefill).  The paper has no counterpart; these settings exist so
+ * that this path can be exercised without faulting or hanging anything:
+ *   CL_DEBUG_WAIT_LIMIT_US   bound of a single wait of the persistent step kernel in microseconds (default 2 000 000)
+ *   CL_DEBUG_BARRIER_EXTRA   extra arrivals its grid barriers wait for (default 0); with 1 no barrier can complete,
+ *                            so the first one runs into the bound
+ *   CL_DEBUG_DEVICE_ERR      sets the device-side error flags to `value`, as an expired wait would */
+enum { CL_DEBUG_WAIT_LIMIT_US = 1, CL_DEBUG_BARRIER_EXTRA = 2, CL_DEBUG_DEVICE_ERR = 3 };
+int cl_debug_set(cl_ctx *ctx, int what, long long value);
 
 /* ---- bookkeeping ----------------------------------------------------------------------------- */
 

@@ -39,12 +39,25 @@ def accept_greedy(drafts: Sequence[int], targets: Sequence[int]):
     return n, [int(t) for t in drafts[:n]] + [int(targets[n])]
 
 
+def top1_probability(logits_row: np.ndarray) -> float:
+    """max of softmax(logits) in double (the draft's own confidence in its greedy token)."""
+    l = logits_row.astype(np.float64)
+    e = np.exp(l - l.max())
+    return float(e.max() / e.sum())
+
+
 def speculative_cycle(model, skip_mask: Optional[np.ndarray], t0: int, ctx: int, K: int,
-                      want_hidden: bool = False) -> Dict[str, object]:
-    """One cycle from the state (cache valid for positions < ctx, pending token t0)."""
+                      want_hidden: bool = False, stop_p: float = 0.0) -> Dict[str, object]:
+    """One cycle from the state (cache valid for positions < ctx, pending token t0).
+
+    stop_p > 0 is the confidence-aware drafting the paper takes over from SWIFT (Section 3): drafting ends after
+    the first candidate whose top-1 probability under the draft model is below stop_p.  That candidate is still
+    handed to the target model (reading: the paper gives neither the threshold nor which side of it the last
+    candidate falls on); stop_p = 0 always drafts K candidates."""
     drafts: List[int] = []
     d_margin: List[float] = []
     d_logits: List[np.ndarray] = []
+    d_pmax: List[float] = []
     tok = int(t0)
     for i in range(K):
         lg = model.forward([tok], ctx + i, skip_mask)["logits"][0]
@@ -52,15 +65,19 @@ def speculative_cycle(model, skip_mask: Optional[np.ndarray], t0: int, ctx: int,
         drafts.append(tok)
         d_margin.append(top2_margin(lg))
         d_logits.append(lg)
+        d_pmax.append(top1_probability(lg))
+        if stop_p > 0.0 and d_pmax[-1] < stop_p:
+            break
+    nd = len(drafts)
     rows = [int(t0)] + drafts
     ver = model.forward(rows, ctx, None, want_hidden=want_hidden)
     vlog = ver["logits"]
-    targets = [greedy_token(vlog[i]) for i in range(K + 1)]
-    v_margin = [top2_margin(vlog[i]) for i in range(K + 1)]
+    targets = [greedy_token(vlog[i]) for i in range(nd + 1)]
+    v_margin = [top2_margin(vlog[i]) for i in range(nd + 1)]
     n, emitted = accept_greedy(drafts, targets)
     return dict(drafts=drafts, targets=targets, n_accepted=n, emitted=emitted, draft_margins=d_margin,
-                verify_margins=v_margin, draft_logits=d_logits, verify_logits=vlog,
-                hid_attn=ver["hid_attn"], hid_ffn=ver["hid_ffn"], new_ctx=ctx + n + 1, next_t0=emitted[-1])
+                verify_margins=v_margin, draft_logits=d_logits, verify_logits=vlog, draft_pmax=d_pmax, n_drafted=nd,
+                hid_attn=ver.get("hid_attn"), hid_ffn=ver.get("hid_ffn"), new_ctx=ctx + n + 1, next_t0=emitted[-1])
 
 
 def prefill(model, prompt: Sequence[int], want_hidden: bool = False):
@@ -84,7 +101,7 @@ def generate_vanilla(model, prompt: Sequence[int], max_new: int) -> Dict[str, ob
 
 
 def generate_speculative(model, prompt: Sequence[int], skip_mask: Optional[np.ndarray], K: int,
-                         max_new: int) -> Dict[str, object]:
+                         max_new: int, stop_p: float = 0.0) -> Dict[str, object]:
     """Self-speculative greedy decoding: prefill, then cycles until max_new tokens are emitted
     (the last cycle's emission is truncated).  Statistics as defined in Section 4.1.2:
     alpha = accepted / drafted, M = mean accepted per cycle, beta = |S| / L."""
@@ -93,13 +110,13 @@ def generate_speculative(model, prompt: Sequence[int], skip_mask: Optional[np.nd
     ctx = len(prompt)
     cycles: List[Dict[str, object]] = []
     while len(out) < max_new:
-        cyc = speculative_cycle(model, skip_mask, out[-1], ctx, K)
+        cyc = speculative_cycle(model, skip_mask, out[-1], ctx, K, stop_p=stop_p)
         cyc["ctx"] = ctx
         cyc["t0"] = out[-1]
         cycles.append(cyc)
         out.extend(cyc["emitted"])
         ctx = cyc["new_ctx"]
-    drafted = K * len(cycles)
+    drafted = sum(c["n_drafted"] for c in cycles)
     accepted = sum(c["n_accepted"] for c in cycles)
     L = model.L
     n_skipped = 0 if skip_mask is None else int(np.count_nonzero(np.asarray(skip_mask)))

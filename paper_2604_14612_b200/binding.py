@@ -46,6 +46,7 @@ class SelectCfg(C.Structure):
 
 
 CL_MAX_ROUNDS = 32
+CL_DEBUG_WAIT_LIMIT_US, CL_DEBUG_BARRIER_EXTRA, CL_DEBUG_DEVICE_ERR = 1, 2, 3
 
 
 class SearchCfg(C.Structure):
@@ -107,6 +108,7 @@ def load_library():
         "cl_score_loop": [vp, C.POINTER(SelectCfg), C.POINTER(vp), C.c_int, C.c_int, vp, vp, C.POINTER(C.c_int), vp, vp],
         "cl_read_hidden_ring": [vp, vp],
         "cl_get_stats": [vp, C.POINTER(Stats)],
+        "cl_debug_set": [vp, C.c_int, C.c_longlong],
         "cl_layer_confidences_static": [vp, vp, C.c_int, C.c_int, C.c_int, C.c_float, vp, C.c_int, vp, vp, vp, vp],
     }
     for name, args in sig.items():
@@ -130,10 +132,20 @@ def cl_layer_confidences_static(lm_head, final_norm, hidden, rms_eps: float = 1e
     returns dict(conf, p_max, argmax) as numpy arrays with hidden's leading shape."""
     L = load_library()
     import torch
-    assert lm_head.is_cuda and hidden.is_cuda and final_norm.is_cuda
-    assert lm_head.is_contiguous() and hidden.is_contiguous() and final_norm.is_contiguous()
-    assert lm_head.dtype == hidden.dtype and final_norm.dtype == torch.float32
+    if not (lm_head.is_cuda and hidden.is_cuda and final_norm.is_cuda):
+        raise ValueError("lm_head, hidden and final_norm must be CUDA tensors")
+    if not (lm_head.is_contiguous() and hidden.is_contiguous() and final_norm.is_contiguous()):
+        raise ValueError("lm_head, hidden and final_norm must be contiguous")
+    dtypes = {torch.float32: 0, torch.bfloat16: 1}          # the storage types the call supports
+    if lm_head.dtype not in dtypes:
+        raise ValueError(f"lm_head dtype {lm_head.dtype} not supported: float32 or bfloat16 only")
+    if hidden.dtype != lm_head.dtype or final_norm.dtype != torch.float32:
+        raise ValueError("hidden must have lm_head's dtype and final_norm must be float32")
+    if lm_head.dim() != 2 or hidden.dim() < 1:
+        raise ValueError("lm_head must be [vocab, d_model] and hidden [..., d_model]")
     V, d = lm_head.shape
+    if hidden.shape[-1] != d or tuple(final_norm.shape) != (d,):
+        raise ValueError(f"hidden's last dimension and final_norm must have d_model = {d} elements")
     lead = tuple(hidden.shape[:-1])
     n = int(np.prod(lead))
     conf = np.zeros(n, np.float32)
@@ -142,7 +154,7 @@ def cl_layer_confidences_static(lm_head, final_norm, hidden, rms_eps: float = 1e
     if stream is None:
         stream = torch.cuda.current_stream().cuda_stream
     rc = L.cl_layer_confidences_static(lm_head.data_ptr(), final_norm.data_ptr(), V, d,
-                                       1 if lm_head.dtype == torch.bfloat16 else 0, rms_eps, hidden.data_ptr(), n,
+                                       dtypes[lm_head.dtype], rms_eps, hidden.data_ptr(), n,
                                        C.c_void_p(stream), _np_ptr(conf), _np_ptr(pm), _np_ptr(am))
     if rc:
         raise ConfLayersError(rc, L.cl_last_error(None).decode())
@@ -336,6 +348,9 @@ class Context:
         out = torch.empty((L, self.taps, P, d), dtype=dt)
         self._ck(self._L.cl_read_hidden_ring(self._h, out.data_ptr()))
         return out if self.taps == 2 else out[:, 0]
+
+    def cl_debug_set(self, what: int, value: int):
+        self._ck(self._L.cl_debug_set(self._h, what, value))
 
     def cl_get_stats(self) -> Stats:
         st = Stats()

@@ -83,7 +83,11 @@ struct cl_ctx {
     int nsplit, per_max;
     // host view of the device state (exact after every call that synchronises)
     int h_ctx, h_ndraft, tapped;
+    int h_filled;                 // positions [0, h_filled) of every layer's cache have been written by full-model passes
     uint64_t launches;
+    // diagnostics (cl_debug_set)
+    unsigned long long wait_ns;   // bound on any single device-side wait of the step kernel
+    int bar_extra;                // extra arrivals the step kernel's grid barriers wait for (0: barriers complete)
 };
 
 static char g_err[512] = "";
@@ -195,6 +199,7 @@ extern "C" int cl_create(const cl_model_cfg *cfg, void *cuda_stream, cl_ctx **ou
     c->esz = cfg->weight_dtype == 0 ? 4 : 2;
     c->taps = cfg->tap_modules == 2 ? 2 : 1;
     c->err[0] = 0;
+    c->wait_ns = 2000000000ull;
     c->mask.assign((size_t)cfg->n_layers, 0);
     *out = c;
     return CL_OK;
@@ -653,7 +658,8 @@ static int forward_wide(cl_ctx *c, const int *tok, int M, int tap) {
 
 // n_steps consecutive single-token steps in one persistent launch (draft steps with the skip set, or
 // vanilla full-model steps that emit and advance on the device).
-static int run_steps(cl_ctx *c, int mode, int n_steps, int row0, bool full_model, float *logits, int *out_tokens) {
+static int run_steps(cl_ctx *c, int mode, int n_steps, int row0, bool full_model, float *logits, int *out_tokens,
+                     float stop_p = 0.f) {
     const cl_model_cfg &g = c->cfg;
     ClStepArgs a;
     memset(&a, 0, sizeof(a));
@@ -668,6 +674,7 @@ static int run_steps(cl_ctx *c, int mode, int n_steps, int row0, bool full_model
     a.x = c->x; a.qkv = c->qkv; a.hff = c->hff;
     a.att_part = c->att_part2; a.head_part = c->head_part2; a.bar = c->bar_dev;
     a.n_steps = n_steps; a.mode = mode; a.row0 = row0; a.out_tokens = out_tokens; a.logits = logits;
+    a.wait_ns = c->wait_ns; a.bar_arrivals = (unsigned)(c->n_sm + c->bar_extra); a.stop_p = stop_p;
     a.cum_w = c->cum_w_ready ? c->cum_w_dev : nullptr;
     a.busy_ns = c->calibrating ? c->busy_dev : nullptr;
     CU(cudaMemsetAsync(c->bar_dev, 0, 2 * sizeof(unsigned), c->stream));   // the arrival counter starts at zero
@@ -775,8 +782,13 @@ extern "C" int cl_prefill(cl_ctx *c, const int32_t *tokens, int n, int tap_hidde
         KL(cl_launch_advance(c->st, T, last ? 1 : 0, c->stream));
     }
     if ((rc = sync_state(c))) return rc;
+    if ((rc = check_device_err(c, "cl_prefill"))) {
+        c->prefilled = 0;   // the cache holds rows of an aborted pass
+        return rc;
+    }
     c->prefilled = 1;
     c->h_ndraft = 0;
+    c->h_filled = n;
     c->tapped = tap_hidden ? n : 0;
     if (first_token) *first_token = c->h_st->cyc_tok[0];
     return CL_OK;
@@ -811,18 +823,18 @@ extern "C" int cl_draft(cl_ctx *c, int K, float stop_p, int32_t *toks, float *p_
     if (K < 1 || K > CL_MAX_K) return fail(c, CL_ERANGE, "cl_draft: K = %d outside 1..%d", K, CL_MAX_K);
     if (c->h_ctx + K + 1 > c->cfg.max_seq) return fail(c, CL_ERANGE, "cl_draft: position %d exceeds max_seq", c->h_ctx + K);
     int n = 0;
-    if (c->use_step && stop_p <= 0.f) {
-        if ((rc = run_steps(c, CL_STEP_DRAFT, K, 0, false, logits ? c->logits : nullptr, nullptr))) return rc;
-        n = K;
+    if (c->use_step) {
+        // one persistent launch; with stop_p > 0 the kernel itself ends the drafting and records how far it got
+        if ((rc = run_steps(c, CL_STEP_DRAFT, K, 0, false, logits ? c->logits : nullptr, nullptr, stop_p > 0.f ? stop_p : 0.f)))
+            return rc;
+        if ((rc = sync_state(c))) return rc;
+        n = c->h_st->n_drafted;
     } else {
         for (int i = 0; i < K; ++i) {
             float *lg = logits ? c->logits + (size_t)i * c->cfg.vocab : nullptr;
-            if (c->use_step)
-                rc = run_steps(c, CL_STEP_DRAFT, 1, i, false, lg, nullptr);
-            else
-                rc = forward_rows(c, ST_FIELD(c, int, cyc_tok) + i, 1, i, c->mask.data(), 0, 1,
-                                  ST_FIELD(c, int, cyc_tok) + i + 1, ST_FIELD(c, float, d_pmax) + i,
-                                  ST_FIELD(c, float, d_conf) + i, lg);
+            rc = forward_rows(c, ST_FIELD(c, int, cyc_tok) + i, 1, i, c->mask.data(), 0, 1,
+                              ST_FIELD(c, int, cyc_tok) + i + 1, ST_FIELD(c, float, d_pmax) + i,
+                              ST_FIELD(c, float, d_conf) + i, lg);
             if (rc) return rc;
             n = i + 1;
             if (stop_p > 0.f) {   // confidence-aware early stop needs the probability on the host
@@ -830,12 +842,13 @@ extern "C" int cl_draft(cl_ctx *c, int K, float stop_p, int32_t *toks, float *p_
                 if (c->h_st->d_pmax[i] < stop_p) break;
             }
         }
+        ClPoke p = poke_none();
+        p.n_drafted = n;
+        if ((rc = poke(c, p))) return rc;
+        if ((rc = sync_state(c))) return rc;
     }
-    ClPoke p = poke_none();
-    p.n_drafted = n;
-    if ((rc = poke(c, p))) return rc;
-    if ((rc = sync_state(c))) return rc;
     if ((rc = check_device_err(c, "cl_draft"))) return rc;
+    if (n < 1 || n > K) return fail(c, CL_ECUDA, "cl_draft: the device reported %d drafted tokens", n);
     c->h_ndraft = n;
     if (logits) CU(cudaMemcpy(logits, c->logits, (size_t)n * c->cfg.vocab * 4, cudaMemcpyDeviceToHost));
     for (int i = 0; i < n; ++i) {
@@ -873,6 +886,8 @@ extern "C" int cl_verify(cl_ctx *c, int tap_hidden, int32_t *target_toks, float 
                       ST_FIELD(c, float, v_pmax), ST_FIELD(c, float, v_conf), logits ? c->logits : nullptr);
     if (rc) return rc;
     if ((rc = sync_state(c))) return rc;
+    if ((rc = check_device_err(c, "cl_verify"))) return rc;   // target tokens of an aborted pass are never handed out
+    if (c->h_ctx + T > c->h_filled) c->h_filled = c->h_ctx + T;
     if (tap_hidden) c->tapped += 1;
     if (logits) CU(cudaMemcpy(logits, c->logits, (size_t)T * c->cfg.vocab * 4, cudaMemcpyDeviceToHost));
     if (target_toks)
@@ -883,6 +898,9 @@ extern "C" int cl_verify(cl_ctx *c, int tap_hidden, int32_t *target_toks, float 
 extern "C" int cl_accept(cl_ctx *c, int *n_accepted, int32_t *emitted) {
     int rc = need_model(c, "cl_accept", true);
     if (rc) return rc;
+    // an error flag left by an earlier pass means its target tokens are invalid: nothing is committed
+    if ((rc = sync_state(c))) return rc;
+    if ((rc = check_device_err(c, "cl_accept"))) return rc;
     KL(cl_launch_accept(c->st, -1, nullptr, c->stream));
     if ((rc = sync_state(c))) return rc;
     c->h_ndraft = 0;
@@ -910,6 +928,7 @@ extern "C" int cl_step_vanilla(cl_ctx *c, int32_t *tok) {
     }
     if ((rc = sync_state(c))) return rc;
     if ((rc = check_device_err(c, "cl_step_vanilla"))) return rc;
+    if (c->h_ctx > c->h_filled) c->h_filled = c->h_ctx;
     c->h_ndraft = 0;
     if (tok) *tok = c->h_st->emitted[0];
     return CL_OK;
@@ -972,6 +991,7 @@ extern "C" int cl_generate(cl_ctx *c, int K, int max_new, int32_t *out, int *n_o
     p.done = 0;
     if ((rc = poke(c, p))) return rc;
     if ((rc = sync_state(c))) return rc;
+    if (c->h_ctx > c->h_filled) c->h_filled = c->h_ctx;
     c->h_ndraft = 0;
     if (n_out) *n_out = max_new;
     if (stats) cl_get_stats(c, stats);
@@ -996,6 +1016,8 @@ extern "C" int cl_generate_search(cl_ctx *c, const cl_search_cfg *sc, const cl_s
     if (sc->interval < 1 || sc->max_rounds < 0 || sc->max_rounds > CL_MAX_ROUNDS)
         return fail(c, CL_ERANGE, "cl_generate_search: interval >= 1 and 0 <= max_rounds <= %d required", CL_MAX_ROUNDS);
     if (!c->ring) return fail(c, CL_ESTATE, "cl_generate_search: the context has no hidden-state ring (tap_positions = 0)");
+    if (c->tapped <= 0)
+        return fail(c, CL_ESTATE, "cl_generate_search: the ring holds no rows of this input; call cl_prefill with tap_hidden = 1");
     if (c->h_ctx + max_new + K > c->cfg.max_seq)
         return fail(c, CL_ERANGE, "cl_generate_search: %d + %d + %d tokens exceed max_seq %d", c->h_ctx, max_new, K, c->cfg.max_seq);
     if ((rc = check_select(c, sel))) return rc;
@@ -1024,8 +1046,10 @@ extern "C" int cl_generate_search(cl_ctx *c, const cl_search_cfg *sc, const cl_s
         const int ncyc = r.searching ? sc->interval : (remaining + K) / (K + 1);
         for (int i = 0; i < ncyc; ++i)
             if ((rc = enqueue_cycle(c, K, r.searching))) return rc;
+        const int ctx_before = c->h_ctx;
         if ((rc = sync_state(c))) return rc;
         if ((rc = check_device_err(c, "cl_generate_search"))) return rc;
+        if (r.searching) c->tapped += c->h_ctx - ctx_before;   // every verify pass of the interval recorded its rows
         if (!r.searching || (int)(c->h_st->cycles - cyc0) < sc->interval) continue;   // no full interval: nothing to check
         // ---- search check (Section 3.3)
         const float score = (float)((double)(c->h_st->accepted - acc0) / (double)sc->interval);
@@ -1041,6 +1065,9 @@ extern "C" int cl_generate_search(cl_ctx *c, const cl_search_cfg *sc, const cl_s
             r.searching = 0;
             cur = best;
         } else {
+            if (c->tapped < P)   // slots never written would enter the per-layer mean as zero vectors
+                return fail(c, CL_ESTATE, "cl_generate_search: the ring holds %d of %d positions at a search check; use a longer prompt or interval",
+                            c->tapped, P);
             if ((rc = score_rows(c, c->ring, L, c->taps * P, c->sc_clayer))) return rc;
             KL(cl_launch_select(*sel, L, c->sc_clayer, c->sel_mask, nullptr, c->stream));
             CU(cudaMemcpyAsync(cur.data(), c->sel_mask, (size_t)L, cudaMemcpyDeviceToHost, c->stream));
@@ -1055,6 +1082,7 @@ extern "C" int cl_generate_search(cl_ctx *c, const cl_search_cfg *sc, const cl_s
     p.done = 0;
     if ((rc = poke(c, p))) return rc;
     if ((rc = sync_state(c))) return rc;
+    if (c->h_ctx > c->h_filled) c->h_filled = c->h_ctx;
     c->h_ndraft = 0;
     if (n_out) *n_out = max_new;
     if (rep) *rep = r;
@@ -1065,6 +1093,8 @@ extern "C" int cl_rollback(cl_ctx *c, int ctx_len, int32_t pending_token) {
     int rc = need_model(c, "cl_rollback", true);
     if (rc) return rc;
     if (ctx_len < 0 || ctx_len > c->cfg.max_seq - 1) return fail(c, CL_ERANGE, "cl_rollback: ctx_len %d out of range", ctx_len);
+    if (ctx_len > c->h_filled)   // rolling forward would make later passes attend over cache rows that were never written
+        return fail(c, CL_ERANGE, "cl_rollback: ctx_len %d beyond the %d positions the cache holds", ctx_len, c->h_filled);
     if (pending_token < 0 || pending_token >= c->cfg.vocab) return fail(c, CL_EINVAL, "cl_rollback: token out of range");
     ClPoke p = poke_none();
     p.ctx = ctx_len; p.pending = pending_token; p.n_drafted = 0; p.done = 0;
@@ -1242,6 +1272,29 @@ extern "C" int cl_read_hidden_ring(cl_ctx *c, void *out) {
     CU(cudaStreamSynchronize(c->stream));
     CU(cudaMemcpy(out, c->ring, (size_t)c->cfg.n_layers * c->taps * c->cfg.tap_positions * c->cfg.d_model * c->esz, cudaMemcpyDeviceToHost));
     return CL_OK;
+}
+
+extern "C" int cl_debug_set(cl_ctx *c, int what, long long value) {
+    if (!c) return fail(c, CL_EINVAL, "cl_debug_set: null context");
+    switch (what) {
+        case CL_DEBUG_WAIT_LIMIT_US:
+            if (value < 1) return fail(c, CL_EINVAL, "cl_debug_set: wait limit must be at least 1 us");
+            c->wait_ns = (unsigned long long)value * 1000ull;
+            return CL_OK;
+        case CL_DEBUG_BARRIER_EXTRA:
+            if (value < 0 || value > 1024) return fail(c, CL_EINVAL, "cl_debug_set: extra arrivals outside 0..1024");
+            c->bar_extra = (int)value;
+            return CL_OK;
+        case CL_DEBUG_DEVICE_ERR: {
+            if (!c->loaded) return fail(c, CL_ESTATE, "cl_debug_set: no weights loaded");
+            const int flags = (int)value;
+            CU(cudaMemcpyAsync(&c->st->err, &flags, sizeof(int), cudaMemcpyHostToDevice, c->stream));
+            CU(cudaStreamSynchronize(c->stream));
+            return CL_OK;
+        }
+        default:
+            return fail(c, CL_EINVAL, "cl_debug_set: unknown setting %d", what);
+    }
 }
 
 extern "C" int cl_get_stats(cl_ctx *c, cl_stats *out) {

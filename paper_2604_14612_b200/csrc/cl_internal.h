@@ -126,6 +126,9 @@ struct ClStepArgs {
     const float *cum_w;                  // [grid + 1] cumulative row shares of the CTAs (null: equal shares)
     unsigned long long *busy_ns;         // [grid], calibration launches only: time each CTA spent in the matrix phases
     int n_steps, mode, row0;
+    unsigned long long wait_ns;          // bound on any single device-side wait
+    unsigned bar_arrivals;               // arrivals that complete a grid barrier (= grid size)
+    float stop_p;                        // draft mode: stop after the first step whose top-1 probability is below it (0: never)
     int *out_tokens;                     // vanilla mode: emitted tokens (may be null)
     float *logits;                       // optional [n_steps, V]
 };

@@ -240,7 +240,7 @@ cudaError_t cl_launch_gemv(int wdtype, int T, int epi, const ClGemvArgs &a, int 
 // ---- confidence scoring without any allocation ------------------------------------------------------
 // Scratch of cl_layer_confidences_static(): one file-scope array that every GPU loading this library holds until
 // the process exits.  Layout (bytes): [0, 256) the LM-head kernel's ticket counter; then the normalised rows
-// xn [CL_MAX_T, CL_STATIC_MAX_D] fp32; the per-block softmax partials [SC_MAX_GRID, CL_MAX_T]; and the three
+// xn [SC_CHUNK, CL_STATIC_MAX_D] fp32; the per-block softmax partials [SC_MAX_GRID, SC_CHUNK]; and the three
 // per-row results (confidence, top-1 probability, greedy token) [CL_STATIC_MAX_ROWS] each.
 namespace {
 
@@ -311,6 +311,11 @@ extern "C" int cl_layer_confidences_static(const void *lm_head, const float *fin
     }
     if (vocab < 2 || d_model <= 0 || d_model % 8 || n_rows <= 0) {
         cl_set_global_error("cl_layer_confidences_static: need vocab >= 2, d_model a positive multiple of 8, n_rows > 0");
+        return CL_EINVAL;
+    }
+    if (((uintptr_t)lm_head | (uintptr_t)final_norm | (uintptr_t)hidden) & 15u) {
+        // the kernels read these with 16-byte vector loads; a misaligned pointer would trap on the device
+        cl_set_global_error("cl_layer_confidences_static: lm_head, final_norm and hidden must be 16-byte aligned");
         return CL_EINVAL;
     }
     if (d_model > CL_STATIC_MAX_D || n_rows > CL_STATIC_MAX_ROWS) {

@@ -25,7 +25,7 @@ constexpr int SLOT_BYTES = 32768;      // ring slot: as many whole weight rows a
 constexpr int NSLOT = 6;               // 192 KB in flight per SM
 constexpr int MAXIT = 4;               // 16-byte chunks per thread per row: rows up to 32 KB (C <= 16384 bf16)
 constexpr int RB = 256;                // rows per epilogue block
-constexpr unsigned long long WAIT_NS = 2000000000ull;   // 2 s bound on any single wait
+// (every single wait is bounded by ClStepArgs::wait_ns, 2 s unless a diagnostic lowered it)
 
 struct Smem {
     unsigned long long full[NSLOT];
@@ -34,7 +34,8 @@ struct Smem {
     float red[NCW];
     ClHeadPartial hp[NCT];
     int abort;
-    int next_tok;
+    int halt;                     // set by the consumers when drafting stops early: the producer issues no more copies
+    unsigned long long wait_ns;   // bound on any single wait (copied from the launch arguments)
 };
 
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -72,7 +73,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
         if (mbar_try(bar, parity)) return true;
         if ((i & 63u) == 0u) {
             if (*(volatile int *)&sm->abort) return false;
-            if (gtime() - t0 > WAIT_NS) {
+            if (gtime() - t0 > sm->wait_ns) {
                 *(volatile int *)&sm->abort = 1;
                 atomicOr(&st->err, 1);
                 return false;
@@ -111,10 +112,12 @@ __device__ __forceinline__ float4 ldcg_f4(const float *p) { return __ldcg((const
 // it before every launch): barrier number i is passed once the counter reaches i * gridDim.x.  One release
 // increment and an acquire poll per CTA; `target` lives in thread 0's registers.  Called by every consumer
 // thread of every CTA; bounded in time.
-__device__ __forceinline__ void grid_barrier(unsigned *bar, unsigned &target, Smem *sm, ClDevState *st) {
+// `bar_arrivals` = arrivals that complete one barrier: the grid size (a diagnostic may ask for more, so that the
+// wait provably runs out).
+__device__ __forceinline__ void grid_barrier(unsigned *bar, unsigned &target, unsigned bar_arrivals, Smem *sm, ClDevState *st) {
     consumer_sync();
     if (threadIdx.x == 0 && !*(volatile int *)&sm->abort) {
-        target += gridDim.x;
+        target += bar_arrivals;
         asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
         unsigned v;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
@@ -124,7 +127,7 @@ __device__ __forceinline__ void grid_barrier(unsigned *bar, unsigned &target, Sm
             do {
                 asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
                 if ((++i & 255u) == 0u) {
-                    if (*(volatile int *)&st->err || gtime() - t0 > WAIT_NS) {
+                    if (*(volatile int *)&st->err || gtime() - t0 > sm->wait_ns) {
                         *(volatile int *)&sm->abort = 1;
                         atomicOr(&st->err, 2);
                         break;
@@ -394,7 +397,21 @@ __device__ void producer_loop(const ClStepArgs &a, unsigned char *ring, Smem *sm
                 }
             }
         }
-        mbar_wait(&sm->empty[rg.slot], rg.par ^ 1u, sm, st);
+        if (!mbar_try(&sm->empty[rg.slot], rg.par ^ 1u)) {
+            // (a slot stays taken for good once the consumers have stopped early: look at their flag while waiting)
+            const unsigned long long t0 = gtime();
+            for (unsigned i = 1; !mbar_try(&sm->empty[rg.slot], rg.par ^ 1u); ++i) {
+                if ((i & 31u) == 0u) {
+                    if (*(volatile int *)&sm->halt || *(volatile int *)&sm->abort) break;
+                    if (gtime() - t0 > sm->wait_ns) {
+                        *(volatile int *)&sm->abort = 1;
+                        atomicOr(&st->err, 1);
+                        break;
+                    }
+                }
+            }
+        }
+        if (*(volatile int *)&sm->halt) break;
         if (!*(volatile int *)&sm->abort) {
             mbar_expect_tx(&sm->full[rg.slot], bytes);
             bulk_g2s_stream(ring + (size_t)rg.slot * SLOT_BYTES, src, bytes, &sm->full[rg.slot], policy);
@@ -409,7 +426,7 @@ __device__ void producer_loop(const ClStepArgs &a, unsigned char *ring, Smem *sm
         if (last_par[i] < 2u) {
             const unsigned long long t0 = gtime();
             while (!mbar_try(&sm->full[i], last_par[i]))
-                if (gtime() - t0 > WAIT_NS) break;
+                if (gtime() - t0 > sm->wait_ns) break;
         }
     }
 }
@@ -908,6 +925,8 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             mbar_init(&sm->empty[i], NCW);
         }
         sm->abort = 0;
+        sm->halt = 0;
+        sm->wait_ns = a.wait_ns;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -936,7 +955,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             const WT *erow = (const WT *)a.embed + (size_t)tok * d;
             for (int i = blockIdx.x * NCT + tid; i < d; i += gridDim.x * NCT) a.x[i] = st_to_f32<WT>(erow[i]);
         }
-        grid_barrier(a.bar, bar_target, sm, st);
+        grid_barrier(a.bar, bar_target, a.bar_arrivals, sm, st);
         for (int ki = 0; ki < a.n_kept; ++ki) {
             const int ent = a.kept[ki], fl = ent >> 16;   // bit 0: this layer's attention half is skipped, bit 1: its FFN half
             const ClLayerDev L = a.layers[ent & 0xffff];
@@ -948,15 +967,15 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             consume_matrix<WT>(d + 2 * a.Hkv * HD, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.qkv[rb0 + r] = row_sum(sm, r);
             }, a.cum_w, busy_p);
-            grid_barrier(a.bar, bar_target, sm, st);
+            grid_barrier(a.bar, bar_target, a.bar_arrivals, sm, st);
             attention_phase<WT, HD>(a, L, pos, sm, att_first);
-            grid_barrier(a.bar, bar_target, sm, st);
+            grid_barrier(a.bar, bar_target, a.bar_arrivals, sm, st);
             // attention output projection + residual
             load_att_merged<EPC, HD>(a, xr);
             consume_matrix<WT>(d, d, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
             }, a.cum_w, busy_p);
-            grid_barrier(a.bar, bar_target, sm, st);
+            grid_barrier(a.bar, bar_target, a.bar_arrivals, sm, st);
             }
             if (!(fl & 2)) {
             // gate/up projections (rows interleaved) + SiLU(gate) * up
@@ -967,13 +986,13 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
                     a.hff[rb0 / 2 + pr] = gt / (1.f + expf(-gt)) * up;
                 }
             }, a.cum_w, busy_p);
-            grid_barrier(a.bar, bar_target, sm, st);
+            grid_barrier(a.bar, bar_target, a.bar_arrivals, sm, st);
             // down projection + residual
             load_x<EPC>(a.hff, F, xr);
             consume_matrix<WT>(d, F, 1, xr, rg, ring, sm, st, [&](int rb0, int nrb) {
                 for (int r = tid; r < nrb; r += NCT) a.x[rb0 + r] = ldcg_f(a.x + rb0 + r) + row_sum(sm, r);
             }, a.cum_w, busy_p);
-            grid_barrier(a.bar, bar_target, sm, st);
+            grid_barrier(a.bar, bar_target, a.bar_arrivals, sm, st);
             }
         }
         // LM head on the normalised stream, fused with clamp + online softmax / entropy / argmax
@@ -989,7 +1008,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
         }, a.cum_w, busy_p);
         run = hp_block_reduce(run, sm);
         if (tid == 0) a.head_part[blockIdx.x] = run;
-        grid_barrier(a.bar, bar_target, sm, st);
+        grid_barrier(a.bar, bar_target, a.bar_arrivals, sm, st);
         // every CTA reduces the per-CTA partials itself (same order everywhere), so all know the token
         ClHeadPartial fin{0.f, 0.f, 0.f, 0x7fffffff};
         for (int b = tid; b < (int)gridDim.x; b += NCT) {
@@ -1000,14 +1019,17 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
         }
         fin = hp_block_reduce(fin, sm);
         tok = min(max(fin.idx, 0), V - 1);   // (only an aborted run can leave the range; keep the next gather in bounds)
+        const float pm = 1.f / fin.z;        // top-1 probability: the same bits in every CTA
+        // confidence-aware drafting: the candidate whose top-1 probability falls below the threshold is the last one
+        const bool stop = a.mode == CL_STEP_DRAFT && a.stop_p > 0.f && pm < a.stop_p;
         if (blockIdx.x == 0 && tid == 0) {
             const float Hh = logf(fin.z) - fin.s / fin.z;   // entropy of the softmax (Eq. 2), from sums relative to the max
             const float conf = 1.f - Hh * a.inv_log_v;      // Eq. 3-4
-            const float pm = 1.f / fin.z;
             if (a.mode == CL_STEP_DRAFT) {
                 st->cyc_tok[a.row0 + step + 1] = tok;
                 st->d_pmax[a.row0 + step] = pm;
                 st->d_conf[a.row0 + step] = conf;
+                if (stop || step == a.n_steps - 1) st->n_drafted = a.row0 + step + 1;
             } else {
                 // vanilla decoding: the token is emitted at once and becomes the next pending token
                 if (a.out_tokens && st->n_out < st->max_new) a.out_tokens[st->n_out] = tok;
@@ -1022,6 +1044,10 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
                 st->cycles += 1ull;
                 st->emitted_total += 1ull;
             }
+        }
+        if (stop) {   // uniform over the grid
+            if (tid == 0) *(volatile int *)&sm->halt = 1;
+            break;
         }
         // the next step's phase 0 writes x, which nobody reads any more in this step: no barrier needed here,
         // and head_part is rewritten only after the next step's grid barriers

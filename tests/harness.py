@@ -25,6 +25,7 @@ class Report:
     cycles: int = 0
     tokens_compared: int = 0
     near_ties: int = 0
+    near_threshold_stops: int = 0
     max_logit_err: float = 0.0
     max_conf_err: float = 0.0
     notes: List[str] = dataclasses.field(default_factory=list)
@@ -58,31 +59,44 @@ def check_logits(rep: Report, got: np.ndarray, want: np.ndarray, what: str, tol:
 
 
 def lockstep_generate(om, ctx, prompt, mask: Optional[np.ndarray], K: int, gen_len: int, tap: bool = False,
-                      check_conf: bool = True, tol: float = TOL, near_tie: float = NEAR_TIE) -> Report:
+                      check_conf: bool = True, tol: float = TOL, near_tie: float = NEAR_TIE, stop_p: float = 0.0) -> Report:
     """Prefill + speculative cycles along the oracle's trajectory.  tol / near_tie default to the stated 1e-2; the
-    full-depth 7B case passes the measured floor of the storage format instead (see its test)."""
+    full-depth cases pass the bound their depth allows instead (see their tests).  stop_p > 0: confidence-aware
+    drafting; the number of candidates per cycle must equal the oracle's, except where the oracle's deciding top-1
+    probability lies within a factor 1 +- 2 tol of the threshold (counted): logits that differ by at most tol move
+    max softmax = exp(l_max) / sum exp(l_i) by at most a factor exp(+-2 tol)."""
     rep = Report()
     V = om.V
-    ref = oracle.generate_speculative(om, prompt, mask, K, gen_len)
+    ref = oracle.generate_speculative(om, prompt, mask, K, gen_len, stop_p=stop_p)
     first = ctx.cl_prefill(prompt, tap_hidden=tap)
     check_token(rep, first, ref["tokens"][0], ref["first_margin"], "prefill", near_tie)
     ctx.cl_set_skip_set(mask if mask is not None else np.zeros(om.L, np.uint8))
     for ci, cyc in enumerate(ref["cycles"]):
         rep.cycles += 1
         ctx.cl_rollback(cyc["ctx"], cyc["t0"])
-        d = ctx.cl_draft(K, want_logits=True)
-        assert d["n_drafted"] == K
-        for i in range(K):
+        d = ctx.cl_draft(K, stop_p=stop_p, want_logits=True)
+        nd = cyc["n_drafted"]
+        if stop_p <= 0.0:
+            assert d["n_drafted"] == K == nd
+        diverged = False
+        for i in range(min(nd, d["n_drafted"])):
             check_logits(rep, d["logits"][i], cyc["draft_logits"][i], f"cycle {ci} draft {i}", tol)
             if check_conf:
                 conf, pm, _ = oracle.confidence_of_logits(cyc["draft_logits"][i])
                 rep.max_conf_err = max(rep.max_conf_err, abs(conf - float(d["conf"][i])), abs(pm - float(d["p_max"][i])))
             if not check_token(rep, d["tokens"][i], cyc["drafts"][i], cyc["draft_margins"][i], f"cycle {ci} draft {i}", near_tie):
+                diverged = True
                 break   # later drafts were conditioned on a different token
+        if stop_p > 0.0 and not diverged and d["n_drafted"] != nd:
+            # the step at which one side stopped and the other went on
+            pm_o = cyc["draft_pmax"][min(nd, d["n_drafted"]) - 1]
+            assert abs(pm_o - stop_p) <= 2 * tol * stop_p, \
+                f"cycle {ci}: {d['n_drafted']} drafts, oracle {nd}, deciding probability {pm_o:.6g} against {stop_p:.6g}"
+            rep.near_threshold_stops += 1
         ctx.cl_force_tokens(cyc["drafts"])
-        v = ctx.cl_verify(K + 1, tap_hidden=tap, want_logits=True)
+        v = ctx.cl_verify(nd + 1, tap_hidden=tap, want_logits=True)
         same = True
-        for i in range(K + 1):
+        for i in range(nd + 1):
             check_logits(rep, v["logits"][i], cyc["verify_logits"][i], f"cycle {ci} verify row {i}", tol)
             same &= check_token(rep, v["targets"][i], cyc["targets"][i], cyc["verify_margins"][i], f"cycle {ci} verify row {i}", near_tie)
         n, em = ctx.cl_accept()

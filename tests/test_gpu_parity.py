@@ -365,6 +365,44 @@ def test_interval_search_matches_oracle_on_c1():
         assert got["final_set"] == ref2["final_set"] and got["searching"] == ref2["searching"]
 
 
+@pytest.mark.parametrize("name", ["C1", "C2"])
+def test_early_stop_matches_oracle(name):
+    """Confidence-aware drafting (Section 3, after SWIFT): with the threshold at the median top-1 probability of the
+    fixed-K drafts, the device stops every cycle after the same candidate as the oracle (a probability within the
+    tolerance of the threshold may decide differently; such cycles are counted), and everything else of the cycle
+    still matches."""
+    w = synth.WORKLOADS[name]
+    gen = 32 if name == "C1" else 24
+    om, ctx, _ = make_pair(w.shape, w.seed)
+    prompt = synth.make_prompt(w.seed, w.prompt_len, w.shape.vocab)
+    layers = [1] if name == "C1" else [3, 6, 9]
+    mask = synth.layers_to_mask(layers, w.shape.n_layers)
+    K = 6
+    fixed = oracle.generate_speculative(om, prompt, mask, K, gen)
+    pms = sorted(p for c in fixed["cycles"] for p in c["draft_pmax"])
+    thr = float(pms[len(pms) // 2])
+    ref = oracle.generate_speculative(om, prompt, mask, K, gen, stop_p=thr)
+    counts = [c["n_drafted"] for c in ref["cycles"]]
+    assert min(counts) < K and len(set(counts)) > 1, "the threshold must cut some cycles short and not others"
+    rep = lockstep_generate(om, ctx, prompt, mask, K, gen, stop_p=thr)
+    print("early stop", name, "threshold", thr, "oracle drafts per cycle", counts, rep)
+    assert rep.near_threshold_stops <= max(1, len(counts) // 4)
+    # free-running on the device with the same threshold stays lossless
+    first = ctx.cl_prefill(prompt)
+    ctx.cl_set_skip_set(mask)
+    toks = [first]
+    while len(toks) < gen:
+        d = ctx.cl_draft(K, stop_p=thr)
+        assert 1 <= d["n_drafted"] <= K
+        ctx.cl_verify(d["n_drafted"] + 1)
+        n, em = ctx.cl_accept()
+        assert n <= d["n_drafted"]
+        toks.extend(int(t) for t in em)
+    van = oracle.generate_vanilla(om, prompt, gen)
+    lim = next((i for i, m in enumerate(van["margins"]) if m < NEAR_TIE), gen)
+    assert toks[:lim] == van["tokens"][:lim]
+
+
 @pytest.mark.parametrize("name,L,mask", [("C1", 4, [0, 1, 2, 0]), ("C1", 4, [0, 3, 1, 2]), ("C3", 4, [0, 2, 1, 0])])
 def test_half_layer_skip_sets(name, L, mask):
     """Attention-only and FFN-only skips (mask bits 0 and 1) in draft steps, lock-step against the oracle."""

@@ -80,6 +80,80 @@ def test_lossless_on_a_bf16_model():
     assert s["tokens"] == van["tokens"]
 
 
+# ---------------------------------------------------------------- confidence-aware drafting (early stop)
+
+class _ScriptedModel:
+    """Stands in for the transformer: the logits after a token are read from a table (one for the draft model, which
+    is called with a skip mask, one for the target model), so every top-1 probability is known in closed form."""
+    L = 4
+
+    def __init__(self, draft_table, target_table):
+        self.draft_table, self.target_table = draft_table, target_table
+
+    def forward(self, tokens, pos, mask=None, want_hidden=False, want_logits=True):
+        tab = self.target_table if mask is None else self.draft_table
+        return {"logits": np.stack([np.asarray(tab[int(t)], np.float32) for t in tokens])}
+
+
+def test_early_stop_on_a_scripted_model_with_known_probabilities():
+    """Token 0 is followed by logits [0, 2, 1, 0] (greedy token 1, top-1 probability e^2 / (e^2 + e + 2) = 0.6103, the
+    value of the confidence golden vector), token 1 by [0, 0, 1, 0] (greedy token 2, probability e / (e + 3) = 0.4754),
+    token 2 by [0, 0, 0, 4] (token 3, e^4 / (e^4 + 3) = 0.9479), token 3 by [9, 0, 0, 0] (token 0, 0.9996)."""
+    tab = {0: [0, 2, 1, 0], 1: [0, 0, 1, 0], 2: [0, 0, 0, 4], 3: [9, 0, 0, 0]}
+    m = _ScriptedModel(tab, tab)
+    mask = np.array([0, 3, 0, 0], np.uint8)
+    c = oracle.speculative_cycle(m, mask, 0, 10, 4)                                  # no early stop: K drafts
+    assert c["drafts"] == [1, 2, 3, 0] and c["n_drafted"] == 4 and c["n_accepted"] == 4
+    assert c["draft_pmax"] == pytest.approx([0.610296, 0.475367, 0.947915, 0.999630], abs=2e-6)
+    c = oracle.speculative_cycle(m, mask, 0, 10, 4, stop_p=0.5)                      # 0.61 >= 0.5 goes on, 0.4754 < 0.5 stops
+    assert c["drafts"] == [1, 2] and c["n_drafted"] == 2
+    assert c["targets"] == [1, 2, 3] and c["n_accepted"] == 2 and c["emitted"] == [1, 2, 3]   # the low-confidence draft is still verified
+    c = oracle.speculative_cycle(m, mask, 0, 10, 4, stop_p=0.7)                      # already the first draft is below
+    assert c["drafts"] == [1] and c["emitted"] == [1, 2] and c["new_ctx"] == 12
+    c = oracle.speculative_cycle(m, mask, 0, 10, 4, stop_p=0.47)                     # 0.4754 >= 0.47: nothing stops
+    assert c["n_drafted"] == 4
+    c = oracle.speculative_cycle(m, mask, 2, 10, 3, stop_p=0.9999)                   # 0.9479 < 0.9999
+    assert c["drafts"] == [3]
+    # a target model that disagrees on the second token: the stop does not change what acceptance means
+    tgt = dict(tab)
+    tgt[1] = [0, 5, 0, 0]
+    c = oracle.speculative_cycle(_ScriptedModel(tab, tgt), mask, 0, 10, 4, stop_p=0.5)
+    assert c["drafts"] == [1, 2] and c["targets"][:2] == [1, 1] and c["n_accepted"] == 1 and c["emitted"] == [1, 1]
+
+
+def test_early_stop_threshold_zero_is_fixed_k_and_counts_fall_with_the_threshold(c1):
+    w, W, p = c1
+    mask = synth.layers_to_mask([1], w.shape.n_layers)
+    om = oracle.OracleModel(w.shape, W)
+    t0 = oracle.prefill(om, p)[0]
+    base = oracle.speculative_cycle(om, mask, t0, len(p), 6)
+    zero = oracle.speculative_cycle(om, mask, t0, len(p), 6, stop_p=0.0)
+    assert zero["drafts"] == base["drafts"] and zero["n_drafted"] == 6 and zero["emitted"] == base["emitted"]
+    pm = base["draft_pmax"]
+    assert all(0.0 < v <= 1.0 for v in pm)
+    prev = 6
+    for thr in sorted(set([0.0] + [v * (1 + 1e-9) for v in pm] + [v * (1 - 1e-9) for v in pm] + [1.0])):
+        c = oracle.speculative_cycle(om, mask, t0, len(p), 6, stop_p=thr)
+        # from the same state the drafts are a prefix of the fixed-K drafts, cut after the first one below the threshold
+        want = next((i + 1 for i, v in enumerate(pm) if thr > 0 and v < thr), 6)
+        assert c["n_drafted"] == want and c["drafts"] == base["drafts"][:want]
+        assert c["n_drafted"] <= prev
+        prev = c["n_drafted"]
+    assert prev == 1                                                               # threshold 1.0 (above every probability here)
+
+
+@pytest.mark.parametrize("stop_p", [0.002, 0.01, 1.0])
+def test_early_stop_keeps_generation_lossless(c1, stop_p):
+    w, W, p = c1
+    van = oracle.generate_vanilla(oracle.OracleModel(w.shape, W), p, w.gen_len)
+    s = oracle.generate_speculative(oracle.OracleModel(w.shape, W), p, synth.layers_to_mask([1, 2], w.shape.n_layers), 5,
+                                    w.gen_len, stop_p=stop_p)
+    assert s["tokens"] == van["tokens"]
+    assert s["drafted"] == sum(c["n_drafted"] for c in s["cycles"]) <= 5 * len(s["cycles"])
+    if stop_p == 1.0:
+        assert all(c["n_drafted"] == 1 for c in s["cycles"])
+
+
 # ---------------------------------------------------------------- confidence (Eq. 1-4)
 
 def _brute(logits):

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2604_14612_b200 as cl
 import synth
 
@@ -48,6 +49,12 @@ def test_static_scoring_matches_context_scoring_twice(dtype, V, d):
         got = cl.cl_layer_confidences_static(head, gain, hidden, rms_eps=1e-5)
         _check(got, want, hidden, head, gain, 1e-5)
         assert (got["conf"] > -1e-6).all() and (got["conf"] < 1 + 1e-6).all()
+        # and against the CPU oracle's Eq. 1-4 on the same rows (the context's call runs different kernels for a
+        # 16-bit head, so the comparison above is a real one, but this one does not lean on the library at all)
+        o = oracle.layer_confidences(hidden.cpu(), head.cpu(), gain.cpu(), 1e-5)
+        assert np.abs(got["conf"] - o["conf"]).max() <= TOL
+        assert np.abs(got["p_max"] - o["p_max"]).max() <= TOL
+        assert not ((got["argmax"] != o["argmax"]) & (o["margin"] >= NEAR_TIE)).any()
 
 
 def test_static_scoring_rejects_sizes_beyond_its_fixed_scratch():
@@ -61,3 +68,26 @@ def test_static_scoring_rejects_sizes_beyond_its_fixed_scratch():
     with pytest.raises(cl.ConfLayersError) as e:
         cl.cl_layer_confidences_static(torch.zeros((16, 8200), device="cuda"), torch.ones(8200, device="cuda"), wide)
     assert e.value.code == 5
+
+
+def test_static_scoring_rejects_unsupported_dtype_shape_and_alignment():
+    """These fail on the host and launch nothing: an fp16 head (the call knows fp32 and bf16 only), a hidden tensor or a
+    gain whose width is not d_model, and -- through the raw C call -- a pointer that is not 16-byte aligned."""
+    head16 = torch.zeros((16, 64), device="cuda", dtype=torch.float16)
+    gain = torch.ones(64, device="cuda")
+    with pytest.raises(ValueError):
+        cl.cl_layer_confidences_static(head16, gain, torch.zeros((2, 64), device="cuda", dtype=torch.float16))
+    head = torch.zeros((16, 64), device="cuda")
+    with pytest.raises(ValueError):
+        cl.cl_layer_confidences_static(head, gain, torch.zeros((2, 32), device="cuda"))
+    with pytest.raises(ValueError):
+        cl.cl_layer_confidences_static(head, torch.ones(32, device="cuda"), torch.zeros((2, 64), device="cuda"))
+    lib = cl.load_library()
+    hidden = torch.zeros((3, 64), device="cuda")
+    out = np.zeros(2, np.float32)
+    rc = lib.cl_layer_confidences_static(head.data_ptr(), gain.data_ptr(), 16, 64, 2, 1e-5, hidden.data_ptr(), 2, None,
+                                         out.ctypes.data, None, None)
+    assert rc == 1 and b"weight_dtype" in lib.cl_last_error(None)
+    rc = lib.cl_layer_confidences_static(head.data_ptr(), gain.data_ptr(), 16, 64, 0, 1e-5, hidden.data_ptr() + 4, 2, None,
+                                         out.ctypes.data, None, None)
+    assert rc == 1 and b"16-byte aligned" in lib.cl_last_error(None)
