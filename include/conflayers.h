@@ -259,6 +259,13 @@ int cl_layer_confidences_static(const void *lm_head, const float *final_norm, in
 enum { CL_DEBUG_WAIT_LIMIT_US = 1, CL_DEBUG_BARRIER_EXTRA = 2, CL_DEBUG_DEVICE_ERR = 3 };
 int cl_debug_set(cl_ctx *ctx, int what, long long value);
 
+/* Reads a diagnostic record into host memory.  CL_DEBUG_ROWS_PHASE_NS: out = uint64[n_SMs * 8], for every CTA of the
+ * persistent T-row pass (verify, short prompt chunks of 16-bit models) the nanoseconds its first thread spent, during
+ * the last pass, in: 0 embedding, 1 QKV, 2 attention, 3 output projection, 4 gate/up, 5 down projection, 6 LM head,
+ * 7 grid barriers.  The first call switches the recording on (and returns zeros). */
+enum { CL_DEBUG_ROWS_PHASE_NS = 1 };
+int cl_debug_read(cl_ctx *ctx, int what, void *out, int n);
+
 /* ---- bookkeeping ----------------------------------------------------------------------------- */
 
 int cl_get_stats(cl_ctx *ctx, cl_stats *out);      /* alpha, beta, M of Section 4.1.2 derive from these */

@@ -109,6 +109,7 @@ def load_library():
         "cl_read_hidden_ring": [vp, vp],
         "cl_get_stats": [vp, C.POINTER(Stats)],
         "cl_debug_set": [vp, C.c_int, C.c_longlong],
+        "cl_debug_read": [vp, C.c_int, vp, C.c_int],
         "cl_layer_confidences_static": [vp, vp, C.c_int, C.c_int, C.c_int, C.c_float, vp, C.c_int, vp, vp, vp, vp],
     }
     for name, args in sig.items():
@@ -351,6 +352,12 @@ class Context:
 
     def cl_debug_set(self, what: int, value: int):
         self._ck(self._L.cl_debug_set(self._h, what, value))
+
+    def cl_debug_read_phase_ns(self) -> np.ndarray:
+        """[n_SMs, 8] nanoseconds per phase of the last persistent T-row pass (see the header)."""
+        out = np.zeros((256, 8), np.uint64)
+        self._ck(self._L.cl_debug_read(self._h, 1, _np_ptr(out), out.size))
+        return out
 
     def cl_get_stats(self) -> Stats:
         st = Stats()

@@ -72,6 +72,18 @@ struct cl_ctx {
     int v_att_S;                         // parts the keys of a head are cut into in the T-row attention
     unsigned *v_tickets;
     ClHeadPartial *v_head_part;
+    // persistent tensor-core pass of the T-row passes (16-bit models): second, k-block-major copy of the matrices
+    int use_rows;
+    char *wtile, *head_tile;             // per layer [Wqkv | Wo | Wgu | Wd] k-block-major; LM head k-block-major
+    ClRowsLayer *rows_layers_dev;
+    unsigned short *r_ax, *r_aatt, *r_ah;
+    float *r_ssq, *r_att_part, *r_ws;
+    unsigned *r_bar;                     // arrival counters of the pass: the grid's, then one per group of CTAs
+    int rows_split;                      // CTAs per group that cut the K range of the output / down projections between them
+    unsigned *r_tickets;
+    ClHeadPartial *r_head_part;
+    int rows_chain;                      // ring slots per accumulation chain in tensor memory
+    unsigned long long *r_phase_ns;      // diagnostics (cl_debug_read): per-CTA time by phase of the last pass
     // wide tensor-core GEMM path of the prompt pass (bf16 models)
     int use_wide;
     ClTensorMap map_wx, map_watt, map_wh;  // activation rows as bf16 hi/lo parts, boxes of 128 rows
@@ -211,7 +223,8 @@ static void free_all(cl_ctx *c) {
                     c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sc_xn, c->sc_part, c->sel_mask, c->sel_margins, c->sel_clayers,
                     c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->head_part2,
                     c->cum_w_dev, c->busy_dev, c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_att_part, c->v_tickets, c->v_head_part,
-                    c->w_ax, c->w_aatt, c->w_ah, c->w_x, c->w_P};
+                    c->w_ax, c->w_aatt, c->w_ah, c->w_x, c->w_P, c->wtile, c->head_tile, c->rows_layers_dev, c->r_ax, c->r_aatt,
+                    c->r_ah, c->r_ssq, c->r_att_part, c->r_tickets, c->r_head_part, c->r_phase_ns, c->r_ws, c->r_bar};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (c->h_st) cudaFreeHost(c->h_st);
@@ -241,6 +254,7 @@ static cudaError_t dmalloc(T **p, size_t bytes) {
     } while (0)
 
 static int calibrate_row_shares(cl_ctx *c);
+static char *ring_slot(cl_ctx *c, int l, int which);
 
 extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
     if (!c || !w) return fail(c, CL_EINVAL, "cl_load: null argument");
@@ -446,6 +460,61 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 }
             }
         }
+        // ---- persistent T-row pass on the tensor cores: k-block-major copies of every matrix, operand buffers, partials
+        c->use_rows = 0;
+        {
+            const char *off = getenv("CL_DISABLE_ROWS_KERNEL");
+            int coop = 0;
+            cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
+            const bool shape_ok = d % 64 == 0 && F % 64 == 0 && (d / 8 + c->n_sm - 1) / c->n_sm <= 16 && g.n_heads <= 8 * c->n_sm &&
+                                  (d + c->n_sm - 1) / c->n_sm + 8 <= 224;
+            if (g.weight_dtype != 0 && coop && shape_ok && L > 0 && !(off && off[0] == '1')) {
+                // the output and down projections give each CTA too few rows for an efficient tensor-core tile: groups of
+                // CTAs share rows and cut K (a group's partial products meet in a workspace)
+                const char *sp = getenv("CL_ROWS_SPLIT");   // tuning knob
+                c->rows_split = (sp && sp[0]) ? atoi(sp) : 4;
+                if (c->rows_split < 1 || c->rows_split > 8) c->rows_split = 1;
+                // (a group's rows must fit one tile of 224 rows: its parts meet in a workspace that holds one tile per CTA)
+                while (c->rows_split > 1 && (c->n_sm % c->rows_split || d / 64 < (size_t)c->rows_split || F / 64 < (size_t)c->rows_split ||
+                                             (d * c->rows_split + c->n_sm - 1) / c->n_sm + 8 > 224))
+                    c->rows_split >>= 1;
+                DM(c->wtile, per_layer * L);
+                DM(c->head_tile, V * d * es);
+                DM(c->r_ws, (size_t)c->n_sm * CL_MAX_T * 224 * 4);
+                DM(c->r_bar, ((size_t)1 + c->n_sm) * 4);
+                std::vector<ClRowsLayer> rl(L);
+                for (size_t l = 0; l < L; ++l) {
+                    const ClLayer &y = c->layers[l];
+                    char *t0 = c->wtile + l * per_layer;
+                    KL(cl_launch_tile_layout(y.wqkv, t0, (int)qkv_rows, (int)d, 1, c->n_sm, c->stream));
+                    KL(cl_launch_tile_layout(y.wo, t0 + b_qkv, (int)d, (int)d, 1, c->n_sm / c->rows_split, c->stream));
+                    KL(cl_launch_tile_layout(y.wgu, t0 + b_qkv + b_o, (int)(2 * F), (int)d, 2, c->n_sm, c->stream));
+                    KL(cl_launch_tile_layout(y.wd, t0 + b_qkv + b_o + b_gu, (int)d, (int)F, 1, c->n_sm / c->rows_split, c->stream));
+                    rl[l] = ClRowsLayer{t0, t0 + b_qkv, t0 + b_qkv + b_o, t0 + b_qkv + b_o + b_gu, y.n1, y.n2, y.kc, y.vc,
+                                        ring_slot(c, (int)l, 0), ring_slot(c, (int)l, 1)};
+                }
+                KL(cl_launch_tile_layout(c->lm_head, c->head_tile, (int)V, (int)d, 1, c->n_sm, c->stream));
+                DM(c->rows_layers_dev, L * sizeof(ClRowsLayer));
+                CU(cudaMemcpyAsync(c->rows_layers_dev, rl.data(), L * sizeof(ClRowsLayer), cudaMemcpyHostToDevice, c->stream));
+                CU(cudaStreamSynchronize(c->stream));   // rl goes out of scope
+                const size_t a_d = (d / 64) * CL_ROWS_AROWS * 64 * 2, a_f = (F / 64) * CL_ROWS_AROWS * 64 * 2;
+                DM(c->r_ax, a_d);
+                DM(c->r_aatt, a_d);
+                DM(c->r_ah, a_f);
+                CU(cudaMemsetAsync(c->r_ax, 0, a_d, c->stream));
+                CU(cudaMemsetAsync(c->r_aatt, 0, a_d, c->stream));
+                CU(cudaMemsetAsync(c->r_ah, 0, a_f, c->stream));
+                DM(c->r_ssq, (size_t)c->n_sm * CL_SLOTS * 4);
+                DM(c->r_att_part, (size_t)cl_rows_att_part_floats(g.n_heads) * 4);
+                DM(c->r_tickets, (size_t)g.n_heads * 4);
+                CU(cudaMemsetAsync(c->r_tickets, 0, (size_t)g.n_heads * 4, c->stream));
+                DM(c->r_head_part, (size_t)c->n_sm * CL_SLOTS * sizeof(ClHeadPartial));
+                const char *ch = getenv("CL_ROWS_CHAIN");   // tuning knob
+                c->rows_chain = (ch && ch[0]) ? atoi(ch) : 4;
+                if (c->rows_chain < 1) c->rows_chain = 1;
+                c->use_rows = 1;
+            }
+        }
         CU(cudaStreamSynchronize(c->stream));   // host staging vector and borrowed pointers are released after this
         if (stage_g) cudaFree(stage_g);
         if (stage_u) cudaFree(stage_u);
@@ -504,12 +573,38 @@ static int head(cl_ctx *c, int T, const float *xin, const ClDevState *st, int *o
 static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, int want_head, int *out_tok, float *out_pmax,
                            float *out_conf, float *logits);
 
+// The same pass as one persistent launch on the tensor cores (16-bit models): all layers and the LM head.
+static int forward_rows_persistent(cl_ctx *c, const int *tok, int T, int row0, int tap, int want_head, int *out_tok,
+                                   float *out_pmax, float *out_conf, float *logits) {
+    const cl_model_cfg &g = c->cfg;
+    ClRowsArgs a;
+    memset(&a, 0, sizeof(a));
+    a.layers = c->rows_layers_dev; a.L = g.n_layers; a.head = c->head_tile; a.embed = c->embed; a.final_norm = c->final_norm;
+    a.d = g.d_model; a.F = g.d_ffn; a.V = g.vocab; a.H = g.n_heads; a.Hkv = g.n_kv_heads; a.hd = g.head_dim; a.max_seq = g.max_seq;
+    a.T = T; a.row0 = row0; a.want_head = want_head; a.f16 = g.weight_dtype == 2;
+    a.att_parts = c->n_sm / g.n_heads;
+    if (a.att_parts < 1) a.att_parts = 1;
+    if (a.att_parts > 8) a.att_parts = 8;
+    a.tap = tap && c->ring; a.tap_P = g.tap_positions;
+    a.chain = c->rows_chain; a.split = c->rows_split; a.ws = c->r_ws;
+    a.eps = g.rms_eps; a.inv_d = 1.0f / (float)g.d_model; a.inv_log_v = (float)(1.0 / log((double)g.vocab));
+    a.rope_cs = c->rope_cs; a.st = c->st; a.tok = tok;
+    a.x = c->x; a.qkv = c->qkv; a.Ax = c->r_ax; a.Aatt = c->r_aatt; a.Ah = c->r_ah;
+    a.ssq = c->r_ssq; a.att_part = c->r_att_part; a.att_tickets = c->r_tickets; a.head_part = c->r_head_part;
+    a.logits = logits; a.out_tok = out_tok; a.out_pmax = out_pmax; a.out_conf = out_conf;
+    a.bar = c->r_bar; a.bar_arrivals = (unsigned)c->n_sm; a.wait_ns = c->wait_ns; a.phase_ns = c->r_phase_ns;
+    CU(cudaMemsetAsync(c->r_bar, 0, ((size_t)1 + c->n_sm / c->rows_split) * 4, c->stream));   // arrival counters start at zero
+    KL(cl_launch_rows_pass(g.weight_dtype, g.head_dim, a, c->n_sm, c->stream));
+    return CL_OK;
+}
+
 // tok: device pointer to the T token ids; rows sit at positions st->ctx + row0 + t.
 static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_t *mask, int tap, int want_head,
                         int *out_tok, float *out_pmax, float *out_conf, float *logits) {
     const cl_model_cfg &g = c->cfg;
     const int d = g.d_model, F = g.d_ffn, wd = g.weight_dtype, qkv_rows = d + 2 * g.n_kv_heads * g.head_dim;
     int rc;
+    if (c->use_rows && !mask) return forward_rows_persistent(c, tok, T, row0, tap, want_head, out_tok, out_pmax, out_conf, logits);
     if (c->use_tc && !mask) return forward_rows_tc(c, tok, T, row0, tap, want_head, out_tok, out_pmax, out_conf, logits);
     KL(cl_launch_embed(wd, c->embed, tok, T, d, c->x, c->st, c->stream));
     for (int l = 0; l < g.n_layers; ++l) {
@@ -1295,6 +1390,22 @@ extern "C" int cl_debug_set(cl_ctx *c, int what, long long value) {
         default:
             return fail(c, CL_EINVAL, "cl_debug_set: unknown setting %d", what);
     }
+}
+
+extern "C" int cl_debug_read(cl_ctx *c, int what, void *out, int n) {
+    if (!c || !out) return fail(c, CL_EINVAL, "cl_debug_read: null argument");
+    if (what == CL_DEBUG_ROWS_PHASE_NS) {
+        if (!c->use_rows) return fail(c, CL_ESTATE, "cl_debug_read: this context does not run the persistent T-row pass");
+        if (n < c->n_sm * 8) return fail(c, CL_ERANGE, "cl_debug_read: room for %d values needed", c->n_sm * 8);
+        if (!c->r_phase_ns) {   // first call: switch the recording on; the next passes fill it
+            DM(c->r_phase_ns, (size_t)c->n_sm * 8 * sizeof(unsigned long long));
+            CU(cudaMemset(c->r_phase_ns, 0, (size_t)c->n_sm * 8 * sizeof(unsigned long long)));
+        }
+        CU(cudaStreamSynchronize(c->stream));
+        CU(cudaMemcpy(out, c->r_phase_ns, (size_t)c->n_sm * 8 * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+        return CL_OK;
+    }
+    return fail(c, CL_EINVAL, "cl_debug_read: unknown item %d", what);
 }
 
 extern "C" int cl_get_stats(cl_ctx *c, cl_stats *out) {

@@ -63,6 +63,29 @@ struct ClHeadPartial {
     int idx;
 };
 
+#ifdef __CUDACC__
+// Merge of two partial softmax statistics (b after a in index order: ties of the maximum keep the lower index).
+__device__ __forceinline__ ClHeadPartial cl_hp_merge(const ClHeadPartial &a, const ClHeadPartial &b) {
+    if (b.z == 0.f) return a;
+    if (a.z == 0.f) return b;
+    ClHeadPartial r;
+    r.m = fmaxf(a.m, b.m);
+    const float ea = expf(a.m - r.m), eb = expf(b.m - r.m);
+    r.z = a.z * ea + b.z * eb;
+    r.s = ea * (a.s + (a.m - r.m) * a.z) + eb * (b.s + (b.m - r.m) * b.z);
+    r.idx = (a.m > b.m) ? a.idx : (b.m > a.m) ? b.idx : min(a.idx, b.idx);
+    return r;
+}
+__device__ __forceinline__ ClHeadPartial cl_hp_shfl_xor(const ClHeadPartial &a, int o) {
+    ClHeadPartial r;
+    r.m = __shfl_xor_sync(0xffffffffu, a.m, o);
+    r.z = __shfl_xor_sync(0xffffffffu, a.z, o);
+    r.s = __shfl_xor_sync(0xffffffffu, a.s, o);
+    r.idx = __shfl_xor_sync(0xffffffffu, a.idx, o);
+    return r;
+}
+#endif
+
 enum { CL_EPI_STORE = 0, CL_EPI_RESID = 1, CL_EPI_SILU = 2, CL_EPI_HEAD = 3 };
 
 struct ClGemvArgs {
@@ -193,6 +216,50 @@ cudaError_t cl_launch_pass_begin(const void *embed, const int *tok, int T, int d
                                  const float *g, float *ssq_out, const ClDevState *st, int f16, cudaStream_t s);
 cudaError_t cl_launch_head_finalize(const ClHeadPartial *part, int tiles, int T, float inv_log_v, int *out_tok, float *out_pmax,
                                     float *out_conf, const ClDevState *st, cudaStream_t s);
+
+// ---- persistent tensor-core pass over T <= CL_MAX_T rows (16-bit models): all layers and the LM head in one launch ----
+#define CL_ROWS_AROWS 32   // rows per k-block of an activation operand buffer: hi part of token t in row t, lo part in row T + t
+struct ClRowsLayer {
+    const char *wqkv, *wo, *wgu, *wd;   // copies in the kernel's streaming order (CTA by CTA, [K / 64][block rows][64], 16-byte pieces permuted by row & 7)
+    const float *n1, *n2;
+    char *kc, *vc;
+    void *tap0, *tap1;                  // this layer's hidden-state ring after the attention add / after the FFN add (or null)
+};
+struct ClRowsArgs {
+    const ClRowsLayer *layers;          // device [L]
+    int L;
+    const char *head;                   // LM head, k-block-major
+    const void *embed;                  // [V, d] row-major
+    const float *final_norm;
+    int d, F, V, H, Hkv, hd, max_seq;
+    int T, row0, want_head, f16, att_parts, tap, tap_P;
+    int split;                          // CTAs of a group that share the rows of an output / down projection and cut K between them
+    int chain;                          // ring slots summed in tensor memory before the accumulator is drained into registers
+    float eps, inv_d, inv_log_v;
+    const float2 *rope_cs;
+    ClDevState *st;
+    const int *tok;                     // device [T] token ids of the rows
+    float *x, *qkv;                     // residual stream [T, d], QKV product [T, d + 2 Hkv hd] (raw: no rotary yet)
+    unsigned short *Ax, *Aatt, *Ah;     // activation operands [d / 64 | d / 64 | F / 64][CL_ROWS_AROWS][64]
+    float *ws;                          // [grid, CL_MAX_T, 224] raw products of the output / down projections, per CTA (K part)
+    float *ssq;                         // [grid, CL_SLOTS] per-CTA sums of squares of the residual rows
+    float *att_part;                    // [H, 8, CL_MAX_T, hd + 2] per-part attention records
+    unsigned *att_tickets;              // [H], zero between launches
+    ClHeadPartial *head_part;           // [grid, CL_SLOTS]
+    float *logits;                      // optional [T, V]
+    int *out_tok;                       // [T] greedy token after each row
+    float *out_pmax, *out_conf;
+    unsigned *bar;                      // [1 + grid / split] arrival counters, zero at launch: the grid's barrier, then one per group
+    unsigned bar_arrivals;
+    unsigned long long wait_ns;
+    unsigned long long *phase_ns;       // diagnostics, optional: [grid, 8] time of each CTA's thread 0 by phase
+};
+size_t cl_rows_smem_bytes();
+int cl_rows_att_part_floats(int H);
+// src: row-major [rows, K] 16-bit elements; dst: the same matrix in the streaming order of a grid of `grid` CTAs
+// (rows split in units of `unit` rows, exactly as the kernel splits them)
+cudaError_t cl_launch_tile_layout(const void *src, void *dst, int rows, int K, int unit, int grid, cudaStream_t s);
+cudaError_t cl_launch_rows_pass(int wdtype, int head_dim, const ClRowsArgs &a, int grid, cudaStream_t s);
 
 // ---- wide tensor-core GEMM of the prompt pass (bf16 models): up to CL_WIDE_MAX_M prompt rows at a time ----
 #define CL_WIDE_MAX_M 512

@@ -1,0 +1,1082 @@
+// Persistent full-model pass over T <= 9 token rows of a model stored in a 16-bit type: the (K+1)-row verify pass of
+// Section 3 (Figure 2: the target model checks the K candidates and the pending token in one forward pass), and the
+// short prompt chunks, which are the same pass.  One cooperative launch runs every layer and the LM head.
+//
+// The pass is bound by HBM weight streaming (at most 9 flop per weight byte), so its shape follows the single-token
+// step kernel: one CTA per SM, every CTA owns a contiguous block of rows of every matrix (single-row granularity, so
+// all SMs stream the same number of bytes), one producer thread walks the static schedule and keeps a 192 KB ring of
+// weight tiles filled straight through the phase boundaries, and the phases of a layer (QKV | attention | O |
+// gate/up | down) are separated by grid barriers, not by launches.  What differs is the arithmetic: 2 T activation
+// rows against every weight row is more than the CUDA cores issue at the HBM rate, so the contraction runs on the
+// tensor cores:
+//
+//   D[m, n] = sum_k A[m, k] * B[n, k]      tcgen05.mma, M = 128, N = the CTA's rows (multiple of 16, <= 224), K = 16
+//
+// A = activation rows: row t holds hi = round16(v), row T + t holds lo = round16(v - hi) of token t, so the product
+//     keeps about 16 mantissa bits of the fp32 activations; rows 2 T .. 127 of the operand are whatever the shared
+//     memory behind the tile holds -- row m of D depends on row m of A only, and those rows of D are never read.
+// B = the CTA's weight rows.  The weights are stored a second time, in the order this kernel streams them: CTA by
+//     CTA (each CTA's row block [r0, r1) of a matrix is one contiguous region, so a CTA walks memory sequentially --
+//     with a k-block-major order over the whole matrix every copy of a CTA started in another 2 MB page and the
+//     stream ran at a third of the HBM rate), inside a block k-block by k-block, [K / 64][r1 - r0][64] elements, with
+//     the 16-byte pieces of a row's 128 bytes permuted by (piece ^ (row & 7)): that is the layout the tensor core's
+//     128-byte-swizzle shared-memory descriptor expects, so the rows [g0, g1) of one k-block arrive with one bulk
+//     copy of exactly the bytes this CTA owns.  The tile in shared memory starts at row g0 & ~7 (keeping row & 7
+//     equal on both sides); rows in front of g0 and behind g1 are stale -- column n of D depends on row n of B
+//     only, and those columns are never read.
+// The accumulator lives in tensor memory (two buffers of 256 columns); it is drained into fp32 registers after
+// every ring slot (64 to 320 elements of K), so a long K is summed in fp32 registers, not in one tensor-core chain.
+// Warp roles: warps 0-13 workers (embedding, attention, epilogues; warps 0, 4, 8, 12 are the four that can read
+// tensor-memory lanes 0-31 and drain the accumulator), warp 14 producer, warp 15 MMA issue and tensor-memory owner.
+// RMSNorm is split around the GEMM as in the other tensor-core kernels: the activation operand holds x * gain,
+// the per-token scale rsqrt(mean x^2 + eps) multiplies the product.
+// Every wait is bounded; on expiry an error flag is raised, later waits fall through, copies in flight are waited
+// for, tensor memory is released and the host reports CL_ETIMEOUT.
+#include <math.h>
+#include <string.h>
+
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int RW = 14;                 // worker warps (16 warps in all: four per scheduler, 128 registers per thread)
+constexpr int RT = RW * 32;            // worker threads
+constexpr int R_THREADS = RT + 64;     // + producer warp + MMA warp
+constexpr int R_SLOT = 32768;          // ring slot
+constexpr int R_NSLOT = 6;             // 192 KB of tiles in flight per SM
+constexpr int R_MAXN = 224;            // most rows of a weight tile (tile + activation rows fill a slot at one k-block)
+constexpr int R_ATT_MAXS = 8;          // most parts the cached keys of a head are cut into
+
+struct RSmem {
+    unsigned long long full[R_NSLOT], empty[R_NSLOT], tfull[2], tempty[2];
+    unsigned long long wait_ns;
+    unsigned tmem_base;
+    int abort;
+    int bars_done;                     // grid barriers this CTA has passed (read by the producer)
+    int is_last;
+    float scale[CL_SLOTS];             // RMSNorm scale of every token row for the current phase
+    float red[4][CL_SLOTS];
+    float esum[16][CL_SLOTS];          // embedding phase: per-chunk sums of squares
+    ClHeadPartial hp[4][CL_SLOTS];
+    float wrec[RW * (128 + 2)];        // attention: per-warp (max, sum, o[hd]) records
+    unsigned long long t_prev, ph_ns[8];   // diagnostics: time of thread 0 by phase
+};
+
+// Diagnostics (a.phase_ns != null): thread 0 adds the time since its last call to phase `idx`
+// (0 embedding, 1 QKV, 2 attention, 3 output projection, 4 gate/up, 5 down, 6 LM head, 7 grid barriers).
+__device__ __forceinline__ void phase_clock(const ClRowsArgs &a, RSmem *sm, int idx) {
+    if (a.phase_ns && threadIdx.x == 0) {
+        const unsigned long long now = gtime_ns();
+        sm->ph_ns[idx] += now - sm->t_prev;
+        sm->t_prev = now;
+    }
+}
+
+// ---- schedule ---------------------------------------------------------------------------------------
+// GEMM jobs in execution order: job 4 l + m = matrix m of layer l (0 QKV, 1 O, 2 gate/up, 3 down), job 4 L = LM head.
+// A CTA's rows [r0, r1) of a job are cut into groups of at most R_MAXN tile rows; a group's K range into ring slots
+// of as many k-blocks as fit.  Producer, MMA issuer and drain warps walk the same sequence.
+struct Job {
+    const char *W;        // k-block-major weights
+    const unsigned short *A;
+    int rows, KB, unit, epi, need;
+    int split;            // CTAs that share a row block and cut its K range between them (1: every CTA owns rows over all of K)
+};
+
+__device__ __forceinline__ Job job_of(const ClRowsArgs &a, int ji) {
+    Job j;
+    const int L = a.L;
+    if (ji < 4 * L) {
+        const int l = ji >> 2, m = ji & 3;
+        const ClRowsLayer &y = a.layers[l];
+        const int base = 1 + 5 * l;   // grid barriers passed when layer l's QKV input is complete
+        if (m == 0) { j.W = y.wqkv; j.A = a.Ax; j.rows = a.d + 2 * a.Hkv * a.hd; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_STORE; j.need = base; j.split = 1; }
+        else if (m == 1) { j.W = y.wo; j.A = a.Aatt; j.rows = a.d; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_RESID; j.need = base + 2; j.split = a.split; }
+        else if (m == 2) { j.W = y.wgu; j.A = a.Ax; j.rows = 2 * a.F; j.KB = a.d >> 6; j.unit = 2; j.epi = CL_VEPI_SILU; j.need = base + 3; j.split = 1; }
+        else { j.W = y.wd; j.A = a.Ah; j.rows = a.d; j.KB = a.F >> 6; j.unit = 1; j.epi = CL_VEPI_RESID; j.need = base + 4; j.split = a.split; }
+    } else {
+        j.W = a.head; j.A = a.Ax; j.rows = a.V; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_HEAD; j.need = 1 + 5 * L; j.split = 1;
+    }
+    return j;
+}
+
+// Rows [r0, r1) of a matrix that CTA c of G owns (a unit is `unit` consecutive rows that stay together).
+__device__ __forceinline__ void rows_of_cta(int rows, int unit, int c, int G, int &r0, int &r1) {
+    const long long units = rows / unit;
+    r0 = (int)(units * c / G) * unit;
+    r1 = (int)(units * (c + 1) / G) * unit;
+}
+// Rows of this CTA (split = 1) or of its group of `split` neighbouring CTAs.
+__device__ __forceinline__ void rows_of(int rows, int unit, int split, int &r0, int &r1) {
+    rows_of_cta(rows, unit, blockIdx.x / split, gridDim.x / split, r0, r1);
+}
+
+// Position in the schedule: (job, group of the CTA's rows, slot).  advance() is a handful of instructions inside a
+// group (the producer, the MMA issuer and the drain warps each run it once per slot, serially, so it has to be);
+// everything that costs a division is worked out once per group.
+struct Cursor {
+    const ClRowsArgs &a;
+    int njobs, ars;
+    // job
+    int ji;
+    const char *W;
+    const unsigned short *A;
+    int rows, KB, unit, epi, need;
+    int kb_begin, kb_end;     // the CTA's k-blocks of the job (all of them unless the job is split over K)
+    int r0, r1;               // the rows of the CTA (of its group, for a job split over K)
+    // group
+    int g0, g1, a0, npad;     // weight rows [g0, g1); first tile row g0 & ~7; tile rows (multiple of 16)
+    int per;                  // k-blocks per ring slot
+    unsigned stride;          // bytes between the k-block tiles of a slot (activation rows + weight rows)
+    size_t wbase;             // byte offset in W of (row g0, k-block 0)
+    unsigned wstep;           // bytes between k-blocks in W (the CTA's block is [K / 64][r1 - r0][64])
+    // slot
+    int kb0, kbs, in_chain;
+    bool done;
+
+    __device__ Cursor(const ClRowsArgs &args) : a(args), ji(-1), in_chain(0), done(false) {
+        njobs = 4 * a.L + (a.want_head ? 1 : 0);
+        ars = (2 * a.T + 7) & ~7;
+        next_job();
+    }
+    __device__ __forceinline__ bool first() const { return kb0 == kb_begin; }
+    __device__ __forceinline__ bool last() const { return kb0 + kbs >= kb_end; }             // last slot of the group
+    __device__ __forceinline__ bool job_last() const { return last() && g1 >= r1; }          // ... of the job, for this CTA
+    __device__ __forceinline__ bool chain_first() const { return in_chain == 0; }
+    __device__ __forceinline__ bool chain_last() const { return last() || in_chain + 1 >= a.chain; }
+    __device__ void open_group(int g) {
+        g0 = g;
+        a0 = g & ~7;
+        g1 = min(r1, a0 + R_MAXN);
+        npad = (g1 - a0 + 15) & ~15;
+        stride = (unsigned)(ars + npad) * 128u;
+        per = R_SLOT / (int)stride;
+        wbase = ((size_t)r0 * KB + (size_t)(g0 - r0)) * 128;
+        wstep = (unsigned)(r1 - r0) * 128u;
+        kb0 = kb_begin;
+        kbs = min(per, kb_end - kb_begin);
+    }
+    __device__ void next_job() {
+        for (++ji; ji < njobs; ++ji) {
+            const Job j = job_of(a, ji);
+            W = j.W; A = j.A; rows = j.rows; KB = j.KB; unit = j.unit; epi = j.epi; need = j.need;
+            rows_of(rows, unit, j.split, r0, r1);
+            const int member = (int)blockIdx.x % j.split;
+            kb_begin = KB * member / j.split;
+            kb_end = KB * (member + 1) / j.split;
+            if (r0 < r1 && kb_begin < kb_end) {
+                open_group(r0);
+                return;
+            }
+        }
+        done = true;
+    }
+    __device__ __forceinline__ void advance() {
+        in_chain = chain_last() ? 0 : in_chain + 1;
+        kb0 += kbs;
+        if (kb0 < kb_end) {
+            kbs = min(per, kb_end - kb0);
+        } else if (g1 < r1) {
+            open_group(g1);
+        } else {
+            next_job();
+        }
+    }
+};
+
+// ---- small helpers -------------------------------------------------------------------------------------
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(RT) : "memory"); }
+__device__ __forceinline__ void drain_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(s_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(s_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_g2s_stream(void *dst, const void *src, unsigned bytes, unsigned long long *bar,
+                                                unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+            s_u32(dst)),
+        "l"(src), "r"(bytes), "r"(s_u32(bar)), "l"(policy)
+        : "memory");
+}
+// Non-blocking look at an mbarrier phase.  (mbarrier.try_wait may suspend the thread for a while before it answers
+// "not yet"; a loop that serves two queues must not sit in it.)
+__device__ __forceinline__ bool bar_test(unsigned long long *b, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(s_u32(b)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Orders this thread's generic-proxy accesses of global memory with async-proxy (bulk copy) accesses.
+__device__ __forceinline__ void proxy_fence_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+
+__device__ __forceinline__ bool r_wait(unsigned long long *b, unsigned parity, RSmem *sm, int *err) {
+    if (bar_try(b, parity)) return true;
+    if (*(volatile int *)&sm->abort) return false;
+    const unsigned long long t0 = gtime_ns();
+    for (unsigned i = 1;; ++i) {
+        if (bar_try(b, parity)) return true;
+        if ((i & 63u) == 0u) {
+            if (*(volatile int *)&sm->abort) return false;
+            if (gtime_ns() - t0 > sm->wait_ns) {
+                *(volatile int *)&sm->abort = 1;
+                atomicOr(err, 8);
+                return false;
+            }
+        }
+    }
+}
+
+// Grid barrier on one arrival counter that only grows during a launch (the host zeroes it before the launch).
+// Called by every worker thread; thread 0 arrives and polls (bounded) and then publishes the count for the producer.
+__device__ __forceinline__ void grid_barrier(const ClRowsArgs &a, unsigned &target, int &passed, RSmem *sm) {
+    proxy_fence_global();   // this thread's global stores are read by other CTAs' bulk copies after the barrier
+    worker_sync();
+    if (threadIdx.x == 0) {
+        if (!*(volatile int *)&sm->abort) {
+            target += a.bar_arrivals;
+            asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.bar) : "memory");
+            unsigned v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.bar) : "memory");
+            if ((int)(v - target) < 0) {
+                const unsigned long long t0 = gtime_ns();
+                unsigned i = 0;
+                do {
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.bar) : "memory");
+                    if ((++i & 255u) == 0u) {
+                        if (*(volatile int *)&a.st->err || gtime_ns() - t0 > sm->wait_ns) {
+                            *(volatile int *)&sm->abort = 1;
+                            atomicOr(&a.st->err, 16);
+                            break;
+                        }
+                    }
+                } while ((int)(v - target) < 0);
+            }
+        }
+        __threadfence();
+        *(volatile int *)&sm->bars_done = passed + 1;
+    }
+    ++passed;
+    worker_sync();
+    phase_clock(a, sm, 7);
+}
+
+__device__ __forceinline__ void tmem_ld16(unsigned taddr, float (&v)[16]) {
+    unsigned r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Index (in 16-bit elements) of element k of activation row r in a k-block-major operand buffer [K / 64][R_AROWS][64].
+__device__ __forceinline__ size_t a_index(int r, int k) {
+    const int kb = k >> 6, c = (k & 63) >> 3, e = k & 7;
+    return ((size_t)kb * CL_ROWS_AROWS + r) * 64 + (size_t)(((c ^ (r & 7)) << 3) + e);
+}
+__device__ __forceinline__ void a_store_split(unsigned short *A, int t, int T, int k, float v, int f16) {
+    unsigned short hi, lo;
+    split_b16(v, f16, hi, lo);
+    A[a_index(t, k)] = hi;
+    A[a_index(T + t, k)] = lo;
+}
+
+__device__ __forceinline__ ClHeadPartial rp_merge(const ClHeadPartial &a, const ClHeadPartial &b) { return cl_hp_merge(a, b); }
+
+// ---- producer ------------------------------------------------------------------------------------------
+// The whole producer warp runs this (uniform control flow; lane j issues the copy of a slot's j-th k-block, so a slot
+// costs the same few instructions however many k-blocks it holds).  Weight tiles are requested as soon as a ring
+// slot is free -- weights never change, so the stream runs ahead of the grid barriers; the activation tiles of a slot
+// are requested once the barrier that completes them has been passed (bars_done), both on the slot's one mbarrier.
+__device__ void producer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, int lane) {
+    unsigned long long policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    Cursor w(a), q(a);                     // weight cursor; head of the queue of slots that still lack their activation tiles
+    const unsigned abytes = (unsigned)w.ars * 128u;
+    unsigned slot = 0, par = 0;            // ring slot of the weight cursor
+    unsigned qslot = 0;                    // ring slot of the queue's head
+    int pn = 0;                            // queue length
+    unsigned used = 0;                     // bit i: slot i has copies in flight of phase parity (used_par >> i) & 1
+    unsigned used_par = 0;
+    int fenced = 0;                        // grid barriers whose writes this warp has ordered before its copies
+    unsigned long long t_idle = 0;
+    unsigned n_idle = 0;
+    while (!w.done || pn > 0) {
+        if (__shfl_sync(0xffffffffu, *(volatile int *)&sm->abort, 0)) break;
+        bool progress = false;
+        if (pn > 0) {
+            const int bars = __shfl_sync(0xffffffffu, *(volatile int *)&sm->bars_done, 0);
+            if (bars >= q.need) {
+                if (bars > fenced) {   // once per barrier: other CTAs' stores before this warp's bulk-copy reads
+                    __threadfence();
+                    proxy_fence_global();
+                    fenced = bars;
+                }
+                if (lane < q.kbs)
+                    bulk_g2s(ring + (size_t)qslot * R_SLOT + (size_t)lane * q.stride,
+                             q.A + (size_t)(q.kb0 + lane) * (CL_ROWS_AROWS * 64), abytes, &sm->full[qslot]);
+                if (++qslot == R_NSLOT) qslot = 0;
+                --pn;
+                q.advance();
+                progress = true;
+            }
+        }
+        // (lane 0's view of the barrier and of the clock is the warp's: control flow stays uniform)
+        if (!w.done && pn < R_NSLOT && __shfl_sync(0xffffffffu, (int)bar_test(&sm->empty[slot], par ^ 1u), 0)) {
+            const unsigned bbytes = (unsigned)(w.g1 - w.g0) * 128u;
+            if (lane == 0) bar_expect(&sm->full[slot], (unsigned)w.kbs * (bbytes + abytes));
+            __syncwarp();
+            if (lane < w.kbs)
+                bulk_g2s_stream(ring + (size_t)slot * R_SLOT + (size_t)lane * w.stride + abytes + (size_t)(w.g0 - w.a0) * 128,
+                                w.W + w.wbase + (size_t)(w.kb0 + lane) * w.wstep, bbytes, &sm->full[slot], policy);
+            used |= 1u << slot;
+            used_par = (used_par & ~(1u << slot)) | (par << slot);
+            ++pn;
+            if (++slot == R_NSLOT) { slot = 0; par ^= 1u; }
+            w.advance();
+            progress = true;
+        }
+        if (progress) {
+            t_idle = 0;
+            n_idle = 0;
+        } else if ((++n_idle & 255u) == 0u) {
+            const unsigned long long now = __shfl_sync(0xffffffffu, gtime_ns(), 0);
+            if (t_idle == 0) t_idle = now;
+            else if (now - t_idle > sm->wait_ns) {
+                if (lane == 0) {
+                    *(volatile int *)&sm->abort = 1;
+                    atomicOr(&a.st->err, 32);
+                }
+                break;
+            }
+        }
+        __syncwarp();
+    }
+    // After an abort some slots expect activation bytes that were never requested: their barrier cannot complete, but the
+    // weight copies still have to land before the CTA may exit.  A copy takes microseconds; wait a bounded moment.
+    if (*(volatile int *)&sm->abort) {
+        const unsigned long long t0 = gtime_ns();
+        while (gtime_ns() - t0 < 200000ull) {
+        }
+    } else {
+        for (int i = 0; i < R_NSLOT; ++i) {
+            if (used & (1u << i)) {
+                const unsigned long long t0 = gtime_ns();
+                while (!bar_try(&sm->full[i], (used_par >> i) & 1u))
+                    if (gtime_ns() - t0 > sm->wait_ns) break;
+            }
+        }
+    }
+}
+
+// The four multiply-adds of one 64-element k-block in one block of instructions (the issuing thread is the bottleneck
+// when a CTA's tile has few rows: the tensor core needs about 46 cycles for a small tile, a thread that computes
+// two descriptors and a predicate per instruction issues one in about 80).  Descriptors advance by 2 units of 16 bytes
+// per 16 elements of K; `acc` = 0 makes the first one overwrite the accumulator.
+__device__ __forceinline__ void umma_kblock(unsigned tmem_d, unsigned long long adesc, unsigned long long bdesc, unsigned idesc,
+                                            unsigned acc) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 q, 0, 0;\n\t"
+        "add.u64 a1, %1, 2;\n\tadd.u64 a2, %1, 4;\n\tadd.u64 a3, %1, 6;\n\t"
+        "add.u64 b1, %2, 2;\n\tadd.u64 b2, %2, 4;\n\tadd.u64 b3, %2, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %3, q;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %3, q;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %3, q;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+
+// ---- MMA issuer ------------------------------------------------------------------------------------------
+__device__ void mma_issuer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, unsigned tmem) {
+    Cursor c(a);
+    unsigned slot = 0, par = 0, n = 0;   // n: accumulation chains so far (buffer n & 1)
+    const unsigned long long desc0 = umma_desc(0);
+    const unsigned ars16 = (unsigned)c.ars * 8u;   // activation rows of a tile in 16-byte units
+    while (!c.done) {
+        const unsigned buf = n & 1u;
+        if (c.chain_first() && !r_wait(&sm->tempty[buf], ((n >> 1) & 1u) ^ 1u, sm, &a.st->err)) return;
+        if (!r_wait(&sm->full[slot], par, sm, &a.st->err)) return;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const unsigned idesc = umma_idesc(128, c.npad, a.f16);
+        const unsigned base = s_u32(ring + (size_t)slot * R_SLOT);
+        unsigned long long adesc = desc0 + (unsigned long long)((base & 0x3ffffu) >> 4);
+        const unsigned stride16 = c.stride >> 4;
+        const unsigned d_tmem = tmem + buf * 256u;
+        unsigned acc = c.chain_first() ? 0u : 1u;
+        for (int j = 0; j < c.kbs; ++j) {
+            umma_kblock(d_tmem, adesc, adesc + ars16, idesc, acc);
+            acc = 1u;
+            adesc += stride16;
+        }
+        umma_commit(&sm->empty[slot]);                     // the slot is free once these multiply-adds have read it
+        if (c.chain_last()) {
+            umma_commit(&sm->tfull[buf]);                  // ... and the accumulator buffer is complete
+            ++n;
+        }
+        if (++slot == R_NSLOT) { slot = 0; par ^= 1u; }
+        c.advance();
+    }
+}
+
+// ---- drain warps: accumulator -> registers, epilogue ---------------------------------------------------------
+// Drain warp dw (0..3) takes the 32-column chunks dw and dw + 4 of the tile (N <= 224: seven chunks).  Lane m of the
+// warp holds row m of D: lanes t < T the hi product of token t, lanes T + t its lo product.
+struct DrainState {
+    float ssq;                 // RESID: running sum of x^2 of this lane's token over the CTA's rows
+    ClHeadPartial run;         // HEAD: running softmax statistics of this lane's token
+};
+
+struct Group {
+    int g0, g1, a0, npad;
+};
+
+__device__ __forceinline__ void epilogue_chunk(const ClRowsArgs &a, int epi, int rows, const Group &s, int ji, int chunk,
+                                               const float (&acc)[32], int lane, RSmem *sm, DrainState &ds, int pos0) {
+    const int T = a.T, t = lane;
+    const bool tok = lane < T;
+    const float sc = (tok && epi != CL_VEPI_RESID) ? sm->scale[t] : 1.f;
+    const int row0 = s.a0 + chunk * 32;
+    if (epi == CL_VEPI_RESID) {
+        // the raw product of this CTA's K range goes to the workspace; resid_phase() adds the group's parts
+        float *wsrow = a.ws + ((size_t)blockIdx.x * CL_MAX_T + t) * R_MAXN + chunk * 32;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const float lo = __shfl_down_sync(0xffffffffu, acc[i], T);   // all lanes take part
+            if (tok && chunk * 32 + i < s.npad) wsrow[i] = acc[i] + lo;
+        }
+        return;
+    }
+    float prev = 0.f;   // SILU: the gate value of the pair (even column)
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const float lo = __shfl_down_sync(0xffffffffu, acc[i], T);   // all lanes take part
+        const int row = row0 + i;
+        const bool live = tok && row >= s.g0 && row < s.g1;
+        const float tot = acc[i] + lo;
+        if (epi == CL_VEPI_STORE) {
+            if (live) a.qkv[(size_t)t * rows + row] = sc * tot;
+        } else if (epi == CL_VEPI_SILU) {
+            const float v = sc * tot;
+            if (i & 1) {   // rows interleave gate (even) and up (odd); a0 is even, so pairs never straddle lanes or chunks
+                if (live) {
+                    const float h = prev / (1.f + expf(-prev)) * v;
+                    a_store_split(a.Ah, t, T, row >> 1, h, a.f16);
+                }
+            } else {
+                prev = v;
+            }
+        } else {
+            if (live) {
+                const float lg = fminf(fmaxf(sc * tot, -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
+                if (a.logits) a.logits[(size_t)t * a.V + row] = lg;
+                ds.run = rp_merge(ds.run, ClHeadPartial{lg, 1.f, 0.f, row});
+            }
+        }
+    }
+}
+
+// Drains every chain of job `ji` that this CTA has (it may own no row of the job) and runs the job's epilogue.
+__device__ void drain_job(const ClRowsArgs &a, RSmem *sm, unsigned tmem, int dw, int lane, int ji, Cursor &c, unsigned &n, int pos0) {
+    if (c.done || c.ji != ji) return;
+    const int epi = c.epi, rows = c.rows;
+    DrainState ds;
+    ds.ssq = 0.f;
+    ds.run = ClHeadPartial{0.f, 0.f, 0.f, 0x7fffffff};
+    bool job_done = false;
+    while (!job_done) {
+        // one group: the sum of its chains
+        float acc[2][32];
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[q][i] = 0.f;
+        const Group g{c.g0, c.g1, c.a0, c.npad};
+        for (;;) {
+            const bool chain_end = c.chain_last(), group_end = c.last();
+            job_done = c.job_last();
+            c.advance();
+            if (!chain_end) continue;   // the accumulator keeps summing in tensor memory
+            const unsigned buf = n & 1u;
+            const bool ok = r_wait(&sm->tfull[buf], (n >> 1) & 1u, sm, &a.st->err);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (ok) {
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int chunk = dw + 4 * q;
+                    if (chunk * 32 < g.npad) {   // uniform over the warp
+#pragma unroll
+                        for (int hlf = 0; hlf < 2; ++hlf) {
+                            float v[16];
+                            tmem_ld16(tmem + buf * 256u + (unsigned)(chunk * 32 + hlf * 16), v);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) acc[q][hlf * 16 + i] += v[i];
+                        }
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) bar_arrive(&sm->tempty[buf]);
+            ++n;
+            if (group_end) break;
+        }
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int chunk = dw + 4 * q;
+            if (chunk * 32 < g.npad) epilogue_chunk(a, epi, rows, g, ji, chunk, acc[q], lane, sm, ds, pos0);
+        }
+    }
+    // per-job reductions over the four drain warps (fixed order)
+    if (epi == CL_VEPI_RESID) {
+        // (nothing per job: resid_phase() follows)
+    } else if (epi == CL_VEPI_HEAD) {
+        if (lane < CL_SLOTS) sm->hp[dw][lane] = ds.run;
+        drain_sync();
+        if (dw == 0 && lane < a.T)
+            a.head_part[(size_t)blockIdx.x * CL_SLOTS + lane] =
+                rp_merge(rp_merge(sm->hp[0][lane], sm->hp[1][lane]), rp_merge(sm->hp[2][lane], sm->hp[3][lane]));
+        drain_sync();
+    }
+}
+
+// A CTA that owns no row of the LM head still has to publish neutral statistics (they are merged by CTA 0).
+__device__ void publish_neutral(const ClRowsArgs &a, int ji) {
+    const Job jb = job_of(a, ji);
+    int r0, r1;
+    rows_of(jb.rows, jb.unit, jb.split, r0, r1);
+    if (r0 < r1) return;
+    if (threadIdx.x < a.T && jb.epi == CL_VEPI_HEAD)
+        a.head_part[(size_t)blockIdx.x * CL_SLOTS + threadIdx.x] = ClHeadPartial{0.f, 0.f, 0.f, 0x7fffffff};
+}
+
+// Barrier of the `split` CTAs of a group (arrival counter per group, growing during a launch like the grid's).
+__device__ __forceinline__ void group_barrier(const ClRowsArgs &a, unsigned &target, RSmem *sm) {
+    worker_sync();
+    if (a.split > 1 && threadIdx.x == 0 && !*(volatile int *)&sm->abort) {
+        unsigned *bar = a.bar + 1 + blockIdx.x / a.split;
+        target += (unsigned)a.split;
+        __threadfence();
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
+        if ((int)(v - target) < 0) {
+            const unsigned long long t0 = gtime_ns();
+            unsigned i = 0;
+            do {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
+                if ((++i & 255u) == 0u) {
+                    if (*(volatile int *)&a.st->err || gtime_ns() - t0 > sm->wait_ns) {
+                        *(volatile int *)&sm->abort = 1;
+                        atomicOr(&a.st->err, 64);
+                        break;
+                    }
+                }
+            } while ((int)(v - target) < 0);
+        }
+    }
+    worker_sync();
+}
+
+// Second half of an output / down projection: the `split` CTAs of a group hold the products of their K ranges in the
+// workspace; after the group's barrier each of them takes a share of the group's rows, adds the parts in member order
+// (fixed: results do not depend on timing), and applies the epilogue, one thread per (token, row): residual add, the
+// next GEMM's operand rows hi/lo(x * gain), hidden tap, and this CTA's sum of x^2 per token.
+__device__ void resid_phase(const ClRowsArgs &a, int ji, int pos0, unsigned &grp_target, RSmem *sm) {
+    group_barrier(a, grp_target, sm);
+    const int T = a.T, l = ji >> 2, g = a.split, tid = threadIdx.x;
+    const Job jb = job_of(a, ji);
+    int r0, r1;
+    rows_of(jb.rows, jb.unit, g, r0, r1);
+    const int member = (int)blockIdx.x % g, first_cta = (int)blockIdx.x - member;
+    const ClRowsLayer &y = a.layers[l];
+    const bool attn_half = (ji & 3) == 1;
+    const float *gain = attn_half ? y.n2 : ((l + 1 < a.L) ? a.layers[l + 1].n1 : a.final_norm);
+    unsigned short *tap = (unsigned short *)(a.tap ? (attn_half ? y.tap0 : y.tap1) : nullptr);
+    float *sq = sm->wrec;   // [T][64] squares of this CTA's new residual values (the attention records are not in use now)
+    for (int t = tid; t < CL_SLOTS; t += RT) sm->red[0][t] = 0.f;
+    // the group's rows in tiles of at most R_MAXN rows, exactly as the GEMM cut them
+    for (int g0 = r0; g0 < r1;) {
+        const int a0 = g0 & ~7, g1 = min(r1, a0 + R_MAXN), n = g1 - g0;
+        const int q0 = g0 + n * member / g, q1 = g0 + n * (member + 1) / g;   // this CTA's share of the tile's rows
+        for (int c0 = q0; c0 < q1; c0 += 64) {                                // ... 64 rows at a time
+            const int nq = min(64, q1 - c0);
+            worker_sync();
+            for (int idx = tid; idx < T * nq; idx += RT) {
+                const int t = idx / nq, i = idx % nq, row = c0 + i;
+                float parts[8];
+#pragma unroll
+                for (int m = 0; m < 8; ++m)
+                    parts[m] = m < g ? __ldcg(a.ws + ((size_t)(first_cta + m) * CL_MAX_T + t) * R_MAXN + (row - a0)) : 0.f;
+                float sum = parts[0];
+#pragma unroll
+                for (int m = 1; m < 8; ++m)
+                    if (m < g) sum += parts[m];
+                float *xp = a.x + (size_t)t * a.d + row;
+                const float xn = __ldcg(xp) + sum;
+                *xp = xn;
+                a_store_split(a.Ax, t, T, row, xn * __ldg(gain + row), a.f16);
+                if (tap && t + a.tap_P >= T)   // (slot = position mod P: of rows that share a slot the last one stays)
+                    tap[(size_t)((pos0 + t) % a.tap_P) * a.d + row] = f32_to_b16(xn, a.f16);
+                sq[t * 64 + i] = xn * xn;
+            }
+            worker_sync();
+            if (tid < T) {
+                float ss = sm->red[0][tid];
+                for (int i = 0; i < nq; ++i) ss += sq[tid * 64 + i];
+                sm->red[0][tid] = ss;
+            }
+        }
+        g0 = g1;
+    }
+    worker_sync();
+    if (tid < T) a.ssq[(size_t)blockIdx.x * CL_SLOTS + tid] = sm->red[0][tid];
+}
+
+// RMSNorm scale of every token row from the per-CTA sums of squares (fixed order: lane-strided, then a shuffle tree).
+__device__ void compute_scales(const ClRowsArgs &a, RSmem *sm) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp < a.T) {
+        float ss = 0.f;
+        for (int c = lane; c < (int)gridDim.x; c += 32) ss += __ldcg(a.ssq + (size_t)c * CL_SLOTS + warp);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) sm->scale[warp] = 1.0f / sqrtf(ss * a.inv_d + a.eps);
+    }
+    worker_sync();
+}
+
+// ---- embedding phase: x[t] = E[token t]; first operand hi/lo(x * g); per-CTA sums of squares ---------------------
+__device__ void embed_phase(const ClRowsArgs &a, RSmem *sm) {
+    const int T = a.T, nch = a.d >> 3, tid = threadIdx.x;
+    const float *g = a.L ? a.layers[0].n1 : a.final_norm;
+    const int per = (nch + gridDim.x - 1) / gridDim.x;   // chunks of 8 columns per CTA (at most 16)
+    for (int idx = tid; idx < 16 * CL_SLOTS; idx += RT) sm->esum[idx / CL_SLOTS][idx % CL_SLOTS] = 0.f;
+    worker_sync();
+    for (int idx = tid; idx < per * T; idx += RT) {
+        const int i = idx / T, t = idx % T, ch = (int)blockIdx.x + i * (int)gridDim.x;
+        if (ch < nch) {
+            const int tok = a.tok[t];
+            const uint4 raw = *(const uint4 *)((const unsigned short *)a.embed + (size_t)tok * a.d + ch * 8);
+            const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) pair16_to_f32(u[e], a.f16, v[2 * e], v[2 * e + 1]);
+            float4 *xp = (float4 *)(a.x + (size_t)t * a.d + ch * 8);
+            xp[0] = make_float4(v[0], v[1], v[2], v[3]);
+            xp[1] = make_float4(v[4], v[5], v[6], v[7]);
+            float ss = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                ss = fmaf(v[e], v[e], ss);
+                a_store_split(a.Ax, t, T, ch * 8 + e, v[e] * g[ch * 8 + e], a.f16);
+            }
+            sm->esum[i][t] = ss;
+        }
+    }
+    worker_sync();
+    if (tid < T) {
+        float ss = 0.f;
+        for (int i = 0; i < per; ++i) ss += sm->esum[i][tid];
+        a.ssq[(size_t)blockIdx.x * CL_SLOTS + tid] = ss;
+    }
+}
+
+// ---- attention of the T rows over the cache ------------------------------------------------------------------
+// Work item (head h, part s of the cached keys [0, base)) -> one CTA.  Inside the CTA warp w serves token row
+// t = w / nsub and the sub-range sub = w % nsub of the part's keys (nsub = 14 / T warps per row).  A warp walks its
+// keys 32 at a time with an online softmax (scores reduced with warp shuffles).  The rows' own keys and values
+// (positions base .. base + t, causal) come raw from the QKV product: the last warp of row t in the last part
+// rotates each key, rounds key and value to the storage type and folds them in; the warp of the last row also
+// appends them to the cache (one query head per key/value head).  The CTA merges its warps per row and writes one
+// record per (h, s, t); the last CTA of a head to finish (ticket) merges the parts in order and writes the
+// normalised output as the output projection's hi/lo operand rows.
+template <typename ST, int HD>
+__device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int base, RSmem *sm) {
+    constexpr int EPL = 8, LPK = HD / EPL, KPW = 32 / LPK, VPL = HD / 32, WSTRIDE = HD + 2, HALF = HD / 2;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int T = a.T, S = a.att_parts, nsub = RW / T;
+    const int t = warp / nsub, sub = warp % nsub;
+    const bool active = warp < T * nsub;
+    const int li = lane % LPK, ksub = lane / LPK;
+    const float scale = rsqrtf((float)HD);
+    const int group = a.H / a.Hkv, kvd = a.Hkv * HD, ld = a.d + 2 * kvd;
+    ST *Kc = (ST *)y.kc, *Vc = (ST *)y.vc;
+    float *wrec = sm->wrec;
+    for (int item = blockIdx.x; item < a.H * S; item += gridDim.x) {
+        const int h = item % a.H, s = item / a.H, kvh = h / group;
+        float m_run = -INFINITY, l_run = 0.f, o_run[VPL];
+#pragma unroll
+        for (int e = 0; e < VPL; ++e) o_run[e] = 0.f;
+        if (active) {
+            const int pos = base + t;
+            const float *qraw = a.qkv + (size_t)t * ld + h * HD;
+            float qr[EPL];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                const int idx = li * EPL + e;
+                const int i = idx < HALF ? idx : idx - HALF;
+                const float2 cs = a.rope_cs[(size_t)pos * HALF + i];
+                const float qa = __ldcg(qraw + i), qb = __ldcg(qraw + i + HALF);
+                qr[e] = idx < HALF ? qa * cs.x - qb * cs.y : qb * cs.x + qa * cs.y;
+            }
+            const int k0 = (int)((long long)base * s / S), k1 = (int)((long long)base * (s + 1) / S);
+            const int kw0 = k0 + (int)((long long)(k1 - k0) * sub / nsub), kw1 = k0 + (int)((long long)(k1 - k0) * (sub + 1) / nsub);
+            const ST *Kh = Kc + (size_t)kvh * a.max_seq * HD, *Vh = Vc + (size_t)kvh * a.max_seq * HD;
+            for (int j0 = kw0; j0 < kw1; j0 += 32) {
+                const int n = min(32, kw1 - j0);
+                float my_score = -INFINITY;
+                constexpr int NPASS = 32 / KPW, PB = NPASS < 8 ? NPASS : 8;
+#pragma unroll
+                for (int b0 = 0; b0 < NPASS; b0 += PB) {
+                    if (b0 * KPW >= n) break;   // uniform
+                    uint4 raw[PB];
+#pragma unroll
+                    for (int p = 0; p < PB; ++p) {
+                        const int j = (b0 + p) * KPW + ksub;
+                        raw[p] = make_uint4(0u, 0u, 0u, 0u);
+                        if (j < n) raw[p] = __ldg((const uint4 *)(Kh + (size_t)(j0 + j) * HD + li * EPL));
+                    }
+#pragma unroll
+                    for (int p = 0; p < PB; ++p) {
+                        const int jb = (b0 + p) * KPW;
+                        if (jb < n) {   // uniform
+                            const unsigned u[4] = {raw[p].x, raw[p].y, raw[p].z, raw[p].w};
+                            float sc = 0.f;
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                float ka, kb;
+                                ClPair16<ST>::get(u[e], ka, kb);
+                                sc = fmaf(qr[2 * e], ka, sc);
+                                sc = fmaf(qr[2 * e + 1], kb, sc);
+                            }
+#pragma unroll
+                            for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                            sc *= scale;
+#pragma unroll
+                            for (int k = 0; k < KPW; ++k) {
+                                const float v = __shfl_sync(0xffffffffu, sc, k * LPK);
+                                if (lane == jb + k && jb + k < n) my_score = v;
+                            }
+                        }
+                    }
+                }
+                float m_new = my_score;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) m_new = fmaxf(m_new, __shfl_xor_sync(0xffffffffu, m_new, o));
+                m_new = fmaxf(m_new, m_run);
+                const float p = (lane < n) ? expf(my_score - m_new) : 0.f;
+                const float resc = (l_run > 0.f) ? expf(m_run - m_new) : 0.f;
+                float ps = p;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+                l_run = fmaf(l_run, resc, ps);
+#pragma unroll
+                for (int e = 0; e < VPL; ++e) o_run[e] *= resc;
+                m_run = m_new;
+#pragma unroll
+                for (int jg = 0; jg < 32; jg += 8) {
+                    if (jg >= n) break;   // uniform
+                    float vv[8][VPL];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const ST *vp = Vh + (size_t)(j0 + min(jg + j, n - 1)) * HD + lane * VPL;
+                        if (VPL == 4) {
+                            const uint2 u = __ldg((const uint2 *)vp);
+                            ClPair16<ST>::get(u.x, vv[j][0], vv[j][1 % VPL]);
+                            ClPair16<ST>::get(u.y, vv[j][2 % VPL], vv[j][3 % VPL]);
+                        } else {
+                            const unsigned u = __ldg((const unsigned *)vp);
+                            ClPair16<ST>::get(u, vv[j][0], vv[j][1 % VPL]);
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float pj = __shfl_sync(0xffffffffu, p, jg + j);
+#pragma unroll
+                        for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(pj, vv[j][e], o_run[e]);
+                    }
+                }
+            }
+            if (s == S - 1 && sub == nsub - 1) {
+                // the pass's own positions base .. base + t
+                const bool writer = (t == T - 1) && (h % group) == 0;
+                for (int jn = 0; jn <= t; ++jn) {
+                    const float *kraw = a.qkv + (size_t)jn * ld + a.d + kvh * HD, *vraw = kraw + kvd;
+                    float sc = 0.f;
+                    unsigned short kst[EPL];
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) {
+                        const int idx = li * EPL + e;
+                        const int i = idx < HALF ? idx : idx - HALF;
+                        const float2 cs = a.rope_cs[(size_t)(base + jn) * HALF + i];
+                        const float ka = __ldcg(kraw + i), kb = __ldcg(kraw + i + HALF);
+                        kst[e] = f32_to_b16(idx < HALF ? ka * cs.x - kb * cs.y : kb * cs.x + ka * cs.y, a.f16);
+                        sc = fmaf(qr[e], b16_to_f32(kst[e], a.f16), sc);
+                    }
+#pragma unroll
+                    for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                    sc = __shfl_sync(0xffffffffu, sc, 0) * scale;
+                    if (ksub == 0 && writer) {
+                        unsigned short *kd = (unsigned short *)Kc + ((size_t)kvh * a.max_seq + base + jn) * HD + li * EPL;
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) kd[e] = kst[e];
+                    }
+                    float vn[VPL];
+#pragma unroll
+                    for (int e = 0; e < VPL; ++e) {
+                        const unsigned short vs = f32_to_b16(__ldcg(vraw + lane * VPL + e), a.f16);
+                        if (writer) ((unsigned short *)Vc)[((size_t)kvh * a.max_seq + base + jn) * HD + lane * VPL + e] = vs;
+                        vn[e] = b16_to_f32(vs, a.f16);
+                    }
+                    const float m_new = fmaxf(m_run, sc);
+                    const float resc = (l_run > 0.f) ? expf(m_run - m_new) : 0.f;
+                    const float pn = expf(sc - m_new);
+                    l_run = fmaf(l_run, resc, pn);
+#pragma unroll
+                    for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(o_run[e], resc, pn * vn[e]);
+                    m_run = m_new;
+                }
+            }
+        }
+        if (lane == 0) {
+            wrec[warp * WSTRIDE] = m_run;
+            wrec[warp * WSTRIDE + 1] = l_run;
+        }
+#pragma unroll
+        for (int e = 0; e < VPL; ++e) wrec[warp * WSTRIDE + 2 + lane * VPL + e] = o_run[e];
+        worker_sync();
+        // merge the nsub warps of every row (fixed order); one record per (h, s, t), or the final output if S == 1
+        float *part = a.att_part + ((size_t)h * R_ATT_MAXS + s) * CL_MAX_T * WSTRIDE;
+        for (int i = tid; i < T * HD; i += RT) {
+            const int tt = i / HD, e = i % HD;
+            float M = -INFINITY;
+            for (int w = 0; w < nsub; ++w) {
+                const float *r = wrec + (tt * nsub + w) * WSTRIDE;
+                if (r[1] > 0.f) M = fmaxf(M, r[0]);
+            }
+            float Ls = 0.f, O = 0.f;
+            for (int w = 0; w < nsub; ++w) {
+                const float *r = wrec + (tt * nsub + w) * WSTRIDE;
+                if (r[1] > 0.f) {
+                    const float f = expf(r[0] - M);
+                    Ls = fmaf(r[1], f, Ls);
+                    O = fmaf(r[2 + e], f, O);
+                }
+            }
+            if (S == 1) {
+                a_store_split(a.Aatt, tt, T, h * HD + e, O / Ls, a.f16);
+            } else {
+                float *rec = part + (size_t)tt * WSTRIDE;
+                if (e == 0) { rec[0] = M; rec[1] = Ls; }
+                rec[2 + e] = O;
+            }
+        }
+        if (S > 1) {
+            worker_sync();
+            if (tid == 0) {
+                const unsigned prev = ticket_acq_rel(a.att_tickets + h);
+                const int last = prev == (unsigned)S - 1;
+                if (last) a.att_tickets[h] = 0u;
+                sm->is_last = last;
+            }
+            worker_sync();
+            if (sm->is_last) {
+                const float *p0 = a.att_part + (size_t)h * R_ATT_MAXS * CL_MAX_T * WSTRIDE;
+                for (int i = tid; i < T * HD; i += RT) {
+                    const int tt = i / HD, e = i % HD;
+                    float pm[R_ATT_MAXS], pl[R_ATT_MAXS], po[R_ATT_MAXS];
+#pragma unroll
+                    for (int s2 = 0; s2 < R_ATT_MAXS; ++s2) {
+                        const float *ps = p0 + ((size_t)min(s2, S - 1) * CL_MAX_T + tt) * WSTRIDE;
+                        pm[s2] = __ldcg(ps);
+                        pl[s2] = (s2 < S) ? __ldcg(ps + 1) : 0.f;
+                        po[s2] = __ldcg(ps + 2 + e);
+                    }
+                    float M = -INFINITY;
+#pragma unroll
+                    for (int s2 = 0; s2 < R_ATT_MAXS; ++s2)
+                        if (pl[s2] > 0.f) M = fmaxf(M, pm[s2]);
+                    float Ls = 0.f, O = 0.f;
+#pragma unroll
+                    for (int s2 = 0; s2 < R_ATT_MAXS; ++s2) {   // part order
+                        if (pl[s2] > 0.f) {
+                            const float f = expf(pm[s2] - M);
+                            Ls = fmaf(pl[s2], f, Ls);
+                            O = fmaf(po[s2], f, O);
+                        }
+                    }
+                    a_store_split(a.Aatt, tt, T, h * HD + e, O / Ls, a.f16);
+                }
+            }
+        }
+        worker_sync();
+    }
+}
+
+// ---- the kernel ---------------------------------------------------------------------------------------------
+template <typename ST, int HD>
+__global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constant__ ClRowsArgs a) {
+    if (a.st->done) return;   // written only between launches: uniform over the grid
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *ring = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // the control block sits behind the ring: the M = 128 operand descriptor of the last tile reads up to 16 KB past
+    // its activation rows, which must stay inside this CTA's shared memory
+    RSmem *sm = (RSmem *)(ring + (size_t)R_NSLOT * R_SLOT);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int i = 0; i < R_NSLOT; ++i) {
+            bar_init(&sm->full[i], 1);
+            bar_init(&sm->empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            bar_init(&sm->tfull[i], 1);
+            bar_init(&sm->tempty[i], 4);
+        }
+        sm->abort = 0;
+        sm->bars_done = 0;
+        sm->wait_ns = a.wait_ns;
+        for (int i = 0; i < 8; ++i) sm->ph_ns[i] = 0ull;
+        sm->t_prev = gtime_ns();
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == RW + 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(s_u32(&sm->tmem_base)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem = *(volatile unsigned *)&sm->tmem_base;
+
+    if (warp == RW) {
+        producer(a, ring, sm, lane);
+    } else if (warp == RW + 1) {
+        if (lane == 0) mma_issuer(a, ring, sm, tmem);
+    } else {
+        const int base = a.st->ctx + a.row0;   // position of row 0
+        const bool drains = (warp & 3) == 0;
+        const int dw = warp >> 2;
+        unsigned bar_target = 0u, grp_target = 0u, n_acc = 0u;
+        int passed = 0;
+        Cursor cur(a);
+        embed_phase(a, sm);
+        phase_clock(a, sm, 0);
+        grid_barrier(a, bar_target, passed, sm);
+        for (int l = 0; l < a.L; ++l) {
+            const ClRowsLayer &y = a.layers[l];
+            compute_scales(a, sm);
+            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * l, cur, n_acc, base);
+            phase_clock(a, sm, 1);
+            grid_barrier(a, bar_target, passed, sm);
+            attention_phase<ST, HD>(a, y, base, sm);
+            phase_clock(a, sm, 2);
+            grid_barrier(a, bar_target, passed, sm);
+            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * l + 1, cur, n_acc, base);
+            resid_phase(a, 4 * l + 1, base, grp_target, sm);
+            phase_clock(a, sm, 3);
+            grid_barrier(a, bar_target, passed, sm);
+            compute_scales(a, sm);
+            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * l + 2, cur, n_acc, base);
+            phase_clock(a, sm, 4);
+            grid_barrier(a, bar_target, passed, sm);
+            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * l + 3, cur, n_acc, base);
+            resid_phase(a, 4 * l + 3, base, grp_target, sm);
+            phase_clock(a, sm, 5);
+            grid_barrier(a, bar_target, passed, sm);
+        }
+        if (a.want_head) {
+            compute_scales(a, sm);
+            publish_neutral(a, 4 * a.L);
+            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * a.L, cur, n_acc, base);
+            phase_clock(a, sm, 6);
+            grid_barrier(a, bar_target, passed, sm);
+            // CTA 0 merges the per-CTA statistics of every token row (one warp per row, fixed order): Eq. 1-4
+            if (blockIdx.x == 0 && warp < a.T) {
+                ClHeadPartial p{0.f, 0.f, 0.f, 0x7fffffff};
+                for (int c = lane; c < (int)gridDim.x; c += 32) {
+                    const ClHeadPartial *src = a.head_part + (size_t)c * CL_SLOTS + warp;
+                    ClHeadPartial q;
+                    q.m = __ldcg(&src->m); q.z = __ldcg(&src->z); q.s = __ldcg(&src->s); q.idx = __ldcg(&src->idx);
+                    p = rp_merge(p, q);
+                }
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const ClHeadPartial other = cl_hp_shfl_xor(p, o);
+                    p = ((lane & o) == 0) ? rp_merge(p, other) : rp_merge(other, p);
+                }
+                if (lane == 0) {
+                    const float H = logf(p.z) - p.s / p.z;
+                    if (a.out_tok) a.out_tok[warp] = min(max(p.idx, 0), a.V - 1);
+                    if (a.out_pmax) a.out_pmax[warp] = 1.f / p.z;
+                    if (a.out_conf) a.out_conf[warp] = 1.f - H * a.inv_log_v;
+                }
+            }
+        }
+    }
+    if (a.phase_ns && tid == 0)
+        for (int i = 0; i < 8; ++i) a.phase_ns[(size_t)blockIdx.x * 8 + i] = sm->ph_ns[i];
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == RW + 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    }
+}
+
+// ---- load-time re-layout: row-major [rows, K] -> the streaming order of this kernel: the row block of CTA 0, of
+// CTA 1, ...; inside a block [K / 64][block rows][64] elements with the 16-byte pieces of a row's 128 bytes permuted
+// by (piece ^ (row & 7)) -----------------------------------------------------------------------------------------
+__global__ void k_tile_layout(const uint4 *src, uint4 *dst, int rows, int KB, int unit, int G) {
+    const size_t total = (size_t)rows * KB * 8;
+    const long long units = rows / unit;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i & 7);
+        const size_t rk = i >> 3;
+        const int kb = (int)(rk % KB);
+        const int r = (int)(rk / KB);
+        int owner = (int)min((long long)G - 1, ((long long)(r / unit) + 1) * G / units);
+        int r0, r1;
+        rows_of_cta(rows, unit, owner, G, r0, r1);
+        while (r < r0) rows_of_cta(rows, unit, --owner, G, r0, r1);
+        while (r >= r1) rows_of_cta(rows, unit, ++owner, G, r0, r1);
+        dst[((size_t)r0 * KB + (size_t)kb * (r1 - r0) + (r - r0)) * 8 + (size_t)(c ^ (r & 7))] = src[i];
+    }
+}
+
+}  // namespace
+
+size_t cl_rows_smem_bytes() { return (size_t)R_NSLOT * R_SLOT + 16384 + 1024; }
+
+int cl_rows_att_part_floats(int H) { return H * R_ATT_MAXS * CL_MAX_T * (128 + 2); }
+
+cudaError_t cl_launch_tile_layout(const void *src, void *dst, int rows, int K, int unit, int grid, cudaStream_t s) {
+    k_tile_layout<<<1184, 256, 0, s>>>((const uint4 *)src, (uint4 *)dst, rows, K / 64, unit, grid);
+    return cudaGetLastError();
+}
+
+cudaError_t cl_launch_rows_pass(int wdtype, int head_dim, const ClRowsArgs &a, int grid, cudaStream_t s) {
+    static_assert(sizeof(RSmem) <= 16384, "control block must fit behind the ring");
+    const void *fn = nullptr;
+    if (wdtype == 1 && head_dim == 64) fn = (const void *)k_rows_pass<__nv_bfloat16, 64>;
+    else if (wdtype == 1 && head_dim == 128) fn = (const void *)k_rows_pass<__nv_bfloat16, 128>;
+    else if (wdtype == 2 && head_dim == 64) fn = (const void *)k_rows_pass<__half, 64>;
+    else if (wdtype == 2 && head_dim == 128) fn = (const void *)k_rows_pass<__half, 128>;
+    else return cudaErrorInvalidValue;
+    const size_t smem = cl_rows_smem_bytes();
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    void *params[] = {(void *)&a};
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(R_THREADS), params, smem, s);
+}

@@ -38,17 +38,6 @@ struct ScoreArgs {
     int f16;                        // 16-bit type of both operands: 0 bf16, 1 fp16
 };
 
-__device__ __forceinline__ ClHeadPartial sc_merge(const ClHeadPartial &a, const ClHeadPartial &b) {
-    if (b.z == 0.f) return a;
-    if (a.z == 0.f) return b;
-    ClHeadPartial r;
-    r.m = fmaxf(a.m, b.m);
-    const float ea = expf(a.m - r.m), eb = expf(b.m - r.m);
-    r.z = a.z * ea + b.z * eb;
-    r.s = ea * (a.s + (a.m - r.m) * a.z) + eb * (b.s + (b.m - r.m) * b.z);
-    r.idx = (a.m > b.m) ? a.idx : (b.m > a.m) ? b.idx : min(a.idx, b.idx);
-    return r;
-}
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_score(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, ScoreArgs a) {
@@ -205,7 +194,7 @@ __global__ void k_score_finalize(const ClHeadPartial *partials, int NCG, int R, 
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= R) return;
     ClHeadPartial f{0.f, 0.f, 0.f, 0x7fffffff};
-    for (int g = 0; g < NCG; ++g) f = sc_merge(f, partials[(size_t)r * NCG + g]);
+    for (int g = 0; g < NCG; ++g) f = cl_hp_merge(f, partials[(size_t)r * NCG + g]);
     const float H = logf(f.z) - f.s / f.z;   // entropy of the softmax from sums relative to the maximum
     conf[r] = 1.f - H * inv_log_v;
     pmax[r] = 1.f / f.z;

@@ -145,34 +145,13 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-__device__ __forceinline__ ClHeadPartial hp_merge(const ClHeadPartial &a, const ClHeadPartial &b) {
-    if (b.z == 0.f) return a;
-    if (a.z == 0.f) return b;
-    ClHeadPartial r;
-    r.m = fmaxf(a.m, b.m);
-    const float ea = expf(a.m - r.m), eb = expf(b.m - r.m);
-    r.z = a.z * ea + b.z * eb;
-    r.s = ea * (a.s + (a.m - r.m) * a.z) + eb * (b.s + (b.m - r.m) * b.z);
-    r.idx = (a.m > b.m) ? a.idx : (b.m > a.m) ? b.idx : min(a.idx, b.idx);
-    return r;
-}
-
-__device__ __forceinline__ ClHeadPartial hp_shfl_xor(const ClHeadPartial &a, int o) {
-    ClHeadPartial r;
-    r.m = __shfl_xor_sync(0xffffffffu, a.m, o);
-    r.z = __shfl_xor_sync(0xffffffffu, a.z, o);
-    r.s = __shfl_xor_sync(0xffffffffu, a.s, o);
-    r.idx = __shfl_xor_sync(0xffffffffu, a.idx, o);
-    return r;
-}
-
 // Fixed-order reduction of one ClHeadPartial per consumer thread; result valid in every thread.
 __device__ ClHeadPartial hp_block_reduce(ClHeadPartial v, Smem *sm) {
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        const ClHeadPartial other = hp_shfl_xor(v, o);
+        const ClHeadPartial other = cl_hp_shfl_xor(v, o);
         // combine in a lane-independent order so every lane ends with identical bits
-        v = ((threadIdx.x & o) == 0) ? hp_merge(v, other) : hp_merge(other, v);
+        v = ((threadIdx.x & o) == 0) ? cl_hp_merge(v, other) : cl_hp_merge(other, v);
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     consumer_sync();
@@ -180,7 +159,7 @@ __device__ ClHeadPartial hp_block_reduce(ClHeadPartial v, Smem *sm) {
     consumer_sync();
     ClHeadPartial r = sm->hp[0];
 #pragma unroll
-    for (int w = 1; w < NCW; ++w) r = hp_merge(r, sm->hp[w]);
+    for (int w = 1; w < NCW; ++w) r = cl_hp_merge(r, sm->hp[w]);
     return r;
 }
 
@@ -1003,7 +982,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             for (int r = tid; r < nrb; r += NCT) {
                 const float l = fminf(fmaxf(row_sum(sm, r), -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
                 if (lg) lg[rb0 + r] = l;
-                run = hp_merge(run, ClHeadPartial{l, 1.f, 0.f, rb0 + r});
+                run = cl_hp_merge(run, ClHeadPartial{l, 1.f, 0.f, rb0 + r});
             }
         }, a.cum_w, busy_p);
         run = hp_block_reduce(run, sm);
@@ -1015,7 +994,7 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
             const ClHeadPartial *p = a.head_part + b;
             ClHeadPartial q;
             q.m = ldcg_f(&p->m); q.z = ldcg_f(&p->z); q.s = ldcg_f(&p->s); q.idx = __ldcg(&p->idx);
-            fin = hp_merge(fin, q);
+            fin = cl_hp_merge(fin, q);
         }
         fin = hp_block_reduce(fin, sm);
         tok = min(max(fin.idx, 0), V - 1);   // (only an aborted run can leave the range; keep the next gather in bounds)

@@ -263,12 +263,13 @@ def test_tensor_core_pass_matches_streaming_pass(monkeypatch, wd):
     prompt = synth.make_prompt(5, 11, sh.vocab)                        # a full chunk of 8 and a ragged one of 3
     out = {}
     for tc in (0, 1):
+        monkeypatch.setenv("CL_DISABLE_ROWS_KERNEL", "0" if tc else "1")
         monkeypatch.setenv("CL_DISABLE_TC_PASS", "0" if tc else "1")
         ctx = cl.Context.from_shape(sh, tap_positions=16)               # longer than any pass: no two rows share a slot
         ctx.cl_load(W)
         first = ctx.cl_prefill(prompt, tap_hidden=True)
         res = [first]
-        for drafts in ([11, 22, 33, 44], [5, 6, 7, 8, 9, 10, 11, 12]):
+        for drafts in ([11, 22, 33, 44], [5, 6, 7, 8, 9, 10, 11, 12], [3], []):
             ctx.cl_rollback(len(prompt), first)
             ctx.cl_force_tokens(drafts)
             v = ctx.cl_verify(len(drafts) + 1, tap_hidden=True, want_logits=True)
@@ -277,11 +278,13 @@ def test_tensor_core_pass_matches_streaming_pass(monkeypatch, wd):
         out[tc] = res
         ctx.close()
     assert out[0][0] == out[1][0]
-    for i in (1, 2):
+    for i in (1, 2, 3, 4):
         assert np.abs(out[0][i][1] - out[1][i][1]).max() <= 2e-3        # both far inside the 1e-2 tolerance
-        assert np.array_equal(out[0][i][0], out[1][i][0])
-    scale = max(1.0, float(np.abs(out[0][3]).max()))
-    assert np.abs(out[0][3] - out[1][3]).max() <= 2 ** -7 * scale        # taps: one bf16 ulp at the top of the range
+        top2 = np.sort(out[0][i][1], axis=1)[:, -2:]
+        clear = (top2[:, 1] - top2[:, 0]) >= NEAR_TIE
+        assert np.array_equal(out[0][i][0][clear], out[1][i][0][clear])
+    scale = max(1.0, float(np.abs(out[0][5]).max()))
+    assert np.abs(out[0][5] - out[1][5]).max() <= 2 ** -7 * scale        # taps: one bf16 ulp at the top of the range
 
 
 @pytest.mark.parametrize("wd", ["bf16", "fp16"])
