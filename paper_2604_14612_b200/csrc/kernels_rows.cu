@@ -33,6 +33,7 @@
 // Every wait is bounded; on expiry an error flag is raised, later waits fall through, copies in flight are waited
 // for, tensor memory is released and the host reports CL_ETIMEOUT.
 #include <math.h>
+#include <stddef.h>
 #include <string.h>
 
 #include "tc_common.cuh"
@@ -45,7 +46,11 @@ constexpr int R_THREADS = RT + 64;     // + producer warp + MMA warp
 constexpr int R_SLOT = 32768;          // ring slot
 constexpr int R_NSLOT = 6;             // 192 KB of tiles in flight per SM
 constexpr int R_MAXN = 224;            // most rows of a weight tile (tile + activation rows fill a slot at one k-block)
+constexpr int R_CTRL_BYTES = 16384;    // control block behind the ring (at least 16 KB: see the kernel)
 constexpr int R_ATT_MAXS = 8;          // most parts the cached keys of a head are cut into
+
+constexpr int R_STAGE_LD = R_MAXN + 1;  // row pitch of the epilogue staging buffer (odd: token rows fall into different banks)
+constexpr int R_STAGE_FLOATS = 2032;   // staging buffer: a GEMM tile's raw products of every token row
 
 struct RSmem {
     unsigned long long full[R_NSLOT], empty[R_NSLOT], tfull[2], tempty[2];
@@ -55,10 +60,12 @@ struct RSmem {
     int bars_done;                     // grid barriers this CTA has passed (read by the producer)
     int is_last;
     float scale[CL_SLOTS];             // RMSNorm scale of every token row for the current phase
-    float red[4][CL_SLOTS];
+    float red[CL_SLOTS];
     float esum[16][CL_SLOTS];          // embedding phase: per-chunk sums of squares
-    ClHeadPartial hp[4][CL_SLOTS];
-    float wrec[RW * (128 + 2)];        // attention: per-warp (max, sum, o[hd]) records
+    ClHeadPartial hpw[RW];             // LM head: per-warp statistics
+    // one buffer, used in turn by: the GEMM epilogues (raw products of a tile, [T][R_STAGE_LD]); the residual epilogue
+    // ([T][64] squares); the attention phase (per-warp (max, sum, o[hd]) records, [RW][hd + 2])
+    alignas(16) float stage[R_STAGE_FLOATS];
     unsigned long long t_prev, ph_ns[8];   // diagnostics: time of thread 0 by phase
 };
 
@@ -430,135 +437,126 @@ __device__ void mma_issuer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, 
     }
 }
 
-// ---- drain warps: accumulator -> registers, epilogue ---------------------------------------------------------
+// ---- GEMM jobs on the worker side: drain the accumulator, epilogue ------------------------------------------------
 // Drain warp dw (0..3) takes the 32-column chunks dw and dw + 4 of the tile (N <= 224: seven chunks).  Lane m of the
-// warp holds row m of D: lanes t < T the hi product of token t, lanes T + t its lo product.
-struct DrainState {
-    float ssq;                 // RESID: running sum of x^2 of this lane's token over the CTA's rows
-    ClHeadPartial run;         // HEAD: running softmax statistics of this lane's token
-};
-
+// warp holds row m of D: lanes t < T the hi product of token t, lanes T + t its lo product.  The sums hi + lo of a
+// finished tile go to a staging buffer in shared memory (to the workspace in global memory for an output / down
+// projection, whose epilogue follows the group's barrier); then all worker warps apply the epilogue, whole warps per
+// token row:
+//   STORE  qkv[t, r] = s_t * acc                     (s_t = RMSNorm scale of token t)
+//   SILU   rows interleave gate / up: h = silu(s_t g) * (s_t u) -> hi/lo(h), the down projection's operand
+//   HEAD   logits = clamp(s_t * acc) -> running softmax statistics and argmax per token (Eq. 1-4)
 struct Group {
     int g0, g1, a0, npad;
 };
 
-__device__ __forceinline__ void epilogue_chunk(const ClRowsArgs &a, int epi, int rows, const Group &s, int ji, int chunk,
-                                               const float (&acc)[32], int lane, RSmem *sm, DrainState &ds, int pos0) {
-    const int T = a.T, t = lane;
-    const bool tok = lane < T;
-    const float sc = (tok && epi != CL_VEPI_RESID) ? sm->scale[t] : 1.f;
-    const int row0 = s.a0 + chunk * 32;
-    if (epi == CL_VEPI_RESID) {
-        // the raw product of this CTA's K range goes to the workspace; resid_phase() adds the group's parts
-        float *wsrow = a.ws + ((size_t)blockIdx.x * CL_MAX_T + t) * R_MAXN + chunk * 32;
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            const float lo = __shfl_down_sync(0xffffffffu, acc[i], T);   // all lanes take part
-            if (tok && chunk * 32 + i < s.npad) wsrow[i] = acc[i] + lo;
-        }
-        return;
-    }
-    float prev = 0.f;   // SILU: the gate value of the pair (even column)
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const float lo = __shfl_down_sync(0xffffffffu, acc[i], T);   // all lanes take part
-        const int row = row0 + i;
-        const bool live = tok && row >= s.g0 && row < s.g1;
-        const float tot = acc[i] + lo;
-        if (epi == CL_VEPI_STORE) {
-            if (live) a.qkv[(size_t)t * rows + row] = sc * tot;
-        } else if (epi == CL_VEPI_SILU) {
-            const float v = sc * tot;
-            if (i & 1) {   // rows interleave gate (even) and up (odd); a0 is even, so pairs never straddle lanes or chunks
-                if (live) {
-                    const float h = prev / (1.f + expf(-prev)) * v;
-                    a_store_split(a.Ah, t, T, row >> 1, h, a.f16);
-                }
-            } else {
-                prev = v;
-            }
-        } else {
-            if (live) {
-                const float lg = fminf(fmaxf(sc * tot, -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
-                if (a.logits) a.logits[(size_t)t * a.V + row] = lg;
-                ds.run = rp_merge(ds.run, ClHeadPartial{lg, 1.f, 0.f, row});
-            }
-        }
-    }
-}
-
-// Drains every chain of job `ji` that this CTA has (it may own no row of the job) and runs the job's epilogue.
-__device__ void drain_job(const ClRowsArgs &a, RSmem *sm, unsigned tmem, int dw, int lane, int ji, Cursor &c, unsigned &n, int pos0) {
-    if (c.done || c.ji != ji) return;
-    const int epi = c.epi, rows = c.rows;
-    DrainState ds;
-    ds.ssq = 0.f;
-    ds.run = ClHeadPartial{0.f, 0.f, 0.f, 0x7fffffff};
+// All worker warps call this with the same cursor state.  `run` carries a thread's LM-head statistics across tiles.
+__device__ __forceinline__ void gemm_job(const ClRowsArgs &a, RSmem *sm, unsigned tmem, int ji, Cursor &c, unsigned &n, ClHeadPartial &run) {
+    if (c.done || c.ji != ji) return;   // this CTA has no part in the job
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool drains = (warp & 3) == 0;
+    const int dw = warp >> 2;
+    const int T = a.T, epi = c.epi, rows = c.rows;
+    const int wpt = RW / T;                                  // warps per token row in the epilogue
+    const int et = warp / wpt, ej = (warp % wpt) * 32 + lane, estride = wpt * 32;
     bool job_done = false;
     while (!job_done) {
-        // one group: the sum of its chains
-        float acc[2][32];
-#pragma unroll
-        for (int q = 0; q < 2; ++q)
-#pragma unroll
-            for (int i = 0; i < 32; ++i) acc[q][i] = 0.f;
         const Group g{c.g0, c.g1, c.a0, c.npad};
-        for (;;) {
-            const bool chain_end = c.chain_last(), group_end = c.last();
+        // walk the tile's slots first (an accumulation chain ends every a.chain slots and at the tile's end), so that
+        // no schedule arithmetic runs while the accumulator registers are live
+        int nchains = 0;
+        for (bool group_end = false; !group_end;) {
+            nchains += c.chain_last() ? 1 : 0;
+            group_end = c.last();
             job_done = c.job_last();
             c.advance();
-            if (!chain_end) continue;   // the accumulator keeps summing in tensor memory
-            const unsigned buf = n & 1u;
-            const bool ok = r_wait(&sm->tfull[buf], (n >> 1) & 1u, sm, &a.st->err);
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (ok) {
+        }
+        float acc[2][32];
+        if (drains) {
 #pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    const int chunk = dw + 4 * q;
-                    if (chunk * 32 < g.npad) {   // uniform over the warp
+            for (int q = 0; q < 2; ++q)
 #pragma unroll
-                        for (int hlf = 0; hlf < 2; ++hlf) {
-                            float v[16];
-                            tmem_ld16(tmem + buf * 256u + (unsigned)(chunk * 32 + hlf * 16), v);
+                for (int i = 0; i < 32; ++i) acc[q][i] = 0.f;
+            for (int ch = 0; ch < nchains; ++ch) {
+                const unsigned buf = (n + ch) & 1u;
+                const bool ok = r_wait(&sm->tfull[buf], ((n + ch) >> 1) & 1u, sm, &a.st->err);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (ok) {
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) acc[q][hlf * 16 + i] += v[i];
+                    for (int q = 0; q < 2; ++q) {
+                        const int chunk = dw + 4 * q;
+                        if (chunk * 32 < g.npad) {   // uniform over the warp
+#pragma unroll
+                            for (int hlf = 0; hlf < 2; ++hlf) {
+                                float v[16];
+                                tmem_ld16(tmem + buf * 256u + (unsigned)(chunk * 32 + hlf * 16), v);
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) acc[q][hlf * 16 + i] += v[i];
+                            }
                         }
                     }
                 }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) bar_arrive(&sm->tempty[buf]);
             }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) bar_arrive(&sm->tempty[buf]);
-            ++n;
-            if (group_end) break;
         }
+        n += (unsigned)nchains;
+        if (drains) {
+            // hi + lo of every token; to the workspace (output / down projection) or to the staging buffer
+            float *dst = (epi == CL_VEPI_RESID) ? a.ws + ((size_t)blockIdx.x * CL_MAX_T + lane) * R_MAXN : sm->stage + lane * R_STAGE_LD;
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int chunk = dw + 4 * q;
-            if (chunk * 32 < g.npad) epilogue_chunk(a, epi, rows, g, ji, chunk, acc[q], lane, sm, ds, pos0);
+            for (int q = 0; q < 2; ++q) {
+                const int chunk = dw + 4 * q;
+                if (chunk * 32 < g.npad) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float lo = __shfl_down_sync(0xffffffffu, acc[q][i], T);   // all lanes take part
+                        if (lane < T && chunk * 32 + i < g.npad) dst[chunk * 32 + i] = acc[q][i] + lo;
+                    }
+                }
+            }
         }
-    }
-    // per-job reductions over the four drain warps (fixed order)
-    if (epi == CL_VEPI_RESID) {
-        // (nothing per job: resid_phase() follows)
-    } else if (epi == CL_VEPI_HEAD) {
-        if (lane < CL_SLOTS) sm->hp[dw][lane] = ds.run;
-        drain_sync();
-        if (dw == 0 && lane < a.T)
-            a.head_part[(size_t)blockIdx.x * CL_SLOTS + lane] =
-                rp_merge(rp_merge(sm->hp[0][lane], sm->hp[1][lane]), rp_merge(sm->hp[2][lane], sm->hp[3][lane]));
-        drain_sync();
+        if (epi == CL_VEPI_RESID) continue;   // resid_phase() follows the job
+        worker_sync();
+        if (et < T) {
+            const float sc = sm->scale[et];
+            const float *st = sm->stage + et * R_STAGE_LD - g.a0;   // st[row] = raw product of (token et, weight row)
+            if (epi == CL_VEPI_STORE) {
+                for (int row = g.g0 + ej; row < g.g1; row += estride) a.qkv[(size_t)et * rows + row] = sc * st[row];
+            } else if (epi == CL_VEPI_SILU) {   // rows interleave gate (even) and up (odd); g0 is even
+                for (int row = g.g0 + 2 * ej; row < g.g1; row += 2 * estride) {
+                    const float gt = sc * st[row], up = sc * st[row + 1];
+                    a_store_split(a.Ah, et, T, row >> 1, gt / (1.f + expf(-gt)) * up, a.f16);
+                }
+            } else {
+                for (int row = g.g0 + ej; row < g.g1; row += estride) {
+                    const float lg = fminf(fmaxf(sc * st[row], -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
+                    if (a.logits) a.logits[(size_t)et * a.V + row] = lg;
+                    run = rp_merge(run, ClHeadPartial{lg, 1.f, 0.f, row});
+                }
+            }
+        }
+        worker_sync();   // the staging buffer is free again
     }
 }
 
-// A CTA that owns no row of the LM head still has to publish neutral statistics (they are merged by CTA 0).
-__device__ void publish_neutral(const ClRowsArgs &a, int ji) {
-    const Job jb = job_of(a, ji);
-    int r0, r1;
-    rows_of(jb.rows, jb.unit, jb.split, r0, r1);
-    if (r0 < r1) return;
-    if (threadIdx.x < a.T && jb.epi == CL_VEPI_HEAD)
-        a.head_part[(size_t)blockIdx.x * CL_SLOTS + threadIdx.x] = ClHeadPartial{0.f, 0.f, 0.f, 0x7fffffff};
+// End of the LM-head job: the statistics of a token row are spread over the threads of its warps; merge them in a
+// fixed order (rows ascend with the lane inside a warp pass, so a tree over lanes then warps is a fixed order too).
+__device__ void head_finish(const ClRowsArgs &a, RSmem *sm, ClHeadPartial run) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wpt = RW / a.T;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const ClHeadPartial other = cl_hp_shfl_xor(run, o);
+        run = ((lane & o) == 0) ? rp_merge(run, other) : rp_merge(other, run);
+    }
+    if (lane == 0) sm->hpw[warp] = run;
+    worker_sync();
+    if (tid < a.T) {
+        ClHeadPartial r = sm->hpw[tid * wpt];
+        for (int w = 1; w < wpt; ++w) r = rp_merge(r, sm->hpw[tid * wpt + w]);
+        a.head_part[(size_t)blockIdx.x * CL_SLOTS + tid] = r;
+    }
 }
 
 // Barrier of the `split` CTAs of a group (arrival counter per group, growing during a launch like the grid's).
@@ -604,8 +602,8 @@ __device__ void resid_phase(const ClRowsArgs &a, int ji, int pos0, unsigned &grp
     const bool attn_half = (ji & 3) == 1;
     const float *gain = attn_half ? y.n2 : ((l + 1 < a.L) ? a.layers[l + 1].n1 : a.final_norm);
     unsigned short *tap = (unsigned short *)(a.tap ? (attn_half ? y.tap0 : y.tap1) : nullptr);
-    float *sq = sm->wrec;   // [T][64] squares of this CTA's new residual values (the attention records are not in use now)
-    for (int t = tid; t < CL_SLOTS; t += RT) sm->red[0][t] = 0.f;
+    float *sq = sm->stage;   // [T][64] squares of this CTA's new residual values
+    for (int t = tid; t < CL_SLOTS; t += RT) sm->red[t] = 0.f;
     // the group's rows in tiles of at most R_MAXN rows, exactly as the GEMM cut them
     for (int g0 = r0; g0 < r1;) {
         const int a0 = g0 & ~7, g1 = min(r1, a0 + R_MAXN), n = g1 - g0;
@@ -633,15 +631,15 @@ __device__ void resid_phase(const ClRowsArgs &a, int ji, int pos0, unsigned &grp
             }
             worker_sync();
             if (tid < T) {
-                float ss = sm->red[0][tid];
+                float ss = sm->red[tid];
                 for (int i = 0; i < nq; ++i) ss += sq[tid * 64 + i];
-                sm->red[0][tid] = ss;
+                sm->red[tid] = ss;
             }
         }
         g0 = g1;
     }
     worker_sync();
-    if (tid < T) a.ssq[(size_t)blockIdx.x * CL_SLOTS + tid] = sm->red[0][tid];
+    if (tid < T) a.ssq[(size_t)blockIdx.x * CL_SLOTS + tid] = sm->red[tid];
 }
 
 // RMSNorm scale of every token row from the per-CTA sums of squares (fixed order: lane-strided, then a shuffle tree).
@@ -713,7 +711,7 @@ __device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int b
     const float scale = rsqrtf((float)HD);
     const int group = a.H / a.Hkv, kvd = a.Hkv * HD, ld = a.d + 2 * kvd;
     ST *Kc = (ST *)y.kc, *Vc = (ST *)y.vc;
-    float *wrec = sm->wrec;
+    float *wrec = sm->stage;
     for (int item = blockIdx.x; item < a.H * S; item += gridDim.x) {
         const int h = item % a.H, s = item / a.H, kvh = h / group;
         float m_run = -INFINITY, l_run = 0.f, o_run[VPL];
@@ -966,9 +964,8 @@ __global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constan
         if (lane == 0) mma_issuer(a, ring, sm, tmem);
     } else {
         const int base = a.st->ctx + a.row0;   // position of row 0
-        const bool drains = (warp & 3) == 0;
-        const int dw = warp >> 2;
         unsigned bar_target = 0u, grp_target = 0u, n_acc = 0u;
+        ClHeadPartial run{0.f, 0.f, 0.f, 0x7fffffff};
         int passed = 0;
         Cursor cur(a);
         embed_phase(a, sm);
@@ -977,29 +974,29 @@ __global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constan
         for (int l = 0; l < a.L; ++l) {
             const ClRowsLayer &y = a.layers[l];
             compute_scales(a, sm);
-            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * l, cur, n_acc, base);
+            gemm_job(a, sm, tmem, 4 * l, cur, n_acc, run);
             phase_clock(a, sm, 1);
             grid_barrier(a, bar_target, passed, sm);
             attention_phase<ST, HD>(a, y, base, sm);
             phase_clock(a, sm, 2);
             grid_barrier(a, bar_target, passed, sm);
-            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * l + 1, cur, n_acc, base);
+            gemm_job(a, sm, tmem, 4 * l + 1, cur, n_acc, run);
             resid_phase(a, 4 * l + 1, base, grp_target, sm);
             phase_clock(a, sm, 3);
             grid_barrier(a, bar_target, passed, sm);
             compute_scales(a, sm);
-            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * l + 2, cur, n_acc, base);
+            gemm_job(a, sm, tmem, 4 * l + 2, cur, n_acc, run);
             phase_clock(a, sm, 4);
             grid_barrier(a, bar_target, passed, sm);
-            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * l + 3, cur, n_acc, base);
+            gemm_job(a, sm, tmem, 4 * l + 3, cur, n_acc, run);
             resid_phase(a, 4 * l + 3, base, grp_target, sm);
             phase_clock(a, sm, 5);
             grid_barrier(a, bar_target, passed, sm);
         }
         if (a.want_head) {
             compute_scales(a, sm);
-            publish_neutral(a, 4 * a.L);
-            if (drains) drain_job(a, sm, tmem, dw, lane, 4 * a.L, cur, n_acc, base);
+            gemm_job(a, sm, tmem, 4 * a.L, cur, n_acc, run);
+            head_finish(a, sm, run);
             phase_clock(a, sm, 6);
             grid_barrier(a, bar_target, passed, sm);
             // CTA 0 merges the per-CTA statistics of every token row (one warp per row, fixed order): Eq. 1-4
@@ -1057,7 +1054,7 @@ __global__ void k_tile_layout(const uint4 *src, uint4 *dst, int rows, int KB, in
 
 }  // namespace
 
-size_t cl_rows_smem_bytes() { return (size_t)R_NSLOT * R_SLOT + 16384 + 1024; }
+size_t cl_rows_smem_bytes() { return (size_t)R_NSLOT * R_SLOT + R_CTRL_BYTES + 1024; }
 
 int cl_rows_att_part_floats(int H) { return H * R_ATT_MAXS * CL_MAX_T * (128 + 2); }
 
@@ -1067,7 +1064,9 @@ cudaError_t cl_launch_tile_layout(const void *src, void *dst, int rows, int K, i
 }
 
 cudaError_t cl_launch_rows_pass(int wdtype, int head_dim, const ClRowsArgs &a, int grid, cudaStream_t s) {
-    static_assert(sizeof(RSmem) <= 16384, "control block must fit behind the ring");
+    static_assert(sizeof(RSmem) <= R_CTRL_BYTES, "control block must fit behind the ring");
+    static_assert(R_STAGE_FLOATS >= CL_MAX_T * R_STAGE_LD && R_STAGE_FLOATS % 4 == 0, "staging buffer holds a tile of every token row");
+    static_assert(R_STAGE_FLOATS >= RW * (128 + 2), "staging buffer holds the attention records");
     const void *fn = nullptr;
     if (wdtype == 1 && head_dim == 64) fn = (const void *)k_rows_pass<__nv_bfloat16, 64>;
     else if (wdtype == 1 && head_dim == 128) fn = (const void *)k_rows_pass<__nv_bfloat16, 128>;
