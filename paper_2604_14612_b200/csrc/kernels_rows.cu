@@ -66,6 +66,8 @@ struct RSmem {
     // one buffer, used in turn by: the GEMM epilogues (raw products of a tile, [T][R_STAGE_LD]); the residual epilogue
     // ([T][64] squares); the attention phase (per-warp (max, sum, o[hd]) records, [RW][hd + 2])
     alignas(16) float stage[R_STAGE_FLOATS];
+    alignas(16) unsigned short knew[CL_MAX_T * 128];   // attention: the pass's own keys (rotated) and values in the storage type
+    alignas(16) unsigned short vnew[CL_MAX_T * 128];
     unsigned long long t_prev, ph_ns[8];   // diagnostics: time of thread 0 by phase
 };
 
@@ -643,16 +645,19 @@ __device__ void resid_phase(const ClRowsArgs &a, int ji, int pos0, unsigned &grp
 }
 
 // RMSNorm scale of every token row from the per-CTA sums of squares (fixed order: lane-strided, then a shuffle tree).
+// The warps that do not drain the accumulator do this while the GEMM runs (token k <-> the k-th of them); the barrier
+// in front of the epilogue, the first reader, orders it.
 __device__ void compute_scales(const ClRowsArgs &a, RSmem *sm) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (warp < a.T) {
+    if ((warp & 3) == 0) return;
+    const int t = warp - 1 - (warp >> 2);
+    if (t < a.T) {
         float ss = 0.f;
-        for (int c = lane; c < (int)gridDim.x; c += 32) ss += __ldcg(a.ssq + (size_t)c * CL_SLOTS + warp);
+        for (int c = lane; c < (int)gridDim.x; c += 32) ss += __ldcg(a.ssq + (size_t)c * CL_SLOTS + t);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if (lane == 0) sm->scale[warp] = 1.0f / sqrtf(ss * a.inv_d + a.eps);
+        if (lane == 0) sm->scale[t] = 1.0f / sqrtf(ss * a.inv_d + a.eps);
     }
-    worker_sync();
 }
 
 // ---- embedding phase: x[t] = E[token t]; first operand hi/lo(x * g); per-CTA sums of squares ---------------------
@@ -695,9 +700,9 @@ __device__ void embed_phase(const ClRowsArgs &a, RSmem *sm) {
 // Work item (head h, part s of the cached keys [0, base)) -> one CTA.  Inside the CTA warp w serves token row
 // t = w / nsub and the sub-range sub = w % nsub of the part's keys (nsub = 14 / T warps per row).  A warp walks its
 // keys 32 at a time with an online softmax (scores reduced with warp shuffles).  The rows' own keys and values
-// (positions base .. base + t, causal) come raw from the QKV product: the last warp of row t in the last part
-// rotates each key, rounds key and value to the storage type and folds them in; the warp of the last row also
-// appends them to the cache (one query head per key/value head).  The CTA merges its warps per row and writes one
+// (positions base .. base + t, causal) come raw from the QKV product: the CTA of the last part first rotates the
+// keys, rounds keys and values to the storage type and keeps them in shared memory (one query head per key/value
+// head also appends them to the cache); the last warp of row t folds them in.  The CTA merges its warps per row and writes one
 // record per (h, s, t); the last CTA of a head to finish (ticket) merges the parts in order and writes the
 // normalised output as the output projection's hi/lo operand rows.
 template <typename ST, int HD>
@@ -714,6 +719,29 @@ __device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int b
     float *wrec = sm->stage;
     for (int item = blockIdx.x; item < a.H * S; item += gridDim.x) {
         const int h = item % a.H, s = item / a.H, kvh = h / group;
+        if (s == S - 1) {
+            // the pass's own keys and values, raw in the QKV product: rotate the keys, round both to the storage type, keep
+            // them for the warps below (one query head per key/value head also appends them to the cache); one thread per
+            // (row, pair of elements i, i + hd / 2), so the whole set costs one memory round trip
+            const bool writer = (h % group) == 0;
+            for (int idx = tid; idx < T * HALF; idx += RT) {
+                const int jn = idx / HALF, i = idx % HALF;
+                const float *kraw = a.qkv + (size_t)jn * ld + a.d + kvh * HD, *vraw = kraw + kvd;
+                const float2 cs = a.rope_cs[(size_t)(base + jn) * HALF + i];
+                const float ka = __ldcg(kraw + i), kb = __ldcg(kraw + i + HALF);
+                const float va = __ldcg(vraw + i), vb = __ldcg(vraw + i + HALF);
+                const unsigned short kk0 = f32_to_b16(ka * cs.x - kb * cs.y, a.f16), kk1 = f32_to_b16(kb * cs.x + ka * cs.y, a.f16);
+                const unsigned short v0 = f32_to_b16(va, a.f16), v1 = f32_to_b16(vb, a.f16);
+                sm->knew[jn * HD + i] = kk0; sm->knew[jn * HD + i + HALF] = kk1;
+                sm->vnew[jn * HD + i] = v0; sm->vnew[jn * HD + i + HALF] = v1;
+                if (writer) {
+                    unsigned short *ck = (unsigned short *)Kc + ((size_t)kvh * a.max_seq + base + jn) * HD;
+                    unsigned short *cv = (unsigned short *)Vc + ((size_t)kvh * a.max_seq + base + jn) * HD;
+                    ck[i] = kk0; ck[i + HALF] = kk1; cv[i] = v0; cv[i + HALF] = v1;
+                }
+            }
+            worker_sync();
+        }
         float m_run = -INFINITY, l_run = 0.f, o_run[VPL];
 #pragma unroll
         for (int e = 0; e < VPL; ++e) o_run[e] = 0.f;
@@ -809,35 +837,20 @@ __device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int b
             }
             if (s == S - 1 && sub == nsub - 1) {
                 // the pass's own positions base .. base + t
-                const bool writer = (t == T - 1) && (h % group) == 0;
                 for (int jn = 0; jn <= t; ++jn) {
-                    const float *kraw = a.qkv + (size_t)jn * ld + a.d + kvh * HD, *vraw = kraw + kvd;
-                    float sc = 0.f;
-                    unsigned short kst[EPL];
+                    float kf[EPL], vn[VPL];
+                    const uint4 raw = *(const uint4 *)(sm->knew + jn * HD + li * EPL);
+                    const unsigned u[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-                    for (int e = 0; e < EPL; ++e) {
-                        const int idx = li * EPL + e;
-                        const int i = idx < HALF ? idx : idx - HALF;
-                        const float2 cs = a.rope_cs[(size_t)(base + jn) * HALF + i];
-                        const float ka = __ldcg(kraw + i), kb = __ldcg(kraw + i + HALF);
-                        kst[e] = f32_to_b16(idx < HALF ? ka * cs.x - kb * cs.y : kb * cs.x + ka * cs.y, a.f16);
-                        sc = fmaf(qr[e], b16_to_f32(kst[e], a.f16), sc);
-                    }
+                    for (int e = 0; e < 4; ++e) pair16_to_f32(u[e], a.f16, kf[2 * e], kf[2 * e + 1]);
+#pragma unroll
+                    for (int e = 0; e < VPL; ++e) vn[e] = b16_to_f32(sm->vnew[jn * HD + lane * VPL + e], a.f16);
+                    float sc = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) sc = fmaf(qr[e], kf[e], sc);
 #pragma unroll
                     for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
                     sc = __shfl_sync(0xffffffffu, sc, 0) * scale;
-                    if (ksub == 0 && writer) {
-                        unsigned short *kd = (unsigned short *)Kc + ((size_t)kvh * a.max_seq + base + jn) * HD + li * EPL;
-#pragma unroll
-                        for (int e = 0; e < EPL; ++e) kd[e] = kst[e];
-                    }
-                    float vn[VPL];
-#pragma unroll
-                    for (int e = 0; e < VPL; ++e) {
-                        const unsigned short vs = f32_to_b16(__ldcg(vraw + lane * VPL + e), a.f16);
-                        if (writer) ((unsigned short *)Vc)[((size_t)kvh * a.max_seq + base + jn) * HD + lane * VPL + e] = vs;
-                        vn[e] = b16_to_f32(vs, a.f16);
-                    }
                     const float m_new = fmaxf(m_run, sc);
                     const float resc = (l_run > 0.f) ? expf(m_run - m_new) : 0.f;
                     const float pn = expf(sc - m_new);
