@@ -78,7 +78,8 @@ struct cl_ctx {
     ClRowsLayer *rows_layers_dev;
     unsigned short *r_ax, *r_aatt, *r_ah;
     float *r_ssq, *r_att_part, *r_ws;
-    unsigned *r_bar;                     // arrival counters of the pass: the grid's, then one per group of CTAs
+    unsigned *r_bar;                     // counters of the pass: the grid barrier, one per group of CTAs, the completion counters
+    int r_sync_words, r_c_ssq, r_c_ax, r_c_ah, r_c_att, r_c_qkv;
     int rows_split;                      // CTAs per group that cut the K range of the output / down projections between them
     unsigned *r_tickets;
     ClHeadPartial *r_head_part;
@@ -481,7 +482,13 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 DM(c->wtile, per_layer * L);
                 DM(c->head_tile, V * d * es);
                 DM(c->r_ws, (size_t)c->n_sm * CL_MAX_T * 224 * 4);
-                DM(c->r_bar, ((size_t)1 + c->n_sm) * 4);
+                c->r_c_ssq = 1 + c->n_sm / c->rows_split;
+                c->r_c_ax = c->r_c_ssq + 1;
+                c->r_c_ah = c->r_c_ax + (int)(d / 64);
+                c->r_c_att = c->r_c_ah + (int)(F / 64);
+                c->r_c_qkv = c->r_c_att + g.n_heads;
+                c->r_sync_words = c->r_c_qkv + (int)(qkv_rows / g.head_dim);
+                DM(c->r_bar, (size_t)c->r_sync_words * 4);
                 std::vector<ClRowsLayer> rl(L);
                 for (size_t l = 0; l < L; ++l) {
                     const ClLayer &y = c->layers[l];
@@ -592,8 +599,9 @@ static int forward_rows_persistent(cl_ctx *c, const int *tok, int T, int row0, i
     a.x = c->x; a.qkv = c->qkv; a.Ax = c->r_ax; a.Aatt = c->r_aatt; a.Ah = c->r_ah;
     a.ssq = c->r_ssq; a.att_part = c->r_att_part; a.att_tickets = c->r_tickets; a.head_part = c->r_head_part;
     a.logits = logits; a.out_tok = out_tok; a.out_pmax = out_pmax; a.out_conf = out_conf;
-    a.bar = c->r_bar; a.bar_arrivals = (unsigned)c->n_sm; a.wait_ns = c->wait_ns; a.phase_ns = c->r_phase_ns;
-    CU(cudaMemsetAsync(c->r_bar, 0, ((size_t)1 + c->n_sm / c->rows_split) * 4, c->stream));   // arrival counters start at zero
+    a.sync = c->r_bar; a.bar_arrivals = (unsigned)c->n_sm; a.wait_ns = c->wait_ns; a.phase_ns = c->r_phase_ns;
+    a.c_ssq = c->r_c_ssq; a.c_ax = c->r_c_ax; a.c_ah = c->r_c_ah; a.c_att = c->r_c_att; a.c_qkv = c->r_c_qkv;
+    CU(cudaMemsetAsync(c->r_bar, 0, (size_t)c->r_sync_words * 4, c->stream));   // every counter starts at zero
     KL(cl_launch_rows_pass(g.weight_dtype, g.head_dim, a, c->n_sm, c->stream));
     return CL_OK;
 }

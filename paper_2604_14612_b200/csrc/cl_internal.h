@@ -249,7 +249,9 @@ struct ClRowsArgs {
     float *logits;                      // optional [T, V]
     int *out_tok;                       // [T] greedy token after each row
     float *out_pmax, *out_conf;
-    unsigned *bar;                      // [1 + grid / split] arrival counters, zero at launch: the grid's barrier, then one per group
+    unsigned *sync;                     // counters, all zero at launch: [0] the grid barrier, [1 .. 1 + grid / split) the groups' barriers,
+                                        // then the completion counters of the buffers that connect the phases, at the offsets below
+    int c_ssq, c_ax, c_ah, c_att, c_qkv;   // offsets in sync: 1 | d / 64 | F / 64 | H | (d + 2 Hkv hd) / hd counters
     unsigned bar_arrivals;
     unsigned long long wait_ns;
     unsigned long long *phase_ns;       // diagnostics, optional: [grid, 8] time of each CTA's thread 0 by phase

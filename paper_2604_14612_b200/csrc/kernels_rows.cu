@@ -57,7 +57,6 @@ struct RSmem {
     unsigned long long wait_ns;
     unsigned tmem_base;
     int abort;
-    int bars_done;                     // grid barriers this CTA has passed (read by the producer)
     int is_last;
     float scale[CL_SLOTS];             // RMSNorm scale of every token row for the current phase
     float red[CL_SLOTS];
@@ -81,6 +80,30 @@ __device__ __forceinline__ void phase_clock(const ClRowsArgs &a, RSmem *sm, int 
     }
 }
 
+// ---- completion counters -------------------------------------------------------------------------------
+// The phases of a layer are not separated by grid barriers.  Every buffer that one phase writes and the next reads has
+// counters in global memory that only grow during a launch (the host zeroes them before it): a writer adds, with
+// release semantics and after its CTA's stores, how much of a piece it has completed; a reader waits (acquire, bounded)
+// until the piece is complete for the pass over the buffer it needs.  a.sync + ...
+//   c_ax  + kb   columns [64 kb, 64 kb + 64) of the operand rows Ax, 64 per pass: pass 1 = embedding, 2 l + 2 = layer l's
+//                output projection, 2 l + 3 = its down projection (so layer l's QKV needs 64 (2 l + 1), its gate/up 64 (2 l + 2))
+//   c_ssq        CTAs that have published their sum of squares of the residual rows, grid size per pass (same passes)
+//   c_qkv + b    rows [hd b, hd b + hd) of the QKV product (one head's q, k or v), hd per layer
+//   c_att + h    head h's attention output in Aatt, 1 per layer
+//   c_ah  + kb   columns [64 kb, 64 kb + 64) of the FFN hidden operand rows Ah, 64 per layer
+// A k-block of a GEMM starts as soon as its 64 activation columns are complete, whatever the rest of the grid is
+// doing; the weight stream never waits.  Overwriting a buffer needs no counter: every phase needs all of K of the one
+// before it to finish, so by the time a CTA can write a buffer again every reader of its previous contents is done.
+// One grid barrier remains, in front of the merge of the LM-head statistics.
+__device__ __forceinline__ void counter_add(unsigned *c, unsigned v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(c), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned counter_read(const unsigned *c) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(c) : "memory");
+    return v;
+}
+
 // ---- schedule ---------------------------------------------------------------------------------------
 // GEMM jobs in execution order: job 4 l + m = matrix m of layer l (0 QKV, 1 O, 2 gate/up, 3 down), job 4 L = LM head.
 // A CTA's rows [r0, r1) of a job are cut into groups of at most R_MAXN tile rows; a group's K range into ring slots
@@ -88,7 +111,9 @@ __device__ __forceinline__ void phase_clock(const ClRowsArgs &a, RSmem *sm, int 
 struct Job {
     const char *W;        // k-block-major weights
     const unsigned short *A;
-    int rows, KB, unit, epi, need;
+    int rows, KB, unit, epi;
+    int dep, dep_shift;   // k-block kb of the activation operand is complete when counter dep + (kb >> dep_shift) ...
+    unsigned dep_target;  // ... has reached this value (see "completion counters" below)
     int split;            // CTAs that share a row block and cut its K range between them (1: every CTA owns rows over all of K)
 };
 
@@ -98,13 +123,13 @@ __device__ __forceinline__ Job job_of(const ClRowsArgs &a, int ji) {
     if (ji < 4 * L) {
         const int l = ji >> 2, m = ji & 3;
         const ClRowsLayer &y = a.layers[l];
-        const int base = 1 + 5 * l;   // grid barriers passed when layer l's QKV input is complete
-        if (m == 0) { j.W = y.wqkv; j.A = a.Ax; j.rows = a.d + 2 * a.Hkv * a.hd; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_STORE; j.need = base; j.split = 1; }
-        else if (m == 1) { j.W = y.wo; j.A = a.Aatt; j.rows = a.d; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_RESID; j.need = base + 2; j.split = a.split; }
-        else if (m == 2) { j.W = y.wgu; j.A = a.Ax; j.rows = 2 * a.F; j.KB = a.d >> 6; j.unit = 2; j.epi = CL_VEPI_SILU; j.need = base + 3; j.split = 1; }
-        else { j.W = y.wd; j.A = a.Ah; j.rows = a.d; j.KB = a.F >> 6; j.unit = 1; j.epi = CL_VEPI_RESID; j.need = base + 4; j.split = a.split; }
+        const int hs = a.hd == 128 ? 1 : 0;   // k-blocks per head: 2 (hd 128) or 1 (hd 64)
+        if (m == 0) { j.W = y.wqkv; j.A = a.Ax; j.rows = a.d + 2 * a.Hkv * a.hd; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_STORE; j.dep = a.c_ax; j.dep_shift = 0; j.dep_target = 64u * (2 * l + 1); j.split = 1; }
+        else if (m == 1) { j.W = y.wo; j.A = a.Aatt; j.rows = a.d; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_RESID; j.dep = a.c_att; j.dep_shift = hs; j.dep_target = (unsigned)(l + 1); j.split = a.split; }
+        else if (m == 2) { j.W = y.wgu; j.A = a.Ax; j.rows = 2 * a.F; j.KB = a.d >> 6; j.unit = 2; j.epi = CL_VEPI_SILU; j.dep = a.c_ax; j.dep_shift = 0; j.dep_target = 64u * (2 * l + 2); j.split = 1; }
+        else { j.W = y.wd; j.A = a.Ah; j.rows = a.d; j.KB = a.F >> 6; j.unit = 1; j.epi = CL_VEPI_RESID; j.dep = a.c_ah; j.dep_shift = 0; j.dep_target = 64u * (l + 1); j.split = a.split; }
     } else {
-        j.W = a.head; j.A = a.Ax; j.rows = a.V; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_HEAD; j.need = 1 + 5 * L; j.split = 1;
+        j.W = a.head; j.A = a.Ax; j.rows = a.V; j.KB = a.d >> 6; j.unit = 1; j.epi = CL_VEPI_HEAD; j.dep = a.c_ax; j.dep_shift = 0; j.dep_target = 64u * (2 * L + 1); j.split = 1;
     }
     return j;
 }
@@ -130,7 +155,9 @@ struct Cursor {
     int ji;
     const char *W;
     const unsigned short *A;
-    int rows, KB, unit, epi, need;
+    int rows, KB, unit, epi;
+    int dep, dep_shift;
+    unsigned dep_target;
     int kb_begin, kb_end;     // the CTA's k-blocks of the job (all of them unless the job is split over K)
     int r0, r1;               // the rows of the CTA (of its group, for a job split over K)
     // group
@@ -168,7 +195,8 @@ struct Cursor {
     __device__ void next_job() {
         for (++ji; ji < njobs; ++ji) {
             const Job j = job_of(a, ji);
-            W = j.W; A = j.A; rows = j.rows; KB = j.KB; unit = j.unit; epi = j.epi; need = j.need;
+            W = j.W; A = j.A; rows = j.rows; KB = j.KB; unit = j.unit; epi = j.epi;
+            dep = j.dep; dep_shift = j.dep_shift; dep_target = j.dep_target;
             rows_of(rows, unit, j.split, r0, r1);
             const int member = (int)blockIdx.x % j.split;
             kb_begin = KB * member / j.split;
@@ -241,36 +269,32 @@ __device__ __forceinline__ bool r_wait(unsigned long long *b, unsigned parity, R
     }
 }
 
-// Grid barrier on one arrival counter that only grows during a launch (the host zeroes it before the launch).
-// Called by every worker thread; thread 0 arrives and polls (bounded) and then publishes the count for the producer.
-__device__ __forceinline__ void grid_barrier(const ClRowsArgs &a, unsigned &target, int &passed, RSmem *sm) {
-    proxy_fence_global();   // this thread's global stores are read by other CTAs' bulk copies after the barrier
-    worker_sync();
-    if (threadIdx.x == 0) {
-        if (!*(volatile int *)&sm->abort) {
-            target += a.bar_arrivals;
-            asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.bar) : "memory");
-            unsigned v;
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.bar) : "memory");
-            if ((int)(v - target) < 0) {
-                const unsigned long long t0 = gtime_ns();
-                unsigned i = 0;
-                do {
-                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.bar) : "memory");
-                    if ((++i & 255u) == 0u) {
-                        if (*(volatile int *)&a.st->err || gtime_ns() - t0 > sm->wait_ns) {
-                            *(volatile int *)&sm->abort = 1;
-                            atomicOr(&a.st->err, 16);
-                            break;
-                        }
-                    }
-                } while ((int)(v - target) < 0);
+// Bounded wait for a completion counter; called by one thread.
+__device__ __forceinline__ bool counter_wait(const unsigned *c, unsigned target, RSmem *sm, int *err) {
+    if ((int)(counter_read(c) - target) >= 0) return true;
+    const unsigned long long t0 = gtime_ns();
+    for (unsigned i = 1;; ++i) {
+        if ((int)(counter_read(c) - target) >= 0) return true;
+        if ((i & 63u) == 0u) {
+            if (*(volatile int *)&sm->abort || *(volatile int *)err) return false;
+            if (gtime_ns() - t0 > sm->wait_ns) {
+                *(volatile int *)&sm->abort = 1;
+                atomicOr(err, 16);
+                return false;
             }
         }
-        __threadfence();
-        *(volatile int *)&sm->bars_done = passed + 1;
     }
-    ++passed;
+}
+
+// Grid barrier on one arrival counter that only grows during a launch (the host zeroes it before the launch).
+// Called by every worker thread; thread 0 arrives and polls (bounded).
+__device__ __forceinline__ void grid_barrier(const ClRowsArgs &a, unsigned &target, RSmem *sm) {
+    worker_sync();
+    if (threadIdx.x == 0 && !*(volatile int *)&sm->abort) {
+        target += a.bar_arrivals;
+        counter_add(a.sync, 1u);
+        counter_wait(a.sync, target, sm, &a.st->err);
+    }
     worker_sync();
     phase_clock(a, sm, 7);
 }
@@ -306,7 +330,7 @@ __device__ __forceinline__ ClHeadPartial rp_merge(const ClHeadPartial &a, const 
 // The whole producer warp runs this (uniform control flow; lane j issues the copy of a slot's j-th k-block, so a slot
 // costs the same few instructions however many k-blocks it holds).  Weight tiles are requested as soon as a ring
 // slot is free -- weights never change, so the stream runs ahead of the grid barriers; the activation tiles of a slot
-// are requested once the barrier that completes them has been passed (bars_done), both on the slot's one mbarrier.
+// are requested once the completion counters of their k-blocks say so, both on the slot's one mbarrier.
 __device__ void producer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, int lane) {
     unsigned long long policy;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
@@ -317,26 +341,39 @@ __device__ void producer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, in
     int pn = 0;                            // queue length
     unsigned used = 0;                     // bit i: slot i has copies in flight of phase parity (used_par >> i) & 1
     unsigned used_par = 0;
-    int fenced = 0;                        // grid barriers whose writes this warp has ordered before its copies
+    bool job_ready = false;                // every k-block of the queue head's job is known to be complete
+    unsigned looks = 0;
     unsigned long long t_idle = 0;
     unsigned n_idle = 0;
     while (!w.done || pn > 0) {
         if (__shfl_sync(0xffffffffu, *(volatile int *)&sm->abort, 0)) break;
         bool progress = false;
         if (pn > 0) {
-            const int bars = __shfl_sync(0xffffffffu, *(volatile int *)&sm->bars_done, 0);
-            if (bars >= q.need) {
-                if (bars > fenced) {   // once per barrier: other CTAs' stores before this warp's bulk-copy reads
-                    __threadfence();
-                    proxy_fence_global();
-                    fenced = bars;
+            // the head of the queue: are the activation columns of its k-blocks complete?  Lane j looks at k-block j's
+            // counter; once a look at the job's whole K range has found everything complete, no more looks for this job.
+            bool ready = job_ready;
+            if (!ready) {
+                const unsigned v = lane < q.kbs ? counter_read(a.sync + q.dep + ((q.kb0 + lane) >> q.dep_shift)) : q.dep_target;
+                ready = __all_sync(0xffffffffu, (int)(v - q.dep_target) >= 0);
+                if (ready) {
+                    if ((++looks & 3u) == 0u) {
+                        bool all = true;
+                        for (int kb = q.kb0 + lane; kb < q.kb_end; kb += 32)
+                            all = all && (int)(counter_read(a.sync + q.dep + (kb >> q.dep_shift)) - q.dep_target) >= 0;
+                        job_ready = __all_sync(0xffffffffu, all);
+                    }
+                    proxy_fence_global();   // other CTAs' stores (acquired above) before this warp's bulk-copy reads
                 }
+            }
+            if (ready) {
                 if (lane < q.kbs)
                     bulk_g2s(ring + (size_t)qslot * R_SLOT + (size_t)lane * q.stride,
                              q.A + (size_t)(q.kb0 + lane) * (CL_ROWS_AROWS * 64), abytes, &sm->full[qslot]);
                 if (++qslot == R_NSLOT) qslot = 0;
                 --pn;
+                const int ji_old = q.ji;
                 q.advance();
+                if (q.done || q.ji != ji_old) job_ready = false;
                 progress = true;
             }
         }
@@ -531,6 +568,7 @@ __device__ __forceinline__ void gemm_job(const ClRowsArgs &a, RSmem *sm, unsigne
                     const float gt = sc * st[row], up = sc * st[row + 1];
                     a_store_split(a.Ah, et, T, row >> 1, gt / (1.f + expf(-gt)) * up, a.f16);
                 }
+                proxy_fence_global();   // these stores are read by other CTAs' bulk copies
             } else {
                 for (int row = g.g0 + ej; row < g.g1; row += estride) {
                     const float lg = fminf(fmaxf(sc * st[row], -CL_LOGIT_CLAMP), CL_LOGIT_CLAMP);
@@ -539,7 +577,17 @@ __device__ __forceinline__ void gemm_job(const ClRowsArgs &a, RSmem *sm, unsigne
                 }
             }
         }
-        worker_sync();   // the staging buffer is free again
+        worker_sync();   // the staging buffer is free again; this tile's results are complete
+        if (tid == 0) {
+            if (epi == CL_VEPI_STORE) {          // rows of the QKV product, counted per head-sized block
+                for (int b = g.g0 / a.hd; b * a.hd < g.g1; ++b)
+                    counter_add(a.sync + a.c_qkv + b, (unsigned)(min(g.g1, (b + 1) * a.hd) - max(g.g0, b * a.hd)));
+            } else if (epi == CL_VEPI_SILU) {    // columns of the FFN hidden operand rows, counted per k-block
+                const int j0 = g.g0 >> 1, j1 = g.g1 >> 1;
+                for (int kb = j0 >> 6; kb * 64 < j1; ++kb)
+                    counter_add(a.sync + a.c_ah + kb, (unsigned)(min(j1, (kb + 1) * 64) - max(j0, kb * 64)));
+            }
+        }
     }
 }
 
@@ -565,7 +613,7 @@ __device__ void head_finish(const ClRowsArgs &a, RSmem *sm, ClHeadPartial run) {
 __device__ __forceinline__ void group_barrier(const ClRowsArgs &a, unsigned &target, RSmem *sm) {
     worker_sync();
     if (a.split > 1 && threadIdx.x == 0 && !*(volatile int *)&sm->abort) {
-        unsigned *bar = a.bar + 1 + blockIdx.x / a.split;
+        unsigned *bar = a.sync + 1 + blockIdx.x / a.split;
         target += (unsigned)a.split;
         __threadfence();
         asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
@@ -642,16 +690,31 @@ __device__ void resid_phase(const ClRowsArgs &a, int ji, int pos0, unsigned &grp
     }
     worker_sync();
     if (tid < T) a.ssq[(size_t)blockIdx.x * CL_SLOTS + tid] = sm->red[tid];
+    proxy_fence_global();   // the operand rows written above are read by other CTAs' bulk copies
+    worker_sync();
+    if (tid == 0) {
+        // this CTA's share of the operand columns, counted per k-block; and its sum of squares
+        for (int g0 = r0; g0 < r1;) {
+            const int a0 = g0 & ~7, g1 = min(r1, a0 + R_MAXN), n = g1 - g0;
+            const int q0 = g0 + n * member / g, q1 = g0 + n * (member + 1) / g;
+            for (int kb = q0 >> 6; kb * 64 < q1; ++kb)
+                counter_add(a.sync + a.c_ax + kb, (unsigned)(min(q1, (kb + 1) * 64) - max(q0, kb * 64)));
+            g0 = g1;
+        }
+        counter_add(a.sync + a.c_ssq, 1u);
+    }
 }
 
 // RMSNorm scale of every token row from the per-CTA sums of squares (fixed order: lane-strided, then a shuffle tree).
 // The warps that do not drain the accumulator do this while the GEMM runs (token k <-> the k-th of them); the barrier
 // in front of the epilogue, the first reader, orders it.
-__device__ void compute_scales(const ClRowsArgs &a, RSmem *sm) {
+__device__ void compute_scales(const ClRowsArgs &a, RSmem *sm, int pass) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if ((warp & 3) == 0) return;
     const int t = warp - 1 - (warp >> 2);
     if (t < a.T) {
+        if (lane == 0) counter_wait(a.sync + a.c_ssq, (unsigned)pass * gridDim.x, sm, &a.st->err);   // every CTA's sum is there
+        __syncwarp();
         float ss = 0.f;
         for (int c = lane; c < (int)gridDim.x; c += 32) ss += __ldcg(a.ssq + (size_t)c * CL_SLOTS + t);
 #pragma unroll
@@ -688,12 +751,19 @@ __device__ void embed_phase(const ClRowsArgs &a, RSmem *sm) {
             sm->esum[i][t] = ss;
         }
     }
+    proxy_fence_global();   // the operand rows written above are read by other CTAs' bulk copies
     worker_sync();
     if (tid < T) {
         float ss = 0.f;
         for (int i = 0; i < per; ++i) ss += sm->esum[i][tid];
         a.ssq[(size_t)blockIdx.x * CL_SLOTS + tid] = ss;
     }
+    worker_sync();
+    if (tid < per) {   // 8 operand columns per chunk, counted per k-block
+        const int ch = (int)blockIdx.x + tid * (int)gridDim.x;
+        if (ch < nch) counter_add(a.sync + a.c_ax + (ch >> 3), 8u);
+    }
+    if (tid == 0) counter_add(a.sync + a.c_ssq, 1u);
 }
 
 // ---- attention of the T rows over the cache ------------------------------------------------------------------
@@ -706,7 +776,7 @@ __device__ void embed_phase(const ClRowsArgs &a, RSmem *sm) {
 // record per (h, s, t); the last CTA of a head to finish (ticket) merges the parts in order and writes the
 // normalised output as the output projection's hi/lo operand rows.
 template <typename ST, int HD>
-__device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int base, RSmem *sm) {
+__device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int layer, int base, RSmem *sm) {
     constexpr int EPL = 8, LPK = HD / EPL, KPW = 32 / LPK, VPL = HD / 32, WSTRIDE = HD + 2, HALF = HD / 2;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int T = a.T, S = a.att_parts, nsub = RW / T;
@@ -719,6 +789,17 @@ __device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int b
     float *wrec = sm->stage;
     for (int item = blockIdx.x; item < a.H * S; item += gridDim.x) {
         const int h = item % a.H, s = item / a.H, kvh = h / group;
+        // this head's q rows and its key/value head's k and v rows of the QKV product: complete? (three counters, one
+        // lane each)
+        if (warp == 0) {
+            if (lane < 3) {
+                const int b = lane == 0 ? h : (lane == 1 ? a.H + kvh : a.H + a.Hkv + kvh);
+                counter_wait(a.sync + a.c_qkv + b, (unsigned)(HD * (layer + 1)), sm, &a.st->err);
+            }
+            __syncwarp();
+        }
+        phase_clock(a, sm, 7);
+        worker_sync();
         if (s == S - 1) {
             // the pass's own keys and values, raw in the QKV product: rotate the keys, round both to the storage type, keep
             // them for the warps below (one query head per key/value head also appends them to the cache); one thread per
@@ -932,7 +1013,11 @@ __device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int b
                 }
             }
         }
+        // the CTA that wrote the head's operand rows says so (its stores are read by other CTAs' bulk copies)
+        const bool wrote = S == 1 || sm->is_last;
+        if (wrote) proxy_fence_global();
         worker_sync();
+        if (wrote && tid == 0) counter_add(a.sync + a.c_att + h, 1u);
     }
 }
 
@@ -956,7 +1041,6 @@ __global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constan
             bar_init(&sm->tempty[i], 4);
         }
         sm->abort = 0;
-        sm->bars_done = 0;
         sm->wait_ns = a.wait_ns;
         for (int i = 0; i < 8; ++i) sm->ph_ns[i] = 0ull;
         sm->t_prev = gtime_ns();
@@ -979,39 +1063,32 @@ __global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constan
         const int base = a.st->ctx + a.row0;   // position of row 0
         unsigned bar_target = 0u, grp_target = 0u, n_acc = 0u;
         ClHeadPartial run{0.f, 0.f, 0.f, 0x7fffffff};
-        int passed = 0;
         Cursor cur(a);
         embed_phase(a, sm);
         phase_clock(a, sm, 0);
-        grid_barrier(a, bar_target, passed, sm);
         for (int l = 0; l < a.L; ++l) {
             const ClRowsLayer &y = a.layers[l];
-            compute_scales(a, sm);
+            compute_scales(a, sm, 2 * l + 1);
             gemm_job(a, sm, tmem, 4 * l, cur, n_acc, run);
             phase_clock(a, sm, 1);
-            grid_barrier(a, bar_target, passed, sm);
-            attention_phase<ST, HD>(a, y, base, sm);
+            attention_phase<ST, HD>(a, y, l, base, sm);
             phase_clock(a, sm, 2);
-            grid_barrier(a, bar_target, passed, sm);
             gemm_job(a, sm, tmem, 4 * l + 1, cur, n_acc, run);
             resid_phase(a, 4 * l + 1, base, grp_target, sm);
             phase_clock(a, sm, 3);
-            grid_barrier(a, bar_target, passed, sm);
-            compute_scales(a, sm);
+            compute_scales(a, sm, 2 * l + 2);
             gemm_job(a, sm, tmem, 4 * l + 2, cur, n_acc, run);
             phase_clock(a, sm, 4);
-            grid_barrier(a, bar_target, passed, sm);
             gemm_job(a, sm, tmem, 4 * l + 3, cur, n_acc, run);
             resid_phase(a, 4 * l + 3, base, grp_target, sm);
             phase_clock(a, sm, 5);
-            grid_barrier(a, bar_target, passed, sm);
         }
         if (a.want_head) {
-            compute_scales(a, sm);
+            compute_scales(a, sm, 2 * a.L + 1);
             gemm_job(a, sm, tmem, 4 * a.L, cur, n_acc, run);
             head_finish(a, sm, run);
             phase_clock(a, sm, 6);
-            grid_barrier(a, bar_target, passed, sm);
+            grid_barrier(a, bar_target, sm);
             // CTA 0 merges the per-CTA statistics of every token row (one warp per row, fixed order): Eq. 1-4
             if (blockIdx.x == 0 && warp < a.T) {
                 ClHeadPartial p{0.f, 0.f, 0.f, 0x7fffffff};
