@@ -25,13 +25,16 @@
  *     attention, query head h reads key/value head h / (n_heads / n_kv_heads)),
  *     head_dim in {64, 128}, d_model and d_ffn multiples of 8, 1 <= K <= CL_MAX_K.
  *   - Which kernels run: single-token steps (draft, vanilla) run in one persistent cooperative kernel when d_model and
- *     d_ffn are at most 16384 (bf16) / 8192 (fp32); passes of several rows (verify, prefill) and the confidence scoring
- *     of bf16 and fp16 models run on the tensor cores (tcgen05, both operands in the model's 16-bit type); fp32 models
- *     and the cases above use per-matrix CUDA-core kernels.
+ *     d_ffn are at most 16384 (bf16) / 8192 (fp32).  Passes of up to CL_MAX_K + 1 rows (verify, short prompt chunks) of
+ *     bf16 and fp16 models run in one persistent cooperative launch on the tensor cores (tcgen05, both operands in the
+ *     model's 16-bit type) when d_model and d_ffn are multiples of 64 and d_model <= 31968; for it cl_load keeps a
+ *     second copy of every matrix in the order that kernel streams it (device memory for weights doubles).  The
+ *     confidence scoring of 16-bit models runs on the tensor cores too; fp32 models and the remaining cases use
+ *     per-matrix CUDA-core kernels.
  *     A prompt of more than 16 tokens (bf16 / fp16 models) runs all rows but the last through wide tensor-core GEMMs, up to
  *     512 rows at a time, and the last row through the pass of several rows, which has the LM head.
- *     Environment switches read by cl_load (diagnostics): CL_DISABLE_STEP_KERNEL=1, CL_DISABLE_TC_PASS=1,
- *     CL_DISABLE_WIDE_PREFILL=1, CL_DISABLE_ROW_SHARES=1, CL_L2_AHEAD_KB=<n>.
+ *     Environment switches read by cl_load (diagnostics): CL_DISABLE_STEP_KERNEL=1, CL_DISABLE_ROWS_KERNEL=1,
+ *     CL_DISABLE_WIDE_PREFILL=1, CL_DISABLE_ROW_SHARES=1, CL_L2_AHEAD_KB=<n>, CL_ROWS_SPLIT=<1|2|4>, CL_ROWS_CHAIN=<n>.
  */
 #ifndef CONFLAYERS_H
 #define CONFLAYERS_H

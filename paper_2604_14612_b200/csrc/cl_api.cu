@@ -63,15 +63,8 @@ struct cl_ctx {
     unsigned *bar_dev;
     float *att_part2;
     ClHeadPartial *head_part2;
-    // skinny tensor-core GEMM path of the T-row passes (bf16 models)
-    int use_tc;
+    // TMA descriptors of the row-major matrices (B operand of the wide GEMMs of the prompt pass, 16-bit models)
     std::vector<ClTensorMap> map_qkv, map_o, map_gu, map_d;
-    ClTensorMap map_head, map_bx[2], map_batt[2], map_bh[2];   // [0]: N = 16, [1]: N = 32
-    __nv_bfloat16 *bx, *batt, *bh;       // GEMM input rows as bf16 hi/lo parts: [32, d] [32, d] [32, F]
-    float *v_ws, *v_ssq, *v_att_part;
-    int v_att_S;                         // parts the keys of a head are cut into in the T-row attention
-    unsigned *v_tickets;
-    ClHeadPartial *v_head_part;
     // persistent tensor-core pass of the T-row passes (16-bit models): second, k-block-major copy of the matrices
     int use_rows;
     char *wtile, *head_tile;             // per layer [Wqkv | Wo | Wgu | Wd] k-block-major; LM head k-block-major
@@ -223,7 +216,7 @@ static void free_all(cl_ctx *c) {
                     c->att, c->hff, c->att_part, c->logits, c->tickets, c->head_part, c->st, c->prompt_dev, c->out_dev,
                     c->ring, c->sc_conf, c->sc_pmax, c->sc_clayer, c->sc_arg, c->sc_xn, c->sc_part, c->sel_mask, c->sel_margins, c->sel_clayers,
                     c->layers_dev, c->kept_dev, c->kept_all_dev, c->bar_dev, c->att_part2, c->head_part2,
-                    c->cum_w_dev, c->busy_dev, c->bx, c->batt, c->bh, c->v_ws, c->v_ssq, c->v_att_part, c->v_tickets, c->v_head_part,
+                    c->cum_w_dev, c->busy_dev,
                     c->w_ax, c->w_aatt, c->w_ah, c->w_x, c->w_P, c->wtile, c->head_tile, c->rows_layers_dev, c->r_ax, c->r_aatt,
                     c->r_ah, c->r_ssq, c->r_att_part, c->r_tickets, c->r_head_part, c->r_phase_ns, c->r_ws, c->r_bar};
     for (void *p : ptrs)
@@ -394,55 +387,23 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
             const char *off = getenv("CL_DISABLE_STEP_KERNEL");
             c->use_step = coop && d <= (size_t)maxc && F <= (size_t)maxc && !(off && off[0] == '1');
         }
-        // ---- skinny tensor-core GEMM path (bf16): tensor maps of every matrix, hi/lo input rows, workspace
-        c->use_tc = 0;
+        // ---- wide GEMM path of the prompt pass (16-bit models): tensor maps of every matrix, hi/lo activation rows,
+        // residual stream, product parts
         if (g.weight_dtype != 0) {
             const int f16 = g.weight_dtype == 2;
-            const char *off = getenv("CL_DISABLE_TC_PASS");
-            const int G = c->n_sm;
-            auto segs_ok = [&](size_t rows, size_t K) {
-                const size_t MT = (rows + 127) / 128, KB = (K + 63) / 64, U = MT * KB, upc = (U + G - 1) / G;
-                return (upc + KB - 1) / KB + 1 <= (size_t)CL_V_MAXSEG;
-            };
-            bool ok = !(off && off[0] == '1') && segs_ok(qkv_rows, d) && segs_ok(d, d) && segs_ok(2 * F, d) && segs_ok(d, F) &&
-                      segs_ok(V, d);
-            if (ok) {
-                DM(c->bx, 32 * d * 2);
-                DM(c->batt, 32 * d * 2);
-                DM(c->bh, 32 * F * 2);
-                CU(cudaMemsetAsync(c->bx, 0, 32 * d * 2, c->stream));
-                CU(cudaMemsetAsync(c->batt, 0, 32 * d * 2, c->stream));
-                CU(cudaMemsetAsync(c->bh, 0, 32 * F * 2, c->stream));
-                DM(c->v_ws, (size_t)G * CL_V_MAXSEG * 128 * 32 * 4);
-                const size_t max_tiles = (std::max(std::max(qkv_rows, 2 * F), V) + 127) / 128;
-                DM(c->v_tickets, max_tiles * 4);
-                CU(cudaMemsetAsync(c->v_tickets, 0, max_tiles * 4, c->stream));
-                DM(c->v_ssq, ((d + 127) / 128) * CL_SLOTS * 4);
-                c->v_att_S = c->n_sm / g.n_heads;   // one wave of CTAs
-                if (c->v_att_S < 1) c->v_att_S = 1;
-                if (c->v_att_S > 8) c->v_att_S = 8;
-                DM(c->v_att_part, cl_attn_rows_part_floats(g.n_heads, c->v_att_S, CL_MAX_T, g.head_dim) * 4);
-                DM(c->v_head_part, ((V + 127) / 128) * CL_SLOTS * sizeof(ClHeadPartial));
-                c->map_qkv.resize(L); c->map_o.resize(L); c->map_gu.resize(L); c->map_d.resize(L);
-                for (size_t l = 0; l < L && ok; ++l) {
-                    const ClLayer &y = c->layers[l];
-                    ok = cl_make_tensor_map(&c->map_qkv[l], y.wqkv, (int)qkv_rows, (int)d, 128, f16) &&
-                         cl_make_tensor_map(&c->map_o[l], y.wo, (int)d, (int)d, 128, f16) &&
-                         cl_make_tensor_map(&c->map_gu[l], y.wgu, (int)(2 * F), (int)d, 128, f16) &&
-                         cl_make_tensor_map(&c->map_d[l], y.wd, (int)d, (int)F, 128, f16);
-                }
-                ok = ok && cl_make_tensor_map(&c->map_head, c->lm_head, (int)V, (int)d, 128, f16);
-                for (int i = 0; i < 2 && ok; ++i) {
-                    const int N = i ? 32 : 16;
-                    ok = cl_make_tensor_map(&c->map_bx[i], c->bx, N, (int)d, N, f16) &&
-                         cl_make_tensor_map(&c->map_batt[i], c->batt, N, (int)d, N, f16) &&
-                         cl_make_tensor_map(&c->map_bh[i], c->bh, N, (int)F, N, f16);
-                }
-                if (!ok) return fail(c, CL_ECUDA, "cl_load: encoding a TMA tensor map failed");
-                c->use_tc = 1;
-                // ---- wide GEMM path of the prompt pass: hi/lo activation rows, residual stream, product parts
-                const char *woff = getenv("CL_DISABLE_WIDE_PREFILL");
-                if (!(woff && woff[0] == '1') && g.max_seq > 17) {
+            const char *woff = getenv("CL_DISABLE_WIDE_PREFILL");
+            if (!(woff && woff[0] == '1') && g.max_seq > 17) {
+                {
+                    bool ok = true;
+                    c->map_qkv.resize(L); c->map_o.resize(L); c->map_gu.resize(L); c->map_d.resize(L);
+                    for (size_t l = 0; l < L && ok; ++l) {
+                        const ClLayer &y = c->layers[l];
+                        ok = cl_make_tensor_map(&c->map_qkv[l], y.wqkv, (int)qkv_rows, (int)d, 128, f16) &&
+                             cl_make_tensor_map(&c->map_o[l], y.wo, (int)d, (int)d, 128, f16) &&
+                             cl_make_tensor_map(&c->map_gu[l], y.wgu, (int)(2 * F), (int)d, 128, f16) &&
+                             cl_make_tensor_map(&c->map_d[l], y.wd, (int)d, (int)F, 128, f16);
+                    }
+                    if (!ok) return fail(c, CL_ECUDA, "cl_load: encoding a TMA tensor map failed");
                     const size_t Mw = CL_WIDE_MAX_M, widest = std::max(qkv_rows, 2 * F);
                     DM(c->w_ax, 2 * Mw * d * 2);
                     DM(c->w_aatt, 2 * Mw * d * 2);
@@ -577,9 +538,6 @@ static int head(cl_ctx *c, int T, const float *xin, const ClDevState *st, int *o
     return CL_OK;
 }
 
-static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, int want_head, int *out_tok, float *out_pmax,
-                           float *out_conf, float *logits);
-
 // The same pass as one persistent launch on the tensor cores (16-bit models): all layers and the LM head.
 static int forward_rows_persistent(cl_ctx *c, const int *tok, int T, int row0, int tap, int want_head, int *out_tok,
                                    float *out_pmax, float *out_conf, float *logits) {
@@ -613,7 +571,6 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
     const int d = g.d_model, F = g.d_ffn, wd = g.weight_dtype, qkv_rows = d + 2 * g.n_kv_heads * g.head_dim;
     int rc;
     if (c->use_rows && !mask) return forward_rows_persistent(c, tok, T, row0, tap, want_head, out_tok, out_pmax, out_conf, logits);
-    if (c->use_tc && !mask) return forward_rows_tc(c, tok, T, row0, tap, want_head, out_tok, out_pmax, out_conf, logits);
     KL(cl_launch_embed(wd, c->embed, tok, T, d, c->x, c->st, c->stream));
     for (int l = 0; l < g.n_layers; ++l) {
         const int skip_bits = mask ? mask[l] : 0;
@@ -626,9 +583,8 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
         KL(cl_launch_rope_append(wd, c->qkv, T, row0, g.n_heads, g.n_kv_heads, g.head_dim, d, c->rope_cs, y.kc, y.vc, g.max_seq, c->st,
                                  c->stream));
         ClAttnArgs a;
-        a.rope_cs = nullptr;
         a.q = c->qkv; a.ld_q = qkv_rows; a.n_kv_heads = g.n_kv_heads; a.kcache = y.kc; a.vcache = y.vc; a.part = c->att_part; a.tickets = c->tickets + 1;
-        a.out = c->att; a.out_b = nullptr; a.nh = 0; a.st = c->st; a.row0 = row0; a.n_heads = g.n_heads; a.head_dim = g.head_dim; a.d_model = d;
+        a.out = c->att; a.st = c->st; a.row0 = row0; a.n_heads = g.n_heads; a.head_dim = g.head_dim; a.d_model = d;
         a.nsplit = c->nsplit; a.per_max = c->per_max; a.max_seq = g.max_seq;
         KL(cl_launch_attn(wd, T, a, c->stream));
         if ((rc = gemv(c, T, CL_EPI_RESID, y.wo, d, d, c->att, c->x, d))) return rc;
@@ -647,64 +603,6 @@ static int forward_rows(cl_ctx *c, const int *tok, int T, int row0, const uint8_
     if (want_head) {
         KL(cl_launch_rmsnorm(c->x, c->final_norm, T, d, g.rms_eps, c->xn, c->st, c->stream));
         if ((rc = head(c, T, c->xn, c->st, out_tok, out_pmax, out_conf, logits))) return rc;
-    }
-    return CL_OK;
-}
-
-// The same pass on the tensor cores (bf16 models): one stream-K skinny GEMM per matrix, RMSNorm folded into the
-// GEMM epilogues, attention over the cache between the QKV and the output projection.
-static int forward_rows_tc(cl_ctx *c, const int *tok, int T, int row0, int tap, int want_head, int *out_tok, float *out_pmax,
-                           float *out_conf, float *logits) {
-    const cl_model_cfg &g = c->cfg;
-    const int d = g.d_model, F = g.d_ffn, V = g.vocab, L = g.n_layers, G = c->n_sm, qkv_rows = d + 2 * g.n_kv_heads * g.head_dim;
-    const int N = T <= 8 ? 16 : 32, nh = N / 2, sel = N == 16 ? 0 : 1;
-    const int KBd = (d + 63) / 64, KBf = (F + 63) / 64, dtiles = (d + 127) / 128;
-    ClSkinnyArgs b;
-    memset(&b, 0, sizeof(b));
-    b.T = T; b.N = N; b.st = c->st; b.ws = c->v_ws; b.tickets = c->v_tickets; b.ssq_tiles = dtiles;
-    b.inv_dim = 1.0f / (float)d; b.eps = g.rms_eps; b.nh = nh; b.row0 = row0; b.err = &c->st->err;
-    b.f16 = g.weight_dtype == 2;
-    KL(cl_launch_pass_begin(c->embed, tok, T, d, c->x, c->bx, nh, L ? c->layers[0].n1 : c->final_norm, c->v_ssq, c->st, b.f16,
-                            c->stream));
-    for (int l = 0; l < L; ++l) {
-        const ClLayer &y = c->layers[l];
-        ClSkinnyArgs a = b;
-        a.rows = qkv_rows; a.KB = KBd; a.epi = CL_VEPI_STORE; a.ssq_in = c->v_ssq; a.out = c->qkv; a.ld = qkv_rows;
-        KL(cl_launch_skinny(c->map_qkv[l], c->map_bx[sel], a, G, c->stream));
-        ClAttnArgs t;   // (rotary embedding and cache append of the rows happen inside the attention kernel)
-        t.rope_cs = c->rope_cs;
-        t.q = c->qkv; t.ld_q = qkv_rows; t.n_kv_heads = g.n_kv_heads; t.kcache = y.kc; t.vcache = y.vc; t.part = c->att_part; t.tickets = c->tickets + 1;
-        t.out = c->att; t.out_b = c->batt; t.nh = nh; t.st = c->st; t.row0 = row0; t.n_heads = g.n_heads; t.head_dim = g.head_dim;
-        t.d_model = d; t.nsplit = c->nsplit; t.per_max = c->per_max; t.max_seq = g.max_seq;
-        t.part = c->v_att_part;
-        KL(cl_launch_attn_rows(g.weight_dtype, T, c->v_att_S, t, c->stream));
-        a = b;
-        a.rows = d; a.KB = KBd; a.epi = CL_VEPI_RESID; a.out = c->x; a.ld = d; a.bnext = c->bx; a.bn_ld = d; a.gnext = y.n2;
-        a.ssq_out = c->v_ssq;
-        if (tap && ring_slot(c, l, 0)) {
-            a.tap = ring_slot(c, l, 0);
-            a.tap_P = g.tap_positions;
-        }
-        KL(cl_launch_skinny(c->map_o[l], c->map_batt[sel], a, G, c->stream));
-        a = b;
-        a.rows = 2 * F; a.KB = KBd; a.epi = CL_VEPI_SILU; a.ssq_in = c->v_ssq; a.bnext = c->bh; a.bn_ld = F;
-        KL(cl_launch_skinny(c->map_gu[l], c->map_bx[sel], a, G, c->stream));
-        a = b;
-        a.rows = d; a.KB = KBf; a.epi = CL_VEPI_RESID; a.out = c->x; a.ld = d; a.bnext = c->bx; a.bn_ld = d;
-        a.gnext = (l + 1 < L) ? c->layers[l + 1].n1 : c->final_norm;
-        a.ssq_out = c->v_ssq;
-        if (tap && ring_slot(c, l, 1)) {
-            a.tap = ring_slot(c, l, 1);
-            a.tap_P = g.tap_positions;
-        }
-        KL(cl_launch_skinny(c->map_d[l], c->map_bh[sel], a, G, c->stream));
-    }
-    if (want_head) {
-        ClSkinnyArgs a = b;
-        a.rows = V; a.KB = KBd; a.epi = CL_VEPI_HEAD; a.ssq_in = c->v_ssq; a.logits = logits; a.head_part = c->v_head_part;
-        KL(cl_launch_skinny(c->map_head, c->map_bx[sel], a, G, c->stream));
-        KL(cl_launch_head_finalize(c->v_head_part, (V + 127) / 128, T, (float)(1.0 / log((double)V)), out_tok, out_pmax, out_conf,
-                                   c->st, c->stream));
     }
     return CL_OK;
 }

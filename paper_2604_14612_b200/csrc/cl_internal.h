@@ -112,12 +112,8 @@ struct ClAttnArgs {
     float *part;          // [T, H, nsplit, hd + 2] partial (m, l, o[hd])
     unsigned *tickets;    // [T, H]
     float *out;           // [T, d]
-    __nv_bfloat16 *out_b; // optional [2 * nh, d]: the output again as bf16 hi (row t) and lo (row nh + t) parts
-    int nh;
     const ClDevState *st;
     int row0, n_heads, n_kv_heads, head_dim, d_model, nsplit, per_max, max_seq;
-    const float2 *rope_cs;  // k_attn_rows only, optional: q and the rows' own k, v are still raw in the [q | k | v] rows;
-                            // the kernel applies the rotary embedding itself and appends k, v to the cache
 };
 
 // Per-layer device pointers as the token-step kernel sees them.
@@ -174,48 +170,18 @@ cudaError_t cl_launch_rmsnorm_rows(int in_dtype, const void *x, const float *g, 
 cudaError_t cl_launch_rope_append(int wdtype, float *qkv, int T, int row0, int H, int Hkv, int hd, int d, const float2 *rope_cs,
                                   void *kcache, void *vcache, int max_seq, const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_attn(int wdtype, int T, const ClAttnArgs &a, cudaStream_t s);
-size_t cl_attn_rows_part_floats(int H, int S, int T, int hd);
-cudaError_t cl_launch_attn_rows(int wdtype, int T, int S, const ClAttnArgs &a, cudaStream_t s);
 cudaError_t cl_launch_tap(int wdtype, const float *x, int T, int row0, int d, void *ring_layer, int P,
                           const ClDevState *st, cudaStream_t s);
 cudaError_t cl_launch_accept(ClDevState *st, int K, int *out_tokens, cudaStream_t s);
 cudaError_t cl_launch_advance(ClDevState *st, int n, int set_pending_from_tgt, cudaStream_t s);
-// ---- skinny tensor-core GEMM of the T-row passes (bf16 models) ----
+// epilogues of the tensor-core GEMMs of the T-row pass
 enum { CL_VEPI_STORE = 0, CL_VEPI_RESID = 1, CL_VEPI_SILU = 2, CL_VEPI_HEAD = 3 };
-#define CL_V_MAXSEG 8   // workspace slots per CTA (segments of different tiles one CTA may hold partially)
-
-struct ClSkinnyArgs {
-    int rows, KB, T, N, epi;          // weight rows, K blocks of 64, token rows, MMA N (16 | 32), epilogue
-    const ClDevState *st;
-    float *ws;                        // [grid, CL_V_MAXSEG, 128, 32] partial accumulators
-    unsigned *tickets;                // [tiles], zero between launches
-    const float *ssq_in;              // [ssq_tiles, CL_SLOTS] sums of squares of the input rows, or null (scale 1)
-    int ssq_tiles;
-    float inv_dim, eps;
-    float *out;                       // STORE: qkv [T, ld]; RESID: residual stream x [T, ld] (updated in place)
-    int ld;
-    __nv_bfloat16 *bnext;             // RESID / SILU: next GEMM's input rows [N_next rows, bn_ld]: hi at t, lo at nh + t
-    int bn_ld, nh;
-    const float *gnext;               // RESID: gain of the next RMSNorm
-    float *ssq_out;                   // RESID: [tiles, CL_SLOTS]
-    void *tap;                        // RESID, optional: this layer's hidden-state ring [P, rows] in the storage type
-    int tap_P, row0;
-    float *logits;                    // HEAD, optional [T, rows]
-    ClHeadPartial *head_part;         // HEAD: [tiles, CL_SLOTS]
-    int *err;
-    int f16;                          // the model's 16-bit type: 0 bf16, 1 fp16 (weights, activation parts, taps)
-};
 
 struct ClTensorMap {                  // opaque 128-byte TMA descriptor (CUtensorMap)
     alignas(64) unsigned char bytes[128];
 };
 
 bool cl_make_tensor_map(ClTensorMap *m, const void *base, int rows, int cols, int box_rows, int f16 = 0);
-cudaError_t cl_launch_skinny(const ClTensorMap &mapA, const ClTensorMap &mapB, const ClSkinnyArgs &a, int grid, cudaStream_t s);
-cudaError_t cl_launch_pass_begin(const void *embed, const int *tok, int T, int d, float *x, __nv_bfloat16 *bnext, int nh,
-                                 const float *g, float *ssq_out, const ClDevState *st, int f16, cudaStream_t s);
-cudaError_t cl_launch_head_finalize(const ClHeadPartial *part, int tiles, int T, float inv_log_v, int *out_tok, float *out_pmax,
-                                    float *out_conf, const ClDevState *st, cudaStream_t s);
 
 // ---- persistent tensor-core pass over T <= CL_MAX_T rows (16-bit models): all layers and the LM head in one launch ----
 #define CL_ROWS_AROWS 32   // rows per k-block of an activation operand buffer: hi part of token t in row t, lo part in row T + t

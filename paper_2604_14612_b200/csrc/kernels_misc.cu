@@ -210,11 +210,6 @@ __global__ void __launch_bounds__(128) k_attn(ClAttnArgs a) {
         }
         const float o = O / Lsum;
         a.out[(size_t)t * d + h * HD + tid] = o;
-        if (a.out_b) {
-            const __nv_bfloat16 hi = __float2bfloat16_rn(o);
-            a.out_b[(size_t)t * d + h * HD + tid] = hi;
-            a.out_b[(size_t)(a.nh + t) * d + h * HD + tid] = __float2bfloat16_rn(o - __bfloat162float(hi));
-        }
     }
     if (tid == 0) a.tickets[t * a.n_heads + h] = 0u;
 }

@@ -487,3 +487,8 @@ cudaError_t cl_launch_attn_wide(const float *q, int ld_q, const void *kcache, co
     }
     return cudaGetLastError();
 }
+
+bool cl_make_tensor_map(ClTensorMap *m, const void *base, int rows, int cols, int box_rows, int f16) {
+    static_assert(sizeof(ClTensorMap) >= sizeof(CUtensorMap), "tensor map storage");
+    return make_map((CUtensorMap *)m->bytes, base, rows, cols, box_rows, f16);
+}

@@ -15,7 +15,7 @@ from oracle.selection import SelectConfig, select_skip_set, selection_details
 
 pytestmark = pytest.mark.gpu
 
-from harness import (NEAR_TIE, TOL, Report, lockstep_generate, make_pair, oracle_prefill_hidden,  # noqa: E402
+from harness import (NEAR_TIE, TOL, Report, depth_tol, lockstep_generate, make_pair, oracle_prefill_hidden,  # noqa: E402
                      ring_in_position_order)
 
 
@@ -255,8 +255,8 @@ def test_generate_to_the_last_cache_slot():
 
 @pytest.mark.parametrize("wd", ["bf16", "fp16"])
 def test_tensor_core_pass_matches_streaming_pass(monkeypatch, wd):
-    """The tcgen05 pass (verify / prefill of 16-bit models) against the CUDA-core T-row path on the same inputs:
-    two independent implementations of the same full-model pass, T = 5 (N = 16) and T = 9 (N = 32)."""
+    """The persistent tcgen05 pass (verify / short prompt chunks of 16-bit models) against the CUDA-core T-row path on the
+    same inputs: two independent implementations of the same full-model pass, T = 5, 9, 2 and 1 rows."""
     base = synth.WORKLOADS["C2"].shape
     sh = dataclasses.replace(base, n_layers=2, max_seq=64, weight_dtype=wd)
     W = synth.make_weights(sh, 5, device="cuda")
@@ -264,7 +264,6 @@ def test_tensor_core_pass_matches_streaming_pass(monkeypatch, wd):
     out = {}
     for tc in (0, 1):
         monkeypatch.setenv("CL_DISABLE_ROWS_KERNEL", "0" if tc else "1")
-        monkeypatch.setenv("CL_DISABLE_TC_PASS", "0" if tc else "1")
         ctx = cl.Context.from_shape(sh, tap_positions=16)               # longer than any pass: no two rows share a slot
         ctx.cl_load(W)
         first = ctx.cl_prefill(prompt, tap_hidden=True)
@@ -366,6 +365,42 @@ def test_interval_search_matches_oracle_on_c1():
         assert got["scores"] == pytest.approx(ref2["scores"], abs=1e-6)
         assert got["sets"] == ref2["sets"] and got["best_round"] == ref2["best_round"]
         assert got["final_set"] == ref2["final_set"] and got["searching"] == ref2["searching"]
+
+
+def test_interval_search_matches_oracle_on_a_bf16_model():
+    """Section 3.3 driver end to end on a 16-bit model (the 12-layer shape cut to 4 layers): the verify passes of the
+    persistent tensor-core kernel write the hidden taps, the tensor-core scoring kernel turns the ring into layer
+    confidences, the selection kernel picks the next set, and drafting goes on with it.  Rounds, scores, sets and tokens
+    equal the oracle's loop; a run whose trajectory meets a near tie is only compared up to it."""
+    w = synth.reduced(synth.WORKLOADS["C2"], n_layers=4, prompt_len=24, gen_len=8)
+    P, K, max_new, interval, max_rounds = 8, 3, 40, 4, 2
+    sh = dataclasses.replace(w.shape, max_seq=128)
+    om, ctx, Wh = make_pair(sh, w.seed + 2, tap_positions=P)
+    prompt = synth.make_prompt(w.seed, 24, sh.vocab)
+    oc = SelectConfig(n_layers=sh.n_layers, lo=1, hi=2, n_skip=1)
+    sc = cl.SelectCfg.make(1, 2, n_skip=1)
+    compared = 0
+    for initial, goal in (([1, 2], 10.0), ([2], 0.0), ([1], 10.0)):
+        ref = oracle.generate_search(om, Wh, prompt, initial, K, max_new, interval, goal, max_rounds, oc, P,
+                                     storage_dtype=torch.bfloat16)
+        van = oracle.generate_vanilla(om, prompt, max_new)
+        first = ctx.cl_prefill(prompt, tap_hidden=True)
+        ctx.cl_set_skip_set(synth.layers_to_mask(initial, sh.n_layers))
+        got = ctx.cl_generate_search(K, max_new - 1, interval, goal, max_rounds, sc)
+        toks = [first] + [int(t) for t in got["tokens"]]
+        lim = next((i for i, m in enumerate(van["margins"]) if m < NEAR_TIE), max_new)
+        assert toks[:lim] == ref["tokens"][:lim]
+        if lim < max_new:
+            continue   # the trajectories may part at the near tie: rounds are no longer comparable
+        compared += 1
+        assert got["scores"] == pytest.approx(ref["scores"], abs=1e-6)
+        assert got["best_round"] == ref["best_round"] and got["searching"] == ref["searching"]
+        if got["sets"] != ref["sets"] or got["final_set"] != ref["final_set"]:
+            # two eligible layers, one to skip: the sets may only differ where their confidences nearly tie
+            h = torch.tensor(ctx.cl_read_hidden_ring().float().numpy())
+            c = oracle.layer_confidences(h.to(torch.bfloat16), Wh["lm_head"], Wh["final_norm"], sh.rms_eps)["c_layer"]
+            assert abs(c[1] - c[2]) < 5e-3, (got["sets"], ref["sets"], c)
+    print("bf16 interval search: runs compared in full:", compared)
 
 
 @pytest.mark.parametrize("name", ["C1", "C2"])
@@ -479,23 +514,23 @@ def test_full_size_properties_in_the_bench_configuration(name, K, ratio, gen, wd
     _first_difference_is_a_near_tie(ctx, w, list(van), list(full), first)
 
 
-def test_c3_full_depth_against_oracle():
-    """All 32 layers of the 7B shape, short prompt: every draft / verify logit row and token against the oracle.
-
-    Tolerance 4e-2 instead of 1e-2, and the same margin for counted near ties.  The KV cache is stored in bf16:
-    a key or value that lands within rounding noise of a bf16 boundary is rounded differently by two correct
-    implementations, which moves that element by 2^-9 relative.  Measured at this shape with an independent fp64
-    reference: perturbing K/V by 1e-7 relative (fp32 rounding noise) before the bf16 rounding moves the logits of
-    an 8-layer model by 3e-3, the oracle itself sits 3.4e-3 from the fp64 reference at 8 layers, and the distance
-    grows like sqrt(depth): at 32 layers the CUDA-core path (fp32 activations) is 1.4e-2 from the oracle and the
-    tensor-core pass 2.5e-2.  The stated 1e-2 is kept wherever the depth is at most 12 layers."""
-    w = synth.reduced(synth.WORKLOADS["C3"], n_layers=32, prompt_len=12, gen_len=5)
+@pytest.mark.parametrize("name,prompt_len,K,ratio", [("C3", 12, 4, 0.5), ("C4", 8, 6, 0.4)])
+def test_full_depth_against_oracle(name, prompt_len, K, ratio):
+    """All 32 layers of the 7B shape and all 40 of the 13B shape, short prompt: every draft / verify logit row, token and
+    accept count against the oracle.  The tolerance on logits, and the near-tie margin with it, is the bound for this
+    depth that tests/test_gpu_depth.py measures and enforces (2.4e-2 at 32 layers, 3.9e-2 at the 13B shape's 40): at this depth the
+    bf16 KV cache, not the kernels, decides how far two correct implementations may sit apart."""
+    w0 = synth.WORKLOADS[name]
+    L = w0.shape.n_layers
+    w = synth.reduced(w0, n_layers=L, prompt_len=prompt_len, gen_len=5 if name == "C3" else 4)
     om, ctx, _ = make_pair(w.shape, w.seed, gen_device="cuda")
     prompt = synth.make_prompt(w.seed, w.prompt_len, w.shape.vocab)
-    n_skip = synth.n_skip_for_ratio(w.lo, w.hi, 0.5)
-    mask = synth.layers_to_mask(synth.uniform_skip_layers(w.lo, w.hi, n_skip), 32)
-    rep = lockstep_generate(om, ctx, prompt, mask, 4, w.gen_len, tol=4e-2, near_tie=4e-2)
-    print("C3 full depth", rep)
+    n_skip = synth.n_skip_for_ratio(w.lo, w.hi, ratio)
+    mask = synth.layers_to_mask(synth.uniform_skip_layers(w.lo, w.hi, n_skip), L)
+    tol = depth_tol(L)
+    rep = lockstep_generate(om, ctx, prompt, mask, K, w.gen_len, tol=tol, near_tie=tol)
+    print(name, "full depth, tolerance", tol, rep)
+    assert rep.cycles >= 1 and rep.tokens_compared >= K + 2
 
 
 @pytest.mark.parametrize("name,L,kv,K", [("C1", 4, 2, 3), ("C1", 4, 1, 4), ("C2", 3, 4, 4), ("C3", 3, 8, 8)])
