@@ -132,6 +132,18 @@ def make_weights(shape: ModelShape, seed: int, device="cpu") -> Dict[str, object
     return w
 
 
+def damp_output_projections(w: Dict[str, object], layers, factor: float) -> Dict[str, object]:
+    """Scales, in place, the attention output projection and the FFN down projection of the given layers by `factor`
+    (and rounds back to the storage type): those layers then add little to the residual stream, which is what a
+    trained model's skippable layers look like to the draft model.  Random-init layers all matter equally, so a model
+    made by ``make_weights`` alone accepts almost no draft once layers are skipped."""
+    for l in layers:
+        for n in ("wo", "wd"):
+            t = w[n][int(l)]
+            w[n][int(l)] = (t.float() * factor).to(t.dtype).contiguous()
+    return w
+
+
 def weights_to(w: Dict[str, object], device) -> Dict[str, object]:
     """Copy a weight dict to another device (bit-identical values)."""
     out: Dict[str, object] = {}
