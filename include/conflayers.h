@@ -199,7 +199,8 @@ int cl_score_loop(cl_ctx *ctx, const cl_select_cfg *cfg, const void *const *hidd
  * max_rounds searched sets, the search ends and the best set drafts for the rest of the call (it stays installed).
  * Otherwise the layers are scored on the hidden-state ring (Section 3.1), a new set is selected with *sel
  * (Section 3.2) and installed.  Needs tap_positions > 0 and a cl_prefill with tap_hidden = 1 (which clears the
- * ring); verify passes record the ring while the search is on.  The emitted tokens do not depend on the search.
+ * ring); while the search is on the verify passes of the last tap_positions cycles of an interval record the ring (earlier
+ * ones would be overwritten before the search check).  The emitted tokens do not depend on the search.
  * out: host [max_new].  rep (may be NULL): scores[i] of round i, i < n_scored; masks (host, may be NULL):
  * [(max_rounds + 1), n_layers], row i = the set of round i. */
 #define CL_MAX_ROUNDS 32

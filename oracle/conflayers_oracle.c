@@ -75,13 +75,24 @@ float orc_fp16_bits_to_f32(uint16_t b) {
     return (float)(sign ? -v : v);
 }
 
-/* all 65536 widenings, filled once (by whichever thread gets there first; every thread writes the same values) */
+/* all 65536 widenings, filled once: under a lock, and published only after the table is complete (threads of a
+ * parallel region may arrive here together) */
 static const float *fp16_table(void) {
     static float table[65536];
-    static volatile int ready = 0;
-    if (!ready) {
-        for (int b = 0; b < 65536; ++b) table[b] = orc_fp16_bits_to_f32((uint16_t)b);
-        ready = 1;
+    static int ready = 0;
+    int r;
+#pragma omp atomic read
+    r = ready;
+    if (!r) {
+#pragma omp critical(orc_fp16_table)
+        {
+            if (!ready) {
+                for (int b = 0; b < 65536; ++b) table[b] = orc_fp16_bits_to_f32((uint16_t)b);
+#pragma omp flush
+#pragma omp atomic write
+                ready = 1;
+            }
+        }
     }
     return table;
 }

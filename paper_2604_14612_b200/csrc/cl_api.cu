@@ -1045,8 +1045,10 @@ extern "C" int cl_generate_search(cl_ctx *c, const cl_search_cfg *sc, const cl_s
         const unsigned long long cyc0 = c->h_st->cycles, acc0 = c->h_st->accepted;
         // while searching: one interval; afterwards: the fewest cycles that can finish (cycles past the end exit at once)
         const int ncyc = r.searching ? sc->interval : (remaining + K) / (K + 1);
+        // Taps while searching: every cycle advances by at least one position, so the last P cycles of an interval rewrite
+        // every slot of the ring (slot = position mod P); what earlier cycles would record is gone by the search check.
         for (int i = 0; i < ncyc; ++i)
-            if ((rc = enqueue_cycle(c, K, r.searching))) return rc;
+            if ((rc = enqueue_cycle(c, K, r.searching && ncyc - i <= P))) return rc;
         const int ctx_before = c->h_ctx;
         if ((rc = sync_state(c))) return rc;
         if ((rc = check_device_err(c, "cl_generate_search"))) return rc;

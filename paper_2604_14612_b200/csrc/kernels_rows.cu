@@ -6,7 +6,8 @@
 // step kernel: one CTA per SM, every CTA owns a contiguous block of rows of every matrix (single-row granularity, so
 // all SMs stream the same number of bytes), one producer thread walks the static schedule and keeps a 192 KB ring of
 // weight tiles filled straight through the phase boundaries, and the phases of a layer (QKV | attention | O |
-// gate/up | down) are separated by grid barriers, not by launches.  What differs is the arithmetic: 2 T activation
+// gate/up | down) follow one another inside the launch, ordered by completion counters per buffer (below), not by
+// launches.  What differs is the arithmetic: 2 T activation
 // rows against every weight row is more than the CUDA cores issue at the HBM rate, so the contraction runs on the
 // tensor cores:
 //
@@ -25,7 +26,8 @@
 //     equal on both sides); rows in front of g0 and behind g1 are stale -- column n of D depends on row n of B
 //     only, and those columns are never read.
 // The accumulator lives in tensor memory (two buffers of 256 columns); it is drained into fp32 registers after
-// every ring slot (64 to 320 elements of K), so a long K is summed in fp32 registers, not in one tensor-core chain.
+// every `chain` ring slots (4 by default; a slot holds 64 to 320 elements of K), so a long K is summed in fp32
+// registers in pieces, not in one tensor-core chain: the pieces bound the rounding error of the chain.
 // Warp roles: warps 0-13 workers (embedding, attention, epilogues; warps 0, 4, 8, 12 are the four that can read
 // tensor-memory lanes 0-31 and drain the accumulator), warp 14 producer, warp 15 MMA issue and tensor-memory owner.
 // RMSNorm is split around the GEMM as in the other tensor-core kernels: the activation operand holds x * gain,
@@ -225,30 +227,6 @@ struct Cursor {
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(RT) : "memory"); }
 __device__ __forceinline__ void drain_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
-__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(s_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(s_u32(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_g2s_stream(void *dst, const void *src, unsigned bytes, unsigned long long *bar,
-                                                unsigned long long policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
-            s_u32(dst)),
-        "l"(src), "r"(bytes), "r"(s_u32(bar)), "l"(policy)
-        : "memory");
-}
-// Non-blocking look at an mbarrier phase.  (mbarrier.try_wait may suspend the thread for a while before it answers
-// "not yet"; a loop that serves two queues must not sit in it.)
-__device__ __forceinline__ bool bar_test(unsigned long long *b, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(s_u32(b)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
 // Orders this thread's generic-proxy accesses of global memory with async-proxy (bulk copy) accesses.
 __device__ __forceinline__ void proxy_fence_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 
@@ -332,8 +310,7 @@ __device__ __forceinline__ ClHeadPartial rp_merge(const ClHeadPartial &a, const 
 // slot is free -- weights never change, so the stream runs ahead of the grid barriers; the activation tiles of a slot
 // are requested once the completion counters of their k-blocks say so, both on the slot's one mbarrier.
 __device__ void producer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, int lane) {
-    unsigned long long policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    const unsigned long long policy = policy_evict_first();
     Cursor w(a), q(a);                     // weight cursor; head of the queue of slots that still lack their activation tiles
     const unsigned abytes = (unsigned)w.ars * 128u;
     unsigned slot = 0, par = 0;            // ring slot of the weight cursor

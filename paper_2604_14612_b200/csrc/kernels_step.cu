@@ -15,7 +15,7 @@
 //
 // Every wait (mbarrier or grid barrier) is bounded in time; on expiry an error flag is set, every later
 // wait falls through, the kernel runs to its end with meaningless data and the host reports CL_ETIMEOUT.
-#include "cl_internal.h"
+#include "tc_common.cuh"
 
 namespace {
 
@@ -38,42 +38,16 @@ struct Smem {
     unsigned long long wait_ns;   // bound on any single wait (copied from the launch arguments)
 };
 
-__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ unsigned long long gtime() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-__device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(unsigned long long *bar, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
 // Bounded wait.  Returns false (and raises the abort flags) if the phase did not complete in time.
 __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, Smem *sm, ClDevState *st) {
-    if (mbar_try(bar, parity)) return true;
+    if (bar_try(bar, parity)) return true;
     if (*(volatile int *)&sm->abort) return false;
-    const unsigned long long t0 = gtime();
+    const unsigned long long t0 = gtime_ns();
     for (unsigned i = 1;; ++i) {
-        if (mbar_try(bar, parity)) return true;
+        if (bar_try(bar, parity)) return true;
         if ((i & 63u) == 0u) {
             if (*(volatile int *)&sm->abort) return false;
-            if (gtime() - t0 > sm->wait_ns) {
+            if (gtime_ns() - t0 > sm->wait_ns) {
                 *(volatile int *)&sm->abort = 1;
                 atomicOr(&st->err, 1);
                 return false;
@@ -83,21 +57,6 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
 }
 
 
-// Bulk asynchronous copy global -> shared (completion counted in bytes on an mbarrier), marking the lines
-// evict-first in L2: streamed weights are used once per token.
-__device__ __forceinline__ void bulk_g2s_stream(void *dst, const void *src, unsigned bytes, unsigned long long *bar,
-                                                unsigned long long policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
-            smem_u32(dst)),
-        "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
-        : "memory");
-}
-__device__ __forceinline__ unsigned long long policy_evict_first() {
-    unsigned long long p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
 // Ask L2 to fetch a 16-byte-aligned range (multiple of 16 bytes); nothing waits for it.
 __device__ __forceinline__ void l2_prefetch_bulk(const void *src, unsigned bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
@@ -122,12 +81,12 @@ __device__ __forceinline__ void grid_barrier(unsigned *bar, unsigned &target, un
         unsigned v;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
         if ((int)(v - target) < 0) {
-            const unsigned long long t0 = gtime();
+            const unsigned long long t0 = gtime_ns();
             unsigned i = 0;
             do {
                 asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
                 if ((++i & 255u) == 0u) {
-                    if (*(volatile int *)&st->err || gtime() - t0 > sm->wait_ns) {
+                    if (*(volatile int *)&st->err || gtime_ns() - t0 > sm->wait_ns) {
                         *(volatile int *)&sm->abort = 1;
                         atomicOr(&st->err, 2);
                         break;
@@ -368,21 +327,21 @@ __device__ void producer_loop(const ClStepArgs &a, unsigned char *ring, Smem *sm
             const char *psrc;
             unsigned pbytes;
             while (fetched < filled + bytes && pf.next(psrc, pbytes)) fetched += pbytes;   // never behind the fill cursor
-            if (!mbar_try(&sm->empty[rg.slot], rg.par ^ 1u)) {
+            if (!bar_try(&sm->empty[rg.slot], rg.par ^ 1u)) {
                 // ring full: the consumers are held up, HBM would go idle; spend the time fetching into L2
-                while (fetched < filled + bytes + ahead && !mbar_try(&sm->empty[rg.slot], rg.par ^ 1u) && pf.next(psrc, pbytes)) {
+                while (fetched < filled + bytes + ahead && !bar_try(&sm->empty[rg.slot], rg.par ^ 1u) && pf.next(psrc, pbytes)) {
                     l2_prefetch_bulk(psrc, pbytes);
                     fetched += pbytes;
                 }
             }
         }
-        if (!mbar_try(&sm->empty[rg.slot], rg.par ^ 1u)) {
+        if (!bar_try(&sm->empty[rg.slot], rg.par ^ 1u)) {
             // (a slot stays taken for good once the consumers have stopped early: look at their flag while waiting)
-            const unsigned long long t0 = gtime();
-            for (unsigned i = 1; !mbar_try(&sm->empty[rg.slot], rg.par ^ 1u); ++i) {
+            const unsigned long long t0 = gtime_ns();
+            for (unsigned i = 1; !bar_try(&sm->empty[rg.slot], rg.par ^ 1u); ++i) {
                 if ((i & 31u) == 0u) {
                     if (*(volatile int *)&sm->halt || *(volatile int *)&sm->abort) break;
-                    if (gtime() - t0 > sm->wait_ns) {
+                    if (gtime_ns() - t0 > sm->wait_ns) {
                         *(volatile int *)&sm->abort = 1;
                         atomicOr(&st->err, 1);
                         break;
@@ -392,7 +351,7 @@ __device__ void producer_loop(const ClStepArgs &a, unsigned char *ring, Smem *sm
         }
         if (*(volatile int *)&sm->halt) break;
         if (!*(volatile int *)&sm->abort) {
-            mbar_expect_tx(&sm->full[rg.slot], bytes);
+            bar_expect(&sm->full[rg.slot], bytes);
             bulk_g2s_stream(ring + (size_t)rg.slot * SLOT_BYTES, src, bytes, &sm->full[rg.slot], policy);
             last_par[rg.slot] = rg.par;
         }
@@ -403,9 +362,9 @@ __device__ void producer_loop(const ClStepArgs &a, unsigned char *ring, Smem *sm
     // consumers have already waited for all of them; after an abort this is the bounded wait for copies in flight.
     for (int i = 0; i < NSLOT; ++i) {
         if (last_par[i] < 2u) {
-            const unsigned long long t0 = gtime();
-            while (!mbar_try(&sm->full[i], last_par[i]))
-                if (gtime() - t0 > sm->wait_ns) break;
+            const unsigned long long t0 = gtime_ns();
+            while (!bar_try(&sm->full[i], last_par[i]))
+                if (gtime_ns() - t0 > sm->wait_ns) break;
         }
     }
 }
@@ -456,7 +415,7 @@ __device__ __forceinline__ void consume_rows(int r0, int r1, int nchunks, int rp
     constexpr int SH = 5 - Log2<R>::v;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned rowbytes = (unsigned)nchunks * 16u;
-    const unsigned ring_addr = smem_u32(ring);
+    const unsigned ring_addr = s_u32(ring);
     // Byte offset of this thread's it-th chunk inside a row.  Chunks past the end of the row are redirected to the
     // row's last chunk: its (finite) weights meet activation registers that hold zeros.
     unsigned coff[NIT];
@@ -491,7 +450,7 @@ __device__ __forceinline__ void consume_rows(int r0, int r1, int nchunks, int rp
                 }
                 if (g + R >= ns) {   // every read of this slot has returned: hand it back to the producer
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm->empty[rg.slot]);
+                    if (lane == 0) bar_arrive(&sm->empty[rg.slot]);
                 }
                 warp_reduce_rows<R>(acc, lane);
                 const int row = sr + g + ((lane >> SH) & (R - 1));
@@ -512,14 +471,14 @@ __device__ __forceinline__ void consume_matrix(int rows, int cols, int unit, con
     constexpr int EPC = Chunk<WT>::EPC;
     int r0, r1;
     my_rows(rows, unit, cum_w, r0, r1);
-    const unsigned long long t_start = busy ? gtime() : 0ull;   // calibration launches only
+    const unsigned long long t_start = busy ? gtime_ns() : 0ull;   // calibration launches only
     const int nchunks = cols / EPC;
     const int rps = rows_per_slot((size_t)nchunks * 16, unit);
     const int nit = (nchunks + NCT - 1) / NCT;   // uniform over the grid
     if (nit <= 1) consume_rows<WT, 1, 4>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
     else if (nit <= 2) consume_rows<WT, 2, 2>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
     else consume_rows<WT, 4, 1>(r0, r1, nchunks, rps, xr, rg, ring, sm, st, epi);
-    if (busy) *busy += gtime() - t_start;
+    if (busy) *busy += gtime_ns() - t_start;
 }
 
 __device__ __forceinline__ float row_sum(const Smem *sm, int r) {
@@ -900,8 +859,8 @@ __global__ void __launch_bounds__(NCT + 32, 1) k_token_steps(ClStepArgs a) {
 
     if (tid == 0) {
         for (int i = 0; i < NSLOT; ++i) {
-            mbar_init(&sm->full[i], 1);
-            mbar_init(&sm->empty[i], NCW);
+            bar_init(&sm->full[i], 1);
+            bar_init(&sm->empty[i], NCW);
         }
         sm->abort = 0;
         sm->halt = 0;

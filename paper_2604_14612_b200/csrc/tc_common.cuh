@@ -51,6 +51,39 @@ __device__ __forceinline__ bool bar_wait(unsigned long long *b, unsigned parity,
     }
 }
 
+// Non-blocking look at an mbarrier phase.  (mbarrier.try_wait may suspend the thread for a while before it answers
+// "not yet"; a loop that serves two queues must not sit in it.)
+__device__ __forceinline__ bool bar_test(unsigned long long *b, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(s_u32(b)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bulk asynchronous copy global -> shared (16-byte aligned addresses, size a multiple of 16 bytes; completion counted
+// in bytes on an mbarrier).  The _stream form marks the lines evict-first in L2: streamed weights are used once per pass.
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(s_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(s_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_g2s_stream(void *dst, const void *src, unsigned bytes, unsigned long long *bar,
+                                                unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+            s_u32(dst)),
+        "l"(src), "r"(bytes), "r"(s_u32(bar)), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ unsigned long long policy_evict_first() {
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
 // Ticket of a "last arrival finishes the job" protocol, taken by ONE thread after a barrier of the threads that wrote
 // the data and before the barrier after which they read other CTAs' data: the release half orders the CTA's earlier
 // writes (made visible to this thread by the barrier) before the increment, the acquire half orders the later reads
