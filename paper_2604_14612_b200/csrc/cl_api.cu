@@ -73,10 +73,11 @@ struct cl_ctx {
     float *r_ssq, *r_att_part, *r_ws;
     unsigned *r_bar;                     // counters of the pass: the grid barrier, one per group of CTAs, the completion counters
     int r_sync_words, r_c_ssq, r_c_ax, r_c_ah, r_c_att, r_c_qkv;
+    int rows_entry;                      // bytes per ring entry of the T-row pass (as many k-blocks as fit, at least one)
     int rows_split;                      // CTAs per group that cut the K range of the output / down projections between them
     unsigned *r_tickets;
     ClHeadPartial *r_head_part;
-    int rows_chain;                      // ring slots per accumulation chain in tensor memory
+    int rows_chain;                      // k-blocks per accumulation chain in tensor memory
     unsigned long long *r_phase_ns;      // diagnostics (cl_debug_read): per-CTA time by phase of the last pass
     // wide tensor-core GEMM path of the prompt pass (bf16 models)
     int use_wide;
@@ -478,8 +479,11 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 CU(cudaMemsetAsync(c->r_tickets, 0, (size_t)g.n_heads * 4, c->stream));
                 DM(c->r_head_part, (size_t)c->n_sm * CL_SLOTS * sizeof(ClHeadPartial));
                 const char *ch = getenv("CL_ROWS_CHAIN");   // tuning knob
-                c->rows_chain = (ch && ch[0]) ? atoi(ch) : 4;
+                c->rows_chain = (ch && ch[0]) ? atoi(ch) : 8;
                 if (c->rows_chain < 1) c->rows_chain = 1;
+                const char *en = getenv("CL_ROWS_ENTRY_KB");   // tuning knob
+                c->rows_entry = ((en && en[0]) ? atoi(en) : 64) * 1024;
+                if (c->rows_entry < 1024) c->rows_entry = 1024;
                 c->use_rows = 1;
             }
         }
@@ -551,7 +555,7 @@ static int forward_rows_persistent(cl_ctx *c, const int *tok, int T, int row0, i
     if (a.att_parts < 1) a.att_parts = 1;
     if (a.att_parts > 8) a.att_parts = 8;
     a.tap = tap && c->ring; a.tap_P = g.tap_positions;
-    a.chain = c->rows_chain; a.split = c->rows_split; a.ws = c->r_ws;
+    a.entry = c->rows_entry; a.chain = c->rows_chain; a.split = c->rows_split; a.ws = c->r_ws;
     a.eps = g.rms_eps; a.inv_d = 1.0f / (float)g.d_model; a.inv_log_v = (float)(1.0 / log((double)g.vocab));
     a.rope_cs = c->rope_cs; a.st = c->st; a.tok = tok;
     a.x = c->x; a.qkv = c->qkv; a.Ax = c->r_ax; a.Aatt = c->r_aatt; a.Ah = c->r_ah;

@@ -200,7 +200,8 @@ struct ClRowsArgs {
     int d, F, V, H, Hkv, hd, max_seq;
     int T, row0, want_head, f16, att_parts, tap, tap_P;
     int split;                          // CTAs of a group that share the rows of an output / down projection and cut K between them
-    int chain;                          // ring slots summed in tensor memory before the accumulator is drained into registers
+    int entry;                          // bytes: a ring entry (one group of bulk copies) takes as many k-blocks of a tile as fit in this, at least one
+    int chain;                          // k-blocks (64 elements of K) summed in tensor memory before the accumulator is drained into registers
     float eps, inv_d, inv_log_v;
     const float2 *rope_cs;
     ClDevState *st;

@@ -45,8 +45,8 @@ namespace {
 constexpr int RW = 14;                 // worker warps (16 warps in all: four per scheduler, 128 registers per thread)
 constexpr int RT = RW * 32;            // worker threads
 constexpr int R_THREADS = RT + 64;     // + producer warp + MMA warp
-constexpr int R_SLOT = 32768;          // ring slot
-constexpr int R_NSLOT = 6;             // 192 KB of tiles in flight per SM
+constexpr int R_RING = 196608;         // ring of tiles in flight per SM, allocated by the byte (multiples of 1 KB)
+constexpr int R_NE = 16;               // most ring entries (bulk-copy groups with their own pair of mbarriers) in flight
 constexpr int R_MAXN = 224;            // most rows of a weight tile (tile + activation rows fill a slot at one k-block)
 constexpr int R_CTRL_BYTES = 16384;    // control block behind the ring (at least 16 KB: see the kernel)
 constexpr int R_ATT_MAXS = 8;          // most parts the cached keys of a head are cut into
@@ -55,7 +55,8 @@ constexpr int R_STAGE_LD = R_MAXN + 1;  // row pitch of the epilogue staging buf
 constexpr int R_STAGE_FLOATS = 2032;   // staging buffer: a GEMM tile's raw products of every token row
 
 struct RSmem {
-    unsigned long long full[R_NSLOT], empty[R_NSLOT], tfull[2], tempty[2];
+    unsigned long long full[R_NE], empty[R_NE], tfull[2], tempty[2];
+    unsigned vstart[R_NE];             // producer: where an entry in flight starts in the ring's running byte count
     unsigned long long wait_ns;
     unsigned tmem_base;
     int abort;
@@ -64,6 +65,7 @@ struct RSmem {
     float red[CL_SLOTS];
     float esum[16][CL_SLOTS];          // embedding phase: per-chunk sums of squares
     ClHeadPartial hpw[RW];             // LM head: per-warp statistics
+    float wsum[RW];                    // residual phase: per-warp sums of squares
     // one buffer, used in turn by: the GEMM epilogues (raw products of a tile, [T][R_STAGE_LD]); the residual epilogue
     // ([T][64] squares); the attention phase (per-warp (max, sum, o[hd]) records, [RW][hd + 2])
     alignas(16) float stage[R_STAGE_FLOATS];
@@ -108,14 +110,14 @@ __device__ __forceinline__ unsigned counter_read(const unsigned *c) {
 
 // ---- schedule ---------------------------------------------------------------------------------------
 // GEMM jobs in execution order: job 4 l + m = matrix m of layer l (0 QKV, 1 O, 2 gate/up, 3 down), job 4 L = LM head.
-// A CTA's rows [r0, r1) of a job are cut into groups of at most R_MAXN tile rows; a group's K range into ring slots
+// A CTA's rows [r0, r1) of a job are cut into groups of at most R_MAXN tile rows; a group's K range into ring entries
 // of as many k-blocks as fit.  Producer, MMA issuer and drain warps walk the same sequence.
 struct Job {
     const char *W;        // k-block-major weights
     const unsigned short *A;
     int rows, KB, unit, epi;
     int dep, dep_shift;   // k-block kb of the activation operand is complete when counter dep + (kb >> dep_shift) ...
-    unsigned dep_target;  // ... has reached this value (see "completion counters" below)
+    unsigned dep_target;  // ... has reached this value (see "completion counters")
     int split;            // CTAs that share a row block and cut its K range between them (1: every CTA owns rows over all of K)
 };
 
@@ -168,27 +170,46 @@ struct Cursor {
     unsigned stride;          // bytes between the k-block tiles of a slot (activation rows + weight rows)
     size_t wbase;             // byte offset in W of (row g0, k-block 0)
     unsigned wstep;           // bytes between k-blocks in W (the CTA's block is [K / 64][r1 - r0][64])
-    // slot
-    int kb0, kbs, in_chain;
+    // slot = ring entry
+    int kb0, kbs, in_chain;   // in_chain: k-blocks of the accumulation chain before this slot
+    // the entry's place in the ring: every role computes the same sequence.  Entries are laid end to end; one that would
+    // cross the end of the ring starts at its beginning instead.  voff counts all bytes so far, the skipped ones too, so
+    // an entry fits once voff + size - (voff of the oldest entry still in use) <= R_RING.
+    unsigned e, par;          // entry index (mbarrier pair) and its phase parity
+    unsigned poff, voff, size;
     bool done;
 
-    __device__ Cursor(const ClRowsArgs &args) : a(args), ji(-1), in_chain(0), done(false) {
+    __device__ Cursor(const ClRowsArgs &args) : a(args), ji(-1), in_chain(0), e(R_NE - 1), par(1u), poff(0u), voff(0u), size(0u), done(false) {
         njobs = 4 * a.L + (a.want_head ? 1 : 0);
         ars = (2 * a.T + 7) & ~7;
         next_job();
+        place();
     }
-    __device__ __forceinline__ bool first() const { return kb0 == kb_begin; }
     __device__ __forceinline__ bool last() const { return kb0 + kbs >= kb_end; }             // last slot of the group
     __device__ __forceinline__ bool job_last() const { return last() && g1 >= r1; }          // ... of the job, for this CTA
     __device__ __forceinline__ bool chain_first() const { return in_chain == 0; }
-    __device__ __forceinline__ bool chain_last() const { return last() || in_chain + 1 >= a.chain; }
+    __device__ __forceinline__ bool chain_last() const { return last() || in_chain + kbs >= a.chain; }
+    __device__ __forceinline__ void place() {
+        if (done) return;
+        const unsigned nsize = (unsigned)kbs * stride;
+        poff += size;
+        voff += size;
+        if (poff + nsize > (unsigned)R_RING) {
+            voff += (unsigned)R_RING - poff;
+            poff = 0u;
+        }
+        size = nsize;
+        if (++e == (unsigned)R_NE) { e = 0u; par ^= 1u; }
+    }
     __device__ void open_group(int g) {
         g0 = g;
         a0 = g & ~7;
         g1 = min(r1, a0 + R_MAXN);
         npad = (g1 - a0 + 15) & ~15;
-        stride = (unsigned)(ars + npad) * 128u;
-        per = R_SLOT / (int)stride;
+        // a tile takes the rows it is sent, rounded up to 8; the multiply-add reads npad rows, up to 8 more: whatever
+        // lies behind the tile (the columns of D they produce are never read)
+        stride = (unsigned)(ars + ((g1 - a0 + 7) & ~7)) * 128u;
+        per = max(1, min(32, a.entry / (int)stride));
         wbase = ((size_t)r0 * KB + (size_t)(g0 - r0)) * 128;
         wstep = (unsigned)(r1 - r0) * 128u;
         kb0 = kb_begin;
@@ -211,7 +232,7 @@ struct Cursor {
         done = true;
     }
     __device__ __forceinline__ void advance() {
-        in_chain = chain_last() ? 0 : in_chain + 1;
+        in_chain = chain_last() ? 0 : in_chain + kbs;
         kb0 += kbs;
         if (kb0 < kb_end) {
             kbs = min(per, kb_end - kb0);
@@ -220,12 +241,12 @@ struct Cursor {
         } else {
             next_job();
         }
+        place();
     }
 };
 
 // ---- small helpers -------------------------------------------------------------------------------------
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(RT) : "memory"); }
-__device__ __forceinline__ void drain_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
 // Orders this thread's generic-proxy accesses of global memory with async-proxy (bulk copy) accesses.
 __device__ __forceinline__ void proxy_fence_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
@@ -311,63 +332,79 @@ __device__ __forceinline__ ClHeadPartial rp_merge(const ClHeadPartial &a, const 
 // are requested once the completion counters of their k-blocks say so, both on the slot's one mbarrier.
 __device__ void producer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, int lane) {
     const unsigned long long policy = policy_evict_first();
-    Cursor w(a), q(a);                     // weight cursor; head of the queue of slots that still lack their activation tiles
+    Cursor w(a), q(a);                     // weight cursor; head of the queue of entries that still lack their activation tiles
     const unsigned abytes = (unsigned)w.ars * 128u;
-    unsigned slot = 0, par = 0;            // ring slot of the weight cursor
-    unsigned qslot = 0;                    // ring slot of the queue's head
-    int pn = 0;                            // queue length
-    unsigned used = 0;                     // bit i: slot i has copies in flight of phase parity (used_par >> i) & 1
+    int pn = 0;                            // entries between q and w: weights requested, activation tiles not yet
+    int nout = 0;                          // entries between the oldest one still in use and w
+    unsigned fe = 0u, fpar = 0u;           // ... that oldest entry: index and parity
+    unsigned used = 0;                     // bit i: entry i has copies in flight of phase parity (used_par >> i) & 1
     unsigned used_par = 0;
-    bool job_ready = false;                // every k-block of the queue head's job is known to be complete
-    unsigned looks = 0;
+    bool job_ready = false;                // every k-block of the queue head's job from its current one on is known to be complete
+    int known = 0;                         // k-blocks from the queue head's first one that are known to be complete
     unsigned long long t_idle = 0;
     unsigned n_idle = 0;
     while (!w.done || pn > 0) {
         if (__shfl_sync(0xffffffffu, *(volatile int *)&sm->abort, 0)) break;
         bool progress = false;
+        // (lane 0's view of a barrier and of the clock is the warp's: control flow stays uniform)
+        // the oldest entry in use: have its multiply-adds read it?  Then its bytes are free.
+        if (nout > 0 && __shfl_sync(0xffffffffu, (int)bar_test(&sm->empty[fe], fpar), 0)) {
+            if (++fe == (unsigned)R_NE) { fe = 0u; fpar ^= 1u; }
+            --nout;
+            progress = true;
+        }
         if (pn > 0) {
-            // the head of the queue: are the activation columns of its k-blocks complete?  Lane j looks at k-block j's
-            // counter; once a look at the job's whole K range has found everything complete, no more looks for this job.
-            bool ready = job_ready;
-            if (!ready) {
-                const unsigned v = lane < q.kbs ? counter_read(a.sync + q.dep + ((q.kb0 + lane) >> q.dep_shift)) : q.dep_target;
-                ready = __all_sync(0xffffffffu, (int)(v - q.dep_target) >= 0);
-                if (ready) {
-                    if ((++looks & 3u) == 0u) {
-                        bool all = true;
-                        for (int kb = q.kb0 + lane; kb < q.kb_end; kb += 32)
-                            all = all && (int)(counter_read(a.sync + q.dep + (kb >> q.dep_shift)) - q.dep_target) >= 0;
-                        job_ready = __all_sync(0xffffffffu, all);
-                    }
+            // the head of the queue: are the activation columns of its k-blocks complete?  `known` k-blocks from the head's
+            // first one are known to be; when that is not enough, lane j looks at the counter of k-block j from there (one
+            // round trip for up to 32 k-blocks: a look per entry would make this loop the bottleneck of the stream)
+            if (!job_ready && known < q.kbs) {
+                const int kb = q.kb0 + lane;
+                const bool ok = kb >= q.kb_end || (int)(counter_read(a.sync + q.dep + (kb >> q.dep_shift)) - q.dep_target) >= 0;
+                const unsigned bal = __ballot_sync(0xffffffffu, ok);
+                const int nk = bal == 0xffffffffu ? 32 : __ffs(~bal) - 1;
+                if (nk > known) {
+                    known = nk;
                     proxy_fence_global();   // other CTAs' stores (acquired above) before this warp's bulk-copy reads
                 }
+                job_ready = q.kb0 + known >= q.kb_end;
             }
-            if (ready) {
+            if (job_ready || known >= q.kbs) {
                 if (lane < q.kbs)
-                    bulk_g2s(ring + (size_t)qslot * R_SLOT + (size_t)lane * q.stride,
-                             q.A + (size_t)(q.kb0 + lane) * (CL_ROWS_AROWS * 64), abytes, &sm->full[qslot]);
-                if (++qslot == R_NSLOT) qslot = 0;
+                    bulk_g2s(ring + q.poff + (size_t)lane * q.stride, q.A + (size_t)(q.kb0 + lane) * (CL_ROWS_AROWS * 64), abytes,
+                             &sm->full[q.e]);
                 --pn;
-                const int ji_old = q.ji;
+                known = max(0, known - q.kbs);
+                const int ji_old = q.ji, g0_old = q.g0;
                 q.advance();
-                if (q.done || q.ji != ji_old) job_ready = false;
+                if (q.done || q.ji != ji_old) {
+                    job_ready = false;
+                    known = 0;
+                } else if (q.g0 != g0_old) {
+                    known = 0;   // the next group of rows starts over at the job's first k-block (job_ready stays)
+                }
                 progress = true;
             }
         }
-        // (lane 0's view of the barrier and of the clock is the warp's: control flow stays uniform)
-        if (!w.done && pn < R_NSLOT && __shfl_sync(0xffffffffu, (int)bar_test(&sm->empty[slot], par ^ 1u), 0)) {
-            const unsigned bbytes = (unsigned)(w.g1 - w.g0) * 128u;
-            if (lane == 0) bar_expect(&sm->full[slot], (unsigned)w.kbs * (bbytes + abytes));
-            __syncwarp();
-            if (lane < w.kbs)
-                bulk_g2s_stream(ring + (size_t)slot * R_SLOT + (size_t)lane * w.stride + abytes + (size_t)(w.g0 - w.a0) * 128,
-                                w.W + w.wbase + (size_t)(w.kb0 + lane) * w.wstep, bbytes, &sm->full[slot], policy);
-            used |= 1u << slot;
-            used_par = (used_par & ~(1u << slot)) | (par << slot);
-            ++pn;
-            if (++slot == R_NSLOT) { slot = 0; par ^= 1u; }
-            w.advance();
-            progress = true;
+        // the next entry's weights, as soon as its bytes and its pair of barriers are free
+        if (!w.done && nout < R_NE) {
+            const unsigned oldest = nout > 0 ? *(volatile unsigned *)&sm->vstart[fe] : w.voff;
+            if (w.voff + w.size - oldest <= (unsigned)R_RING) {
+                const unsigned bbytes = (unsigned)(w.g1 - w.g0) * 128u;
+                if (lane == 0) {
+                    sm->vstart[w.e] = w.voff;
+                    bar_expect(&sm->full[w.e], (unsigned)w.kbs * (bbytes + abytes));
+                }
+                __syncwarp();
+                if (lane < w.kbs)
+                    bulk_g2s_stream(ring + w.poff + (size_t)lane * w.stride + abytes + (size_t)(w.g0 - w.a0) * 128,
+                                    w.W + w.wbase + (size_t)(w.kb0 + lane) * w.wstep, bbytes, &sm->full[w.e], policy);
+                used |= 1u << w.e;
+                used_par = (used_par & ~(1u << w.e)) | (w.par << w.e);
+                ++pn;
+                ++nout;
+                w.advance();
+                progress = true;
+            }
         }
         if (progress) {
             t_idle = 0;
@@ -385,14 +422,14 @@ __device__ void producer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, in
         }
         __syncwarp();
     }
-    // After an abort some slots expect activation bytes that were never requested: their barrier cannot complete, but the
+    // After an abort some entries expect activation bytes that were never requested: their barrier cannot complete, but the
     // weight copies still have to land before the CTA may exit.  A copy takes microseconds; wait a bounded moment.
     if (*(volatile int *)&sm->abort) {
         const unsigned long long t0 = gtime_ns();
         while (gtime_ns() - t0 < 200000ull) {
         }
     } else {
-        for (int i = 0; i < R_NSLOT; ++i) {
+        for (int i = 0; i < R_NE; ++i) {
             if (used & (1u << i)) {
                 const unsigned long long t0 = gtime_ns();
                 while (!bar_try(&sm->full[i], (used_par >> i) & 1u))
@@ -424,16 +461,17 @@ __device__ __forceinline__ void umma_kblock(unsigned tmem_d, unsigned long long 
 // ---- MMA issuer ------------------------------------------------------------------------------------------
 __device__ void mma_issuer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, unsigned tmem) {
     Cursor c(a);
-    unsigned slot = 0, par = 0, n = 0;   // n: accumulation chains so far (buffer n & 1)
+    unsigned n = 0;   // accumulation chains so far (buffer n & 1)
     const unsigned long long desc0 = umma_desc(0);
     const unsigned ars16 = (unsigned)c.ars * 8u;   // activation rows of a tile in 16-byte units
+    const unsigned ring0 = s_u32(ring);
     while (!c.done) {
         const unsigned buf = n & 1u;
         if (c.chain_first() && !r_wait(&sm->tempty[buf], ((n >> 1) & 1u) ^ 1u, sm, &a.st->err)) return;
-        if (!r_wait(&sm->full[slot], par, sm, &a.st->err)) return;
+        if (!r_wait(&sm->full[c.e], c.par, sm, &a.st->err)) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const unsigned idesc = umma_idesc(128, c.npad, a.f16);
-        const unsigned base = s_u32(ring + (size_t)slot * R_SLOT);
+        const unsigned base = ring0 + c.poff;
         unsigned long long adesc = desc0 + (unsigned long long)((base & 0x3ffffu) >> 4);
         const unsigned stride16 = c.stride >> 4;
         const unsigned d_tmem = tmem + buf * 256u;
@@ -443,12 +481,11 @@ __device__ void mma_issuer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, 
             acc = 1u;
             adesc += stride16;
         }
-        umma_commit(&sm->empty[slot]);                     // the slot is free once these multiply-adds have read it
+        umma_commit(&sm->empty[c.e]);                      // the entry is free once these multiply-adds have read it
         if (c.chain_last()) {
             umma_commit(&sm->tfull[buf]);                  // ... and the accumulator buffer is complete
             ++n;
         }
-        if (++slot == R_NSLOT) { slot = 0; par ^= 1u; }
         c.advance();
     }
 }
@@ -478,7 +515,7 @@ __device__ __forceinline__ void gemm_job(const ClRowsArgs &a, RSmem *sm, unsigne
     bool job_done = false;
     while (!job_done) {
         const Group g{c.g0, c.g1, c.a0, c.npad};
-        // walk the tile's slots first (an accumulation chain ends every a.chain slots and at the tile's end), so that
+        // walk the tile's slots first (an accumulation chain ends after a.chain k-blocks and at the tile's end), so that
         // no schedule arithmetic runs while the accumulator registers are live
         int nchains = 0;
         for (bool group_end = false; !group_end;) {
@@ -586,60 +623,37 @@ __device__ void head_finish(const ClRowsArgs &a, RSmem *sm, ClHeadPartial run) {
     }
 }
 
-// Barrier of the `split` CTAs of a group (arrival counter per group, growing during a launch like the grid's).
-__device__ __forceinline__ void group_barrier(const ClRowsArgs &a, unsigned &target, RSmem *sm) {
-    worker_sync();
-    if (a.split > 1 && threadIdx.x == 0 && !*(volatile int *)&sm->abort) {
-        unsigned *bar = a.sync + 1 + blockIdx.x / a.split;
-        target += (unsigned)a.split;
-        __threadfence();
-        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
-        unsigned v;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
-        if ((int)(v - target) < 0) {
-            const unsigned long long t0 = gtime_ns();
-            unsigned i = 0;
-            do {
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(bar) : "memory");
-                if ((++i & 255u) == 0u) {
-                    if (*(volatile int *)&a.st->err || gtime_ns() - t0 > sm->wait_ns) {
-                        *(volatile int *)&sm->abort = 1;
-                        atomicOr(&a.st->err, 64);
-                        break;
-                    }
-                }
-            } while ((int)(v - target) < 0);
-        }
-    }
-    worker_sync();
-}
-
 // Second half of an output / down projection: the `split` CTAs of a group hold the products of their K ranges in the
-// workspace; after the group's barrier each of them takes a share of the group's rows, adds the parts in member order
-// (fixed: results do not depend on timing), and applies the epilogue, one thread per (token, row): residual add, the
-// next GEMM's operand rows hi/lo(x * gain), hidden tap, and this CTA's sum of x^2 per token.
-__device__ void resid_phase(const ClRowsArgs &a, int ji, int pos0, unsigned &grp_target, RSmem *sm) {
-    group_barrier(a, grp_target, sm);
-    const int T = a.T, l = ji >> 2, g = a.split, tid = threadIdx.x;
+// workspace.  Nobody waits for anybody: each member takes a ticket of its group when its products are stored, and the
+// member that draws the last one does the group's rows -- adds the parts in member order (fixed: results do not depend
+// on who came last), residual add, the next GEMM's operand rows hi/lo(x * gain), hidden tap, sum of x^2 per token.
+// Whole warps per token row (RW / T of them), a thread's rows 32 apart, so a row's sum of squares is a fixed tree.
+__device__ void resid_phase(const ClRowsArgs &a, int ji, int pos0, RSmem *sm) {
+    const int T = a.T, l = ji >> 2, g = a.split, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Job jb = job_of(a, ji);
     int r0, r1;
     rows_of(jb.rows, jb.unit, g, r0, r1);
-    const int member = (int)blockIdx.x % g, first_cta = (int)blockIdx.x - member;
-    const ClRowsLayer &y = a.layers[l];
-    const bool attn_half = (ji & 3) == 1;
-    const float *gain = attn_half ? y.n2 : ((l + 1 < a.L) ? a.layers[l + 1].n1 : a.final_norm);
-    unsigned short *tap = (unsigned short *)(a.tap ? (attn_half ? y.tap0 : y.tap1) : nullptr);
-    float *sq = sm->stage;   // [T][64] squares of this CTA's new residual values
-    for (int t = tid; t < CL_SLOTS; t += RT) sm->red[t] = 0.f;
-    // the group's rows in tiles of at most R_MAXN rows, exactly as the GEMM cut them
-    for (int g0 = r0; g0 < r1;) {
-        const int a0 = g0 & ~7, g1 = min(r1, a0 + R_MAXN), n = g1 - g0;
-        const int q0 = g0 + n * member / g, q1 = g0 + n * (member + 1) / g;   // this CTA's share of the tile's rows
-        for (int c0 = q0; c0 < q1; c0 += 64) {                                // ... 64 rows at a time
-            const int nq = min(64, q1 - c0);
-            worker_sync();
-            for (int idx = tid; idx < T * nq; idx += RT) {
-                const int t = idx / nq, i = idx % nq, row = c0 + i;
+    const int first_cta = (int)blockIdx.x - (int)blockIdx.x % g;
+    worker_sync();   // the drain warps' stores to the workspace are done
+    if (tid == 0) {
+        int last = 1;
+        if (g > 1) {
+            const unsigned prev = ticket_acq_rel(a.sync + 1 + blockIdx.x / g);   // (counts up during a launch: g tickets per job)
+            last = (prev % (unsigned)g) == (unsigned)g - 1u;
+        }
+        sm->is_last = last;
+    }
+    worker_sync();
+    const bool mine = sm->is_last != 0;
+    if (mine) {
+        const ClRowsLayer &y = a.layers[l];
+        const bool attn_half = (ji & 3) == 1;
+        const float *gain = attn_half ? y.n2 : ((l + 1 < a.L) ? a.layers[l + 1].n1 : a.final_norm);
+        unsigned short *tap = (unsigned short *)(a.tap ? (attn_half ? y.tap0 : y.tap1) : nullptr);
+        const int wpt = RW / T, t = warp / wpt, a0 = r0 & ~7;   // (the group's rows are one tile of the GEMM)
+        float ss = 0.f;
+        if (t < T) {
+            for (int row = r0 + (warp % wpt) * 32 + lane; row < r1; row += wpt * 32) {
                 float parts[8];
 #pragma unroll
                 for (int m = 0; m < 8; ++m)
@@ -654,31 +668,31 @@ __device__ void resid_phase(const ClRowsArgs &a, int ji, int pos0, unsigned &grp
                 a_store_split(a.Ax, t, T, row, xn * __ldg(gain + row), a.f16);
                 if (tap && t + a.tap_P >= T)   // (slot = position mod P: of rows that share a slot the last one stays)
                     tap[(size_t)((pos0 + t) % a.tap_P) * a.d + row] = f32_to_b16(xn, a.f16);
-                sq[t * 64 + i] = xn * xn;
-            }
-            worker_sync();
-            if (tid < T) {
-                float ss = sm->red[tid];
-                for (int i = 0; i < nq; ++i) ss += sq[tid * 64 + i];
-                sm->red[tid] = ss;
+                ss = fmaf(xn, xn, ss);
             }
         }
-        g0 = g1;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) sm->wsum[warp] = ss;
+        proxy_fence_global();   // the operand rows written above are read by other CTAs' bulk copies
+    }
+    if (!mine) return;   // (uniform over the CTA)
+    worker_sync();
+    // the group's sum of squares goes to its first member's slot and zeros to the others', whoever computed it: the order
+    // in which the slots are added up later must not depend on who came last
+    if (tid < T) {
+        const int wpt = RW / T;
+        float ss = 0.f;
+        for (int w = 0; w < wpt; ++w) ss += sm->wsum[tid * wpt + w];
+        a.ssq[(size_t)first_cta * CL_SLOTS + tid] = ss;
+        for (int m = 1; m < g; ++m) a.ssq[(size_t)(first_cta + m) * CL_SLOTS + tid] = 0.f;
     }
     worker_sync();
-    if (tid < T) a.ssq[(size_t)blockIdx.x * CL_SLOTS + tid] = sm->red[tid];
-    proxy_fence_global();   // the operand rows written above are read by other CTAs' bulk copies
-    worker_sync();
     if (tid == 0) {
-        // this CTA's share of the operand columns, counted per k-block; and its sum of squares
-        for (int g0 = r0; g0 < r1;) {
-            const int a0 = g0 & ~7, g1 = min(r1, a0 + R_MAXN), n = g1 - g0;
-            const int q0 = g0 + n * member / g, q1 = g0 + n * (member + 1) / g;
-            for (int kb = q0 >> 6; kb * 64 < q1; ++kb)
-                counter_add(a.sync + a.c_ax + kb, (unsigned)(min(q1, (kb + 1) * 64) - max(q0, kb * 64)));
-            g0 = g1;
-        }
-        counter_add(a.sync + a.c_ssq, 1u);
+        // the group's columns of the operand rows, counted per k-block; and the sums of squares of its g slots
+        for (int kb = r0 >> 6; kb * 64 < r1; ++kb)
+            counter_add(a.sync + a.c_ax + kb, (unsigned)(min(r1, (kb + 1) * 64) - max(r0, kb * 64)));
+        counter_add(a.sync + a.c_ssq, (unsigned)g);
     }
 }
 
@@ -1006,10 +1020,10 @@ __global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constan
     unsigned char *ring = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     // the control block sits behind the ring: the M = 128 operand descriptor of the last tile reads up to 16 KB past
     // its activation rows, which must stay inside this CTA's shared memory
-    RSmem *sm = (RSmem *)(ring + (size_t)R_NSLOT * R_SLOT);
+    RSmem *sm = (RSmem *)(ring + (size_t)R_RING);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int i = 0; i < R_NSLOT; ++i) {
+        for (int i = 0; i < R_NE; ++i) {
             bar_init(&sm->full[i], 1);
             bar_init(&sm->empty[i], 1);
         }
@@ -1038,7 +1052,7 @@ __global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constan
         if (lane == 0) mma_issuer(a, ring, sm, tmem);
     } else {
         const int base = a.st->ctx + a.row0;   // position of row 0
-        unsigned bar_target = 0u, grp_target = 0u, n_acc = 0u;
+        unsigned bar_target = 0u, n_acc = 0u;
         ClHeadPartial run{0.f, 0.f, 0.f, 0x7fffffff};
         Cursor cur(a);
         embed_phase(a, sm);
@@ -1051,13 +1065,13 @@ __global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constan
             attention_phase<ST, HD>(a, y, l, base, sm);
             phase_clock(a, sm, 2);
             gemm_job(a, sm, tmem, 4 * l + 1, cur, n_acc, run);
-            resid_phase(a, 4 * l + 1, base, grp_target, sm);
+            resid_phase(a, 4 * l + 1, base, sm);
             phase_clock(a, sm, 3);
             compute_scales(a, sm, 2 * l + 2);
             gemm_job(a, sm, tmem, 4 * l + 2, cur, n_acc, run);
             phase_clock(a, sm, 4);
             gemm_job(a, sm, tmem, 4 * l + 3, cur, n_acc, run);
-            resid_phase(a, 4 * l + 3, base, grp_target, sm);
+            resid_phase(a, 4 * l + 3, base, sm);
             phase_clock(a, sm, 5);
         }
         if (a.want_head) {
@@ -1121,7 +1135,7 @@ __global__ void k_tile_layout(const uint4 *src, uint4 *dst, int rows, int KB, in
 
 }  // namespace
 
-size_t cl_rows_smem_bytes() { return (size_t)R_NSLOT * R_SLOT + R_CTRL_BYTES + 1024; }
+size_t cl_rows_smem_bytes() { return (size_t)R_RING + R_CTRL_BYTES + 1024; }
 
 int cl_rows_att_part_floats(int H) { return H * R_ATT_MAXS * CL_MAX_T * (128 + 2); }
 
