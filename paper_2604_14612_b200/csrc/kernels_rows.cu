@@ -766,6 +766,21 @@ __device__ void embed_phase(const ClRowsArgs &a, RSmem *sm) {
 // head also appends them to the cache); the last warp of row t folds them in.  The CTA merges its warps per row and writes one
 // record per (h, s, t); the last CTA of a head to finish (ticket) merges the parts in order and writes the
 // normalised output as the output projection's hi/lo operand rows.
+// Ahead of a layer's QKV job: ask for the cached keys and values this CTA's attention item will read, so that they wait
+// in L2 when the attention phase starts (the worker warps have nothing else to do while the job's weights stream).
+template <int HD>
+__device__ __forceinline__ void attention_prefetch(const ClRowsArgs &a, const ClRowsLayer &y, int base) {
+    const int S = a.att_parts, item = blockIdx.x;
+    if (item >= a.H * S) return;
+    const int h = item % a.H, s = item / a.H, kvh = h / (a.H / a.Hkv);
+    const int k0 = (int)((long long)base * s / S), k1 = (int)((long long)base * (s + 1) / S);
+    const size_t off = ((size_t)kvh * a.max_seq + k0) * HD * 2, bytes = (size_t)(k1 - k0) * HD * 2;
+    for (size_t b = (size_t)threadIdx.x * 128; b < bytes; b += (size_t)RT * 128) {
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(y.kc + off + b));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(y.vc + off + b));
+    }
+}
+
 template <typename ST, int HD>
 __device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int layer, int base, RSmem *sm) {
     constexpr int EPL = 8, LPK = HD / EPL, KPW = 32 / LPK, VPL = HD / 32, WSTRIDE = HD + 2, HALF = HD / 2;
@@ -1059,6 +1074,7 @@ __global__ void __launch_bounds__(R_THREADS, 1) k_rows_pass(const __grid_constan
         phase_clock(a, sm, 0);
         for (int l = 0; l < a.L; ++l) {
             const ClRowsLayer &y = a.layers[l];
+            attention_prefetch<HD>(a, y, base);
             compute_scales(a, sm, 2 * l + 1);
             gemm_job(a, sm, tmem, 4 * l, cur, n_acc, run);
             phase_clock(a, sm, 1);
