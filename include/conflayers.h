@@ -34,7 +34,8 @@
  *     A prompt of more than 16 tokens (bf16 / fp16 models) runs all rows but the last through wide tensor-core GEMMs, up to
  *     512 rows at a time, and the last row through the pass of several rows, which has the LM head.
  *     Environment switches read by cl_load (diagnostics): CL_DISABLE_STEP_KERNEL=1, CL_DISABLE_ROWS_KERNEL=1,
- *     CL_DISABLE_WIDE_PREFILL=1, CL_DISABLE_ROW_SHARES=1, CL_L2_AHEAD_KB=<n>, CL_ROWS_SPLIT=<1|2|4>, CL_ROWS_CHAIN=<n>.
+ *     CL_DISABLE_WIDE_PREFILL=1, CL_DISABLE_ROW_SHARES=1, CL_L2_AHEAD_KB=<n>, CL_ROWS_SPLIT=<1|2|4>, CL_ROWS_CHAIN=<k-blocks
+ *     of 64 elements per tensor-memory accumulation chain>, CL_ROWS_ENTRY_KB=<size of a ring entry of that pass>.
  */
 #ifndef CONFLAYERS_H
 #define CONFLAYERS_H
