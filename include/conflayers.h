@@ -174,7 +174,8 @@ int cl_force_tokens(cl_ctx *ctx, const int32_t *toks, int n);
 /* Early-exit confidence of hidden states (Section 3.1, Eq. 1-4): each row goes through the final
  * RMSNorm and the shared LM head; logits are clamped in fp32; per row the entropy confidence
  * 1 - H/log(vocab), the top-1 probability and the greedy token are reduced on the fly (logits are
- * never stored).  hidden: DEVICE pointer [rows, P, d_model] in the model's storage type, or NULL to
+ * never stored).  hidden: DEVICE pointer [rows, P, d_model] in the model's storage type (16-byte aligned for
+ * 16-bit models, CL_EINVAL otherwise; cl_score_loop's tensors likewise), or NULL to
  * score the context's own ring (rows = n_layers, P = taps * tap_positions with taps = 1 or 2, see tap_modules).
  * Outputs (host, may be NULL): conf_rows, p_max, argmax [rows, P]; c_layer [rows] = mean over P. */
 int cl_layer_confidences(cl_ctx *ctx, const void *hidden, int rows, int P, float *conf_rows, float *p_max,

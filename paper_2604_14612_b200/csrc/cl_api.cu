@@ -1153,6 +1153,8 @@ static int score_rows(cl_ctx *c, const void *hidden, int rows, int P, float *c_l
     if (rc) return rc;
     if (c->cfg.weight_dtype != 0) {
         // 16-bit head: one dense contraction on the tensor cores with the softmax statistics fused into its epilogue
+        if (((uintptr_t)hidden & 15u) != 0 || d % 8 != 0)
+            return fail(c, CL_EINVAL, "confidence scoring: hidden rows must be 16-byte aligned and d_model a multiple of 8");
         const int f16 = c->cfg.weight_dtype == 2;
         KL(cl_launch_rmsnorm_bf16(c->cfg.weight_dtype, hidden, c->final_norm, (int)n, (int)d, c->cfg.rms_eps, c->sc_xn, f16, c->stream));
         KL(cl_launch_score_tc(c->sc_xn, c->lm_head, (int)n, c->cfg.vocab, (int)d, c->sc_part, c->n_sm, &c->st->err, c->sc_conf,

@@ -284,49 +284,56 @@ __device__ __forceinline__ double dmul(double a, double b) { return __dmul_rn(a,
 __device__ __forceinline__ double dadd(double a, double b) { return __dadd_rn(a, b); }
 __device__ __forceinline__ double dsub(double a, double b) { return __dadd_rn(a, -b); }
 
-__device__ void sel_gradient(const double *x, double *out, int n) {
-    if (n < 2) {
-        for (int i = 0; i < n; ++i) out[i] = 0.0;
-        return;
-    }
-    out[0] = dsub(x[1], x[0]);
-    out[n - 1] = dsub(x[n - 1], x[n - 2]);
-    for (int i = 1; i < n - 1; ++i) out[i] = dmul(dsub(x[i + 1], x[i - 1]), 0.5);
+// One element of the discrete gradient (central differences inside, one-sided at the ends).
+__device__ __forceinline__ double sel_gradient_at(const double *x, int i, int n) {
+    if (n < 2) return 0.0;
+    if (i == 0) return dsub(x[1], x[0]);
+    if (i == n - 1) return dsub(x[n - 1], x[n - 2]);
+    return dmul(dsub(x[i + 1], x[i - 1]), 0.5);
 }
 
+// One warp.  Everything that is a sum over layers in a stated order (Eq. 5, the local statistics of Eq. 8-9) is added
+// in that order by one lane, every operation rounded on its own, so the margins are those of a sequential evaluation
+// bit for bit; the layers themselves (lane i takes layers i, i + 32, ...) run side by side, and the sequential
+// selection of the smallest margins becomes a rank by counting (ties -> lower layer index, as picking minima does).
 __global__ void k_select(cl_select_cfg cfg, int L, const float *c_layer, uint8_t *mask, double *margins) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (blockIdx.x != 0 || threadIdx.x >= 32) return;
     __shared__ double c[CL_SEL_MAX], chat[CL_SEL_MAX], g[CL_SEL_MAX], tmp[CL_SEL_MAX], mg[CL_SEL_MAX];
-    __shared__ unsigned char chosen[CL_SEL_MAX];
+    const int lane = threadIdx.x;
     const int lo = cfg.lo, n = cfg.hi - cfg.lo + 1;
-    for (int l = 0; l < L; ++l) {
+    for (int l = lane; l < L; l += 32) {
         mask[l] = 0;
         if (margins) margins[l] = 0.0;
     }
     if (n <= 0) return;
-    for (int i = 0; i < n; ++i) c[i] = (double)c_layer[lo + i];
-    // Eq. 5
+    for (int i = lane; i < n; i += 32) c[i] = (double)c_layer[lo + i];
+    __syncwarp();
+    // Eq. 5 (every lane adds up the same sequence: no broadcast needed)
     double s = 0.0;
     for (int i = 0; i < n; ++i) s = dadd(s, c[i]);
     const double mu = s / (double)n;
     s = 0.0;
     for (int i = 0; i < n; ++i) s = dadd(s, dmul(dsub(c[i], mu), dsub(c[i], mu)));
     const double sigma = sqrt(s / (double)n);
-    for (int i = 0; i < n; ++i) chat[i] = dsub(c[i], mu) / dadd(sigma, cfg.eps);
+    for (int i = lane; i < n; i += 32) chat[i] = dsub(c[i], mu) / dadd(sigma, cfg.eps);
+    __syncwarp();
     // Eq. 6
-    if (n >= 3) {
-        sel_gradient(chat, tmp, n);
-        sel_gradient(tmp, g, n);
-        for (int i = 0; i < n; ++i) g[i] = fabs(g[i]);
-    } else {
-        for (int i = 0; i < n; ++i) g[i] = 0.0;
-    }
-    double gmin = g[0], gmax = g[0];
-    for (int i = 1; i < n; ++i) {
+    for (int i = lane; i < n; i += 32) tmp[i] = n >= 3 ? sel_gradient_at(chat, i, n) : 0.0;
+    __syncwarp();
+    for (int i = lane; i < n; i += 32) g[i] = n >= 3 ? fabs(sel_gradient_at(tmp, i, n)) : 0.0;
+    __syncwarp();
+    double gmin = g[0], gmax = g[0];   // (minimum and maximum do not depend on the order)
+    for (int i = lane; i < n; i += 32) {
         gmin = fmin(gmin, g[i]);
         gmax = fmax(gmax, g[i]);
     }
-    for (int i = 0; i < n; ++i) g[i] = dsub(g[i], gmin) / dadd(dsub(gmax, gmin), cfg.eps);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        gmin = fmin(gmin, __shfl_xor_sync(0xffffffffu, gmin, o));
+        gmax = fmax(gmax, __shfl_xor_sync(0xffffffffu, gmax, o));
+    }
+    __syncwarp();
+    for (int i = lane; i < n; i += 32) g[i] = dsub(g[i], gmin) / dadd(dsub(gmax, gmin), cfg.eps);
     // w_max
     double w_max = cfg.w_max;
     if (!(w_max > 0.0)) {
@@ -337,8 +344,9 @@ __global__ void k_select(cl_select_cfg cfg, int L, const float *c_layer, uint8_t
         }
         w_max = (double)(cnt > 1 ? cnt : 1);
     }
+    __syncwarp();
     // Eq. 7-10
-    for (int i = 0; i < n; ++i) {
+    for (int i = lane; i < n; i += 32) {
         const double w = dadd(cfg.w_base, dmul(dmul(w_max, g[i]), (double)(lo + i) / (double)L));
         const int W = cfg.fixed_window > 0 ? cfg.fixed_window : (int)floor(dadd(w, 0.5));
         int half = (W + 1) / 2;
@@ -363,31 +371,31 @@ __global__ void k_select(cl_select_cfg cfg, int L, const float *c_layer, uint8_t
             sd_i = sqrt(sum / (double)cnt);
         }
         mg[i] = dsub(chat[i], dsub(m_i, dmul(cfg.lambda, sd_i)));
-        chosen[i] = 0;
     }
+    __syncwarp();
     // Eq. 10 and the ratio post-step: smallest margins first, ties -> lower layer index
-    int n_chosen = 0, need;
-    if (cfg.n_skip >= 0) {
+    int n_fixed = 0, need;
+    const bool by_sign = cfg.n_skip < 0;   // layers with a negative margin are in; then the smallest others up to the ratio
+    if (!by_sign) {
         need = cfg.n_skip < n ? cfg.n_skip : n;
     } else {
-        for (int i = 0; i < n; ++i)
-            if (mg[i] < 0.0) {
-                chosen[i] = 1;
-                ++n_chosen;
-            }
+        for (int i = 0; i < n; ++i) n_fixed += mg[i] < 0.0 ? 1 : 0;
         need = (int)floor(dadd(dmul(cfg.min_ratio, (double)n), 0.5));
     }
-    while (n_chosen < need) {
-        int best = -1;
-        for (int i = 0; i < n; ++i)
-            if (!chosen[i] && (best < 0 || mg[i] < mg[best])) best = i;
-        if (best < 0) break;
-        chosen[best] = 1;
-        ++n_chosen;
-    }
-    for (int i = 0; i < n; ++i) {
-        if (chosen[i]) mask[lo + i] = 3;
-        if (margins) margins[lo + i] = mg[i];
+    for (int i = lane; i < n; i += 32) {
+        const double m = mg[i];
+        bool in = by_sign && m < 0.0;
+        if (!in) {
+            int rank = 0;   // candidates (layers not in yet) that would be picked before this one
+            for (int j = 0; j < n; ++j) {
+                const double q = mg[j];
+                if (by_sign && q < 0.0) continue;
+                rank += (q < m || (j < i && !(m < q))) ? 1 : 0;
+            }
+            in = n_fixed + rank < need;
+        }
+        if (in) mask[lo + i] = 3;
+        if (margins) margins[lo + i] = m;
     }
 }
 

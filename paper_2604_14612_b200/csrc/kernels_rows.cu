@@ -847,41 +847,46 @@ __device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int l
             const int k0 = (int)((long long)base * s / S), k1 = (int)((long long)base * (s + 1) / S);
             const int kw0 = k0 + (int)((long long)(k1 - k0) * sub / nsub), kw1 = k0 + (int)((long long)(k1 - k0) * (sub + 1) / nsub);
             const ST *Kh = Kc + (size_t)kvh * a.max_seq * HD, *Vh = Vc + (size_t)kvh * a.max_seq * HD;
-            for (int j0 = kw0; j0 < kw1; j0 += 32) {
-                const int n = min(32, kw1 - j0);
+            // CH keys per iteration: the key rows and the value rows of the iteration are requested together (the values do
+            // not depend on the scores), so an iteration costs one memory round trip; lane j < CH keeps key j's score
+            constexpr int CH = 16, NPASS = CH / KPW;
+            for (int j0 = kw0; j0 < kw1; j0 += CH) {
+                const int n = min(CH, kw1 - j0);
+                uint4 raw[NPASS];
+#pragma unroll
+                for (int p = 0; p < NPASS; ++p) {
+                    const int j = p * KPW + ksub;
+                    raw[p] = make_uint4(0u, 0u, 0u, 0u);
+                    if (j < n) raw[p] = __ldg((const uint4 *)(Kh + (size_t)(j0 + j) * HD + li * EPL));
+                }
+                uint2 vraw[CH];   // the value rows stay in their storage type until they are used
+#pragma unroll
+                for (int j = 0; j < CH; ++j) {
+                    const ST *vp = Vh + (size_t)(j0 + min(j, n - 1)) * HD + lane * VPL;
+                    if (VPL == 4) vraw[j] = __ldg((const uint2 *)vp);
+                    else vraw[j] = make_uint2(__ldg((const unsigned *)vp), 0u);
+                }
                 float my_score = -INFINITY;
-                constexpr int NPASS = 32 / KPW, PB = NPASS < 8 ? NPASS : 8;
 #pragma unroll
-                for (int b0 = 0; b0 < NPASS; b0 += PB) {
-                    if (b0 * KPW >= n) break;   // uniform
-                    uint4 raw[PB];
+                for (int p = 0; p < NPASS; ++p) {
+                    const int jb = p * KPW;
+                    if (jb < n) {   // uniform
+                        const unsigned u[4] = {raw[p].x, raw[p].y, raw[p].z, raw[p].w};
+                        float sc = 0.f;
 #pragma unroll
-                    for (int p = 0; p < PB; ++p) {
-                        const int j = (b0 + p) * KPW + ksub;
-                        raw[p] = make_uint4(0u, 0u, 0u, 0u);
-                        if (j < n) raw[p] = __ldg((const uint4 *)(Kh + (size_t)(j0 + j) * HD + li * EPL));
-                    }
+                        for (int e = 0; e < 4; ++e) {
+                            float ka, kb;
+                            ClPair16<ST>::get(u[e], ka, kb);
+                            sc = fmaf(qr[2 * e], ka, sc);
+                            sc = fmaf(qr[2 * e + 1], kb, sc);
+                        }
 #pragma unroll
-                    for (int p = 0; p < PB; ++p) {
-                        const int jb = (b0 + p) * KPW;
-                        if (jb < n) {   // uniform
-                            const unsigned u[4] = {raw[p].x, raw[p].y, raw[p].z, raw[p].w};
-                            float sc = 0.f;
+                        for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                        sc *= scale;
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                float ka, kb;
-                                ClPair16<ST>::get(u[e], ka, kb);
-                                sc = fmaf(qr[2 * e], ka, sc);
-                                sc = fmaf(qr[2 * e + 1], kb, sc);
-                            }
-#pragma unroll
-                            for (int o = LPK >> 1; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
-                            sc *= scale;
-#pragma unroll
-                            for (int k = 0; k < KPW; ++k) {
-                                const float v = __shfl_sync(0xffffffffu, sc, k * LPK);
-                                if (lane == jb + k && jb + k < n) my_score = v;
-                            }
+                        for (int k = 0; k < KPW; ++k) {
+                            const float v = __shfl_sync(0xffffffffu, sc, k * LPK);
+                            if (lane == jb + k && jb + k < n) my_score = v;
                         }
                     }
                 }
@@ -899,27 +904,13 @@ __device__ void attention_phase(const ClRowsArgs &a, const ClRowsLayer &y, int l
                 for (int e = 0; e < VPL; ++e) o_run[e] *= resc;
                 m_run = m_new;
 #pragma unroll
-                for (int jg = 0; jg < 32; jg += 8) {
-                    if (jg >= n) break;   // uniform
-                    float vv[8][VPL];
+                for (int j = 0; j < CH; ++j) {
+                    const float pj = __shfl_sync(0xffffffffu, p, j);   // (0 for j >= n: the repeated last row adds nothing)
+                    float v[4];
+                    ClPair16<ST>::get(vraw[j].x, v[0], v[1]);
+                    ClPair16<ST>::get(vraw[j].y, v[2], v[3]);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const ST *vp = Vh + (size_t)(j0 + min(jg + j, n - 1)) * HD + lane * VPL;
-                        if (VPL == 4) {
-                            const uint2 u = __ldg((const uint2 *)vp);
-                            ClPair16<ST>::get(u.x, vv[j][0], vv[j][1 % VPL]);
-                            ClPair16<ST>::get(u.y, vv[j][2 % VPL], vv[j][3 % VPL]);
-                        } else {
-                            const unsigned u = __ldg((const unsigned *)vp);
-                            ClPair16<ST>::get(u, vv[j][0], vv[j][1 % VPL]);
-                        }
-                    }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float pj = __shfl_sync(0xffffffffu, p, jg + j);
-#pragma unroll
-                        for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(pj, vv[j][e], o_run[e]);
-                    }
+                    for (int e = 0; e < VPL; ++e) o_run[e] = fmaf(pj, v[e], o_run[e]);
                 }
             }
             if (s == S - 1 && sub == nsub - 1) {

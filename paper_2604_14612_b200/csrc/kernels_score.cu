@@ -203,14 +203,39 @@ __global__ void k_score_finalize(const ClHeadPartial *partials, int NCG, int R, 
 
 // Final RMSNorm of hidden rows in the storage type -> rows in the 16-bit type of the LM head (the A operand of the
 // contraction).
+// Eight consecutive elements of a row as floats (one or two 16-byte loads).
+template <typename ST>
+__device__ __forceinline__ void load8(const ST *p, float (&v)[8]) {
+    if (sizeof(ST) == 4) {
+        const float4 a = *(const float4 *)p, b = *((const float4 *)p + 1);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
+        const uint4 u = *(const uint4 *)p;
+        const unsigned w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) ClPair16<ST>::get(w[e], v[2 * e], v[2 * e + 1]);
+    }
+}
+
+// One CTA per row, 16-byte accesses (d is a multiple of 8).  A thread's first chunks stay in registers between the two
+// passes; the sum of squares is added in a fixed order (per thread, shuffle tree, warps in order).
 template <typename ST>
 __global__ void k_rmsnorm_to_bf16(const ST *x, const float *g, int d, float eps, unsigned short *out, int f16) {
     __shared__ float red[32];
+    constexpr int KEEP = 2;
     const ST *xr = x + (size_t)blockIdx.x * d;
+    const int nch = d >> 3;
+    float keep[KEEP][8];
     float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        const float v = (float)xr[i];
-        ss = fmaf(v, v, ss);
+    for (int c = threadIdx.x, k = 0; c < nch; c += blockDim.x, ++k) {
+        float v[8];
+        load8<ST>(xr + (size_t)c * 8, v);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ss = fmaf(v[e], v[e], ss);
+        if (k < KEEP) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) keep[k < KEEP ? k : 0][e] = v[e];
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -219,8 +244,22 @@ __global__ void k_rmsnorm_to_bf16(const ST *x, const float *g, int d, float eps,
     float tot = 0.f;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];   // fixed order
     const float sc = 1.0f / sqrtf(tot / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x)
-        out[(size_t)blockIdx.x * d + i] = f32_to_b16((float)xr[i] * sc * g[i], f16);
+    for (int c = threadIdx.x, k = 0; c < nch; c += blockDim.x, ++k) {
+        float v[8];
+        if (k < KEEP) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = keep[k < KEEP ? k : 0][e];
+        } else {
+            load8<ST>(xr + (size_t)c * 8, v);
+        }
+        const float4 g0 = *(const float4 *)(g + (size_t)c * 8), g1 = *((const float4 *)(g + (size_t)c * 8) + 1);
+        const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+        unsigned w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            w[e] = (unsigned)f32_to_b16(v[2 * e] * sc * gg[2 * e], f16) | ((unsigned)f32_to_b16(v[2 * e + 1] * sc * gg[2 * e + 1], f16) << 16);
+        *(uint4 *)(out + (size_t)blockIdx.x * d + (size_t)c * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
 }
 
 }  // namespace
