@@ -484,6 +484,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 const char *en = getenv("CL_ROWS_ENTRY_KB");   // tuning knob
                 c->rows_entry = ((en && en[0]) ? atoi(en) : 64) * 1024;
                 if (c->rows_entry < 1024) c->rows_entry = 1024;
+                if (c->rows_entry > 96 * 1024) c->rows_entry = 96 * 1024;   // (two entries must fit the ring of 192 KB)
                 c->use_rows = 1;
             }
         }

@@ -286,6 +286,46 @@ def test_tensor_core_pass_matches_streaming_pass(monkeypatch, wd):
     assert np.abs(out[0][5] - out[1][5]).max() <= 2 ** -7 * scale        # taps: one bf16 ulp at the top of the range
 
 
+def test_ring_geometry_of_the_row_pass_does_not_change_its_results(monkeypatch):
+    """The persistent pass lays its weight tiles end to end in a ring and wraps where one would cross the end; how many
+    k-blocks share an entry (and with it where entries wrap, how many are in flight, where an accumulation chain ends) is a
+    tuning parameter.  7B layer shapes, where a layer's tiles go round the ring many times: entries of one k-block (as many
+    in flight as there are barriers), the default, the largest allowed size, and a short accumulation chain must all give
+    the logits of the CUDA-core pass."""
+    base = synth.WORKLOADS["C3"].shape
+    sh = dataclasses.replace(base, n_layers=2, max_seq=64)
+    W = synth.make_weights(sh, 7, device="cuda")
+    prompt = synth.make_prompt(7, 11, sh.vocab)
+    drafts = [11, 22, 33, 44]
+
+    def run(env):
+        for k in ("CL_DISABLE_ROWS_KERNEL", "CL_ROWS_ENTRY_KB", "CL_ROWS_CHAIN"):
+            monkeypatch.delenv(k, raising=False)
+        for k, v in env.items():
+            monkeypatch.setenv(k, v)
+        ctx = cl.Context.from_shape(sh, tap_positions=16)
+        ctx.cl_load(W)
+        first = ctx.cl_prefill(prompt)
+        ctx.cl_force_tokens(drafts)
+        v = ctx.cl_verify(5, want_logits=True)
+        ctx.close()
+        return first, v["targets"].copy(), v["logits"].copy()
+
+    ref = run({"CL_DISABLE_ROWS_KERNEL": "1"})
+    top2 = np.sort(ref[2], axis=1)[:, -2:]
+    clear = (top2[:, 1] - top2[:, 0]) >= NEAR_TIE
+    dflt = run({})
+    assert np.abs(dflt[2] - ref[2]).max() <= 5e-3                      # two implementations, d = 4096: inside the 1e-2 tolerance
+    assert np.array_equal(dflt[1][clear], ref[1][clear])
+    for env in ({"CL_ROWS_ENTRY_KB": "8"}, {"CL_ROWS_ENTRY_KB": "24"}, {"CL_ROWS_ENTRY_KB": "1000"},
+                {"CL_ROWS_ENTRY_KB": "40", "CL_ROWS_CHAIN": "2"}):
+        got = run(env)
+        # the same kernel: only the places where the accumulator is drained into registers move (an entry is never cut,
+        # so large entries make longer tensor-core chains, which round a little differently)
+        assert got[0] == dflt[0] and np.abs(got[2] - dflt[2]).max() <= 4e-3, env
+        assert np.array_equal(got[1][clear], ref[1][clear]), env
+
+
 @pytest.mark.parametrize("wd", ["bf16", "fp16"])
 def test_wide_prompt_pass_matches_chunked_prompt_pass(monkeypatch, wd):
     """The wide tcgen05 GEMMs of the prompt pass (up to 512 rows at a time) against the 8-row passes on the same
