@@ -190,6 +190,34 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def c5_scoring(torch, cl, peaks, peak_kind):
+    """The all-layer confidence scoring workload (C5): 8 rounds of score -> select -> best; tensor-core bound."""
+    cc = synth.C5
+    L5, P5, d5, V5 = cc["n_layers"], cc["positions"], cc["d_model"], cc["vocab"]
+    head5 = synth.make_lm_head(cc["seed"], V5, d5, device="cuda")
+    ctx5 = cl.Context(L5, d5, d5 // 128, 11008, V5, 8, "bf16", rms_eps=cc["rms_eps"])
+    ctx5.cl_load(dict(lm_head=head5, final_norm=torch.ones(d5, device="cuda")), head_only=True)
+    hid5 = [synth.make_hidden(cc["seed"], t, L5, P5, d5, device="cuda") for t in range(cc["iters"])]
+    sc5 = synth.make_round_scores(cc["seed"], cc["iters"])
+    sel5 = cl.SelectCfg.make(cc["lo"], cc["hi"], n_skip=cc["n_skip"])
+    for _ in range(3):
+        ctx5.cl_score_loop(sel5, hid5, sc5)
+    t5 = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx5.cl_score_loop(sel5, hid5, sc5)
+        e1.record()
+        torch.cuda.synchronize()
+        t5.append(e0.elapsed_time(e1))
+    ms5 = statistics.median(t5)
+    tf5 = cc["iters"] * 2.0 * L5 * P5 * d5 * V5 / (ms5 * 1e-3) / 1e12
+    out = {"score_loop_ms": ms5, "tflops": tf5, "bound": "tensor", "frac_of_bf16_burst": tf5 / float(peaks["bf16_tflops"]),
+           "frac_of_bf16_sustained": tf5 / float(peaks["bf16_tflops_sustained"]), "peak_kind": f"of {peak_kind}"}
+    ctx5.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -201,6 +229,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the extra measurements under config.extra (profiling runs)")
     ap.add_argument("--layers", type=int, default=0, help="fewer layers of the same shape (profiling captures only)")
     ap.add_argument("--gen", type=int, default=0, help="fewer generated tokens per step (profiling captures only)")
+    ap.add_argument("--c5-only", action="store_true", help="only the C5 scoring loop; prints its object (profiling captures)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -221,6 +250,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks, peak_kind = measured_peaks()
     peak = float(peaks["hbm_gbs"])
+    if args.c5_only:
+        print(json.dumps({"c5_scoring": c5_scoring(torch, cl, peaks, peak_kind)}), flush=True)
+        return
 
     def barrier():
         if dist is not None:
@@ -407,31 +439,7 @@ def main():
                            vanilla_tokens_per_s=w4.gen_len / (v4["ms"] * 1e-3), vanilla_frac_of_peak=v4_gbs / peak)
         ctx4.close()
         torch.cuda.empty_cache()
-        # the all-layer confidence scoring workload (C5): 8 rounds of score -> select -> best, tensor-core bound
-        cc = synth.C5
-        L5, P5, d5, V5 = cc["n_layers"], cc["positions"], cc["d_model"], cc["vocab"]
-        head5 = synth.make_lm_head(cc["seed"], V5, d5, device="cuda")
-        ctx5 = cl.Context(L5, d5, d5 // 128, 11008, V5, 8, "bf16", rms_eps=cc["rms_eps"])
-        ctx5.cl_load(dict(lm_head=head5, final_norm=torch.ones(d5, device="cuda")), head_only=True)
-        hid5 = [synth.make_hidden(cc["seed"], t, L5, P5, d5, device="cuda") for t in range(cc["iters"])]
-        sc5 = synth.make_round_scores(cc["seed"], cc["iters"])
-        sel5 = cl.SelectCfg.make(cc["lo"], cc["hi"], n_skip=cc["n_skip"])
-        for _ in range(3):
-            ctx5.cl_score_loop(sel5, hid5, sc5)
-        t5 = []
-        for _ in range(5):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            ctx5.cl_score_loop(sel5, hid5, sc5)
-            e1.record()
-            torch.cuda.synchronize()
-            t5.append(e0.elapsed_time(e1))
-        ms5 = statistics.median(t5)
-        tf5 = cc["iters"] * 2.0 * L5 * P5 * d5 * V5 / (ms5 * 1e-3) / 1e12
-        extra["c5_scoring"] = {"score_loop_ms": ms5, "tflops": tf5, "bound": "tensor",
-                               "frac_of_bf16_burst": tf5 / float(peaks["bf16_tflops"]),
-                               "frac_of_bf16_sustained": tf5 / float(peaks["bf16_tflops_sustained"]), "peak_kind": f"of {peak_kind}"}
-        ctx5.close()
+        extra["c5_scoring"] = c5_scoring(torch, cl, peaks, peak_kind)
 
     if rank == 0:
         line = {
