@@ -26,8 +26,8 @@
 //     equal on both sides); rows in front of g0 and behind g1 are stale -- column n of D depends on row n of B
 //     only, and those columns are never read.
 // The accumulator lives in tensor memory (two buffers of 256 columns); it is drained into fp32 registers after
-// every `chain` ring slots (4 by default; a slot holds 64 to 320 elements of K), so a long K is summed in fp32
-// registers in pieces, not in one tensor-core chain: the pieces bound the rounding error of the chain.
+// at most `chain` k-blocks (8 by default: 512 elements of K, more where a ring entry holds more), so a long K is summed
+// in fp32 registers in pieces, not in one tensor-core chain: the pieces bound the rounding error of the chain.
 // Warp roles: warps 0-13 workers (embedding, attention, epilogues; warps 0, 4, 8, 12 are the four that can read
 // tensor-memory lanes 0-31 and drain the accumulator), warp 14 producer, warp 15 MMA issue and tensor-memory owner.
 // RMSNorm is split around the GEMM as in the other tensor-core kernels: the activation operand holds x * gain,
@@ -47,7 +47,7 @@ constexpr int RT = RW * 32;            // worker threads
 constexpr int R_THREADS = RT + 64;     // + producer warp + MMA warp
 constexpr int R_RING = 196608;         // ring of tiles in flight per SM, allocated by the byte (multiples of 1 KB)
 constexpr int R_NE = 16;               // most ring entries (bulk-copy groups with their own pair of mbarriers) in flight
-constexpr int R_MAXN = 224;            // most rows of a weight tile (tile + activation rows fill a slot at one k-block)
+constexpr int R_MAXN = 224;            // most rows of a weight tile (an accumulator buffer has 256 columns)
 constexpr int R_CTRL_BYTES = 16384;    // control block behind the ring (at least 16 KB: see the kernel)
 constexpr int R_ATT_MAXS = 8;          // most parts the cached keys of a head are cut into
 
@@ -149,8 +149,8 @@ __device__ __forceinline__ void rows_of(int rows, int unit, int split, int &r0, 
     rows_of_cta(rows, unit, blockIdx.x / split, gridDim.x / split, r0, r1);
 }
 
-// Position in the schedule: (job, group of the CTA's rows, slot).  advance() is a handful of instructions inside a
-// group (the producer, the MMA issuer and the drain warps each run it once per slot, serially, so it has to be);
+// Position in the schedule: (job, group of the CTA's rows, ring entry).  advance() is a handful of instructions inside a
+// group (the producer, the MMA issuer and the drain warps each run it once per entry, serially, so it has to be);
 // everything that costs a division is worked out once per group.
 struct Cursor {
     const ClRowsArgs &a;
@@ -166,12 +166,12 @@ struct Cursor {
     int r0, r1;               // the rows of the CTA (of its group, for a job split over K)
     // group
     int g0, g1, a0, npad;     // weight rows [g0, g1); first tile row g0 & ~7; tile rows (multiple of 16)
-    int per;                  // k-blocks per ring slot
-    unsigned stride;          // bytes between the k-block tiles of a slot (activation rows + weight rows)
+    int per;                  // k-blocks per ring entry
+    unsigned stride;          // bytes between the k-block tiles of an entry (activation rows + weight rows)
     size_t wbase;             // byte offset in W of (row g0, k-block 0)
     unsigned wstep;           // bytes between k-blocks in W (the CTA's block is [K / 64][r1 - r0][64])
-    // slot = ring entry
-    int kb0, kbs, in_chain;   // in_chain: k-blocks of the accumulation chain before this slot
+    // ring entry
+    int kb0, kbs, in_chain;   // the entry's k-blocks; in_chain: k-blocks of the accumulation chain before this entry
     // the entry's place in the ring: every role computes the same sequence.  Entries are laid end to end; one that would
     // cross the end of the ring starts at its beginning instead.  voff counts all bytes so far, the skipped ones too, so
     // an entry fits once voff + size - (voff of the oldest entry still in use) <= R_RING.
@@ -185,7 +185,7 @@ struct Cursor {
         next_job();
         place();
     }
-    __device__ __forceinline__ bool last() const { return kb0 + kbs >= kb_end; }             // last slot of the group
+    __device__ __forceinline__ bool last() const { return kb0 + kbs >= kb_end; }             // last entry of the group
     __device__ __forceinline__ bool job_last() const { return last() && g1 >= r1; }          // ... of the job, for this CTA
     __device__ __forceinline__ bool chain_first() const { return in_chain == 0; }
     __device__ __forceinline__ bool chain_last() const { return last() || in_chain + kbs >= a.chain; }
@@ -326,10 +326,10 @@ __device__ __forceinline__ void a_store_split(unsigned short *A, int t, int T, i
 __device__ __forceinline__ ClHeadPartial rp_merge(const ClHeadPartial &a, const ClHeadPartial &b) { return cl_hp_merge(a, b); }
 
 // ---- producer ------------------------------------------------------------------------------------------
-// The whole producer warp runs this (uniform control flow; lane j issues the copy of a slot's j-th k-block, so a slot
-// costs the same few instructions however many k-blocks it holds).  Weight tiles are requested as soon as a ring
-// slot is free -- weights never change, so the stream runs ahead of the grid barriers; the activation tiles of a slot
-// are requested once the completion counters of their k-blocks say so, both on the slot's one mbarrier.
+// The whole producer warp runs this (uniform control flow; lane j issues the copy of an entry's j-th k-block, so an entry
+// costs the same few instructions however many k-blocks it holds).  Weight tiles are requested as soon as the ring
+// has room for the entry -- weights never change, so the stream runs ahead of the phases; the activation tiles of an
+// entry are requested once the completion counters of their k-blocks say so, both on the entry's one mbarrier.
 __device__ void producer(const ClRowsArgs &a, unsigned char *ring, RSmem *sm, int lane) {
     const unsigned long long policy = policy_evict_first();
     Cursor w(a), q(a);                     // weight cursor; head of the queue of entries that still lack their activation tiles
@@ -515,7 +515,7 @@ __device__ __forceinline__ void gemm_job(const ClRowsArgs &a, RSmem *sm, unsigne
     bool job_done = false;
     while (!job_done) {
         const Group g{c.g0, c.g1, c.a0, c.npad};
-        // walk the tile's slots first (an accumulation chain ends after a.chain k-blocks and at the tile's end), so that
+        // walk the tile's entries first (an accumulation chain ends after a.chain k-blocks and at the tile's end), so that
         // no schedule arithmetic runs while the accumulator registers are live
         int nchains = 0;
         for (bool group_end = false; !group_end;) {
