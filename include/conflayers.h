@@ -258,8 +258,9 @@ int cl_layer_confidences_static(const void *lm_head, const float *final_norm, in
  * flight and returns; the host call that finds the flag returns CL_ETIMEOUT, clears it, commits nothing of the
  * call, and the context stays usable (re-run cl_prefill).  The paper has no counterpart; these settings exist so
  * that this path can be exercised without faulting or hanging anything:
- *   CL_DEBUG_WAIT_LIMIT_US   bound of a single wait of the persistent step kernel in microseconds (default 2 000 000)
- *   CL_DEBUG_BARRIER_EXTRA   extra arrivals its grid barriers wait for (default 0); with 1 no barrier can complete,
+ *   CL_DEBUG_WAIT_LIMIT_US   bound of a single wait of the persistent kernels (token steps, T-row pass) in microseconds
+ *                            (default 2 000 000)
+ *   CL_DEBUG_BARRIER_EXTRA   extra arrivals their grid barriers wait for (default 0); with 1 no barrier can complete,
  *                            so the first one runs into the bound
  *   CL_DEBUG_DEVICE_ERR      sets the device-side error flags to `value`, as an expired wait would */
 enum { CL_DEBUG_WAIT_LIMIT_US = 1, CL_DEBUG_BARRIER_EXTRA = 2, CL_DEBUG_DEVICE_ERR = 3 };

@@ -94,7 +94,7 @@ struct cl_ctx {
     uint64_t launches;
     // diagnostics (cl_debug_set)
     unsigned long long wait_ns;   // bound on any single device-side wait of the step kernel
-    int bar_extra;                // extra arrivals the step kernel's grid barriers wait for (0: barriers complete)
+    int bar_extra;                // extra arrivals the persistent kernels' grid barriers wait for (0: barriers complete)
 };
 
 static char g_err[512] = "";
@@ -562,7 +562,7 @@ static int forward_rows_persistent(cl_ctx *c, const int *tok, int T, int row0, i
     a.x = c->x; a.qkv = c->qkv; a.Ax = c->r_ax; a.Aatt = c->r_aatt; a.Ah = c->r_ah;
     a.ssq = c->r_ssq; a.att_part = c->r_att_part; a.att_tickets = c->r_tickets; a.head_part = c->r_head_part;
     a.logits = logits; a.out_tok = out_tok; a.out_pmax = out_pmax; a.out_conf = out_conf;
-    a.sync = c->r_bar; a.bar_arrivals = (unsigned)c->n_sm; a.wait_ns = c->wait_ns; a.phase_ns = c->r_phase_ns;
+    a.sync = c->r_bar; a.bar_arrivals = (unsigned)(c->n_sm + c->bar_extra); a.wait_ns = c->wait_ns; a.phase_ns = c->r_phase_ns;
     a.c_ssq = c->r_c_ssq; a.c_ax = c->r_c_ax; a.c_ah = c->r_c_ah; a.c_att = c->r_c_att; a.c_qkv = c->r_c_qkv;
     CU(cudaMemsetAsync(c->r_bar, 0, (size_t)c->r_sync_words * 4, c->stream));   // every counter starts at zero
     KL(cl_launch_rows_pass(g.weight_dtype, g.head_dim, a, c->n_sm, c->stream));

@@ -52,6 +52,31 @@ def test_expired_wait_returns_timeout_and_the_context_recovers():
     assert ctx2.cl_prefill(prompt) == first
 
 
+def test_expired_wait_in_the_row_pass_returns_timeout_and_the_context_recovers():
+    """The same in the persistent T-row pass of a 16-bit model: its one grid barrier (in front of the LM-head merge) waits
+    for one arrival too many and gives up after 3 ms; the launch winds down by itself (copies in flight awaited, tensor
+    memory released), cl_verify reports CL_ETIMEOUT and commits nothing, and the next pass in the same context is correct."""
+    w = synth.reduced(synth.WORKLOADS["C2"], n_layers=2, prompt_len=10, gen_len=4)
+    sh = dataclasses.replace(w.shape, max_seq=64)
+    om, ctx, _ = make_pair(sh, 8)
+    prompt = synth.make_prompt(8, 10, sh.vocab)
+    first = ctx.cl_prefill(prompt)
+    ctx.cl_force_tokens([5, 6, 7])
+    good = ctx.cl_verify(4, want_logits=True)
+    ctx.cl_debug_set(CL_DEBUG_WAIT_LIMIT_US, 3000)
+    ctx.cl_debug_set(CL_DEBUG_BARRIER_EXTRA, 1)
+    with pytest.raises(cl.ConfLayersError) as e:
+        ctx.cl_verify(4)
+    assert e.value.code == 6
+    assert ctx.cl_get_stats().ctx_len == len(prompt)
+    ctx.cl_debug_set(CL_DEBUG_BARRIER_EXTRA, 0)
+    ctx.cl_debug_set(CL_DEBUG_WAIT_LIMIT_US, 2_000_000)
+    assert ctx.cl_prefill(prompt) == first
+    ctx.cl_force_tokens([5, 6, 7])
+    again = ctx.cl_verify(4, want_logits=True)
+    assert np.array_equal(again["targets"], good["targets"]) and np.array_equal(again["logits"], good["logits"])
+
+
 @pytest.mark.parametrize("name", ["C1", "C2"])
 def test_error_flag_stops_verify_accept_and_prefill_from_committing(name):
     """A device-side error flag (what an expired wait leaves) found by cl_verify, cl_accept or cl_prefill makes the call
