@@ -482,7 +482,7 @@ extern "C" int cl_load(cl_ctx *c, const cl_weights *w) {
                 c->rows_chain = (ch && ch[0]) ? atoi(ch) : 8;
                 if (c->rows_chain < 1) c->rows_chain = 1;
                 const char *en = getenv("CL_ROWS_ENTRY_KB");   // tuning knob
-                c->rows_entry = ((en && en[0]) ? atoi(en) : 64) * 1024;
+                c->rows_entry = ((en && en[0]) ? atoi(en) : 70) * 1024;   // (a third of the ring)
                 if (c->rows_entry < 1024) c->rows_entry = 1024;
                 if (c->rows_entry > 96 * 1024) c->rows_entry = 96 * 1024;   // (two entries must fit the ring of 192 KB)
                 c->use_rows = 1;

@@ -4,7 +4,7 @@
 //
 // The pass is bound by HBM weight streaming (at most 9 flop per weight byte), so its shape follows the single-token
 // step kernel: one CTA per SM, every CTA owns a contiguous block of rows of every matrix (single-row granularity, so
-// all SMs stream the same number of bytes), one producer thread walks the static schedule and keeps a 192 KB ring of
+// all SMs stream the same number of bytes), one producer warp walks the static schedule and keeps a 210 KB ring of
 // weight tiles filled straight through the phase boundaries, and the phases of a layer (QKV | attention | O |
 // gate/up | down) follow one another inside the launch, ordered by completion counters per buffer (below), not by
 // launches.  What differs is the arithmetic: 2 T activation
@@ -45,7 +45,8 @@ namespace {
 constexpr int RW = 14;                 // worker warps (16 warps in all: four per scheduler, 128 registers per thread)
 constexpr int RT = RW * 32;            // worker threads
 constexpr int R_THREADS = RT + 64;     // + producer warp + MMA warp
-constexpr int R_RING = 196608;         // ring of tiles in flight per SM, allocated by the byte (multiples of 1 KB)
+constexpr int R_RING = 215040;         // ring of tiles in flight per SM, allocated by the byte (multiples of 1 KB): 210 KB,
+                                       // with the control block and the alignment slack all the shared memory a CTA can have
 constexpr int R_NE = 16;               // most ring entries (bulk-copy groups with their own pair of mbarriers) in flight
 constexpr int R_MAXN = 224;            // most rows of a weight tile (an accumulator buffer has 256 columns)
 constexpr int R_CTRL_BYTES = 16384;    // control block behind the ring (at least 16 KB: see the kernel)
